@@ -1,0 +1,189 @@
+/*
+ * eagle2.h -- C ABI of the B200 (sm_100a) library for the data-parallel hot path of EAGLE-2's
+ * draft-and-verify cycle: draft-tree expansion, reranking, tree mask, tree-masked attention,
+ * acceptance and KV compaction.
+ *
+ * Conventions that hold for every entry point
+ *   - Every array pointer is a DEVICE pointer owned by the caller unless marked [host].  The
+ *     library allocates nothing: scratch memory comes from a caller-supplied workspace whose size
+ *     eagle2_workspace_bytes() reports.  A workspace must be 256-byte aligned and must have been
+ *     passed through eagle2_workspace_init() once after allocation (it zeroes the arrival counters
+ *     that the kernels leave zeroed again on exit).  Calls that share a workspace must be ordered
+ *     on one stream.
+ *   - Every call only enqueues work on `stream` and returns; nothing synchronises, so a sequence of
+ *     calls can be captured in a CUDA graph.
+ *   - Return value: EAGLE2_OK, or a negative EAGLE2_ERR_* found on the host before anything was
+ *     launched.  Conditions found on the device are OR-ed into *d_status (EAGLE2_STATUS_* bits, an
+ *     int32 in device memory that the caller zeroes); the kernel still ends normally.
+ *   - Tree layout (part of the interface).  k children per expanded node and k frontier nodes per
+ *     level, depth D, N = k + (D-1)k^2 candidate nodes, R = 1 + (D-1)k draft-logit rows per cycle.
+ *     Level-1 nodes have candidate index c in [0,k); a node of level l >= 2 has index
+ *     k + (l-2)k^2 + j*k + c with j the frontier slot of its parent and c the rank of the child in
+ *     its parent's draft distribution.  parent = -1 is the root (the last committed token).  Draft
+ *     row 0 produces level 1; row 1 + (s-1)k + j belongs to frontier slot j of step s >= 1.
+ *     Lower index implies shallower-or-equal level, so "ties to the lower index" is the paper's
+ *     "ties to the shallower node", and ascending index is a topological order.
+ */
+#ifndef EAGLE2_H_
+#define EAGLE2_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct CUstream_st* eagle2_stream_t; /* a cudaStream_t */
+
+/* host-side errors (return values) */
+#define EAGLE2_OK 0
+#define EAGLE2_ERR_NULL (-1)        /* a required pointer is NULL */
+#define EAGLE2_ERR_SHAPE (-2)       /* a size is outside the supported range */
+#define EAGLE2_ERR_ALIGN (-3)       /* a base pointer or stride breaks the stated alignment */
+#define EAGLE2_ERR_WORKSPACE (-4)   /* workspace missing, misaligned or too small */
+#define EAGLE2_ERR_CUDA (-5)        /* the CUDA runtime refused the launch */
+
+/* device-side conditions (bits of *d_status) */
+#define EAGLE2_STATUS_NONFINITE_LOGIT 1 /* NaN or +Inf logit, or a row of only -Inf */
+#define EAGLE2_STATUS_NOT_CLOSED 2      /* a selected node's parent was not selected */
+#define EAGLE2_STATUS_KV_OVERFLOW 4     /* a sequence's rows exceed the stated cache capacity */
+#define EAGLE2_STATUS_TIMEOUT 8         /* a bounded device-side wait ran out */
+#define EAGLE2_STATUS_BOUNDS 16         /* an index check failed in a checked build */
+#define EAGLE2_STATUS_BAD_TREE 32       /* parent/path arrays are not a valid topological tree */
+
+/* limits */
+#define EAGLE2_MAX_K 32        /* children per node / frontier size */
+#define EAGLE2_MAX_M 128       /* rerank budget */
+#define EAGLE2_MAX_NODES 4096  /* N = k + (D-1)k^2 */
+#define EAGLE2_MAX_DEPTH 64
+
+/* operations, for eagle2_workspace_bytes */
+#define EAGLE2_OP_EXPAND 0
+#define EAGLE2_OP_RERANK 1
+#define EAGLE2_OP_TREE_MASK 2
+#define EAGLE2_OP_TREE_ATTENTION 3
+#define EAGLE2_OP_ACCEPT 4
+#define EAGLE2_OP_KV_COMPACT 5
+
+int eagle2_version(void);
+const char* eagle2_strerror(int code);
+
+/* Bytes of workspace the given operation needs at these sizes (0 if it needs none; sizes that do
+ * not apply to the operation are ignored).  max_kv_len is the largest kv_len of any sequence. */
+size_t eagle2_workspace_bytes(int op, int B, int V, int k, int D, int m, int Hq, int Hkv, int d,
+                              int max_kv_len);
+
+/* Zero a freshly allocated workspace (asynchronous on `stream`). */
+int eagle2_workspace_init(void* ws, size_t ws_bytes, eagle2_stream_t stream);
+
+/*
+ * Step 1 -- expansion (paper Section 4.1, the value equation V_i = prod c_j over Path(root, t_i)).
+ * Called for s = 0..D-1.  For each of the n_s input rows (n_s = 1 at s = 0, else k; row j belongs
+ * to frontier[b][j]) it takes the log-softmax over the vocabulary, makes the k most probable tokens
+ * the node's children (ties: lower token id) and gives each the value parent value + log-probability,
+ * i.e. the log of the product of draft confidences on the path (the root counts as 1).  The k best
+ * new candidates by value (ties: lower index) become the next frontier.
+ *   draft_logits  fp32 [B][n_s][V]; sequence b starts at draft_logits + b*batch_stride (elements).
+ *                 16-byte aligned base and V % 4 == 0 select the vectorised path; anything else is
+ *                 still handled.
+ *   tree_token, tree_parent  int32 [B][N], tree_value fp64 [B][N]: level s+1 is written; earlier
+ *                 levels are read (values of the frontier nodes).
+ *   frontier      int32 [B][k]: read when s > 0, overwritten with the new frontier.
+ * Limits: 1 <= k <= min(V, EAGLE2_MAX_K), N <= EAGLE2_MAX_NODES.
+ */
+int eagle2_expand(const float* draft_logits, long long batch_stride, int B, int V, int k, int D, int s,
+                  int32_t* tree_token, int32_t* tree_parent, double* tree_value, int32_t* frontier,
+                  void* ws, size_t ws_bytes, int32_t* d_status, eagle2_stream_t stream);
+
+/*
+ * Step 2a -- reranking (paper Section 4.2): the n_sel = min(m, N) nodes with the highest value among
+ * ALL candidates, equal values preferring the shallower (lower-index) node, which keeps the set
+ * closed under parents.  Values are clamped to the parent's effective value first, which changes
+ * nothing for trees made by eagle2_expand and keeps closure for arbitrary values.  The selection is
+ * flattened in ascending candidate index.
+ *   sel_index [B][m] candidate index, sel_parent [B][m] flat position of the parent (-1: root),
+ *   sel_token [B][m], sel_depth [B][m] (level - 1), n_sel [B].  Rows >= n_sel are padding
+ *   (index -1, parent -1, token 0, depth 0).
+ * Limits: 1 <= m <= EAGLE2_MAX_M, N <= EAGLE2_MAX_NODES.  Needs no workspace.
+ */
+int eagle2_rerank(const int32_t* tree_token, const int32_t* tree_parent, const double* tree_value,
+                  int B, int k, int D, int m, int32_t* sel_index, int32_t* sel_parent,
+                  int32_t* sel_token, int32_t* sel_depth, int32_t* n_sel, int32_t* d_status,
+                  eagle2_stream_t stream);
+
+/*
+ * Step 2b -- tree attention mask and position ids (paper Section 4.2: a draft token sees only its
+ * ancestors).  Row i of the mask has bit i and the bits of all ancestors of flat node i set; padding
+ * rows have only their own bit.  pos_ids = kv_len + depth (the root is the last committed token).
+ *   mask_bits  uint64 [B][m][ceil(m/64)], bit j of row i = token i sees token j.
+ *   mask_dense uint8 [B][m][m], optional (NULL to skip).
+ *   pos_ids    int32 [B][m].
+ */
+int eagle2_tree_mask(const int32_t* sel_parent, const int32_t* sel_depth, const int32_t* n_sel,
+                     const int32_t* kv_len, int B, int m, uint64_t* mask_bits, uint8_t* mask_dense,
+                     int32_t* pos_ids, int32_t* d_status, eagle2_stream_t stream);
+
+/*
+ * Step 3 -- tree-masked attention of the verification pass (paper Section 4.2), one layer per call:
+ *   out[b,i,h,:] = sum_j softmax_j(scale * q[b,i,h,:].k[j,h/g,:]) v[j,h/g,:]
+ * over the keys token i may see: every committed cache row [0, kv_len[b]) of its sequence and the
+ * tree rows j whose bit is set in mask row i.  bf16 operands, fp32 accumulation, bf16 result.
+ *   q        bf16 [B][m][Hq][d]
+ *   k_cache, v_cache  bf16 [rows][Hkv][d]; sequence b owns rows kv_off[b] .. kv_off[b]+kv_len[b]+m-1,
+ *            the K/V of tree token j at local row kv_len[b]+j.
+ *   kv_off   int64 [B], kv_len int32 [B], mask_bits as written by eagle2_tree_mask.
+ *   out      bf16 [B][m][Hq][d];  lse fp32 [B][Hq][m], optional natural-log sum of exponentials.
+ *   max_kv_len [host value] upper bound of kv_len[], used only to size the launch.
+ * Limits: d in {64,128}; Hq % Hkv == 0 with Hq/Hkv <= 8; 16-byte aligned q, caches and out.
+ */
+int eagle2_tree_attention(const void* q, const void* k_cache, const void* v_cache,
+                          const int64_t* kv_off, const int32_t* kv_len, const uint64_t* mask_bits,
+                          int B, int m, int Hq, int Hkv, int d, int max_kv_len, float scale, void* out,
+                          float* lse, void* ws, size_t ws_bytes, int32_t* d_status,
+                          eagle2_stream_t stream);
+
+/*
+ * Step 4 -- acceptance (paper Section 2.1 rule, walked over the tree as in Section 2.2).
+ * Rows of target_logits: row 0 belongs to the root, row 1+x to flat node x.  The children of a node
+ * are the selected nodes whose sel_parent is that node, in ascending flat position.
+ *   temperature == 0: follow the child whose token is the arg-max (lowest id on ties) of the target
+ *     row of the current node; the extra token is the arg-max at the node where the walk stops.
+ *   temperature  > 0: at the current node p = softmax(target/T), q = softmax(draft/T) with the draft
+ *     row that produced the node's children; child x is accepted iff u_accept[x] < min(1, p(x)/q(x));
+ *     after a rejection p <- norm(max(p-q,0)) and q loses the rejected token and is renormalised.
+ *     With draft_logits_all == NULL the proposal is the point mass on the candidate (accept with
+ *     probability p(x), then remove x from p), which is lossless for deterministic top-k children.
+ *     The extra token is drawn from the p in force when the walk stops, by inverse CDF in ascending
+ *     token id: the first t with sum_{v<=t} p(v) > u_bonus * sum_v p(v).
+ *   target_logits     fp32 [B][m+1][V], sequence stride t_stride elements (0 shares one set).
+ *   draft_logits_all  fp32 [B][R][V], stride d_stride; may be NULL (see above).
+ *   u_accept fp32 [B][m] indexed by flat node, u_bonus fp32 [B], both in [0,1); unused at T == 0.
+ *   acc_len [B] accepted draft tokens, acc_path [B][D] their flat positions (-1 padded),
+ *   bonus_token [B].
+ */
+int eagle2_accept(const float* target_logits, long long t_stride, const float* draft_logits_all,
+                  long long d_stride, const int32_t* sel_index, const int32_t* sel_parent,
+                  const int32_t* sel_token, const int32_t* n_sel, int B, int V, int k, int D, int m,
+                  float temperature, const float* u_accept, const float* u_bonus, int32_t* acc_len,
+                  int32_t* acc_path, int32_t* bonus_token, void* ws, size_t ws_bytes,
+                  int32_t* d_status, eagle2_stream_t stream);
+
+/*
+ * Step 5 -- KV compaction (paper Section 2.1: rejected draft tokens are discarded; Appendix A: the
+ * cache is pre-allocated).  For every layer, K and V, the accepted tree rows move to the front of
+ * the tree region: local row kv_len+acc_path[j] -> kv_len+j for j < acc_len, then kv_len += acc_len.
+ *   k_layers, v_layers  device arrays of n_layers device pointers to bf16 [rows][Hkv][d] caches.
+ *   kv_len in/out.  acc_path must be strictly increasing with acc_path[j] >= j (a root path in
+ *   topological order); otherwise EAGLE2_STATUS_BAD_TREE is raised and that sequence is left alone.
+ * Limits: Hkv*d*2 bytes per row a multiple of 16; D <= 16.
+ */
+int eagle2_kv_compact(void* const* k_layers, void* const* v_layers, int n_layers,
+                      const int64_t* kv_off, int32_t* kv_len, const int32_t* acc_path,
+                      const int32_t* acc_len, int B, int m, int D, int Hkv, int d, int32_t* d_status,
+                      eagle2_stream_t stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* EAGLE2_H_ */

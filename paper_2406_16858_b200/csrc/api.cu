@@ -1,0 +1,49 @@
+// Library-level entry points: version, error strings, workspace sizing and initialisation.
+#include "common.cuh"
+
+namespace eagle2 {
+size_t expand_workspace_bytes(int B, int V, int k);
+size_t accept_workspace_bytes(int B, int V, int k, int D, int m);
+size_t attention_workspace_bytes(int B, int m, int Hq, int Hkv, int d, int max_kv_len);
+}  // namespace eagle2
+
+extern "C" int eagle2_version(void) { return 100; }
+
+extern "C" const char* eagle2_strerror(int code) {
+    switch (code) {
+        case EAGLE2_OK: return "ok";
+        case EAGLE2_ERR_NULL: return "a required pointer is NULL";
+        case EAGLE2_ERR_SHAPE: return "a size is outside the supported range";
+        case EAGLE2_ERR_ALIGN: return "a pointer or stride is not aligned as required";
+        case EAGLE2_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case EAGLE2_ERR_CUDA: return "the CUDA runtime refused the launch";
+        default: return "unknown error code";
+    }
+}
+
+extern "C" size_t eagle2_workspace_bytes(int op, int B, int V, int k, int D, int m, int Hq, int Hkv, int d,
+                                         int max_kv_len) {
+    if (B < 1) return 0;
+    switch (op) {
+        case EAGLE2_OP_EXPAND:
+            if (V < 1 || k < 1 || k > EAGLE2_MAX_K) return 0;
+            return eagle2::expand_workspace_bytes(B, V, k);
+        case EAGLE2_OP_ACCEPT:
+            if (V < 1 || k < 1 || D < 1 || m < 1) return 0;
+            return eagle2::accept_workspace_bytes(B, V, k, D, m);
+        case EAGLE2_OP_TREE_ATTENTION:
+            if (m < 1 || Hq < 1 || Hkv < 1 || Hq % Hkv || (d != 64 && d != 128) || max_kv_len < 0) return 0;
+            return eagle2::attention_workspace_bytes(B, m, Hq, Hkv, d, max_kv_len);
+        default:
+            return 0;  // rerank, tree mask and KV compaction work in place
+    }
+}
+
+extern "C" int eagle2_workspace_init(void* ws, size_t ws_bytes, eagle2_stream_t stream) {
+    if (ws_bytes == 0) return EAGLE2_OK;
+    if (!ws) return EAGLE2_ERR_NULL;
+    if (!eagle2::aligned(ws, eagle2::kWsAlign)) return EAGLE2_ERR_WORKSPACE;
+    return cudaMemsetAsync(ws, 0, ws_bytes, reinterpret_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? EAGLE2_OK
+               : EAGLE2_ERR_CUDA;
+}

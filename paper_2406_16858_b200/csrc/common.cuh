@@ -1,0 +1,100 @@
+// Shared device/host helpers of the sm_100a library (no arithmetic of the method lives here).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "eagle2.h"
+
+namespace eagle2 {
+
+constexpr int kWarp = 32;
+constexpr size_t kWsAlign = 256;
+
+__host__ __device__ inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+__host__ __device__ inline long long nodes_of(int k, int D) {
+    return (long long)k + (long long)(D - 1) * k * k;
+}
+
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+inline int launch_result() { return cudaGetLastError() == cudaSuccess ? EAGLE2_OK : EAGLE2_ERR_CUDA; }
+
+#ifdef __CUDACC__
+
+__device__ __forceinline__ void raise_status(int32_t* d_status, int bits) {
+    if (bits) atomicOr(d_status, bits);
+}
+
+// Monotone map float -> uint32 (larger float, larger code).  -0 is folded onto +0 first so that
+// equal values always get equal codes; NaN maps to 0, the lowest code.
+__device__ __forceinline__ uint32_t order_code(float x) {
+    if (x != x) return 0u;
+    const uint32_t u = __float_as_uint(x + 0.0f);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float order_decode(uint32_t c) {
+    const uint32_t u = (c & 0x80000000u) ? (c & 0x7fffffffu) : ~c;
+    return __uint_as_float(u);
+}
+// 64-bit selection key: value code in the high word, complemented index in the low word, so the
+// maximum key is the largest value and, among equal values, the lowest index.  Valid keys are > 0.
+__device__ __forceinline__ unsigned long long make_key(float x, uint32_t idx) {
+    return ((unsigned long long)order_code(x) << 32) | (unsigned long long)(0xffffffffu - idx);
+}
+__device__ __forceinline__ uint32_t key_index(unsigned long long key) {
+    return 0xffffffffu - (uint32_t)(key & 0xffffffffu);
+}
+__device__ __forceinline__ float key_value(unsigned long long key) {
+    return order_decode((uint32_t)(key >> 32));
+}
+
+__device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const unsigned long long other = __shfl_xor_sync(0xffffffffu, v, o);
+        v = other > v ? other : v;
+    }
+    return v;
+}
+__device__ __forceinline__ float warp_max_f32(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+__device__ __forceinline__ float warp_sum_f32(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ double warp_sum_f64(double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ double warp_max_f64(double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmax(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+
+// Arrival ticket: returns true in exactly one block, the last of `expected` to arrive, after every
+// other block's earlier global writes are visible to it.  The counter is left at zero.
+__device__ __forceinline__ bool last_block_arrives(int* counter, int expected, int* smem_flag) {
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const int t = atomicAdd(counter, 1);
+        const int last = (t == expected - 1);
+        if (last) *counter = 0;
+        *smem_flag = last;
+    }
+    __syncthreads();
+    const bool last = *smem_flag != 0;
+    if (last) __threadfence();
+    return last;
+}
+
+#endif  // __CUDACC__
+
+}  // namespace eagle2

@@ -1,0 +1,192 @@
+// Step 2 of the hot path (paper Section 4.2): reranking of all candidate nodes by value, flattening
+// of the selected subtree, and the ancestor attention mask with position ids.  The data is a few
+// kilobytes per sequence, so each sequence is one thread block working in shared memory.
+#include <math.h>
+
+#include "common.cuh"
+
+namespace eagle2 {
+
+constexpr int kRerankThreads = 512;
+
+__global__ void __launch_bounds__(kRerankThreads)
+rerank_kernel(const int32_t* __restrict__ tree_token, const int32_t* __restrict__ tree_parent,
+              const double* __restrict__ tree_value, int k, int N, int m, int keep,
+              int32_t* __restrict__ sel_index, int32_t* __restrict__ sel_parent,
+              int32_t* __restrict__ sel_token, int32_t* __restrict__ sel_depth,
+              int32_t* __restrict__ n_sel, int32_t* d_status) {
+    extern __shared__ __align__(16) unsigned char s_dyn[];
+    double* s_val = reinterpret_cast<double*>(s_dyn);            // [N] value, then effective value
+    double* s_eff = s_val + N;                                   // [N]
+    int32_t* s_par = reinterpret_cast<int32_t*>(s_eff + N);      // [N]
+    int32_t* s_flat = s_par + N;                                 // [N] flat position or -1
+    __shared__ int s_scan[kRerankThreads];
+
+    const int b = blockIdx.x, tid = threadIdx.x;
+    const int32_t* tok = tree_token + (long long)b * N;
+    const int32_t* par = tree_parent + (long long)b * N;
+    const double* val = tree_value + (long long)b * N;
+    int status = 0;
+
+    for (int i = tid; i < N; i += kRerankThreads) {
+        int p = par[i];
+        if (p < -1 || p >= i) {
+            status |= EAGLE2_STATUS_BAD_TREE;
+            p = -1;
+        }
+        double v = val[i];
+        if (v != v) {
+            status |= EAGLE2_STATUS_NONFINITE_LOGIT;
+            v = -INFINITY;
+        }
+        s_par[i] = p;
+        s_val[i] = v;
+    }
+    __syncthreads();
+    // effective value = minimum of the values on the path from the root (parents have lower
+    // indices, so the walk ends)
+    for (int i = tid; i < N; i += kRerankThreads) {
+        double v = s_val[i];
+        for (int a = s_par[i]; a >= 0; a = s_par[a]) v = fmin(v, s_val[a]);
+        s_eff[i] = v;
+    }
+    __syncthreads();
+    // rank by (effective value desc, index asc); the first `keep` are selected
+    const int per = (N + kRerankThreads - 1) / kRerankThreads;
+    const int lo = tid * per, hi = min(N, lo + per);
+    int mine = 0;
+    for (int i = lo; i < hi; ++i) {
+        const double vi = s_eff[i];
+        int rank = 0;
+        for (int j = 0; j < N; ++j) {
+            const double vj = s_eff[j];
+            rank += (vj > vi) || (vj == vi && j < i);
+        }
+        const int chosen = rank < keep;
+        s_flat[i] = chosen ? 0 : -1;
+        mine += chosen;
+    }
+    // exclusive scan of the per-thread counts -> flat positions in ascending index
+    s_scan[tid] = mine;
+    __syncthreads();
+    for (int o = 1; o < kRerankThreads; o <<= 1) {
+        const int add = tid >= o ? s_scan[tid - o] : 0;
+        __syncthreads();
+        s_scan[tid] += add;
+        __syncthreads();
+    }
+    int pos = s_scan[tid] - mine;
+    for (int i = lo; i < hi; ++i)
+        if (s_flat[i] == 0) s_flat[i] = pos++;
+    __syncthreads();
+
+    int32_t* o_idx = sel_index + (long long)b * m;
+    int32_t* o_par = sel_parent + (long long)b * m;
+    int32_t* o_tok = sel_token + (long long)b * m;
+    int32_t* o_dep = sel_depth + (long long)b * m;
+    for (int i = tid; i < N; i += kRerankThreads) {
+        const int j = s_flat[i];
+        if (j < 0) continue;
+        const int p = s_par[i];
+        int fp = -1;
+        if (p >= 0) {
+            fp = s_flat[p];
+            if (fp < 0) status |= EAGLE2_STATUS_NOT_CLOSED;
+        }
+        o_idx[j] = i;
+        o_par[j] = fp;
+        o_tok[j] = tok[i];
+        o_dep[j] = i < k ? 0 : 1 + (i - k) / (k * k);
+    }
+    for (int j = keep + tid; j < m; j += kRerankThreads) {
+        o_idx[j] = -1;
+        o_par[j] = -1;
+        o_tok[j] = 0;
+        o_dep[j] = 0;
+    }
+    if (tid == 0) n_sel[b] = keep;
+    if (status) raise_status(d_status, status);
+}
+
+__global__ void __launch_bounds__(EAGLE2_MAX_M)
+tree_mask_kernel(const int32_t* __restrict__ sel_parent, const int32_t* __restrict__ sel_depth,
+                 const int32_t* __restrict__ n_sel, const int32_t* __restrict__ kv_len, int m,
+                 uint64_t* __restrict__ mask_bits, uint8_t* __restrict__ mask_dense,
+                 int32_t* __restrict__ pos_ids, int32_t* d_status) {
+    __shared__ int32_t s_par[EAGLE2_MAX_M];
+    const int b = blockIdx.x, i = threadIdx.x;
+    const int W = (m + 63) / 64;
+    const int ns = n_sel[b];
+    if (i < m) s_par[i] = sel_parent[(long long)b * m + i];
+    __syncthreads();
+    if (i >= m) return;
+    uint64_t row[(EAGLE2_MAX_M + 63) / 64] = {0, 0};
+    int status = 0;
+    row[i >> 6] |= 1ull << (i & 63);
+    if (i < ns) {
+        int a = i;
+        for (;;) {
+            const int p = s_par[a];
+            if (p < 0) {
+                if (p < -1) status |= EAGLE2_STATUS_BAD_TREE;
+                break;
+            }
+            if (p >= a) {  // parents precede children: also bounds the walk
+                status |= EAGLE2_STATUS_BAD_TREE;
+                break;
+            }
+            row[p >> 6] |= 1ull << (p & 63);
+            a = p;
+        }
+    }
+    for (int w = 0; w < W; ++w) mask_bits[((long long)b * m + i) * W + w] = row[w];
+    pos_ids[(long long)b * m + i] = kv_len[b] + (i < ns ? sel_depth[(long long)b * m + i] : 0);
+    if (mask_dense) {
+        uint8_t* d = mask_dense + ((long long)b * m + i) * m;
+        for (int j = 0; j < m; ++j) d[j] = (uint8_t)((row[j >> 6] >> (j & 63)) & 1ull);
+    }
+    if (status) raise_status(d_status, status);
+}
+
+}  // namespace eagle2
+
+using namespace eagle2;
+
+extern "C" int eagle2_rerank(const int32_t* tree_token, const int32_t* tree_parent,
+                             const double* tree_value, int B, int k, int D, int m, int32_t* sel_index,
+                             int32_t* sel_parent, int32_t* sel_token, int32_t* sel_depth,
+                             int32_t* n_sel, int32_t* d_status, eagle2_stream_t stream) {
+    if (!tree_token || !tree_parent || !tree_value || !sel_index || !sel_parent || !sel_token ||
+        !sel_depth || !n_sel || !d_status)
+        return EAGLE2_ERR_NULL;
+    if (B < 0 || k < 1 || k > EAGLE2_MAX_K || D < 1 || D > EAGLE2_MAX_DEPTH || m < 1 ||
+        m > EAGLE2_MAX_M || nodes_of(k, D) > EAGLE2_MAX_NODES)
+        return EAGLE2_ERR_SHAPE;
+    if (!aligned(tree_value, 8)) return EAGLE2_ERR_ALIGN;
+    if (B == 0) return EAGLE2_OK;
+    const int N = (int)nodes_of(k, D);
+    const int keep = m < N ? m : N;
+    const size_t dyn = (size_t)N * (2 * sizeof(double) + 2 * sizeof(int32_t));
+    if (dyn > 40 * 1024 &&
+        cudaFuncSetAttribute(rerank_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) !=
+            cudaSuccess)
+        return EAGLE2_ERR_CUDA;
+    rerank_kernel<<<B, kRerankThreads, dyn, reinterpret_cast<cudaStream_t>(stream)>>>(
+        tree_token, tree_parent, tree_value, k, N, m, keep, sel_index, sel_parent, sel_token, sel_depth,
+        n_sel, d_status);
+    return launch_result();
+}
+
+extern "C" int eagle2_tree_mask(const int32_t* sel_parent, const int32_t* sel_depth,
+                                const int32_t* n_sel, const int32_t* kv_len, int B, int m,
+                                uint64_t* mask_bits, uint8_t* mask_dense, int32_t* pos_ids,
+                                int32_t* d_status, eagle2_stream_t stream) {
+    if (!sel_parent || !sel_depth || !n_sel || !kv_len || !mask_bits || !pos_ids || !d_status)
+        return EAGLE2_ERR_NULL;
+    if (B < 0 || m < 1 || m > EAGLE2_MAX_M) return EAGLE2_ERR_SHAPE;
+    if (!aligned(mask_bits, 8)) return EAGLE2_ERR_ALIGN;
+    if (B == 0) return EAGLE2_OK;
+    tree_mask_kernel<<<B, EAGLE2_MAX_M, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
+        sel_parent, sel_depth, n_sel, kv_len, m, mask_bits, mask_dense, pos_ids, d_status);
+    return launch_result();
+}

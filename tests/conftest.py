@@ -24,3 +24,12 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(scope="session", autouse=True)
+def _built_libraries():
+    """The C-ABI library and the oracle are compiled once per test session (nvcc / gcc)."""
+    from paper_2406_16858_b200 import build as build_lib
+    build_lib.build()
+    from oracle import ref
+    ref.build()

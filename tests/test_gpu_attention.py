@@ -1,0 +1,133 @@
+"""GPU parity: tree-masked attention against the CPU oracle, within 2e-2 absolute (bf16 output,
+fp32 accumulation), through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2406_16858_b200 as e2
+from oracle import ref
+from workloads import get_config
+from workloads import generators as gen
+
+from harness import DEV, dev, gpu_attention, host, make_ws, new_status
+
+pytestmark = pytest.mark.gpu
+TOL = 2e-2
+
+
+def _random_forest_mask(rng, B, m, kv_len, n_sel=None):
+    parent = np.full((B, m), -1, np.int32)
+    depth = np.zeros((B, m), np.int32)
+    for b in range(B):
+        for i in range(1, m):
+            parent[b, i] = rng.integers(-1, i)
+            depth[b, i] = 0 if parent[b, i] < 0 else depth[b, parent[b, i]] + 1
+    ns = np.full(B, m, np.int32) if n_sel is None else n_sel
+    bits, _, _, st = ref.tree_mask(parent, depth, ns, kv_len, m)
+    assert st == 0
+    return bits
+
+
+def _inputs(seed, B, m, Hq, Hkv, d, lens):
+    rng = np.random.default_rng(seed)
+    kv_len = np.array(lens, np.int32)
+    kv_off = gen.kv_offsets(kv_len, m)
+    rows = int(kv_off[-1] + kv_len[-1] + m)
+    q = gen.f32_to_bf16_bits(rng.standard_normal((B, m, Hq, d)).astype(np.float32))
+    kc = gen.f32_to_bf16_bits(rng.standard_normal((rows, Hkv, d)).astype(np.float32))
+    vc = gen.f32_to_bf16_bits(rng.standard_normal((rows, Hkv, d)).astype(np.float32))
+    return q, kc, vc, kv_off, kv_len, _random_forest_mask(rng, B, m, kv_len)
+
+
+def _compare(q, kc, vc, kv_off, kv_len, bits, scale, samples=None):
+    got, lse, st = gpu_attention(q, kc, vc, kv_off, kv_len, bits, scale, want_lse=True)
+    assert st == 0
+    gf = gen.bf16_bits_to_f32(got).astype(np.float64)
+    if samples is None:
+        _, want, wlse = ref.tree_attention(q, kc, vc, kv_off, kv_len, bits, scale, want_lse=True)
+        assert np.abs(gf - want).max() <= TOL
+        assert np.abs(lse - wlse).max() <= 2e-2
+    else:
+        _, want, wlse = ref.tree_attention(q, kc, vc, kv_off, kv_len, bits, scale, samples=samples,
+                                           want_lse=True)
+        for t, (b, h, i) in enumerate(samples):
+            assert np.abs(gf[b, i, h] - want[t]).max() <= TOL
+            assert abs(lse[b, h, i] - wlse[t]) <= 2e-2
+    return gf
+
+
+@pytest.mark.parametrize("seed", range(5))
+def test_tiny_config(seed):
+    cfg = get_config("tiny")
+    q, kc, vc, off, kl, bits = _inputs(seed, 1, cfg.m, cfg.Hq, cfg.Hkv, cfg.d, [cfg.kv_len])
+    _compare(q, kc, vc, off, kl, bits, 1.0 / np.sqrt(cfg.d))
+
+
+@pytest.mark.parametrize("m,Hq,Hkv,d,lens", [
+    (16, 4, 4, 64, [0]),            # no cache at all: tree rows only
+    (16, 4, 4, 64, [1]),
+    (60, 8, 2, 128, [63]),          # GQA g=4, a single partly filled tile
+    (60, 8, 2, 128, [64, 65, 4]),   # tile boundaries, ragged batch
+    (60, 8, 1, 128, [300]),         # g=8: two row blocks
+    (128, 4, 1, 64, [777]),         # largest m, two mask words
+    (7, 2, 2, 64, [129, 1000]),
+    (60, 32, 8, 128, [2050, 31]),
+    (1, 1, 1, 128, [500]),
+])
+def test_shapes_tails_and_gqa(m, Hq, Hkv, d, lens):
+    q, kc, vc, off, kl, bits = _inputs(11, len(lens), m, Hq, Hkv, d, lens)
+    _compare(q, kc, vc, off, kl, bits, 1.0 / np.sqrt(d))
+
+
+def test_padding_rows_see_only_themselves_and_cache():
+    rng = np.random.default_rng(0)
+    m, H, d, L = 16, 2, 64, 40
+    q, kc, vc, off, kl, _ = _inputs(5, 1, m, H, H, d, [L])
+    bits = _random_forest_mask(rng, 1, m, kl, n_sel=np.array([9], np.int32))
+    _compare(q, kc, vc, off, kl, bits, 0.125)
+
+
+def test_large_scores_do_not_overflow():
+    q, kc, vc, off, kl, bits = _inputs(6, 1, 16, 2, 2, 64, [200])
+    _compare(q, kc, vc, off, kl, bits, 3.0)  # sharply peaked softmax
+
+
+@pytest.mark.parametrize("name", ["vicuna7b", "llama3_8b", "llama2_70b"])
+def test_full_size_one_layer_sampled(name):
+    """BASELINE sizes, the launch configuration the benchmark times; the oracle computes sampled
+    (sequence, head, query) rows one by one."""
+    cfg = get_config(name)
+    g = torch.Generator(device=DEV).manual_seed(1234)
+    kv_len = gen.kv_lengths(cfg, 0)
+    kv_off = gen.kv_offsets(kv_len, cfg.m)
+    rows = int(kv_off[-1] + kv_len[-1] + cfg.m)
+    tq = torch.randn((cfg.B, cfg.m, cfg.Hq, cfg.d), generator=g, device=DEV).to(torch.bfloat16)
+    tk = torch.randn((rows, cfg.Hkv, cfg.d), generator=g, device=DEV).to(torch.bfloat16)
+    tv = torch.randn((rows, cfg.Hkv, cfg.d), generator=g, device=DEV).to(torch.bfloat16)
+    draft = gen.draft_rows(cfg, 0)
+    tree = ref.build_tree(draft, cfg.V, cfg.k, cfg.D)
+    sel = ref.rerank(tree.token, tree.parent, tree.value, cfg.k, cfg.D, cfg.m)
+    bits, _, _, _ = ref.tree_mask(sel.parent, sel.depth, sel.n_sel, kv_len, cfg.m)
+    out = torch.zeros_like(tq)
+    st = new_status()
+    ws = make_ws(e2.workspace_bytes(e2.OP_TREE_ATTENTION, B=cfg.B, m=cfg.m, Hq=cfg.Hq, Hkv=cfg.Hkv,
+                                    d=cfg.d, max_kv_len=int(kv_len.max())))
+    e2.tree_attention(tq, tk, tv, dev(kv_off), dev(kv_len), dev(bits), cfg.B, cfg.m, cfg.Hq, cfg.Hkv,
+                      cfg.d, int(kv_len.max()), 1.0 / np.sqrt(cfg.d), out, None, ws, st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    rng = np.random.default_rng(1)
+    n = 48
+    samples = np.stack([rng.integers(0, cfg.B, n), rng.integers(0, cfg.Hq, n),
+                        rng.integers(0, cfg.m, n)], axis=1).astype(np.int32)
+    samples[0] = (0, 0, 0)
+    samples[1] = (cfg.B - 1, cfg.Hq - 1, cfg.m - 1)
+    _, want, _ = ref.tree_attention(host(tq.view(torch.int16), np.uint16), host(tk.view(torch.int16), np.uint16),
+                                    host(tv.view(torch.int16), np.uint16), kv_off, kv_len, bits,
+                                    1.0 / np.sqrt(cfg.d), samples=samples)
+    got = out.float().cpu().numpy().astype(np.float64)
+    for t, (b, h, i) in enumerate(samples):
+        assert np.abs(got[b, i, h] - want[t]).max() <= TOL
+    # property that holds at any size: rows are finite and bounded by the largest |v|
+    assert torch.isfinite(out.float()).all()
+    assert out.float().abs().max() <= tv.float().abs().max()
