@@ -1,0 +1,405 @@
+#!/usr/bin/env python
+"""Benchmark of the draft-and-verify hot path: microseconds per draft-tree cycle.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload llama3_8b] [--impl ours|reference]
+
+A step is one whole cycle (D x expand, rerank, tree mask, one tree attention per layer, accept, KV
+compaction) on seeded synthetic inputs that are resident in HBM, replayed as one CUDA graph.  Rank 0
+prints one JSON line.  With N > 1 every rank runs an independent replica (the path has no exchange
+step); the value is then the time per cycle over all replicas.
+
+``--impl reference`` times the CPU oracle, as it stands, on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from workloads import generators as gen  # noqa: E402
+from workloads import get_config  # noqa: E402
+
+METRIC = "us_per_draft_tree_cycle"
+N_SETS = 4  # rotating logit sets: 4 x (draft + target rows) is larger than the 126 MB L2
+
+# dram__bytes_read.sum + dram__bytes_write.sum of one tree-attention launch, from the ncu capture
+# summarised under profiles/ (None: not captured for that workload)
+NCU_DRAM_BYTES_PER_LAUNCH = {}
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return float(p["hbm_gbs"]), float(p.get("bf16_tflops_sustained", 1400.0)), "measured"
+    return 6650.0, 1400.0, "fallback"
+
+
+# ------------------------------------------------------------------------------------------------
+# clocks during the timed region
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML (read-only) while the timed work runs."""
+
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown",
+               0x4: "sw_power_cap"}
+
+    def __init__(self, index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            self._h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self._nv = None
+
+    def _run(self):
+        nv = self._nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                bits = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self._h))
+                for bit, name in self.REASONS.items():
+                    if bits & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            self._stop.wait(0.02)
+
+    def __enter__(self):
+        if self._nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        med = int(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU oracle timing (cpu_baseline leg and --impl reference)
+
+def oracle_cycle_seconds(cfg, seed: int = 0, attn_samples: int = 96):
+    """Times the oracle on a bounded sample of one cycle and extrapolates to the whole cycle.
+    Logit steps and tree steps run whole; attention runs `attn_samples` query rows of one layer and is
+    scaled to n_layers * m * Hq rows; compaction runs on one layer and is scaled to n_layers."""
+    from oracle import ref
+    small = cfg.with_(B=1)
+    t = {}
+    draft = gen.draft_rows(small, seed)
+    t0 = time.perf_counter()
+    tree = ref.build_tree(draft, small.V, small.k, small.D)
+    t["expand"] = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    sel = ref.rerank(tree.token, tree.parent, tree.value, small.k, small.D, small.m)
+    kv_len = gen.kv_lengths(small, seed)
+    bits, _, _, _ = ref.tree_mask(sel.parent, sel.depth, sel.n_sel, kv_len, small.m)
+    t["rerank_mask"] = time.perf_counter() - t0
+    kv_off = gen.kv_offsets(kv_len, small.m)
+    q, kc, vc = gen.qkv_bf16(small, seed, kv_len, kv_off)
+    rng = np.random.default_rng(seed)
+    samples = np.stack([np.zeros(attn_samples, np.int64), rng.integers(0, small.Hq, attn_samples),
+                        rng.integers(0, small.m, attn_samples)], axis=1).astype(np.int32)
+    t0 = time.perf_counter()
+    ref.tree_attention(q, kc, vc, kv_off, kv_len, bits, 1.0 / math.sqrt(small.d), samples=samples)
+    per_row = (time.perf_counter() - t0) / attn_samples
+    t["attention_extrapolated"] = per_row * small.m * small.Hq * small.n_layers
+    target = gen.target_rows(small, seed, draft, tree.parent, sel.index)
+    ua, ub = gen.uniforms(small, seed)
+    t0 = time.perf_counter()
+    acc = ref.accept(target, draft if small.temperature > 0 else None, sel, small.V, small.k, small.D,
+                     small.m, small.temperature, ua, ub)
+    t["accept"] = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    ref.kv_compact([kc], [vc], kv_off, kv_len.copy(), acc.acc_path, acc.acc_len, small.m, small.D)
+    t["kv_compact_extrapolated"] = (time.perf_counter() - t0) * small.n_layers
+    total = sum(t.values())
+    sample = (f"B=1 of {cfg.name}: expand/rerank/mask/accept whole; attention {attn_samples} of "
+              f"{small.m * small.Hq * small.n_layers} query rows (1 layer) scaled; compaction 1 of "
+              f"{small.n_layers} layers scaled")
+    return total, t, sample, ref.num_threads()
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cfg = get_config(args.workload)
+    steps, warmup = max(1, min(args.steps, 3)), min(args.warmup, 1)
+    for _ in range(warmup):
+        oracle_cycle_seconds(cfg, attn_samples=32)
+    t0 = time.perf_counter()
+    last = None
+    for _ in range(steps):
+        last = oracle_cycle_seconds(cfg)
+    wall = (time.perf_counter() - t0) / steps
+    total, parts, sample, cores = last
+    us = total * 1e6
+    line = {
+        "impl": "reference", "metric": METRIC, "value": us, "unit": "us", "n_gpus": args.gpus,
+        "steps": steps, "warmup": warmup, "ms_per_step": wall * 1e3, "higher_is_better": False,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": cfg.name, "B": 1, "note": "oracle cycle time extrapolated from a bounded sample"},
+        "cpu_baseline": {"value": us, "unit": "us", "cores": cores, "kind": "oracle", "sample": sample,
+                         "parts_us": {k: v * 1e6 for k, v in parts.items()}},
+        "e2e": {"value": us, "unit": "us", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------------
+# the CUDA path
+
+def run_ours(args):
+    import torch
+
+    import paper_2406_16858_b200 as e2
+    from paper_2406_16858_b200.cycle import CycleBuffers, CycleShape, enqueue_cycle
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    cfg = get_config(args.workload)
+    if args.batch:
+        cfg = cfg.with_(B=args.batch)
+    seed = 1000 * rank
+    kv_len_h = gen.kv_lengths(cfg, seed)
+    kv_off_h = gen.kv_offsets(kv_len_h, cfg.m)
+    rows = int(kv_off_h[-1] + kv_len_h[-1] + cfg.m)
+    max_len = int(kv_len_h.max())
+    shape = CycleShape(cfg.B, cfg.V, cfg.k, cfg.D, cfg.m, cfg.n_layers, cfg.Hq, cfg.Hkv, cfg.d, max_len,
+                       cfg.temperature)
+    scale = 1.0 / math.sqrt(cfg.d)
+    g = torch.Generator(device=dev).manual_seed(seed + 1)
+
+    # ---- inputs resident in HBM ------------------------------------------------------------------
+    def randn_bf16(*shape_):
+        return torch.randn(shape_, generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
+
+    k_layers = [randn_bf16(rows, cfg.Hkv, cfg.d) for _ in range(cfg.n_layers)]
+    v_layers = [randn_bf16(rows, cfg.Hkv, cfg.d) for _ in range(cfg.n_layers)]
+    q_layers = [randn_bf16(cfg.B, cfg.m, cfg.Hq, cfg.d) for _ in range(cfg.n_layers)]
+    out_layers = [torch.zeros_like(qq) for qq in q_layers]
+    k_ptrs = torch.tensor([t.data_ptr() for t in k_layers], dtype=torch.int64, device=dev)
+    v_ptrs = torch.tensor([t.data_ptr() for t in v_layers], dtype=torch.int64, device=dev)
+    kv_off = torch.from_numpy(kv_off_h).to(dev)
+    kv_len0 = torch.from_numpy(kv_len_h).to(dev)
+    kv_len = kv_len0.clone()
+
+    buf = CycleBuffers(shape, dev)
+    sets = []
+    for i in range(N_SETS):
+        draft_h = gen.draft_rows(cfg, seed + 17 * i)
+        draft = torch.from_numpy(draft_h).to(dev)
+        # the target rows depend on which nodes were selected: build the tree once to find them
+        buf.expand_all(draft)
+        buf.rerank_and_mask(kv_len)
+        torch.cuda.synchronize()
+        nd = gen.node_draft_rows(buf.tree_parent.cpu().numpy(), cfg.k, cfg.D)
+        sel_index = buf.sel_index.cpu().numpy()
+        src_rows = np.zeros((cfg.B, cfg.m + 1), np.int64)
+        for b in range(cfg.B):
+            for x in range(cfg.m):
+                r = nd[b, sel_index[b, x]] if sel_index[b, x] >= 0 else -1
+                src_rows[b, 1 + x] = r if r >= 0 else (x * 7 + 3) % cfg.R  # stand-in row for unexpanded nodes
+        base = torch.gather(draft, 1, torch.from_numpy(src_rows).to(dev)[:, :, None].expand(-1, -1, cfg.V))
+        target = base + 0.5 * torch.randn(base.shape, generator=g, device=dev)
+        ua_h, ub_h = gen.uniforms(cfg, seed + 17 * i)
+        sets.append(dict(draft=draft, target=target.contiguous(), ua=torch.from_numpy(ua_h).to(dev),
+                         ub=torch.from_numpy(ub_h).to(dev)))
+    assert int(buf.status.item()) == 0, "device status raised while preparing inputs"
+
+    def one_cycle(s):
+        kv_len.copy_(kv_len0)  # the cache length is caller state: start every cycle from the same prefix
+        enqueue_cycle(buf, s["draft"], s["target"], s["ua"], s["ub"], q_layers, k_layers, v_layers,
+                      out_layers, k_ptrs, v_ptrs, kv_off, kv_len, scale)
+
+    stream = torch.cuda.Stream(device=dev)
+    graphs = []
+    with torch.cuda.stream(stream):
+        one_cycle(sets[0])  # warm every kernel (lazy module load) before capture
+        stream.synchronize()
+        for s in sets:
+            gr = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(gr, stream=stream):
+                one_cycle(s)
+            graphs.append(gr)
+        # attention alone (all layers) for the roofline of the dominant kernel
+        attn_graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(attn_graph, stream=stream):
+            for qq, kc, vc, oo in zip(q_layers, k_layers, v_layers, out_layers):
+                buf.attention(qq, kc, vc, kv_off, kv_len0, oo, scale)
+    torch.cuda.synchronize()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, steps):
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        with torch.cuda.stream(stream):
+            ev0.record(stream)
+            for i in range(steps):
+                fn(i)
+            ev1.record(stream)
+        barrier()
+        ms = ev0.elapsed_time(ev1)
+        if world > 1:
+            t = torch.tensor([ms], device=dev, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms
+
+    K, W = args.steps, max(args.warmup, 3)
+    with ClockSampler(local) as clocks:
+        timed(lambda i: graphs[i % N_SETS].replay(), W)
+        ms_total = timed(lambda i: graphs[i % N_SETS].replay(), K)
+        attn_reps = max(20, min(K, 400))
+        timed(lambda i: attn_graph.replay(), 3)
+        ms_attn = timed(lambda i: attn_graph.replay(), attn_reps)
+
+        # ---- end to end: inputs start in pinned host memory, results end in host memory -------------
+        host_in = {
+            "draft": sets[0]["draft"].cpu().pin_memory(), "target": sets[0]["target"].cpu().pin_memory(),
+            "ua": sets[0]["ua"].cpu().pin_memory(), "ub": sets[0]["ub"].cpu().pin_memory(),
+            "q": [t.cpu().pin_memory() for t in q_layers],
+        }
+        # the K/V of the m tree tokens are this cycle's new cache rows, one block per layer
+        tree_rows = [(b, int(kv_off_h[b] + kv_len_h[b])) for b in range(cfg.B)]
+        host_in["tree_k"] = [torch.stack([kc[r:r + cfg.m] for _, r in tree_rows]).cpu().pin_memory()
+                             for kc in k_layers]
+        host_in["tree_v"] = [torch.stack([vc[r:r + cfg.m] for _, r in tree_rows]).cpu().pin_memory()
+                             for vc in v_layers]
+        host_out = {"acc_len": torch.zeros(cfg.B, dtype=torch.int32).pin_memory(),
+                    "acc_path": torch.zeros((cfg.B, cfg.D), dtype=torch.int32).pin_memory(),
+                    "bonus": torch.zeros(cfg.B, dtype=torch.int32).pin_memory(),
+                    "o": [torch.zeros_like(t, device="cpu").pin_memory() for t in out_layers]}
+        h2d = sum(t.numel() * t.element_size() for t in
+                  [host_in["draft"], host_in["target"], host_in["ua"], host_in["ub"], *host_in["q"],
+                   *host_in["tree_k"], *host_in["tree_v"]])
+        d2h = sum(t.numel() * t.element_size() for t in
+                  [host_out["acc_len"], host_out["acc_path"], host_out["bonus"], *host_out["o"]])
+
+        def e2e_step(i):
+            s = sets[0]
+            s["draft"].copy_(host_in["draft"], non_blocking=True)
+            s["target"].copy_(host_in["target"], non_blocking=True)
+            s["ua"].copy_(host_in["ua"], non_blocking=True)
+            s["ub"].copy_(host_in["ub"], non_blocking=True)
+            for layer in range(cfg.n_layers):
+                q_layers[layer].copy_(host_in["q"][layer], non_blocking=True)
+                for j, (_, r) in enumerate(tree_rows):
+                    k_layers[layer][r:r + cfg.m].copy_(host_in["tree_k"][layer][j], non_blocking=True)
+                    v_layers[layer][r:r + cfg.m].copy_(host_in["tree_v"][layer][j], non_blocking=True)
+            graphs[0].replay()
+            host_out["acc_len"].copy_(buf.acc_len, non_blocking=True)
+            host_out["acc_path"].copy_(buf.acc_path, non_blocking=True)
+            host_out["bonus"].copy_(buf.bonus_token, non_blocking=True)
+            for layer in range(cfg.n_layers):
+                host_out["o"][layer].copy_(out_layers[layer], non_blocking=True)
+
+        e2e_steps = max(5, min(K, 50))
+        timed(e2e_step, 3)
+        ms_e2e = timed(e2e_step, e2e_steps)
+    assert int(buf.status.item()) == 0, "device status raised during the timed region"
+
+    us_cycle = ms_total * 1e3 / (K * world)
+    us_attn = ms_attn * 1e3 / (attn_reps * cfg.n_layers)
+    hbm_peak, _, peak_kind = _peaks()
+    kv_bytes = float(sum(2 * (int(L) + cfg.m) * cfg.Hkv * cfg.d * 2 for L in kv_len_h))
+    qo_bytes = float(2 * cfg.B * cfg.m * cfg.Hq * cfg.d * 2)
+    attn_bytes = kv_bytes + qo_bytes
+    achieved = attn_bytes / (us_attn * 1e-6) / 1e9
+    # accepted length of the synthetic workload (tokens per cycle = accepted draft tokens + 1)
+    acc = []
+    with torch.cuda.stream(stream):
+        for gr in graphs:
+            gr.replay()
+            stream.synchronize()
+            acc.append(buf.acc_len.float().mean().item())
+    tau = float(np.mean(acc)) + 1.0
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    line = {
+        "metric": METRIC, "value": us_cycle, "unit": "us", "n_gpus": world, "steps": K, "warmup": W,
+        "ms_per_step": ms_total / K, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16 attention (fp32 accumulate), fp32 logits, fp64 node values", "data": "synthetic",
+        "config": {"workload": cfg.name, "B": cfg.B, "V": cfg.V, "k": cfg.k, "D": cfg.D, "m": cfg.m,
+                   "n_layers": cfg.n_layers, "Hq": cfg.Hq, "Hkv": cfg.Hkv, "d": cfg.d,
+                   "kv_len": [int(x) for x in kv_len_h[:8]], "temperature": cfg.temperature,
+                   "l2": f"inputs larger than L2: {cfg.n_layers} distinct KV layers "
+                         f"({kv_bytes * cfg.n_layers / 1e6:.0f} MB) and {N_SETS} rotating logit sets",
+                   "replicas": world, "synthetic_tau": tau},
+        "clocks": clocks.summary(),
+        "e2e": {"value": ms_e2e * 1e3 / (e2e_steps * world), "unit": "us", "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h},
+        "gpu_launches": buf.launches_per_cycle() * K,
+        "roofline": {"kernel": "tree_attention (+ split merge), one launch per layer", "bound": "hbm",
+                     "achieved": achieved, "peak": hbm_peak, "unit": "GB/s", "frac": achieved / hbm_peak,
+                     "peak_kind": f"of {peak_kind}", "traffic": None, "us_per_launch": us_attn,
+                     "algorithmic_bytes_per_launch": attn_bytes},
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        total, parts, sample, cores = oracle_cycle_seconds(cfg)
+        line["cpu_baseline"] = {"value": total * 1e6, "unit": "us", "cores": cores, "kind": "oracle",
+                                "sample": sample, "parts_us": {k: v * 1e6 for k, v in parts.items()}}
+    line["roofline"]["traffic"] = NCU_DRAM_BYTES_PER_LAUNCH.get(cfg.name)
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llama3_8b")
+    ap.add_argument("--batch", type=int, default=0, help="override the number of sequences")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

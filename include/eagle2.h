@@ -8,8 +8,9 @@
  *     library allocates nothing: scratch memory comes from a caller-supplied workspace whose size
  *     eagle2_workspace_bytes() reports.  A workspace must be 256-byte aligned and must have been
  *     passed through eagle2_workspace_init() once after allocation (it zeroes the arrival counters
- *     that the kernels leave zeroed again on exit).  Calls that share a workspace must be ordered
- *     on one stream.
+ *     that the kernels leave zeroed again on exit; they occupy the first 4*B bytes, rounded up to
+ *     256, in every operation's layout, so one workspace of the largest reported size serves all
+ *     operations).  Calls that share a workspace must be ordered on one stream.
  *   - Every call only enqueues work on `stream` and returns; nothing synchronises, so a sequence of
  *     calls can be captured in a CUDA graph.
  *   - Return value: EAGLE2_OK, or a negative EAGLE2_ERR_* found on the host before anything was

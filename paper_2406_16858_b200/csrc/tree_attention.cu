@@ -50,7 +50,9 @@ struct AttnWs {
 static size_t attention_ws_layout(int B, int Hkv, int d, const AttnPlan& p, void* base, AttnWs* w) {
     if (p.splits == 1) return 0;
     const size_t rows = (size_t)B * Hkv * p.splits * p.n_rb * p.RB;
-    size_t off = 0;
+    // every operation keeps its arrival counters (B ints) at the start of the workspace and leaves
+    // them zero; the partials go behind that region so that a shared workspace stays valid
+    size_t off = round_up(sizeof(int) * (size_t)B, kWsAlign);
     char* c = static_cast<char*>(base);
     if (w) w->o_part = reinterpret_cast<float*>(c + off);
     off += round_up(rows * d * sizeof(float), kWsAlign);
