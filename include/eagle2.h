@@ -131,14 +131,20 @@ int eagle2_tree_mask(const int32_t* sel_parent, const int32_t* sel_depth, const 
  * over the keys token i may see: every committed cache row [0, kv_len[b]) of its sequence and the
  * tree rows j whose bit is set in mask row i.  bf16 operands, fp32 accumulation, bf16 result.
  *   q        bf16 [B][m][Hq][d]
- *   k_cache, v_cache  bf16 [rows][Hkv][d]; sequence b owns rows kv_off[b] .. kv_off[b]+kv_len[b]+m-1,
- *            the K/V of tree token j at local row kv_len[b]+j.
+ *   k_cache, v_cache  bf16 [cache_rows][Hkv][d]; sequence b owns rows kv_off[b] ..
+ *            kv_off[b]+kv_len[b]+m-1, the K/V of tree token j at local row kv_len[b]+j.
+ *   cache_rows [host value] rows allocated in k_cache and in v_cache.  The kernel streams whole
+ *            128-row tiles, so it may read (and ignore) rows of the allocation that follow a
+ *            sequence's last key; rows at or beyond cache_rows are never touched.
  *   kv_off   int64 [B], kv_len int32 [B], mask_bits as written by eagle2_tree_mask.
  *   out      bf16 [B][m][Hq][d];  lse fp32 [B][Hq][m], optional natural-log sum of exponentials.
- *   max_kv_len [host value] upper bound of kv_len[], used only to size the launch.
- * Limits: d in {64,128}; Hq % Hkv == 0 with Hq/Hkv <= 8; 16-byte aligned q, caches and out.
+ *   max_kv_len [host value] upper bound of kv_len[], used to size the launch and the workspace.
+ * A sequence with kv_len outside [0, max_kv_len] or whose rows do not fit in cache_rows raises
+ * EAGLE2_STATUS_KV_OVERFLOW and its output rows are left untouched.
+ * Limits: d in {64,128}; Hq % Hkv == 0 with Hq/Hkv <= 8; scale > 0; cache_rows < 2^31; 16-byte
+ * aligned q, caches and out.
  */
-int eagle2_tree_attention(const void* q, const void* k_cache, const void* v_cache,
+int eagle2_tree_attention(const void* q, const void* k_cache, const void* v_cache, long long cache_rows,
                           const int64_t* kv_off, const int32_t* kv_len, const uint64_t* mask_bits,
                           int B, int m, int Hq, int Hkv, int d, int max_kv_len, float scale, void* out,
                           float* lse, void* ws, size_t ws_bytes, int32_t* d_status,

@@ -55,8 +55,8 @@ def lib() -> C.CDLL:
         h.eagle2_expand.argtypes = [vp, i64, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, sz, vp, vp]
         h.eagle2_rerank.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp]
         h.eagle2_tree_mask.argtypes = [vp, vp, vp, vp, i32, i32, vp, vp, vp, vp, vp]
-        h.eagle2_tree_attention.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, f32,
-                                            vp, vp, vp, sz, vp, vp]
+        h.eagle2_tree_attention.argtypes = [vp, vp, vp, i64, vp, vp, vp, i32, i32, i32, i32, i32, i32,
+                                            f32, vp, vp, vp, sz, vp, vp]
         h.eagle2_accept.argtypes = [vp, i64, vp, i64, vp, vp, vp, vp, i32, i32, i32, i32, i32, f32,
                                     vp, vp, vp, vp, vp, vp, sz, vp, vp]
         h.eagle2_kv_compact.argtypes = [vp, vp, i32, vp, vp, vp, vp, i32, i32, i32, i32, i32, vp, vp]
@@ -134,12 +134,14 @@ def tree_mask(sel_parent, sel_depth, n_sel, kv_len, B: int, m: int, mask_bits, m
         _ptr(mask_dense), _ptr(pos_ids), _ptr(d_status), _stream(stream)))
 
 
-def tree_attention(q, k_cache, v_cache, kv_off, kv_len, mask_bits, B: int, m: int, Hq: int, Hkv: int,
-                   d: int, max_kv_len: int, scale: float, out, lse, ws, d_status, stream=None) -> None:
+def tree_attention(q, k_cache, v_cache, cache_rows: int, kv_off, kv_len, mask_bits, B: int, m: int,
+                   Hq: int, Hkv: int, d: int, max_kv_len: int, scale: float, out, lse, ws, d_status,
+                   stream=None) -> None:
     p, n = _ws(ws)
     _check("eagle2_tree_attention", lib().eagle2_tree_attention(
-        _ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(kv_off), _ptr(kv_len), _ptr(mask_bits), B, m, Hq,
-        Hkv, d, max_kv_len, scale, _ptr(out), _ptr(lse), p, n, _ptr(d_status), _stream(stream)))
+        _ptr(q), _ptr(k_cache), _ptr(v_cache), cache_rows, _ptr(kv_off), _ptr(kv_len), _ptr(mask_bits),
+        B, m, Hq, Hkv, d, max_kv_len, scale, _ptr(out), _ptr(lse), p, n, _ptr(d_status),
+        _stream(stream)))
 
 
 def accept(target_logits, t_stride: int, draft_logits_all, d_stride: int, sel_index, sel_parent,

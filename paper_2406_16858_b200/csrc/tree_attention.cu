@@ -1,55 +1,85 @@
 // Step 3 of the hot path: tree-masked attention of the verification pass (paper Section 4.2: each
 // draft token sees the committed cache and its own ancestors only).
 //
-// Split-KV flash decoding.  The m tree tokens of one sequence and the g = Hq/Hkv query heads that
-// share a KV head are packed into M = m*g query rows, so each K/V tile read from HBM serves all of
-// them.  A block owns (sequence, KV head, row block, KV split): it keeps its query rows in shared
-// memory, streams 64-key K/V tiles through a 3-stage cp.async pipeline, computes Q.K^T and P.V on
-// the tensor cores (bf16 in, fp32 accumulate) with an online softmax in registers, and writes either
-// the final rows (one split) or an unnormalised partial plus (max, sum) that a merge kernel combines.
+// Split-KV flash decoding on the Blackwell tensor path.  The m tree tokens of one sequence and the
+// g = Hq/Hkv query heads that share a KV head are packed into M = m*g query rows, so every K/V tile
+// read from HBM serves all of them.  A block owns (sequence, KV head, row block, KV split) with up
+// to 256 packed rows (two 128-row UMMA tiles) and is warp specialised:
+//   softmax warps  one thread per query row.  S = Q.K^T arrives in tensor memory; the thread reads
+//                  its row, applies scale, tree mask and a lazily rescaled running maximum, and
+//                  writes P as bf16 back into tensor memory over the scores it consumed.
+//   TMA warp       streams 128-key K and V tiles (128-byte swizzled) through a ring of stages.
+//   MMA warp       one thread issues tcgen05.mma: S = Q.K^T (operands in shared memory) and
+//                  O += P.V (P from tensor memory, V in shared memory, MN-major), two score slots
+//                  in flight so that the tensor pipe and the softmax warps overlap.
+// The block writes final rows when its sequence needs a single split, otherwise an unnormalised
+// fp32 partial plus (max, sum) that a merge kernel combines.
+//
+// Every wait on an mbarrier is bounded: when it runs out the block raises EAGLE2_STATUS_TIMEOUT,
+// drains its own copies, frees its tensor memory and returns.
+#include <cuda.h>
 #include <cuda_bf16.h>
 #include <math.h>
+
+#include <mutex>
 
 #include "common.cuh"
 
 namespace eagle2 {
 
-constexpr int kTileKeys = 64;
-constexpr int kStages = 3;
-constexpr int kMaxRowsPerBlock = 256;
+constexpr int kTK = 128;              // keys per K/V tile = N of the Q.K^T instruction
+constexpr int kRowsPerTile = 128;     // M of every tcgen05.mma
+constexpr int kMaxTilesPerSplit = 16; // a block never streams more than 2048 keys
+constexpr int kTmemCols = 512;
+constexpr int kSlots = 2;             // score slots in tensor memory
+constexpr long long kWaitCycles = 1LL << 31;  // ~1 s bound of a barrier wait
+constexpr uint32_t kSuspendNs = 20000;        // a waiting thread sleeps in hardware at most this long per try
 
 struct AttnPlan {
-    int g, M, n_rb, RB, warps, splits;
+    int g, M;
+    int n_rb;       // row blocks per (sequence, KV head)
+    int per_tok;    // tree tokens per row block (the last may hold fewer)
+    int per;        // packed rows per row block = per_tok * g
+    int q_tma;      // 1: query rows arrive by TMA (g divides 128), 0: by cp.async
+    int mt;         // 128-row tiles per block: 1 or 2
+    int splits;     // KV splits per sequence (blocks of the launch)
+    int per_split;  // K/V tiles per split
+    int stages;     // K/V ring depth
     size_t smem;
 };
 
 static void attention_plan(int B, int m, int Hq, int Hkv, int d, int max_kv_len, AttnPlan* p) {
     p->g = Hq / Hkv;
     p->M = m * p->g;
-    p->n_rb = (p->M + kMaxRowsPerBlock - 1) / kMaxRowsPerBlock;
-    const int per = (p->M + p->n_rb - 1) / p->n_rb;
-    p->RB = (per + 15) / 16 * 16;
-    p->warps = p->RB / 16;
+    p->n_rb = (p->M + 2 * kRowsPerTile - 1) / (2 * kRowsPerTile);
+    p->per_tok = (m + p->n_rb - 1) / p->n_rb;
+    p->per = p->per_tok * p->g;  // never above 256: n_rb >= m*g/256
+    p->mt = p->per > kRowsPerTile ? 2 : 1;
+    p->q_tma = (kRowsPerTile % p->g) == 0;
     const long long items = (long long)B * Hkv * p->n_rb;
-    const int per_sm = p->warps <= 4 ? 2 : 1;
-    const long long target = 148LL * per_sm;
-    const int tiles = (max_kv_len + m + kTileKeys - 1) / kTileKeys;
-    long long s = target / (items > 0 ? items : 1);
+    const int tiles = (max_kv_len + m + kTK - 1) / kTK;
+    long long s = 148 / (items > 0 ? items : 1);
     if (s < 1) s = 1;
-    if (s > (tiles + 1) / 2) s = (tiles + 1) / 2;
-    if (s < 1) s = 1;
-    p->splits = (int)s;
-    p->smem = (size_t)p->RB * d * 2 + (size_t)kStages * 2 * kTileKeys * d * 2;
+    if (s > tiles) s = tiles;
+    int per_split = (int)((tiles + s - 1) / s);
+    if (per_split > kMaxTilesPerSplit) per_split = kMaxTilesPerSplit;
+    if (per_split < 1) per_split = 1;
+    p->per_split = per_split;
+    p->splits = (tiles + per_split - 1) / per_split;
+    const size_t unit = (size_t)(d / 64) * kTK * 128;  // one 128-row operand tile
+    int stages = (int)((220 * 1024 - p->mt * unit) / (2 * unit));
+    p->stages = stages > 4 ? 4 : (stages < 2 ? 2 : stages);
+    p->smem = (p->mt + 2 * (size_t)p->stages) * unit + 1024;
 }
 
 struct AttnWs {
-    float* o_part;   // [B][Hkv][splits][n_rb*RB][d]
-    float2* ml;      // [B][Hkv][splits][n_rb*RB]  (running max in log2 units, running sum)
+    float* o_part;  // [B][Hkv][splits][n_rb][mt*128][d]
+    float2* ml;     // [B][Hkv][splits][n_rb][mt*128]  (reference maximum in log2 units, sum)
 };
 
 static size_t attention_ws_layout(int B, int Hkv, int d, const AttnPlan& p, void* base, AttnWs* w) {
     if (p.splits == 1) return 0;
-    const size_t rows = (size_t)B * Hkv * p.splits * p.n_rb * p.RB;
+    const size_t rows = (size_t)B * Hkv * p.splits * p.n_rb * p.mt * kRowsPerTile;
     // every operation keeps its arrival counters (B ints) at the start of the workspace and leaves
     // them zero; the partials go behind that region so that a shared workspace stays valid
     size_t off = round_up(sizeof(int) * (size_t)B, kWsAlign);
@@ -67,60 +97,327 @@ size_t attention_workspace_bytes(int B, int m, int Hq, int Hkv, int d, int max_k
     return attention_ws_layout(B, Hkv, d, p, nullptr, nullptr);
 }
 
-// ---- small PTX wrappers --------------------------------------------------------------------------
+// ---- tensor maps ---------------------------------------------------------------------------------
+// K and V caches are 3-D tensors [rows][Hkv][d] of bf16; a box is 128 rows of one head and 64
+// columns (128 bytes, the swizzle span).  Rows beyond the cache read as zero.
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                   CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                   CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+        else
+            cudaGetLastError();
+    });
+    return fn;
+}
+
+static bool make_cache_map(CUtensorMap* map, const void* base, long long rows, int Hkv, int d) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)Hkv, (cuuint64_t)rows};
+    const cuuint64_t strides[2] = {(cuuint64_t)d * 2, (cuuint64_t)Hkv * d * 2};
+    const cuuint32_t box[3] = {64, 1, (cuuint32_t)kTK};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Queries [B][m][Hq][d] seen as a 4-D tensor (d, head in group, token, KV head): a box of 128/g
+// tokens of one KV head lands as 128 packed rows (token-major, head in group fastest).
+static bool make_query_map(CUtensorMap* map, const void* base, int B, int m, int Hq, int Hkv, int d) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const int g = Hq / Hkv;
+    const cuuint64_t dims[4] = {(cuuint64_t)d, (cuuint64_t)g, (cuuint64_t)B * m, (cuuint64_t)Hkv};
+    const cuuint64_t strides[3] = {(cuuint64_t)d * 2, (cuuint64_t)Hq * d * 2, (cuuint64_t)g * d * 2};
+    const cuuint32_t box[4] = {64, (cuuint32_t)g, (cuuint32_t)(kRowsPerTile / g), 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// ---- PTX wrappers ----------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return (uint32_t)__cvta_generic_to_shared(p);
 }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.b32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity), "r"(kSuspendNs)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait for the phase of the given parity.  Returns false when the bound ran out or another
+// role of the block has already given up (*abort != 0).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (int spin = 1;; ++spin) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((spin & 15) == 0 && (*abort || clock64() - t0 > kWaitCycles)) {
+            *abort = 1;
+            return false;
+        }
+    }
+}
+__device__ __forceinline__ void fence_proxy_async() {
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void fence_barrier_init() {
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2,
+                                            uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes "
+        "[%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, int c3,
+                                            uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes "
+        "[%0], [%1, {%2, %3, %4, %5}], [%6];"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar)
+        : "memory");
+}
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, bool valid) {
     const int n = valid ? 16 : 0;  // 0 source bytes: the 16 destination bytes are zero-filled
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(n));
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(n) : "memory");
 }
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() {
-    asm volatile("cp.async.wait_group %0;\n" ::"n"(N));
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols)
+                 : "memory");
 }
-__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
-                 : "r"(addr));
+__device__ __forceinline__ void tmem_relinquish() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
 }
-__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t addr) {
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];\n"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
-                 : "r"(addr));
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
 }
-__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+__device__ __forceinline__ void tc_fence_before() {
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_after() {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+}
+// Waits for this thread's tensor-memory loads.  The registers of the load are tied to the statement
+// so that no use of them can be scheduled above it.
+__device__ __forceinline__ void tc_wait_ld(uint32_t (&r)[32]) {
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+                   "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]),
+                   "+r"(r[15]), "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]),
+                   "+r"(r[22]), "+r"(r[23]), "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]),
+                   "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+                 :
+                 : "memory");
+}
+__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
+                 : "memory");
+}
+// D[tmem] (+)= A[smem] . B[smem]
+__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                       uint32_t accumulate) {
     asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
-        "{%0,%1,%2,%3};\n"
-        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// D[tmem] (+)= A[tmem] . B[smem]
+__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                       uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// 32 consecutive 32-bit columns of this thread's tensor-memory lane
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]),
+          "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]),
+          "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]),
+          "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+          "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+          "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+          "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+        : "memory");
+}
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
 }
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<const uint32_t*>(&v);
 }
 
-// Shared-memory tiles are [row][DH] bf16 with the 16-byte chunks of a row XOR-swizzled by the row
-// number, so that the 8 rows an ldmatrix touches fall into 8 different bank groups.
-template <int DH>
-__device__ __forceinline__ uint32_t tile_off(int row, int chunk) {
-    return (uint32_t)(row * DH * 2 + ((chunk ^ (row & 7)) << 4));
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float r;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+    return r;
+}
+// Largest raw score of a 32-column chunk (TAIL: only over the columns whose visibility bit is set).
+template <bool TAIL>
+__device__ __forceinline__ float chunk_rowmax(const uint32_t (&r)[32], uint32_t visw, float mx) {
+    float m0 = mx, m1 = -INFINITY;
+#pragma unroll
+    for (int c = 0; c < 32; c += 4) {
+        float a[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            a[e] = __uint_as_float(r[c + e]);
+            if (TAIL && !((visw >> (c + e)) & 1u)) a[e] = -INFINITY;
+        }
+        m0 = max3(m0, a[0], a[1]);
+        m1 = max3(m1, a[2], a[3]);
+    }
+    return fmaxf(m0, m1);
+}
+// p = 2^(s * scale - reference) for a 32-column chunk, packed to 16 bf16 pairs; the sums of the
+// unrounded probabilities accumulate in two packed registers.
+template <bool TAIL>
+__device__ __forceinline__ void chunk_probs(const uint32_t (&r)[32], uint32_t visw, float2 scale2, float2 neg_ref2,
+                                            float2& sum_a, float2& sum_b, uint32_t* pk) {
+#pragma unroll
+    for (int c = 0; c < 32; c += 4) {
+        float2 a = __ffma2_rn(make_float2(__uint_as_float(r[c]), __uint_as_float(r[c + 1])), scale2, neg_ref2);
+        float2 bq = __ffma2_rn(make_float2(__uint_as_float(r[c + 2]), __uint_as_float(r[c + 3])), scale2, neg_ref2);
+        if (TAIL) {
+            if (!((visw >> c) & 1u)) a.x = -INFINITY;
+            if (!((visw >> (c + 1)) & 1u)) a.y = -INFINITY;
+            if (!((visw >> (c + 2)) & 1u)) bq.x = -INFINITY;
+            if (!((visw >> (c + 3)) & 1u)) bq.y = -INFINITY;
+        }
+        const float2 pa = make_float2(ex2(a.x), ex2(a.y)), pb = make_float2(ex2(bq.x), ex2(bq.y));
+        sum_a = __fadd2_rn(sum_a, pa);
+        sum_b = __fadd2_rn(sum_b, pb);
+        pk[c >> 1] = pack_bf16(pa.x, pa.y);
+        pk[(c >> 1) + 1] = pack_bf16(pb.x, pb.y);
+    }
 }
 
-template <int DH>
-__global__ void __launch_bounds__(512)
-tree_attention_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k_cache,
-                      const __nv_bfloat16* __restrict__ v_cache, const int64_t* __restrict__ kv_off,
-                      const int32_t* __restrict__ kv_len, const uint64_t* __restrict__ mask_bits, int m,
-                      int Hq, int Hkv, AttnPlan plan, float scale_log2, __nv_bfloat16* __restrict__ out,
-                      float* __restrict__ lse, AttnWs ws) {
-    constexpr int CH = DH / 8;  // 16-byte chunks per row
-    extern __shared__ __align__(128) unsigned char smem[];
-    __shared__ uint64_t s_mask[EAGLE2_MAX_M * 2];
+// Shared-memory matrix descriptor of a 128-byte swizzled operand tile (8-row groups 1024 bytes apart).
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes) {
+    return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) |
+           ((uint64_t)(1024u >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, M = 128, A K-major; B K-major or MN-major.
+__host__ __device__ constexpr uint32_t instr_desc(int n, bool b_mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((uint32_t)(n >> 3) << 17) |
+           ((uint32_t)(kRowsPerTile >> 4) << 24);
+}
 
-    const int g = plan.g, M = plan.M, RB = plan.RB, S = plan.splits;
+// A sequence is served only if its length is within the plan and its rows lie inside the cache.
+__device__ __forceinline__ bool sequence_ok(int L, long long row_base, int m, int max_kv_len, long long cache_rows) {
+    return L >= 0 && L <= max_kv_len && row_base >= 0 && row_base + L + m <= cache_rows;
+}
+
+struct AttnBarriers {
+    unsigned long long q_full;
+    unsigned long long k_full[4], k_empty[4], v_full[4], v_empty[4];
+    unsigned long long s_full[kSlots], p_full[kSlots];
+    // Per row tile, two barriers used by alternate K/V tiles: P.V of tile j completes a phase of
+    // o_done[t][j & 1].  A waiter may skip phases (it only looks when it must rescale O, and at the
+    // end); with two barriers the one it consults is never more than one phase ahead of it.
+    unsigned long long o_done[2][2];
+};
+
+// Visibility of the 128 keys of a tile that reaches past the committed cache, as four 32-bit words:
+// bit c set = key0 + c is a cache key, or a tree key whose bit is set in the row's mask.
+__device__ __forceinline__ void tile_visibility(unsigned long long mlo, unsigned long long mhi, int key0, int L,
+                                                int n_keys, uint32_t (&vis)[4]) {
+    unsigned long long lo, hi;
+    const int off = key0 - L;  // tree index of column 0
+    if (off >= 0) {
+        if (off >= 128) lo = 0, hi = 0;
+        else if (off >= 64) lo = mhi >> (off - 64), hi = 0;
+        else if (off == 0) lo = mlo, hi = mhi;
+        else lo = (mlo >> off) | (mhi << (64 - off)), hi = mhi >> off;
+    } else {
+        const int sh = -off;  // columns [0, sh) are cache keys
+        if (sh >= 128) lo = ~0ull, hi = ~0ull;
+        else if (sh >= 64) lo = ~0ull, hi = (sh == 64 ? 0ull : ((1ull << (sh - 64)) - 1)) | (mlo << (sh - 64));
+        else lo = ((1ull << sh) - 1) | (mlo << sh), hi = (mlo >> (64 - sh)) | (mhi << sh);
+    }
+    const int nv = n_keys - key0;  // columns that exist at all
+    if (nv < 128) {
+        if (nv <= 0) lo = 0, hi = 0;
+        else if (nv < 64) lo &= (1ull << nv) - 1, hi = 0;
+        else if (nv > 64) hi &= (1ull << (nv - 64)) - 1;
+        else hi = 0;
+    }
+    vis[0] = (uint32_t)lo, vis[1] = (uint32_t)(lo >> 32), vis[2] = (uint32_t)hi, vis[3] = (uint32_t)(hi >> 32);
+}
+
+template <int DH, int MT>
+__global__ void __launch_bounds__(MT * 128 + 64, 1)
+tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map,
+                      const __grid_constant__ CUtensorMap q_map, const __nv_bfloat16* __restrict__ q, const int64_t* __restrict__ kv_off,
+                      const int32_t* __restrict__ kv_len, const uint64_t* __restrict__ mask_bits, int m, int Hq,
+                      int Hkv, long long cache_rows, int max_kv_len, AttnPlan plan, float scale_log2,
+                      __nv_bfloat16* __restrict__ out, float* __restrict__ lse, AttnWs ws, int32_t* d_status) {
+    constexpr int HALVES = DH / 64;                    // 64-column (128-byte) panels per operand tile
+    constexpr uint32_t kPanel = kTK * 128;             // bytes of one panel: 128 rows x 128 bytes
+    constexpr uint32_t kTile = HALVES * kPanel;
+    constexpr int kSoftmaxThreads = MT * 128;
+    constexpr int kTmaWarp = MT * 4, kMmaWarp = MT * 4 + 1;
+    constexpr uint32_t kIdescQK = instr_desc(kTK, false);
+    constexpr uint32_t kIdescPV = instr_desc(DH, true);
+    constexpr uint32_t kOCol = kSlots * kTK;           // first accumulator column of O
+
+    extern __shared__ unsigned char smem_raw[];
+    __shared__ AttnBarriers bars;
+    __shared__ uint32_t s_tmem_base;
+    __shared__ int s_abort;
+
+    const int g = plan.g, M = plan.M, S = plan.splits, NST = plan.stages;
     int bid = blockIdx.x;
     const int split = bid % S;
     bid /= S;
@@ -129,199 +426,380 @@ tree_attention_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* 
     const int hk = bid % Hkv;
     const int b = bid / Hkv;
 
-    const int tid = threadIdx.x, nthreads = blockDim.x;
-    const int warp = tid >> 5, lane = tid & 31;
-    const int L = kv_len[b];
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int L_raw = kv_len[b];
+    const long long row_base = kv_off[b];
+    const bool overflow = !sequence_ok(L_raw, row_base, m, max_kv_len, cache_rows);
+    const int L = overflow ? 0 : L_raw;
     const int n_keys = L + m;
-    const int W = (m + 63) / 64;
-    const int tiles = (n_keys + kTileKeys - 1) / kTileKeys;
-    const int per_split = (tiles + S - 1) / S;
-    const int t_begin = min(split * per_split, tiles);
-    const int t_end = min(t_begin + per_split, tiles);
-    const int nt = t_end - t_begin;
+    const int tiles = (n_keys + kTK - 1) / kTK;
+    const int S_b = (tiles + plan.per_split - 1) / plan.per_split;  // splits this sequence uses
+    const int t_begin = min(split * plan.per_split, tiles);
+    const int nt = overflow ? 0 : min(plan.per_split, tiles - t_begin);
+    const bool direct = S_b <= 1;  // a single split writes final rows
 
-    unsigned char* s_q = smem;
-    unsigned char* s_kv = smem + (size_t)RB * DH * 2;
-    const uint32_t s_q_u32 = smem_u32(s_q);
-    const uint32_t s_kv_u32 = smem_u32(s_kv);
-    constexpr uint32_t kTileBytes = kTileKeys * DH * 2;
+    const int row0 = rb * plan.per;                      // first packed row of this block
+    const int rows_here = min(plan.per, M - row0);       // rows that exist
+    const size_t part_row0 = ((((size_t)b * Hkv + hk) * S + split) * plan.n_rb + rb) * (size_t)(MT * 128);
 
-    const int row0 = rb * RB;  // first packed query row of this block
-    const __nv_bfloat16* kbase = k_cache + (kv_off[b] * Hkv + hk) * (long long)DH;
-    const __nv_bfloat16* vbase = v_cache + (kv_off[b] * Hkv + hk) * (long long)DH;
-    const long long kv_row_stride = (long long)Hkv * DH;
+    if (overflow && tid == 0 && split == 0 && rb == 0 && hk == 0) raise_status(d_status, EAGLE2_STATUS_KV_OVERFLOW);
+    if (nt <= 0 || rows_here <= 0) return;  // a split past the sequence's last tile (never merged), or a rejected sequence
 
-    auto load_tile = [&](int t, int stage) {
-        const int key0 = (t_begin + t) * kTileKeys;
-        const uint32_t kdst = s_kv_u32 + (uint32_t)stage * 2 * kTileBytes;
-        const uint32_t vdst = kdst + kTileBytes;
-        for (int idx = tid; idx < kTileKeys * CH; idx += nthreads) {
-            const int r = idx / CH, c = idx % CH;
-            const int key = key0 + r;
-            const bool ok = key < n_keys;
-            const long long src = (long long)(ok ? key : 0) * kv_row_stride + c * 8;
-            cp_async16(kdst + tile_off<DH>(r, c), kbase + src, ok);
-            cp_async16(vdst + tile_off<DH>(r, c), vbase + src, ok);
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t sQ = smem_base;
+    const uint32_t sK = sQ + MT * kTile;
+    const uint32_t sV = sK + (uint32_t)NST * kTile;
+    unsigned char* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+
+    // ---- set-up: barriers, tensor memory --------------------------------------------------------
+    if (tid == 0) {
+        s_abort = 0;
+        mbar_init(smem_u32(&bars.q_full), plan.q_tma ? 1 : kSoftmaxThreads);
+        for (int s = 0; s < 4; ++s) {
+            mbar_init(smem_u32(&bars.k_full[s]), 1);
+            mbar_init(smem_u32(&bars.k_empty[s]), 1);
+            mbar_init(smem_u32(&bars.v_full[s]), 1);
+            mbar_init(smem_u32(&bars.v_empty[s]), 1);
         }
-    };
-
-    // ---- prologue: query rows and mask into shared memory, first K/V tiles in flight ------------
-    for (int idx = tid; idx < RB * CH; idx += nthreads) {
-        const int r = idx / CH, c = idx % CH;
-        const int pr = row0 + r;  // packed row = token * g + head-in-group
-        const bool ok = pr < M;
-        const int tok = ok ? pr / g : 0, gq = ok ? pr % g : 0;
-        const __nv_bfloat16* src = q + (((long long)b * m + tok) * Hq + hk * g + gq) * DH + c * 8;
-        cp_async16(s_q_u32 + tile_off<DH>(r, c), src, ok);
+        for (int s = 0; s < kSlots; ++s) {
+            mbar_init(smem_u32(&bars.s_full[s]), 1);
+            mbar_init(smem_u32(&bars.p_full[s]), 128);
+        }
+        for (int s = 0; s < 4; ++s) mbar_init(smem_u32(&bars.o_done[s >> 1][s & 1]), 1);
+        fence_barrier_init();
     }
-    cp_async_commit();
-    for (int i = tid; i < m * W; i += nthreads) s_mask[i] = mask_bits[(long long)b * m * W + i];
-#pragma unroll
-    for (int t = 0; t < kStages - 1; ++t) {
-        if (t < nt) load_tile(t, t);
-        cp_async_commit();
+    if (warp == kMmaWarp) {
+        tmem_alloc(smem_u32(&s_tmem_base), kTmemCols);
+        tmem_relinquish();
     }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = s_tmem_base;
+    volatile int* abort_flag = &s_abort;
+    const int n_items = nt * MT;  // item i = (tile i / MT, row tile i % MT), score slot i % 2
 
-    // per-thread rows: r_lo = 16*warp + lane/4, r_hi = r_lo + 8
-    const int qrow_lo = row0 + warp * 16 + (lane >> 2);
-    const int tok_lo = min(qrow_lo, M - 1) / g, tok_hi = min(qrow_lo + 8, M - 1) / g;
-    float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
-    float oacc[DH / 8][4];
+    if (warp == kTmaWarp) {
+        // ===== TMA producer =======================================================================
+        if (lane == 0) {
+            int issued = 0;
+            bool ok = true;
+            if (plan.q_tma) {
+                mbar_expect_tx(smem_u32(&bars.q_full), MT * kTile);
 #pragma unroll
-    for (int n = 0; n < DH / 8; ++n) oacc[n][0] = oacc[n][1] = oacc[n][2] = oacc[n][3] = 0.f;
-
-    for (int it = 0; it < nt; ++it) {
-        cp_async_wait<kStages - 2>();
-        __syncthreads();
-        if (it + kStages - 1 < nt) load_tile(it + kStages - 1, (it + kStages - 1) % kStages);
-        cp_async_commit();
-
-        const uint32_t ks = s_kv_u32 + (uint32_t)(it % kStages) * 2 * kTileBytes;
-        const uint32_t vs = ks + kTileBytes;
-        const int key0 = (t_begin + it) * kTileKeys;
-        const bool need_mask = key0 + kTileKeys > L;
-
+                for (int t = 0; t < MT; ++t)
 #pragma unroll
-        for (int half = 0; half < 2; ++half) {  // 32 keys at a time keeps the register count down
-            float sacc[4][4];
+                    for (int h = 0; h < HALVES; ++h)
+                        tma_load_4d(sQ + t * kTile + h * kPanel, &q_map, h * 64, 0,
+                                    b * m + rb * plan.per_tok + t * (kRowsPerTile / g), hk, smem_u32(&bars.q_full));
+            }
+            for (int j = 0; j < nt && ok; ++j) {
+                const int st = j % NST;
+                const uint32_t ph = (uint32_t)((j / NST) & 1);
+                const int row = (int)(row_base + (long long)(t_begin + j) * kTK);
+                if (j >= NST) ok = mbar_wait(smem_u32(&bars.k_empty[st]), ph ^ 1u, abort_flag);
+                if (!ok) break;
+                mbar_expect_tx(smem_u32(&bars.k_full[st]), kTile);
 #pragma unroll
-            for (int n = 0; n < 4; ++n) sacc[n][0] = sacc[n][1] = sacc[n][2] = sacc[n][3] = 0.f;
+                for (int h = 0; h < HALVES; ++h)
+                    tma_load_3d(sK + st * kTile + h * kPanel, &k_map, h * 64, hk, row, smem_u32(&bars.k_full[st]));
+                if (j >= NST) ok = mbar_wait(smem_u32(&bars.v_empty[st]), ph ^ 1u, abort_flag);
+                if (!ok) {  // K of this tile is in flight, V is not
+                    mbar_wait(smem_u32(&bars.k_full[st]), ph, abort_flag);
+                    break;
+                }
+                mbar_expect_tx(smem_u32(&bars.v_full[st]), kTile);
 #pragma unroll
-            for (int kk = 0; kk < DH / 16; ++kk) {
-                uint32_t a[4];
-                ldmatrix_x4(a, s_q_u32 + tile_off<DH>(warp * 16 + (lane & 15), kk * 2 + (lane >> 4)));
-#pragma unroll
-                for (int np = 0; np < 2; ++np) {  // pairs of 8-key blocks
-                    uint32_t bfr[4];
-                    const int krow = half * 32 + np * 16 + (lane & 7) + ((lane >> 4) << 3);
-                    ldmatrix_x4(bfr, ks + tile_off<DH>(krow, kk * 2 + ((lane >> 3) & 1)));
-                    mma_bf16(sacc[np * 2 + 0], a, bfr[0], bfr[1]);
-                    mma_bf16(sacc[np * 2 + 1], a, bfr[2], bfr[3]);
+                for (int h = 0; h < HALVES; ++h)
+                    tma_load_3d(sV + st * kTile + h * kPanel, &v_map, h * 64, hk, row, smem_u32(&bars.v_full[st]));
+                issued = j + 1;
+            }
+            if (*abort_flag) {
+                if (plan.q_tma) {
+                    const long long t0 = clock64();
+                    while (!mbar_try_wait(smem_u32(&bars.q_full), 0) && clock64() - t0 < kWaitCycles) {}
+                }
+                // drain: every copy issued for the newest tile of each stage must have landed before
+                // the block may leave (bounded by the clock only, the flag is already up)
+                for (int j = max(0, issued - NST); j < issued; ++j) {
+                    const int st = j % NST;
+                    const uint32_t ph = (uint32_t)((j / NST) & 1);
+                    const long long t0 = clock64();
+                    while (!mbar_try_wait(smem_u32(&bars.k_full[st]), ph) && clock64() - t0 < kWaitCycles) {}
+                    while (!mbar_try_wait(smem_u32(&bars.v_full[st]), ph) && clock64() - t0 < kWaitCycles) {}
                 }
             }
-            // scale, mask, online softmax
-            float mx[2] = {-INFINITY, -INFINITY};
+        }
+    } else if (warp == kMmaWarp) {
+        // ===== MMA issuer (whole warp walks the loop, lane 0 waits and issues) =====================
+        auto wait_all = [&](uint32_t bar, uint32_t parity) {  // lane 0 polls, the warp gets the outcome
+            int r = 1;
+            if (lane == 0) r = mbar_wait(bar, parity, abort_flag) ? 1 : 0;
+            r = __shfl_sync(0xffffffffu, r, 0);
+            __syncwarp();
+            return r != 0;
+        };
+        bool ok = wait_all(smem_u32(&bars.q_full), 0);
+        auto issue_qk = [&](int i) {  // S[slot] = Q[row tile] . K[tile]^T
+            const int j = i / MT, t = i % MT, st = j % NST;
+            if (t == 0) ok = ok && wait_all(smem_u32(&bars.k_full[st]), (uint32_t)((j / NST) & 1));
+            if (!ok) return;
+            tc_fence_after();
+            if (lane == 0) {
+                const uint32_t d_tmem = tmem + (uint32_t)(i % kSlots) * kTK;
 #pragma unroll
-            for (int n = 0; n < 4; ++n) {
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    float sv = sacc[n][e] * scale_log2;
-                    if (need_mask) {
-                        const int key = key0 + half * 32 + n * 8 + (lane & 3) * 2 + (e & 1);
-                        bool vis = key < L;
-                        if (!vis && key < n_keys) {
-                            const int j = key - L;
-                            const int tok = (e & 2) ? tok_hi : tok_lo;
-                            vis = (s_mask[tok * W + (j >> 6)] >> (j & 63)) & 1ull;
-                        }
-                        if (!vis) sv = -INFINITY;
+                for (int ks = 0; ks < DH / 16; ++ks) {
+                    const uint32_t koff = (uint32_t)(ks / 4) * kPanel + (uint32_t)(ks % 4) * 32u;
+                    mma_ss(d_tmem, smem_desc(sQ + t * kTile + koff, 16), smem_desc(sK + st * kTile + koff, 16),
+                           kIdescQK, ks > 0);
+                }
+                tc_commit(smem_u32(&bars.s_full[i % kSlots]));
+                if (t == MT - 1) tc_commit(smem_u32(&bars.k_empty[st]));
+            }
+            __syncwarp();
+        };
+        auto issue_pv = [&](int i) {  // O[row tile] += P[slot] . V[tile]
+            const int j = i / MT, t = i % MT, st = j % NST;
+            if (t == 0) {
+                ok = ok && wait_all(smem_u32(&bars.v_full[st]), (uint32_t)((j / NST) & 1));
+                if (!ok) return;
+                const int valid = n_keys - (t_begin + j) * kTK;
+                if (valid < kTK) {
+                    // rows past the sequence's last key hold whatever follows it in the cache: clear
+                    // them so that a zero probability times a non-finite value cannot reach O
+                    const int chunks = (kTK - valid) * 8;
+                    for (int idx = lane; idx < chunks * HALVES; idx += 32) {
+                        const int h = idx / chunks, rem = idx % chunks;
+                        const int r = valid + rem / 8, c = rem % 8;
+                        *reinterpret_cast<uint4*>(smem_gen + (sV - smem_base) + st * kTile + h * kPanel + r * 128 +
+                                                  c * 16) = make_uint4(0, 0, 0, 0);
                     }
-                    sacc[n][e] = sv;
-                    mx[e >> 1] = fmaxf(mx[e >> 1], sv);
+                    fence_proxy_async();
+                    __syncwarp();
                 }
             }
-            float corr[2];
+            ok = ok && wait_all(smem_u32(&bars.p_full[i % kSlots]), (uint32_t)((i / kSlots) & 1));
+            if (!ok) return;
+            tc_fence_after();
+            if (lane == 0) {
+                const uint32_t d_tmem = tmem + kOCol + (uint32_t)t * DH;
+                const uint32_t a_tmem = tmem + (uint32_t)(i % kSlots) * kTK;
 #pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                mx[h] = fmaxf(mx[h], __shfl_xor_sync(0xffffffffu, mx[h], 1));
-                mx[h] = fmaxf(mx[h], __shfl_xor_sync(0xffffffffu, mx[h], 2));
-                const float m_new = fmaxf(m_run[h], mx[h]);
-                corr[h] = (m_new == -INFINITY) ? 1.f : exp2f(m_run[h] - m_new);
-                m_run[h] = m_new;
-                l_run[h] *= corr[h];
+                for (int ks = 0; ks < kTK / 16; ++ks)
+                    mma_ts(d_tmem, a_tmem + ks * 8, smem_desc(sV + st * kTile + ks * 2048u, kPanel), kIdescPV,
+                           (j > 0 || ks > 0) ? 1u : 0u);
+                tc_commit(smem_u32(&bars.o_done[t][j & 1]));
+                if (t == MT - 1) tc_commit(smem_u32(&bars.v_empty[st]));
             }
-            const float base_lo = m_run[0] == -INFINITY ? 0.f : m_run[0];
-            const float base_hi = m_run[1] == -INFINITY ? 0.f : m_run[1];
-            uint32_t pf[2][4];
-#pragma unroll
-            for (int n = 0; n < 4; ++n) {
-                const float p0 = exp2f(sacc[n][0] - base_lo), p1 = exp2f(sacc[n][1] - base_lo);
-                const float p2 = exp2f(sacc[n][2] - base_hi), p3 = exp2f(sacc[n][3] - base_hi);
-                l_run[0] += p0 + p1;
-                l_run[1] += p2 + p3;
-                pf[n >> 1][(n & 1) * 2 + 0] = pack_bf16(p0, p1);
-                pf[n >> 1][(n & 1) * 2 + 1] = pack_bf16(p2, p3);
-            }
-#pragma unroll
-            for (int n = 0; n < DH / 8; ++n) {
-                oacc[n][0] *= corr[0], oacc[n][1] *= corr[0];
-                oacc[n][2] *= corr[1], oacc[n][3] *= corr[1];
-            }
-            // O += P.V over these 32 keys
-#pragma unroll
-            for (int kk = 0; kk < 2; ++kk) {
-#pragma unroll
-                for (int np = 0; np < DH / 16; ++np) {
-                    uint32_t bfr[4];
-                    const int vrow = half * 32 + kk * 16 + (lane & 7) + (((lane >> 3) & 1) << 3);
-                    ldmatrix_x4_trans(bfr, vs + tile_off<DH>(vrow, np * 2 + (lane >> 4)));
-                    mma_bf16(oacc[np * 2 + 0], pf[kk], bfr[0], bfr[1]);
-                    mma_bf16(oacc[np * 2 + 1], pf[kk], bfr[2], bfr[3]);
-                }
-            }
+            __syncwarp();
+        };
+        for (int i = 0; i < kSlots && i < n_items && ok; ++i) issue_qk(i);
+        for (int i = 0; i < n_items && ok; ++i) {
+            issue_pv(i);
+            if (ok && i + kSlots < n_items) issue_qk(i + kSlots);
         }
-    }
-    cp_async_wait<0>();
+    } else {
+        // ===== softmax warps: thread = packed query row ============================================
+        const int wg = warp >> 2;                         // row tile of this warp group
+        const int r_tile = ((warp & 3) << 5) | lane;      // row inside the tile = tensor-memory lane
+        const int r_blk = wg * 128 + r_tile;              // row inside the block
+        const bool row_ok = r_blk < rows_here;
+        const int pr = row0 + (row_ok ? r_blk : 0);       // packed row = token * g + head in group
+        const int tok = pr / g, hq = hk * g + pr % g;
+        const uint32_t lane_sel = (uint32_t)((warp & 3) << 5) << 16;
 
-    // ---- epilogue ----------------------------------------------------------------------------
+        const int W = (m + 63) >> 6;
+        const unsigned long long mlo = mask_bits[((long long)b * m + tok) * W];
+        const unsigned long long mhi = W > 1 ? mask_bits[((long long)b * m + tok) * W + 1] : 0ull;
+        if (!plan.q_tma) {
+            // query rows into shared memory by hand, 128-byte swizzled (chunk c of row r at
+            // c ^ (r & 7)); all copies of a thread are in flight together, absent rows zero-filled
 #pragma unroll
-    for (int h = 0; h < 2; ++h) {
-        l_run[h] += __shfl_xor_sync(0xffffffffu, l_run[h], 1);
-        l_run[h] += __shfl_xor_sync(0xffffffffu, l_run[h], 2);
-    }
-#pragma unroll
-    for (int h = 0; h < 2; ++h) {
-        const int pr = qrow_lo + h * 8;
-        if (pr >= M || pr >= row0 + RB) continue;
-        if (S == 1) {
-            const int tok = pr / g, gq = pr % g, hq = hk * g + gq;
-            const float inv = l_run[h] > 0.f ? 1.f / l_run[h] : 0.f;
-            __nv_bfloat16* dst = out + (((long long)b * m + tok) * Hq + hq) * DH;
-#pragma unroll
-            for (int n = 0; n < DH / 8; ++n) {
-                const uint32_t v = pack_bf16(oacc[n][2 * h] * inv, oacc[n][2 * h + 1] * inv);
-                *reinterpret_cast<uint32_t*>(dst + n * 8 + (lane & 3) * 2) = v;
+            for (int it = 0; it < DH / 8; ++it) {
+                const int idx = tid + it * kSoftmaxThreads;
+                const int r = idx / (DH / 8), c = idx % (DH / 8);
+                const bool live = r < rows_here;
+                const int p2 = row0 + (live ? r : 0);
+                const __nv_bfloat16* src = q + (((long long)b * m + p2 / g) * Hq + hk * g + p2 % g) * DH + c * 8;
+                const int t = r >> 7, rr = r & 127, h = c >> 3, cc = c & 7;
+                cp_async16(sQ + t * kTile + h * kPanel + rr * 128 + ((cc ^ (rr & 7)) << 4), src, live);
             }
-            if (lse && (lane & 3) == 0)
-                lse[((long long)b * Hq + hq) * m + tok] =
-                    (m_run[h] + log2f(l_run[h])) * 0.69314718055994531f;
-        } else {
-            const size_t prow = (((size_t)b * Hkv + hk) * S + split) * ((size_t)plan.n_rb * RB) + (pr);
-            float* dst = ws.o_part + prow * DH;
+            cp_async_commit();
+            cp_async_wait_all();
+            fence_proxy_async();
+            mbar_arrive(smem_u32(&bars.q_full));
+        }
+
+        float m_ref = -INFINITY, l_run = 0.f;
+        bool ok = true;
+        for (int j = 0; j < nt; ++j) {
+            const int i = j * MT + wg, slot = i % kSlots;
+            ok = mbar_wait(smem_u32(&bars.s_full[slot]), (uint32_t)((i / kSlots) & 1), abort_flag);
+            ok = __all_sync(0xffffffffu, ok);  // the tensor-memory accesses below need the whole warp
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t s_addr = tmem + lane_sel + (uint32_t)slot * kTK;
+            const int key0 = (t_begin + j) * kTK;
+            const bool tail = key0 + kTK > L;  // the tile holds tree keys or runs past the last key
+            uint32_t vis[4] = {~0u, ~0u, ~0u, ~0u};
+            if (tail) tile_visibility(mlo, mhi, key0, L, n_keys, vis);
+
+            // Both passes walk the row in four 32-column chunks through two register buffers: the
+            // load of the next chunk is in flight while the current one is processed.  A tile that
+            // lies wholly inside the committed cache takes the branch without mask arithmetic.
+            uint32_t bufa[32], bufb[32];
+            // pass 1: row maximum of the raw scores (the scale is positive)
+            float mx = -INFINITY;
+            tmem_ld32(s_addr, bufa);
+            tc_wait_ld(bufa);
+            tmem_ld32(s_addr + 32, bufb);
+            mx = tail ? chunk_rowmax<true>(bufa, vis[0], mx) : chunk_rowmax<false>(bufa, 0, mx);
+            tc_wait_ld(bufb);
+            tmem_ld32(s_addr + 64, bufa);
+            mx = tail ? chunk_rowmax<true>(bufb, vis[1], mx) : chunk_rowmax<false>(bufb, 0, mx);
+            tc_wait_ld(bufa);
+            tmem_ld32(s_addr + 96, bufb);
+            mx = tail ? chunk_rowmax<true>(bufa, vis[2], mx) : chunk_rowmax<false>(bufa, 0, mx);
+            tc_wait_ld(bufb);
+            tmem_ld32(s_addr, bufa);  // first chunk of pass 2
+            mx = tail ? chunk_rowmax<true>(bufb, vis[3], mx) : chunk_rowmax<false>(bufb, 0, mx);
+            mx *= scale_log2;
+
+            // lazily rescaled reference maximum: probabilities stay below 2^8 in between
+            const float m_new = fmaxf(m_ref, mx);
+            const bool grow = m_new > m_ref + 8.f;
+            if (__any_sync(0xffffffffu, grow)) {
+                const float factor = !grow ? 1.f : (m_ref == -INFINITY ? 0.f : ex2(m_ref - m_new));
+                if (grow) m_ref = m_new, l_run *= factor;
+                // O may be rescaled once the previous P.V of this row tile has finished
+                if (j > 0)
+                    ok = mbar_wait(smem_u32(&bars.o_done[wg][(j - 1) & 1]), (uint32_t)(((j - 1) >> 1) & 1), abort_flag);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                if (j > 0) {
+                    tc_fence_after();
+                    const uint32_t o_addr = tmem + lane_sel + kOCol + (uint32_t)wg * DH;
 #pragma unroll
-            for (int n = 0; n < DH / 8; ++n)
-                *reinterpret_cast<float2*>(dst + n * 8 + (lane & 3) * 2) =
-                    make_float2(oacc[n][2 * h], oacc[n][2 * h + 1]);
-            if ((lane & 3) == 0) ws.ml[prow] = make_float2(m_run[h], l_run[h]);
+                    for (int c4 = 0; c4 < DH / 32; ++c4) {
+                        tmem_ld32(o_addr + c4 * 32, bufb);
+                        tc_wait_ld(bufb);
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) bufb[c] = __float_as_uint(__uint_as_float(bufb[c]) * factor);
+                        tmem_st32(o_addr + c4 * 32, bufb);
+                    }
+                }
+            }
+            // pass 2: P = 2^(s * scale - reference) as bf16 over the first 64 columns of the slot;
+            // packed columns [0,32) are written once score columns [0,64) are in registers, [32,64)
+            // after the rest
+            const float neg_ref = m_ref == -INFINITY ? 0.f : -m_ref;
+            const float2 scale2 = make_float2(scale_log2, scale_log2), neg_ref2 = make_float2(neg_ref, neg_ref);
+            float2 sum_a = make_float2(0.f, 0.f), sum_b = make_float2(0.f, 0.f);
+            uint32_t pk[32];
+            tc_wait_ld(bufa);
+            tmem_ld32(s_addr + 32, bufb);
+            if (tail) chunk_probs<true>(bufa, vis[0], scale2, neg_ref2, sum_a, sum_b, pk);
+            else chunk_probs<false>(bufa, 0, scale2, neg_ref2, sum_a, sum_b, pk);
+            tc_wait_ld(bufb);
+            tmem_ld32(s_addr + 64, bufa);
+            if (tail) chunk_probs<true>(bufb, vis[1], scale2, neg_ref2, sum_a, sum_b, pk + 16);
+            else chunk_probs<false>(bufb, 0, scale2, neg_ref2, sum_a, sum_b, pk + 16);
+            tc_wait_ld(bufa);
+            tmem_ld32(s_addr + 96, bufb);
+            tmem_st32(s_addr, pk);
+            if (tail) chunk_probs<true>(bufa, vis[2], scale2, neg_ref2, sum_a, sum_b, pk);
+            else chunk_probs<false>(bufa, 0, scale2, neg_ref2, sum_a, sum_b, pk);
+            tc_wait_ld(bufb);
+            if (tail) chunk_probs<true>(bufb, vis[3], scale2, neg_ref2, sum_a, sum_b, pk + 16);
+            else chunk_probs<false>(bufb, 0, scale2, neg_ref2, sum_a, sum_b, pk + 16);
+            tmem_st32(s_addr + 32, pk);
+            l_run += (sum_a.x + sum_a.y) + (sum_b.x + sum_b.y);
+            tc_wait_st();
+            tc_fence_before();
+            mbar_arrive(smem_u32(&bars.p_full[slot]));
+        }
+
+        // ---- epilogue: O rows leave tensor memory through shared memory, so that the global
+        // stores are whole contiguous rows.  Row tile 0 stages in the query region (both row tiles'
+        // Q.K^T are complete once any last P.V is), the other one - and a single tile - in the K ring.
+        ok = ok && mbar_wait(smem_u32(&bars.o_done[wg][(nt - 1) & 1]), (uint32_t)(((nt - 1) >> 1) & 1), abort_flag);
+        ok = __all_sync(0xffffffffu, ok);
+        if (ok) {
+            tc_fence_after();
+            const uint32_t o_addr = tmem + lane_sel + kOCol + (uint32_t)wg * DH;
+            const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+            unsigned char* stage = smem_gen + ((MT == 2 && wg == 0) ? 0u : (sK - smem_base));
+            // a staged row is DH fp32 (partial) or DH bf16 (final); 16-byte chunk c of row r sits at
+            // chunk c ^ (r mod chunks-per-row), which keeps both the row-wise writes and the
+            // chunk-wise reads free of bank conflicts
+            const int row_bytes = direct ? DH * 2 : DH * 4;
+            const int cmask = row_bytes / 16 - 1;
+#pragma unroll
+            for (int c4 = 0; c4 < DH / 32; ++c4) {
+                uint32_t orow[32];
+                tmem_ld32(o_addr + c4 * 32, orow);
+                tc_wait_ld(orow);
+                unsigned char* srow = stage + (size_t)r_tile * row_bytes;
+                if (direct) {
+#pragma unroll
+                    for (int c = 0; c < 32; c += 8) {
+                        uint4 v;
+                        v.x = pack_bf16(__uint_as_float(orow[c + 0]) * inv, __uint_as_float(orow[c + 1]) * inv);
+                        v.y = pack_bf16(__uint_as_float(orow[c + 2]) * inv, __uint_as_float(orow[c + 3]) * inv);
+                        v.z = pack_bf16(__uint_as_float(orow[c + 4]) * inv, __uint_as_float(orow[c + 5]) * inv);
+                        v.w = pack_bf16(__uint_as_float(orow[c + 6]) * inv, __uint_as_float(orow[c + 7]) * inv);
+                        const int chunk = c4 * 4 + (c >> 3);
+                        *reinterpret_cast<uint4*>(srow + (((chunk ^ r_tile) & cmask) << 4)) = v;
+                    }
+                } else {
+#pragma unroll
+                    for (int c = 0; c < 32; c += 4) {
+                        const int chunk = c4 * 8 + (c >> 2);
+                        *reinterpret_cast<uint4*>(srow + (((chunk ^ r_tile) & cmask) << 4)) =
+                            make_uint4(orow[c], orow[c + 1], orow[c + 2], orow[c + 3]);
+                    }
+                }
+            }
+            if (row_ok) {
+                if (direct) {
+                    if (lse) lse[((long long)b * Hq + hq) * m + tok] = (m_ref + log2f(l_run)) * 0.69314718055994531f;
+                } else {
+                    ws.ml[part_row0 + r_blk] = make_float2(m_ref, l_run);
+                }
+            }
+            asm volatile("bar.sync %0, 128;" ::"r"(1 + wg) : "memory");  // the row tile's four warps
+            const int rows_tile = min(128, rows_here - wg * 128);
+            const int lanes_per_row = row_bytes / 16;       // 16 or 32 (8 for a 64-wide bf16 row)
+            const int rows_per_pass = 32 / lanes_per_row;
+            const int sub = lane / lanes_per_row, cl = lane % lanes_per_row;
+            for (int r = (warp & 3) * rows_per_pass + sub; r < rows_tile; r += 4 * rows_per_pass) {
+                const uint4 v = *reinterpret_cast<const uint4*>(stage + (size_t)r * row_bytes + (((cl ^ r) & cmask) << 4));
+                if (direct) {
+                    const int p2 = row0 + wg * 128 + r;
+                    __nv_bfloat16* dst = out + (((long long)b * m + p2 / g) * Hq + hk * g + p2 % g) * DH;
+                    *reinterpret_cast<uint4*>(reinterpret_cast<unsigned char*>(dst) + cl * 16) = v;
+                } else {
+                    float* dst = ws.o_part + (part_row0 + wg * 128 + r) * DH;
+                    *reinterpret_cast<uint4*>(reinterpret_cast<unsigned char*>(dst) + cl * 16) = v;
+                }
+            }
         }
     }
+
+    // ---- teardown ----------------------------------------------------------------------------------
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (warp == kMmaWarp) tmem_dealloc(tmem, kTmemCols);
+    if (tid == 0 && s_abort) raise_status(d_status, EAGLE2_STATUS_TIMEOUT);
 }
 
-// One warp per output row: combine the splits' partials.
+// One warp per output row of a sequence that used several splits: combine their partials.
 template <int DH>
 __global__ void __launch_bounds__(256)
-tree_attention_merge_kernel(int B, int m, int Hq, int Hkv, AttnPlan plan, AttnWs ws,
-                            __nv_bfloat16* __restrict__ out, float* __restrict__ lse) {
+tree_attention_merge_kernel(const int64_t* __restrict__ kv_off, const int32_t* __restrict__ kv_len, int B, int m,
+                            int Hq, int Hkv, long long cache_rows, int max_kv_len, AttnPlan plan, AttnWs ws, __nv_bfloat16* __restrict__ out,
+                            float* __restrict__ lse) {
     const int warp_global = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
     const int g = plan.g, S = plan.splits;
     const long long total = (long long)B * Hkv * plan.M;
@@ -329,21 +807,28 @@ tree_attention_merge_kernel(int B, int m, int Hq, int Hkv, AttnPlan plan, AttnWs
     const int pr = warp_global % plan.M;
     const int hk = (warp_global / plan.M) % Hkv;
     const int b = warp_global / (plan.M * Hkv);
-    const size_t rows_per_split = (size_t)plan.n_rb * plan.RB;
-    const size_t first = (((size_t)b * Hkv + hk) * S) * rows_per_split + pr;
+    const int L = kv_len[b];
+    if (!sequence_ok(L, kv_off[b], m, max_kv_len, cache_rows)) return;
+    const int tiles = (L + m + kTK - 1) / kTK;
+    const int S_b = (tiles + plan.per_split - 1) / plan.per_split;
+    if (S_b <= 1) return;  // the attention kernel wrote these rows itself
+    const int rb = pr / plan.per, r = pr % plan.per;
+    const size_t rows_per_block = (size_t)plan.mt * kRowsPerTile;
+    const size_t stride = (size_t)plan.n_rb * rows_per_block;  // rows between consecutive splits
+    const size_t first = (((size_t)b * Hkv + hk) * S) * stride + rb * rows_per_block + r;
     float mmax = -INFINITY;
-    for (int s = 0; s < S; ++s) mmax = fmaxf(mmax, ws.ml[first + s * rows_per_split].x);
+    for (int s = 0; s < S_b; ++s) mmax = fmaxf(mmax, ws.ml[first + s * stride].x);
     constexpr int PER = DH / 32;
     float acc[PER];
 #pragma unroll
     for (int e = 0; e < PER; ++e) acc[e] = 0.f;
     float l = 0.f;
-    for (int s = 0; s < S; ++s) {
-        const float2 ml = ws.ml[first + s * rows_per_split];
+    for (int s = 0; s < S_b; ++s) {
+        const float2 ml = ws.ml[first + s * stride];
         if (ml.x == -INFINITY) continue;
         const float w = exp2f(ml.x - mmax);
         l += ml.y * w;
-        const float* src = ws.o_part + (first + s * rows_per_split) * DH + lane * PER;
+        const float* src = ws.o_part + (first + s * stride) * DH + lane * PER;
 #pragma unroll
         for (int e = 0; e < PER; ++e) acc[e] += src[e] * w;
     }
@@ -357,28 +842,32 @@ tree_attention_merge_kernel(int B, int m, int Hq, int Hkv, AttnPlan plan, AttnWs
         lse[((long long)b * Hq + hq) * m + tok] = (mmax + log2f(l)) * 0.69314718055994531f;
 }
 
-template <int DH>
-static int launch_attention(const void* q, const void* k_cache, const void* v_cache, const int64_t* kv_off,
-                            const int32_t* kv_len, const uint64_t* mask_bits, int B, int m, int Hq, int Hkv,
-                            const AttnPlan& plan, float scale, void* out, float* lse, const AttnWs& ws,
+template <int DH, int MT>
+static int launch_attention(const CUtensorMap& k_map, const CUtensorMap& v_map, const CUtensorMap& q_map,
+                            const void* q,
+                            const int64_t* kv_off, const int32_t* kv_len, const uint64_t* mask_bits, int B,
+                            int m, int Hq, int Hkv, long long cache_rows, int max_kv_len, const AttnPlan& plan,
+                            float scale, void* out, float* lse, const AttnWs& ws, int32_t* d_status,
                             cudaStream_t st) {
-    auto kern = tree_attention_kernel<DH>;
+    auto kern = tree_attention_kernel<DH, MT>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem) !=
-        cudaSuccess)
+        cudaSuccess) {
+        cudaGetLastError();
         return EAGLE2_ERR_CUDA;
+    }
     const long long blocks = (long long)B * Hkv * plan.n_rb * plan.splits;
     if (blocks > 0x7fffffffLL) return EAGLE2_ERR_SHAPE;
-    kern<<<(unsigned)blocks, plan.warps * 32, plan.smem, st>>>(
-        static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(k_cache),
-        static_cast<const __nv_bfloat16*>(v_cache), kv_off, kv_len, mask_bits, m, Hq, Hkv, plan,
-        scale * 1.4426950408889634f, static_cast<__nv_bfloat16*>(out), lse, ws);
+    kern<<<(unsigned)blocks, MT * 128 + 64, plan.smem, st>>>(
+        k_map, v_map, q_map, static_cast<const __nv_bfloat16*>(q), kv_off, kv_len, mask_bits, m, Hq, Hkv, cache_rows,
+        max_kv_len, plan, scale * 1.4426950408889634f, static_cast<__nv_bfloat16*>(out), lse, ws, d_status);
     if (launch_result() != EAGLE2_OK) return EAGLE2_ERR_CUDA;
     if (plan.splits > 1) {
         const long long warps = (long long)B * Hkv * plan.M;
         const long long mblocks = (warps + 7) / 8;
         if (mblocks > 0x7fffffffLL) return EAGLE2_ERR_SHAPE;
         tree_attention_merge_kernel<DH><<<(unsigned)mblocks, 256, 0, st>>>(
-            B, m, Hq, Hkv, plan, ws, static_cast<__nv_bfloat16*>(out), lse);
+            kv_off, kv_len, B, m, Hq, Hkv, cache_rows, max_kv_len, plan, ws, static_cast<__nv_bfloat16*>(out),
+            lse);
         return launch_result();
     }
     return EAGLE2_OK;
@@ -389,14 +878,15 @@ static int launch_attention(const void* q, const void* k_cache, const void* v_ca
 using namespace eagle2;
 
 extern "C" int eagle2_tree_attention(const void* q, const void* k_cache, const void* v_cache,
-                                     const int64_t* kv_off, const int32_t* kv_len,
+                                     long long cache_rows, const int64_t* kv_off, const int32_t* kv_len,
                                      const uint64_t* mask_bits, int B, int m, int Hq, int Hkv, int d,
                                      int max_kv_len, float scale, void* out, float* lse, void* ws,
                                      size_t ws_bytes, int32_t* d_status, eagle2_stream_t stream) {
     if (!q || !k_cache || !v_cache || !kv_off || !kv_len || !mask_bits || !out || !d_status)
         return EAGLE2_ERR_NULL;
     if (B < 0 || m < 1 || m > EAGLE2_MAX_M || Hq < 1 || Hkv < 1 || Hq % Hkv || Hq / Hkv > 8 ||
-        (d != 64 && d != 128) || max_kv_len < 0)
+        (d != 64 && d != 128) || max_kv_len < 0 || cache_rows < 1 || cache_rows > 0x7fffffffLL ||
+        (long long)max_kv_len + m > cache_rows || !(scale > 0.f))
         return EAGLE2_ERR_SHAPE;
     if (!aligned(q, 16) || !aligned(k_cache, 16) || !aligned(v_cache, 16) || !aligned(out, 16) ||
         !aligned(mask_bits, 8))
@@ -409,10 +899,23 @@ extern "C" int eagle2_tree_attention(const void* q, const void* k_cache, const v
         if (!ws || !aligned(ws, kWsAlign)) return EAGLE2_ERR_WORKSPACE;
         if (attention_ws_layout(B, Hkv, d, plan, ws, &w) > ws_bytes) return EAGLE2_ERR_WORKSPACE;
     }
+    CUtensorMap k_map, v_map, q_map;
+    if (!make_cache_map(&k_map, k_cache, cache_rows, Hkv, d) || !make_cache_map(&v_map, v_cache, cache_rows, Hkv, d))
+        return EAGLE2_ERR_CUDA;
+    if (plan.q_tma) {
+        if (!make_query_map(&q_map, q, B, m, Hq, Hkv, d)) return EAGLE2_ERR_CUDA;
+    } else {
+        q_map = k_map;  // unused by the kernel
+    }
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-    if (d == 64)
-        return launch_attention<64>(q, k_cache, v_cache, kv_off, kv_len, mask_bits, B, m, Hq, Hkv, plan,
-                                    scale, out, lse, w, st);
-    return launch_attention<128>(q, k_cache, v_cache, kv_off, kv_len, mask_bits, B, m, Hq, Hkv, plan, scale,
-                                 out, lse, w, st);
+#define EAGLE2_ATTN_CASE(DH_, MT_)                                                                        \
+    return launch_attention<DH_, MT_>(k_map, v_map, q_map, q, kv_off, kv_len, mask_bits, B, m, Hq, Hkv, cache_rows, \
+                                      max_kv_len, plan, scale, out, lse, w, d_status, st)
+    if (d == 64) {
+        if (plan.mt == 1) EAGLE2_ATTN_CASE(64, 1);
+        EAGLE2_ATTN_CASE(64, 2);
+    }
+    if (plan.mt == 1) EAGLE2_ATTN_CASE(128, 1);
+    EAGLE2_ATTN_CASE(128, 2);
+#undef EAGLE2_ATTN_CASE
 }

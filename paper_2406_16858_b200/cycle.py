@@ -86,8 +86,8 @@ class CycleBuffers:
 
     def attention(self, q, k_cache, v_cache, kv_off, kv_len, out, scale: float) -> None:
         s = self.shape
-        e2.tree_attention(q, k_cache, v_cache, kv_off, kv_len, self.mask_bits, s.B, s.m, s.Hq, s.Hkv,
-                          s.d, s.max_kv_len, scale, out, None, self.ws, self.status)
+        e2.tree_attention(q, k_cache, v_cache, k_cache.shape[0], kv_off, kv_len, self.mask_bits, s.B,
+                          s.m, s.Hq, s.Hkv, s.d, s.max_kv_len, scale, out, None, self.ws, self.status)
 
     def accept(self, target_logits, draft_rows, u_accept, u_bonus) -> None:
         s = self.shape

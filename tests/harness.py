@@ -89,7 +89,7 @@ def gpu_attention(q, kc, vc, kv_off, kv_len, mask_bits, scale, want_lse=False):
     st = new_status()
     ws = make_ws(e2.workspace_bytes(e2.OP_TREE_ATTENTION, B=B, m=m, Hq=Hq, Hkv=Hkv, d=d,
                                     max_kv_len=max_len))
-    e2.tree_attention(tq, tk, tv, dev(kv_off.astype(np.int64)), dev(kv_len.astype(np.int32)),
+    e2.tree_attention(tq, tk, tv, kc.shape[0], dev(kv_off.astype(np.int64)), dev(kv_len.astype(np.int32)),
                       dev(mask_bits), B, m, Hq, Hkv, d, max_len, scale, out, lse, ws, st)
     torch.cuda.synchronize()
     return host(out, np.uint16), (host(lse) if want_lse else None), int(st.item())

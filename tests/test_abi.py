@@ -62,8 +62,8 @@ def test_null_and_shape_errors_are_found_on_the_host():
     assert _code(e2.tree_mask, FAKE, FAKE, FAKE, FAKE, 1, 0, FAKE, None, FAKE, FAKE) == -2
     # attention: head_dim, group size, alignment
     att = lambda **kw: e2.tree_attention(  # noqa: E731
-        kw.get("q", FAKE), FAKE, FAKE, FAKE, FAKE, FAKE, 1, 16, kw.get("Hq", 4), kw.get("Hkv", 4),
-        kw.get("d", 64), 128, 0.125, FAKE, None, None, FAKE)
+        kw.get("q", FAKE), FAKE, FAKE, kw.get("rows", 1024), FAKE, FAKE, FAKE, 1, 16, kw.get("Hq", 4),
+        kw.get("Hkv", 4), kw.get("d", 64), 128, 0.125, FAKE, None, None, FAKE)
     assert _code(att) == -4  # two KV splits at this size: a workspace is required
     with pytest.raises(e2.Eagle2Error) as exc:
         att(d=96)
@@ -74,6 +74,9 @@ def test_null_and_shape_errors_are_found_on_the_host():
     with pytest.raises(e2.Eagle2Error) as exc:
         att(q=FAKE + 2)
     assert exc.value.code == -3
+    with pytest.raises(e2.Eagle2Error) as exc:
+        att(rows=100)  # the longest sequence (128 + 16 rows) does not fit in the cache
+    assert exc.value.code == -2
     # accept: sampling needs the uniforms
     assert _code(e2.accept, FAKE, 0, None, 0, FAKE, FAKE, FAKE, FAKE, 1, 100, 4, 3, 16, 1.0, None, None,
                  FAKE, FAKE, FAKE, None, FAKE) == -1

@@ -79,6 +79,59 @@ def test_shapes_tails_and_gqa(m, Hq, Hkv, d, lens):
     _compare(q, kc, vc, off, kl, bits, 1.0 / np.sqrt(d))
 
 
+@pytest.mark.parametrize("m,Hq,Hkv,d,lens", [
+    # many (sequence, KV head) pairs leave one split per sequence: several tiles per block, so the
+    # K/V ring and the score slots are reused; ragged lengths leave some blocks a single tile
+    (60, 16, 16, 128, [700, 100, 1500, 40, 2100, 300, 900, 5]),      # one 128-row tile per block
+    (60, 32, 8, 128, [2300, 64, 513, 1200, 1, 0, 777, 1800, 130, 260, 2047, 90, 400, 33, 1024, 640]),
+    (33, 8, 8, 64, [1500, 257, 900, 31, 2000, 5, 640, 128, 129, 1100]),  # head_dim 64, deeper ring
+])
+def test_many_tiles_per_block(m, Hq, Hkv, d, lens):
+    q, kc, vc, off, kl, bits = _inputs(23, len(lens), m, Hq, Hkv, d, lens)
+    rng = np.random.default_rng(5)
+    n = 400
+    samples = np.stack([rng.integers(0, len(lens), n), rng.integers(0, Hq, n),
+                        rng.integers(0, m, n)], axis=1).astype(np.int32)
+    _compare(q, kc, vc, off, kl, bits, 1.0 / np.sqrt(d), samples=samples)
+
+
+def test_rows_after_a_sequence_may_hold_anything():
+    """The kernel streams whole tiles, so it reads cache rows that follow a sequence's last key; their
+    contents (here NaN and Inf bit patterns) must not reach the output."""
+    m, Hq, Hkv, d = 16, 4, 2, 64
+    kv_len = np.array([70, 3], np.int32)
+    kv_off = np.array([0, 200], np.int64)  # slack between and after the sequences
+    rows = 400
+    rng = np.random.default_rng(2)
+    q = gen.f32_to_bf16_bits(rng.standard_normal((2, m, Hq, d)).astype(np.float32))
+    kc = np.full((rows, Hkv, d), 0x7FC0, np.uint16)  # NaN
+    vc = np.full((rows, Hkv, d), 0x7F80, np.uint16)  # +Inf
+    for b in range(2):
+        lo, hi = int(kv_off[b]), int(kv_off[b] + kv_len[b] + m)
+        kc[lo:hi] = gen.f32_to_bf16_bits(rng.standard_normal((hi - lo, Hkv, d)).astype(np.float32))
+        vc[lo:hi] = gen.f32_to_bf16_bits(rng.standard_normal((hi - lo, Hkv, d)).astype(np.float32))
+    bits = _random_forest_mask(rng, 2, m, kv_len)
+    _compare(q, kc, vc, kv_off, kv_len, bits, 0.125)
+
+
+def test_sequence_outside_the_cache_is_reported_and_skipped():
+    m, Hq, Hkv, d = 16, 2, 2, 64
+    q, kc, vc, off, kl, bits = _inputs(3, 2, m, Hq, Hkv, d, [50, 60])
+    tq, tk, tv = dev(q), dev(kc), dev(vc)
+    out = torch.full((2, m, Hq, d), 0x1234, dtype=torch.int16, device=DEV)
+    st = new_status()
+    ws = make_ws(e2.workspace_bytes(e2.OP_TREE_ATTENTION, B=2, m=m, Hq=Hq, Hkv=Hkv, d=d, max_kv_len=60))
+    bad_len = np.array([50, 61], np.int32)  # sequence 1 claims more rows than max_kv_len allows
+    e2.tree_attention(tq, tk, tv, kc.shape[0], dev(off), dev(bad_len), dev(bits), 2, m, Hq, Hkv, d, 60,
+                      0.125, out, None, ws, st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == e2.STATUS_KV_OVERFLOW
+    got = host(out, np.uint16)
+    assert (got[1] == 0x1234).all()  # untouched
+    _, want, _ = ref.tree_attention(q, kc, vc, off, kl, bits, 0.125)
+    assert np.abs(gen.bf16_bits_to_f32(got[0]).astype(np.float64) - want[0]).max() <= TOL
+
+
 def test_padding_rows_see_only_themselves_and_cache():
     rng = np.random.default_rng(0)
     m, H, d, L = 16, 2, 64, 40
@@ -112,7 +165,7 @@ def test_full_size_one_layer_sampled(name):
     st = new_status()
     ws = make_ws(e2.workspace_bytes(e2.OP_TREE_ATTENTION, B=cfg.B, m=cfg.m, Hq=cfg.Hq, Hkv=cfg.Hkv,
                                     d=cfg.d, max_kv_len=int(kv_len.max())))
-    e2.tree_attention(tq, tk, tv, dev(kv_off), dev(kv_len), dev(bits), cfg.B, cfg.m, cfg.Hq, cfg.Hkv,
+    e2.tree_attention(tq, tk, tv, rows, dev(kv_off), dev(kv_len), dev(bits), cfg.B, cfg.m, cfg.Hq, cfg.Hkv,
                       cfg.d, int(kv_len.max()), 1.0 / np.sqrt(cfg.d), out, None, ws, st)
     torch.cuda.synchronize()
     assert int(st.item()) == 0
