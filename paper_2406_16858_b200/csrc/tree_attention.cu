@@ -472,6 +472,13 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
         tmem_alloc(smem_u32(&s_tmem_base), kTmemCols);
         tmem_relinquish();
     }
+    if (warp == kTmaWarp && lane == 0) {
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&k_map) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&v_map) : "memory");
+        if (plan.q_tma) asm volatile("prefetch.tensormap [%0];" ::"l"(&q_map) : "memory");
+    }
+    // the merge kernel of this call may be scheduled from here on (it waits for this grid to finish)
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -794,12 +801,16 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
     if (tid == 0 && s_abort) raise_status(d_status, EAGLE2_STATUS_TIMEOUT);
 }
 
-// One warp per output row of a sequence that used several splits: combine their partials.
+// One warp per output row of a sequence that used several splits: combine their partials.  The
+// lanes first fetch the splits' (maximum, sum) pairs side by side, then every lane owns DH/32
+// columns and the partial rows are fetched eight splits at a time before any is used.
 template <int DH>
 __global__ void __launch_bounds__(256)
 tree_attention_merge_kernel(const int64_t* __restrict__ kv_off, const int32_t* __restrict__ kv_len, int B, int m,
                             int Hq, int Hkv, long long cache_rows, int max_kv_len, AttnPlan plan, AttnWs ws, __nv_bfloat16* __restrict__ out,
                             float* __restrict__ lse) {
+    // launched with programmatic stream serialisation: wait for the attention kernel's writes
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int warp_global = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
     const int g = plan.g, S = plan.splits;
     const long long total = (long long)B * Hkv * plan.M;
@@ -817,21 +828,46 @@ tree_attention_merge_kernel(const int64_t* __restrict__ kv_off, const int32_t* _
     const size_t stride = (size_t)plan.n_rb * rows_per_block;  // rows between consecutive splits
     const size_t first = (((size_t)b * Hkv + hk) * S) * stride + rb * rows_per_block + r;
     float mmax = -INFINITY;
-    for (int s = 0; s < S_b; ++s) mmax = fmaxf(mmax, ws.ml[first + s * stride].x);
-    constexpr int PER = DH / 32;
+    for (int s0 = 0; s0 < S_b; s0 += 32)
+        if (s0 + lane < S_b) mmax = fmaxf(mmax, ws.ml[first + (size_t)(s0 + lane) * stride].x);
+    mmax = warp_max_f32(mmax);
+    constexpr int PER = DH / 32;  // 4 or 2 consecutive columns per lane
     float acc[PER];
 #pragma unroll
     for (int e = 0; e < PER; ++e) acc[e] = 0.f;
     float l = 0.f;
-    for (int s = 0; s < S_b; ++s) {
-        const float2 ml = ws.ml[first + s * stride];
-        if (ml.x == -INFINITY) continue;
-        const float w = exp2f(ml.x - mmax);
-        l += ml.y * w;
-        const float* src = ws.o_part + (first + s * stride) * DH + lane * PER;
+    for (int s0 = 0; s0 < S_b; s0 += 32) {
+        float w = 0.f;  // weight of split s0 + lane
+        if (s0 + lane < S_b) {
+            const float2 ml = ws.ml[first + (size_t)(s0 + lane) * stride];
+            if (ml.x != -INFINITY) w = exp2f(ml.x - mmax), l += ml.y * w;
+        }
+        const int n = min(32, S_b - s0);
+        for (int s1 = 0; s1 < n; s1 += 8) {
+            float v[8][PER];
 #pragma unroll
-        for (int e = 0; e < PER; ++e) acc[e] += src[e] * w;
+            for (int u = 0; u < 8; ++u) {
+                const int sl = min(s1 + u, n - 1);  // clamped: a repeated row gets weight 0 below
+                const float* src = ws.o_part + (first + (size_t)(s0 + sl) * stride) * DH + lane * PER;
+                if (PER == 4) {
+                    const float4 t = *reinterpret_cast<const float4*>(src);
+                    v[u][0] = t.x, v[u][1] = t.y, v[u][PER - 2] = t.z, v[u][PER - 1] = t.w;
+                } else {
+                    const float2 t = *reinterpret_cast<const float2*>(src);
+                    v[u][0] = t.x, v[u][1] = t.y;
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                float wu = __shfl_sync(0xffffffffu, w, min(s1 + u, 31));
+                if (s1 + u >= n) wu = 0.f;
+                // a split without visible keys leaves its partial row unwritten: never multiply it
+#pragma unroll
+                for (int e = 0; e < PER; ++e) acc[e] += wu != 0.f ? v[u][e] * wu : 0.f;
+            }
+        }
     }
+    l = warp_sum_f32(l);
     const float inv = l > 0.f ? 1.f / l : 0.f;
     const int tok = pr / g, hq = hk * g + pr % g;
     __nv_bfloat16* dst = out + (((long long)b * m + tok) * Hq + hq) * DH + lane * PER;
@@ -865,10 +901,23 @@ static int launch_attention(const CUtensorMap& k_map, const CUtensorMap& v_map, 
         const long long warps = (long long)B * Hkv * plan.M;
         const long long mblocks = (warps + 7) / 8;
         if (mblocks > 0x7fffffffLL) return EAGLE2_ERR_SHAPE;
-        tree_attention_merge_kernel<DH><<<(unsigned)mblocks, 256, 0, st>>>(
-            kv_off, kv_len, B, m, Hq, Hkv, cache_rows, max_kv_len, plan, ws, static_cast<__nv_bfloat16*>(out),
-            lse);
-        return launch_result();
+        // the merge kernel may be scheduled while the attention kernel still runs; it starts with
+        // griddepcontrol.wait, which holds it until that kernel's writes are complete
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)mblocks, 1, 1);
+        cfg.blockDim = dim3(256, 1, 1);
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        if (cudaLaunchKernelEx(&cfg, tree_attention_merge_kernel<DH>, kv_off, kv_len, B, m, Hq, Hkv, cache_rows,
+                               max_kv_len, plan, ws, static_cast<__nv_bfloat16*>(out), lse) != cudaSuccess) {
+            cudaGetLastError();
+            return EAGLE2_ERR_CUDA;
+        }
+        return EAGLE2_OK;
     }
     return EAGLE2_OK;
 }
