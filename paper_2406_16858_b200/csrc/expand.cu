@@ -16,7 +16,7 @@ struct ExpandPlan {
     int chunks;  // chunks per row
 };
 
-constexpr int kMergeKeysMax = 3200;  // per-row partial keys the merging block can hold per warp
+constexpr int kMergeKeysMax = 1024;  // chunk winners per row that the merging warp holds in registers (32 per lane)
 
 static bool expand_plan(long long rows, int V, int k, ExpandPlan* p) {
     int vpt = scan_pick_vpt(rows, V);
@@ -55,27 +55,35 @@ size_t expand_workspace_bytes(int B, int V, int k) {
     return need;
 }
 
+// Monotone map double -> uint64 (larger value, larger code; -0 folded onto +0; NaN lowest).
+__device__ __forceinline__ unsigned long long order_code_f64(double x) {
+    if (x != x) return 0ull;
+    const unsigned long long u = (unsigned long long)__double_as_longlong(x + 0.0);
+    return (u >> 63) ? ~u : (u | 0x8000000000000000ull);
+}
+
 template <int VPT, bool VEC>
-__global__ void __launch_bounds__(kScanThreads)
+__global__ void __launch_bounds__(kScanThreads, 3)
 expand_kernel(const float* __restrict__ draft_logits, long long batch_stride, int V, int k, int D,
               int s, int n_s, int chunks, int32_t* __restrict__ tree_token,
               int32_t* __restrict__ tree_parent, double* __restrict__ tree_value,
               int32_t* __restrict__ frontier, ExpandWs ws, int32_t* d_status) {
     constexpr int NE = 4 * VPT;
-    __shared__ float s_redf[kScanWarps];
-    __shared__ double s_redd[kScanWarps];
-    __shared__ unsigned long long s_keys[kScanWarps * EAGLE2_MAX_K];
+    __shared__ TopkScratch s_topk;
+    __shared__ float s_wmax[kScanWarps], s_wsum[kScanWarps];
     __shared__ int s_flag;
-    extern __shared__ __align__(16) unsigned char s_dyn[];
+    __shared__ unsigned long long s_rank[EAGLE2_MAX_K * EAGLE2_MAX_K];  // the new candidates' value codes
 
     const int chunk = blockIdx.x % chunks;
     const int row = (blockIdx.x / chunks) % n_s;
     const int b = blockIdx.x / (chunks * n_s);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const float* zrow = draft_logits + (long long)b * batch_stride + (long long)row * V;
 
-    // ---- scan this chunk -------------------------------------------------------------------
+    // ---- scan this chunk: per-warp (max, sum of exponentials), block top-k -----------------------
     float x[NE];
     scan_load<VPT, VEC>(zrow, V, chunk, x);
+    if (threadIdx.x == 0) s_topk.count = 0, s_topk.overflow = 0;
     float tmax = -INFINITY;
     int bad = 0;
 #pragma unroll
@@ -83,46 +91,70 @@ expand_kernel(const float* __restrict__ draft_logits, long long batch_stride, in
         bad |= !(x[j] < INFINITY);  // NaN or +Inf
         tmax = fmaxf(tmax, x[j]);
     }
-    const float cmax = block_max_f32(tmax, s_redf);
+    const float wmax = warp_max_f32(tmax);
     float tsum = 0.f;
-    if (cmax > -INFINITY) {
+    if (wmax > -INFINITY) {
 #pragma unroll
-        for (int j = 0; j < NE; ++j) tsum += expf(x[j] - cmax);
+        for (int j = 0; j < NE; ++j) tsum += expf(x[j] - wmax);
     }
-    const double csum = block_sum_f64((double)tsum, s_redd);
+    tsum = warp_sum_f32(tsum);
+    if (lane == 0) s_wmax[warp] = wmax, s_wsum[warp] = tsum;
     unsigned long long key[NE];
 #pragma unroll
     for (int j = 0; j < NE; ++j) {
         const int e = scan_elem_index<VPT, VEC>(chunk, j);
         key[j] = e < V ? make_key(x[j], (uint32_t)e) : 0ull;
     }
+    __syncthreads();
     const size_t part = ((size_t)b * n_s + row) * chunks + chunk;
-    block_topk<NE>(key, k, s_keys, ws.keys + part * k);
-    if (threadIdx.x == 0) ws.stats[part] = make_double2((double)cmax, csum);
+    block_topk_filtered<NE>(key, k, &s_topk, ws.keys + part * k);
+    if (threadIdx.x == 0) {
+        float cmax = s_wmax[0];
+#pragma unroll
+        for (int w = 1; w < kScanWarps; ++w) cmax = fmaxf(cmax, s_wmax[w]);
+        double csum = 0.0;
+        if (cmax > -INFINITY) {
+#pragma unroll
+            for (int w = 0; w < kScanWarps; ++w)
+                if (s_wmax[w] > -INFINITY) csum += (double)s_wsum[w] * (double)expf(s_wmax[w] - cmax);
+        }
+        ws.stats[part] = make_double2((double)cmax, csum);
+    }
     if (bad) raise_status(d_status, EAGLE2_STATUS_NONFINITE_LOGIT);
 
     // ---- the last block of this sequence merges ---------------------------------------------
     if (!last_block_arrives(ws.counters + b, chunks * n_s, &s_flag)) return;
 
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const long long N = nodes_of(k, D);
     const long long base = s ? (long long)k + (long long)(s - 1) * k * k : 0;
     const long long prev_base = s >= 2 ? (long long)k + (long long)(s - 2) * k * k : 0;
     const long long prev_count = s >= 2 ? (long long)k * k : k;
     const int n_new = n_s * k;
-    const int keys_per_row = chunks * k;
-    // dynamic shared memory: per-warp key staging, then the new candidates' values
-    unsigned long long* s_stage = reinterpret_cast<unsigned long long*>(s_dyn) + (size_t)warp * keys_per_row;
-    double* s_val = reinterpret_cast<double*>(reinterpret_cast<unsigned long long*>(s_dyn) +
-                                              (size_t)kScanWarps * keys_per_row);
+    const int keys_per_row = chunks * k;  // at most kMergeKeysMax = 32 per lane
     int32_t* tok = tree_token + (long long)b * N;
     int32_t* par = tree_parent + (long long)b * N;
     double* val = tree_value + (long long)b * N;
     int32_t* fr = frontier + (long long)b * k;
     int status = 0;
 
+    // a warp per row; everything a row needs is fetched before any of it is used
     for (int r = warp; r < n_s; r += kScanWarps) {
         const size_t p0 = ((size_t)b * n_s + r) * chunks;
+        constexpr int BATCH = 16;  // chunk winners per lane and pass
+        unsigned long long cand[BATCH + 1];
+#pragma unroll
+        for (int t = 0; t < BATCH; ++t)
+            cand[t] = lane + 32 * t < keys_per_row ? ws.keys[p0 * k + lane + 32 * t] : 0ull;
+        int parent = -1;
+        double parent_value = 0.0;
+        if (s) {
+            parent = fr[r];
+            if (parent < prev_base || parent >= prev_base + prev_count) {
+                status |= EAGLE2_STATUS_BAD_TREE;
+                parent = (int)prev_base;
+            }
+            parent_value = val[parent];
+        }
         // log-sum-exp of the row from the chunk partials, in double
         double m = -INFINITY;
         for (int c = lane; c < chunks; c += 32) m = fmax(m, ws.stats[p0 + c].x);
@@ -135,45 +167,46 @@ expand_kernel(const float* __restrict__ draft_logits, long long batch_stride, in
         sum = warp_sum_f64(sum);
         if (!(m > -INFINITY)) status |= EAGLE2_STATUS_NONFINITE_LOGIT;
         const double lse = m + log(sum);
-        // top-k of the chunk winners
-        for (int e = lane; e < keys_per_row; e += 32) s_stage[e] = ws.keys[p0 * k + e];
-        __syncwarp();
-        int parent = -1;
-        double parent_value = 0.0;
-        if (s) {
-            parent = fr[r];
-            if (parent < prev_base || parent >= prev_base + prev_count) {
-                status |= EAGLE2_STATUS_BAD_TREE;
-                parent = (int)prev_base;
+        // top-k of the chunk winners, 32*BATCH at a time together with the best so far: lane c
+        // ends up holding the c-th
+        unsigned long long mine = 0;
+        for (int e0 = 0; e0 < keys_per_row; e0 += 32 * BATCH) {
+            if (e0) {
+#pragma unroll
+                for (int t = 0; t < BATCH; ++t)
+                    cand[t] = e0 + lane + 32 * t < keys_per_row ? ws.keys[p0 * k + e0 + lane + 32 * t] : 0ull;
             }
-            parent_value = val[parent];
+            cand[BATCH] = mine;
+            unsigned long long next = 0;
+            for (int c = 0; c < k; ++c) {
+                unsigned long long best = 0;
+#pragma unroll
+                for (int t = 0; t <= BATCH; ++t) best = cand[t] > best ? cand[t] : best;
+                const unsigned long long top = warp_max_u64(best);
+#pragma unroll
+                for (int t = 0; t <= BATCH; ++t) cand[t] = (cand[t] == top) ? 0ull : cand[t];
+                if (lane == c) next = top;
+            }
+            mine = next;
         }
-        for (int c = 0; c < k; ++c) {
-            unsigned long long best = 0;
-            for (int e = lane; e < keys_per_row; e += 32) best = s_stage[e] > best ? s_stage[e] : best;
-            const unsigned long long top = warp_max_u64(best);
-            for (int e = lane; e < keys_per_row; e += 32)
-                if (s_stage[e] == top) s_stage[e] = 0ull;
-            __syncwarp();
-            if (lane == 0) {
-                const long long node = base + (long long)r * k + c;
-                const double v = parent_value + ((double)key_value(top) - lse);
-                tok[node] = (int32_t)key_index(top);
-                par[node] = parent;
-                val[node] = v;
-                s_val[r * k + c] = (v == v) ? v : -INFINITY;
-            }
+        if (lane < k) {
+            const long long node = base + (long long)r * k + lane;
+            const double v = parent_value + ((double)key_value(mine) - lse);
+            tok[node] = (int32_t)key_index(mine);
+            par[node] = parent;
+            val[node] = v;
+            s_rank[r * k + lane] = order_code_f64(v);
         }
     }
     __syncthreads();  // all rows merged; every read of the old frontier is done
 
     // next frontier: rank the new candidates by (value desc, index asc); ranks < k are kept
     for (int i = threadIdx.x; i < n_new; i += kScanThreads) {
-        const double vi = s_val[i];
+        const unsigned long long ci = s_rank[i];
         int rank = 0;
         for (int j = 0; j < n_new; ++j) {
-            const double vj = s_val[j];
-            rank += (vj > vi) || (vj == vi && j < i);
+            const unsigned long long cj = s_rank[j];
+            rank += (cj > ci) || (cj == ci && j < i);
         }
         if (rank < k) fr[rank] = (int32_t)(base + i);
     }
@@ -185,14 +218,9 @@ static int launch_expand(const float* draft_logits, long long batch_stride, int 
                          int s, int n_s, int chunks, int32_t* tree_token, int32_t* tree_parent,
                          double* tree_value, int32_t* frontier, const ExpandWs& ws, int32_t* d_status,
                          cudaStream_t stream) {
-    const size_t dyn = sizeof(unsigned long long) * (size_t)kScanWarps * chunks * k +
-                       sizeof(double) * (size_t)n_s * k;
     auto kern = expand_kernel<VPT, VEC>;
-    if (dyn > 40 * 1024 &&
-        cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) != cudaSuccess)
-        return EAGLE2_ERR_CUDA;
     const long long blocks = (long long)B * n_s * chunks;
-    kern<<<(unsigned)blocks, kScanThreads, dyn, stream>>>(draft_logits, batch_stride, V, k, D, s, n_s,
+    kern<<<(unsigned)blocks, kScanThreads, 0, stream>>>(draft_logits, batch_stride, V, k, D, s, n_s,
                                                           chunks, tree_token, tree_parent, tree_value,
                                                           frontier, ws, d_status);
     return launch_result();

@@ -9,17 +9,28 @@ namespace eagle2 {
 
 constexpr int kRerankThreads = 512;
 
+// Monotone map double -> uint64 (larger value, larger code; -0 folded onto +0).  The caller has
+// already replaced NaN.
+__device__ __forceinline__ unsigned long long value_code(double x) {
+    const unsigned long long u = (unsigned long long)__double_as_longlong(x + 0.0);
+    return (u >> 63) ? ~u : (u | 0x8000000000000000ull);
+}
+
+// Values are compared as integer codes throughout (fp64 compares are slow on this part).  The
+// ranking is a bitonic sort of (code, index) pairs, padded to a power of two with code 0, which
+// sorts behind every real value.
 __global__ void __launch_bounds__(kRerankThreads)
 rerank_kernel(const int32_t* __restrict__ tree_token, const int32_t* __restrict__ tree_parent,
-              const double* __restrict__ tree_value, int k, int N, int m, int keep,
+              const double* __restrict__ tree_value, int k, int N, int P, int m, int keep,
               int32_t* __restrict__ sel_index, int32_t* __restrict__ sel_parent,
               int32_t* __restrict__ sel_token, int32_t* __restrict__ sel_depth,
               int32_t* __restrict__ n_sel, int32_t* d_status) {
     extern __shared__ __align__(16) unsigned char s_dyn[];
-    double* s_val = reinterpret_cast<double*>(s_dyn);            // [N] value, then effective value
-    double* s_eff = s_val + N;                                   // [N]
-    int32_t* s_par = reinterpret_cast<int32_t*>(s_eff + N);      // [N]
-    int32_t* s_flat = s_par + N;                                 // [N] flat position or -1
+    unsigned long long* s_code = reinterpret_cast<unsigned long long*>(s_dyn);  // [N] value codes
+    unsigned long long* s_key = s_code + N;                                     // [P] sort keys
+    int32_t* s_idx = reinterpret_cast<int32_t*>(s_key + P);                     // [P] sort payload
+    int32_t* s_par = s_idx + P;                                                 // [N]
+    int32_t* s_flat = s_par + N;                                                // [N] flat position or -1
     __shared__ int s_scan[kRerankThreads];
 
     const int b = blockIdx.x, tid = threadIdx.x;
@@ -40,42 +51,68 @@ rerank_kernel(const int32_t* __restrict__ tree_token, const int32_t* __restrict_
             v = -INFINITY;
         }
         s_par[i] = p;
-        s_val[i] = v;
+        s_code[i] = value_code(v);
+        s_flat[i] = -1;
     }
     __syncthreads();
     // effective value = minimum of the values on the path from the root (parents have lower
     // indices, so the walk ends)
-    for (int i = tid; i < N; i += kRerankThreads) {
-        double v = s_val[i];
-        for (int a = s_par[i]; a >= 0; a = s_par[a]) v = fmin(v, s_val[a]);
-        s_eff[i] = v;
-    }
-    __syncthreads();
-    // rank by (effective value desc, index asc); the first `keep` are selected
-    const int per = (N + kRerankThreads - 1) / kRerankThreads;
-    const int lo = tid * per, hi = min(N, lo + per);
-    int mine = 0;
-    for (int i = lo; i < hi; ++i) {
-        const double vi = s_eff[i];
-        int rank = 0;
-        for (int j = 0; j < N; ++j) {
-            const double vj = s_eff[j];
-            rank += (vj > vi) || (vj == vi && j < i);
+    for (int i = tid; i < P; i += kRerankThreads) {
+        unsigned long long c = 0;
+        if (i < N) {
+            c = s_code[i];
+            for (int a = s_par[i]; a >= 0; a = s_par[a]) c = s_code[a] < c ? s_code[a] : c;
         }
-        const int chosen = rank < keep;
-        s_flat[i] = chosen ? 0 : -1;
-        mine += chosen;
+        s_key[i] = c;
+        s_idx[i] = i;
     }
-    // exclusive scan of the per-thread counts -> flat positions in ascending index
-    s_scan[tid] = mine;
     __syncthreads();
-    for (int o = 1; o < kRerankThreads; o <<= 1) {
-        const int add = tid >= o ? s_scan[tid - o] : 0;
-        __syncthreads();
-        s_scan[tid] += add;
-        __syncthreads();
+    // order: effective value descending, index ascending
+    for (int size = 2; size <= P; size <<= 1) {
+        for (int stride = size >> 1; stride > 0; stride >>= 1) {
+            for (int i = tid; i < P; i += kRerankThreads) {
+                const int j = i ^ stride;
+                if (j > i) {
+                    const unsigned long long ki = s_key[i], kj = s_key[j];
+                    const int ii = s_idx[i], ij = s_idx[j];
+                    const bool i_first = ki > kj || (ki == kj && ii < ij);  // i belongs before j
+                    const bool forward = (i & size) == 0;
+                    if (i_first != forward) {
+                        s_key[i] = kj, s_key[j] = ki;
+                        s_idx[i] = ij, s_idx[j] = ii;
+                    }
+                }
+            }
+            __syncthreads();
+        }
     }
-    int pos = s_scan[tid] - mine;
+    for (int r = tid; r < keep; r += kRerankThreads) s_flat[s_idx[r]] = 0;
+    __syncthreads();
+    // exclusive scan of the per-thread counts -> flat positions in ascending index
+    const int per = (N + kRerankThreads - 1) / kRerankThreads;
+    const int lo = min(N, tid * per), hi = min(N, lo + per);
+    int mine = 0;
+    for (int i = lo; i < hi; ++i) mine += s_flat[i] == 0;
+    const int lane = tid & 31, warp = tid >> 5;
+    int incl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int up = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += up;
+    }
+    if (lane == 31) s_scan[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+        int w = lane < kRerankThreads / 32 ? s_scan[lane] : 0;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int up = __shfl_up_sync(0xffffffffu, w, o);
+            if (lane >= o) w += up;
+        }
+        if (lane < kRerankThreads / 32) s_scan[lane] = w;  // inclusive totals of the warps
+    }
+    __syncthreads();
+    int pos = incl - mine + (warp ? s_scan[warp - 1] : 0);
     for (int i = lo; i < hi; ++i)
         if (s_flat[i] == 0) s_flat[i] = pos++;
     __syncthreads();
@@ -166,13 +203,16 @@ extern "C" int eagle2_rerank(const int32_t* tree_token, const int32_t* tree_pare
     if (B == 0) return EAGLE2_OK;
     const int N = (int)nodes_of(k, D);
     const int keep = m < N ? m : N;
-    const size_t dyn = (size_t)N * (2 * sizeof(double) + 2 * sizeof(int32_t));
+    int P = 1;
+    while (P < N) P <<= 1;
+    const size_t dyn = (size_t)N * (sizeof(unsigned long long) + 2 * sizeof(int32_t)) +
+                       (size_t)P * (sizeof(unsigned long long) + sizeof(int32_t));
     if (dyn > 40 * 1024 &&
         cudaFuncSetAttribute(rerank_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) !=
             cudaSuccess)
         return EAGLE2_ERR_CUDA;
     rerank_kernel<<<B, kRerankThreads, dyn, reinterpret_cast<cudaStream_t>(stream)>>>(
-        tree_token, tree_parent, tree_value, k, N, m, keep, sel_index, sel_parent, sel_token, sel_depth,
+        tree_token, tree_parent, tree_value, k, N, P, m, keep, sel_index, sel_parent, sel_token, sel_depth,
         n_sel, d_status);
     return launch_result();
 }

@@ -100,6 +100,81 @@ __device__ __forceinline__ void block_topk(unsigned long long (&key)[NKEY], int 
     }
 }
 
+// Sorts one key per lane across the warp, descending (lane 0 ends with the largest).
+__device__ __forceinline__ unsigned long long warp_sort_desc_u64(unsigned long long v) {
+    const int lane = threadIdx.x & 31;
+#pragma unroll
+    for (int size = 2; size <= 32; size <<= 1) {
+#pragma unroll
+        for (int stride = size >> 1; stride > 0; stride >>= 1) {
+            const unsigned long long other = __shfl_xor_sync(0xffffffffu, v, stride);
+            const bool desc = (lane & size) == 0, lower = (lane & stride) == 0;
+            const unsigned long long hi = v > other ? v : other, lo = v > other ? other : v;
+            v = (lower == desc) ? hi : lo;
+        }
+    }
+    return v;
+}
+
+constexpr int kCandCap = 512;  // candidate keys a block can stage for the filtered selection
+
+struct TopkScratch {
+    unsigned long long cand[kCandCap];
+    unsigned long long exact[kScanWarps * EAGLE2_MAX_K];
+    int count;
+    int overflow;
+};
+
+// Block-level top-k (k <= 32) of the keys held in registers, written by warp 0 to out[0..k)
+// (descending; 0 = none).  Each warp takes the k-th largest of its lanes' maxima as a threshold: at
+// least k of its keys reach it, and no key below it can be among the warp's k best, so only the
+// keys at or above it are staged and ranked.  If a block stages more than kCandCap keys (possible
+// for heavily ordered input) it falls back to k rounds of exact warp selection.
+// The caller zeroes scratch->count and scratch->overflow and synchronises before the call.
+template <int NKEY>
+__device__ __forceinline__ void block_topk_filtered(unsigned long long (&key)[NKEY], int k, TopkScratch* scratch,
+                                                    unsigned long long* out) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    unsigned long long lane_max = 0;
+#pragma unroll
+    for (int j = 0; j < NKEY; ++j) lane_max = key[j] > lane_max ? key[j] : lane_max;
+    const unsigned long long sorted = warp_sort_desc_u64(lane_max);
+    const unsigned long long thr = __shfl_sync(0xffffffffu, sorted, k - 1);
+    int cnt = 0;
+#pragma unroll
+    for (int j = 0; j < NKEY; ++j) cnt += (key[j] >= thr && key[j] != 0ull);
+    int incl = cnt;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int up = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += up;
+    }
+    const int total = __shfl_sync(0xffffffffu, incl, 31);
+    int base = 0;
+    if (lane == 0) base = atomicAdd(&scratch->count, total);
+    base = __shfl_sync(0xffffffffu, base, 0);
+    if (base + total <= kCandCap) {
+        int pos = base + incl - cnt;
+#pragma unroll
+        for (int j = 0; j < NKEY; ++j)
+            if (key[j] >= thr && key[j] != 0ull) scratch->cand[pos++] = key[j];
+    } else if (lane == 0) {
+        scratch->overflow = 1;
+    }
+    __syncthreads();
+    if (scratch->overflow) {  // uniform over the block
+        block_topk<NKEY>(key, k, scratch->exact, out);
+        return;
+    }
+    if (warp == 0) {
+        const int n = scratch->count;
+        unsigned long long mine[kCandCap / 32];
+#pragma unroll
+        for (int t = 0; t < kCandCap / 32; ++t) mine[t] = lane + 32 * t < n ? scratch->cand[lane + 32 * t] : 0ull;
+        warp_select<kCandCap / 32>(mine, k, out);
+    }
+}
+
 // Choose elements per chunk (as float4 per thread: 1, 2 or 4) so that a launch fills the GPU when
 // it can and no row is cut into more pieces than the merge step can hold.
 inline int scan_pick_vpt(long long rows, int V) {
