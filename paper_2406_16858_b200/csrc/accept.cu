@@ -248,20 +248,36 @@ accept_chain_kernel(const float* __restrict__ target_logits, long long t_stride,
     __shared__ int s_nchild, s_parent;
 
     // ---- which selected nodes are children produced by draft row r (same in every block) ------
+    // every candidate is looked at by its own thread; ballots keep the ascending order
+    __shared__ unsigned s_ballot[EAGLE2_MAX_M / 32];
     const int ns = min(n_sel[b], m);
-    if (tid == 0) {
-        int c = 0, parent = -1;
-        for (int x = 0; x < ns; ++x) {
+    if (tid < EAGLE2_MAX_M) {
+        const int x = tid;
+        int tokx = 0, parx = -1;
+        bool match = false;
+        if (x < ns) {
             const int idx = sel_index[(long long)b * m + x];
-            if (idx >= 0 && draft_row_of_child(idx, k) == r && c < EAGLE2_MAX_K) {
-                s_child[c] = x;
-                s_ctok[c] = sel_token[(long long)b * m + x];
-                parent = sel_parent[(long long)b * m + x];
-                ++c;
+            match = idx >= 0 && draft_row_of_child(idx, k) == r;
+            if (match) {
+                tokx = sel_token[(long long)b * m + x];
+                parx = sel_parent[(long long)b * m + x];
             }
         }
-        s_nchild = c;
-        s_parent = parent;
+        const unsigned bal = __ballot_sync(0xffffffffu, match);
+        if ((tid & 31) == 0) s_ballot[tid >> 5] = bal;
+        asm volatile("bar.sync 1, %0;" ::"n"(EAGLE2_MAX_M) : "memory");  // the first four warps
+        int before = __popc(bal & ((1u << (tid & 31)) - 1u)), total = 0;
+        for (int w = 0; w < EAGLE2_MAX_M / 32; ++w) {
+            const int c = __popc(s_ballot[w]);
+            if (w < (tid >> 5)) before += c;
+            total += c;
+        }
+        if (match && before < EAGLE2_MAX_K) {
+            s_child[before] = x;
+            s_ctok[before] = tokx;
+            if (before == 0) s_parent = parx;
+        }
+        if (tid == 0) s_nchild = min(total, EAGLE2_MAX_K);
     }
     __syncthreads();
     const int nc = s_nchild;
@@ -333,11 +349,28 @@ accept_chain_kernel(const float* __restrict__ target_logits, long long t_stride,
     double sum_p = chain_block_sum((double)tp, s_redd), sum_q = chain_block_sum((double)tq, s_redd);
     cluster_allreduce2<false>(cluster, sum_p, sum_q, s_xchg, parity);
     const float c_p = (float)(1.0 / sum_p), c_q = full_q ? (float)(1.0 / sum_q) : 0.f;
+    // The first rejection always leads to alpha = 1 (alpha_0 = 0, beta_0 = 1, nothing removed from
+    // q yet), so its residual mass F(1) = sum max(p_0 - q_0, 0) is taken in this same sweep.
+    float part_f1 = 0.f;
     if (RESIDENT) {
         for (int e = tid; e < n_local; e += kChainThreads) {
-            sp[e] = __fmul_rn(sp[e], c_p);
-            if (full_q) sq[e] = __fmul_rn(sq[e], c_q);
+            const float pe = __fmul_rn(sp[e], c_p);
+            sp[e] = pe;
+            if (full_q) {
+                const float qe = __fmul_rn(sq[e], c_q);
+                sq[e] = qe;
+                part_f1 += fmaxf(fmaf(-1.0f, qe, pe), 0.f);
+            }
         }
+    } else if (full_q && nc > 1) {
+        for (int e = tid; e < n_local; e += kChainThreads)
+            part_f1 += fmaxf(fmaf(-1.0f, prob_of(zq[lo + e], inv_t, gmax_q, c_q), prob_of(zp[lo + e], inv_t, gmax_p, c_p)), 0.f);
+    }
+    double f_one = 0.0;
+    if (full_q && nc > 1) {
+        double unused = 0.0;
+        f_one = chain_block_sum((double)part_f1, s_redd);
+        cluster_allreduce2<false>(cluster, f_one, unused, s_xchg, parity);
     }
     // the children's own probabilities, computed exactly like the resident values
     if (tid < nc) {
@@ -394,14 +427,27 @@ accept_chain_kernel(const float* __restrict__ target_logits, long long t_stride,
         // residual after rejecting child j: alpha grows by beta * s for every token still in q
         const double alpha_new = alpha + beta * s;
         const float an = (float)alpha_new;
-        float part = 0.f;
-        for (int e = tid; e < n_local; e += kChainThreads) {
-            const float pe = RESIDENT ? sp[e] : prob_of(zp[lo + e], inv_t, gmax_p, c_p);
-            const float qe = RESIDENT ? sq[e] : prob_of(zq[lo + e], inv_t, gmax_q, c_q);
-            part += fmaxf(fmaf(-an, qe, pe), 0.f);
+        if (j == nc - 1) {
+            // nothing is tested after the last child: only alpha is needed (by the extra token's
+            // law).  A rejection implies p < q at the rejected token, hence mass left elsewhere.
+            alpha = alpha_new;
+            if (tid == 0) s_frozen[j] = alpha;
+            break;
         }
-        double f_new = chain_block_sum((double)part, s_redd), unused = 0.0;
-        cluster_allreduce2<false>(cluster, f_new, unused, s_xchg, parity);
+        double f_new;
+        if (j == 0) {
+            f_new = f_one;  // alpha_new == 1
+        } else {
+            float part = 0.f;
+            for (int e = tid; e < n_local; e += kChainThreads) {
+                const float pe = RESIDENT ? sp[e] : prob_of(zp[lo + e], inv_t, gmax_p, c_p);
+                const float qe = RESIDENT ? sq[e] : prob_of(zq[lo + e], inv_t, gmax_q, c_q);
+                part += fmaxf(fmaf(-an, qe, pe), 0.f);
+            }
+            double unused = 0.0;
+            f_new = chain_block_sum((double)part, s_redd);
+            cluster_allreduce2<false>(cluster, f_new, unused, s_xchg, parity);
+        }
         // tokens removed in earlier rounds keep the alpha in force when they were removed
         for (int i = 0; i < j; ++i) {
             const float pi = s_pf[i], qi = s_qf[i];

@@ -99,15 +99,9 @@ expand_kernel(const float* __restrict__ draft_logits, long long batch_stride, in
     }
     tsum = warp_sum_f32(tsum);
     if (lane == 0) s_wmax[warp] = wmax, s_wsum[warp] = tsum;
-    unsigned long long key[NE];
-#pragma unroll
-    for (int j = 0; j < NE; ++j) {
-        const int e = scan_elem_index<VPT, VEC>(chunk, j);
-        key[j] = e < V ? make_key(x[j], (uint32_t)e) : 0ull;
-    }
     __syncthreads();
     const size_t part = ((size_t)b * n_s + row) * chunks + chunk;
-    block_topk_filtered<NE>(key, k, &s_topk, ws.keys + part * k);
+    block_topk_filtered<VPT, VEC>(x, chunk, V, k, &s_topk, ws.keys + part * k);
     if (threadIdx.x == 0) {
         float cmax = s_wmax[0];
 #pragma unroll

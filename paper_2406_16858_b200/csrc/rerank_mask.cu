@@ -68,25 +68,58 @@ rerank_kernel(const int32_t* __restrict__ tree_token, const int32_t* __restrict_
     }
     __syncthreads();
     // order: effective value descending, index ascending
-    for (int size = 2; size <= P; size <<= 1) {
-        for (int stride = size >> 1; stride > 0; stride >>= 1) {
-            for (int i = tid; i < P; i += kRerankThreads) {
-                const int j = i ^ stride;
-                if (j > i) {
-                    const unsigned long long ki = s_key[i], kj = s_key[j];
-                    const int ii = s_idx[i], ij = s_idx[j];
-                    const bool i_first = ki > kj || (ki == kj && ii < ij);  // i belongs before j
-                    const bool forward = (i & size) == 0;
-                    if (i_first != forward) {
-                        s_key[i] = kj, s_key[j] = ki;
-                        s_idx[i] = ij, s_idx[j] = ii;
+    if (P <= kRerankThreads) {
+        // one element per thread (threads past P hold padding): exchanges closer than a warp go
+        // through shuffles, the others through a double-buffered shared-memory copy
+        __shared__ unsigned long long s_xk[2][kRerankThreads];
+        __shared__ int32_t s_xi[2][kRerankThreads];
+        unsigned long long key = tid < P ? s_key[tid] : 0ull;
+        int idx = tid;
+        int flip = 0;
+#pragma unroll 1
+        for (int size = 2; size <= kRerankThreads; size <<= 1) {
+#pragma unroll 1
+            for (int stride = size >> 1; stride > 0; stride >>= 1) {
+                unsigned long long ok;
+                int oi;
+                if (stride < 32) {
+                    ok = __shfl_xor_sync(0xffffffffu, key, stride);
+                    oi = __shfl_xor_sync(0xffffffffu, idx, stride);
+                } else {
+                    s_xk[flip][tid] = key;
+                    s_xi[flip][tid] = idx;
+                    __syncthreads();
+                    ok = s_xk[flip][tid ^ stride];
+                    oi = s_xi[flip][tid ^ stride];
+                    flip ^= 1;
+                }
+                const bool mine_first = key > ok || (key == ok && idx < oi);
+                const bool keep_first = ((tid & stride) == 0) == ((tid & size) == 0);
+                if (mine_first != keep_first) key = ok, idx = oi;
+            }
+        }
+        if (tid < keep) s_flat[idx] = 0;
+    } else {
+        for (int size = 2; size <= P; size <<= 1) {
+            for (int stride = size >> 1; stride > 0; stride >>= 1) {
+                for (int i = tid; i < P; i += kRerankThreads) {
+                    const int j = i ^ stride;
+                    if (j > i) {
+                        const unsigned long long ki = s_key[i], kj = s_key[j];
+                        const int ii = s_idx[i], ij = s_idx[j];
+                        const bool i_first = ki > kj || (ki == kj && ii < ij);  // i belongs before j
+                        const bool forward = (i & size) == 0;
+                        if (i_first != forward) {
+                            s_key[i] = kj, s_key[j] = ki;
+                            s_idx[i] = ij, s_idx[j] = ii;
+                        }
                     }
                 }
+                __syncthreads();
             }
-            __syncthreads();
         }
+        for (int r = tid; r < keep; r += kRerankThreads) s_flat[s_idx[r]] = 0;
     }
-    for (int r = tid; r < keep; r += kRerankThreads) s_flat[s_idx[r]] = 0;
     __syncthreads();
     // exclusive scan of the per-thread counts -> flat positions in ascending index
     const int per = (N + kRerankThreads - 1) / kRerankThreads;

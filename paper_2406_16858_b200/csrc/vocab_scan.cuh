@@ -100,17 +100,17 @@ __device__ __forceinline__ void block_topk(unsigned long long (&key)[NKEY], int 
     }
 }
 
-// Sorts one key per lane across the warp, descending (lane 0 ends with the largest).
-__device__ __forceinline__ unsigned long long warp_sort_desc_u64(unsigned long long v) {
+// Sorts one value per lane across the warp, descending (lane 0 ends with the largest); NaN never
+// wins a comparison and so sinks.
+__device__ __forceinline__ float warp_sort_desc_f32(float v) {
     const int lane = threadIdx.x & 31;
 #pragma unroll
     for (int size = 2; size <= 32; size <<= 1) {
 #pragma unroll
         for (int stride = size >> 1; stride > 0; stride >>= 1) {
-            const unsigned long long other = __shfl_xor_sync(0xffffffffu, v, stride);
+            const float other = __shfl_xor_sync(0xffffffffu, v, stride);
             const bool desc = (lane & size) == 0, lower = (lane & stride) == 0;
-            const unsigned long long hi = v > other ? v : other, lo = v > other ? other : v;
-            v = (lower == desc) ? hi : lo;
+            v = (lower == desc) ? fmaxf(v, other) : fminf(v, other);
         }
     }
     return v;
@@ -125,24 +125,26 @@ struct TopkScratch {
     int overflow;
 };
 
-// Block-level top-k (k <= 32) of the keys held in registers, written by warp 0 to out[0..k)
-// (descending; 0 = none).  Each warp takes the k-th largest of its lanes' maxima as a threshold: at
-// least k of its keys reach it, and no key below it can be among the warp's k best, so only the
-// keys at or above it are staged and ranked.  If a block stages more than kCandCap keys (possible
-// for heavily ordered input) it falls back to k rounds of exact warp selection.
+// Block-level top-k (k <= 32) of the chunk elements x[] held in registers, written by warp 0 to
+// out[0..k) as selection keys (descending; 0 = none).  Each warp takes the k-th largest of its lanes'
+// maxima as a threshold: at least k of its elements reach it and none below it can be among the
+// warp's k best, so only elements at or above it get a key and are staged and ranked.  If a block
+// stages more than kCandCap keys (possible for heavily ordered input) it falls back to k rounds of
+// exact warp selection over all keys.
 // The caller zeroes scratch->count and scratch->overflow and synchronises before the call.
-template <int NKEY>
-__device__ __forceinline__ void block_topk_filtered(unsigned long long (&key)[NKEY], int k, TopkScratch* scratch,
-                                                    unsigned long long* out) {
+template <int VPT, bool VEC>
+__device__ __forceinline__ void block_topk_filtered(const float (&x)[4 * VPT], int chunk, int V, int k,
+                                                    TopkScratch* scratch, unsigned long long* out) {
+    constexpr int NE = 4 * VPT;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    unsigned long long lane_max = 0;
+    float lane_max = -INFINITY;  // positions beyond V were loaded as -inf
 #pragma unroll
-    for (int j = 0; j < NKEY; ++j) lane_max = key[j] > lane_max ? key[j] : lane_max;
-    const unsigned long long sorted = warp_sort_desc_u64(lane_max);
-    const unsigned long long thr = __shfl_sync(0xffffffffu, sorted, k - 1);
+    for (int j = 0; j < NE; ++j) lane_max = fmaxf(lane_max, x[j]);
+    const float sorted = warp_sort_desc_f32(lane_max);
+    const float thr = __shfl_sync(0xffffffffu, sorted, k - 1);
     int cnt = 0;
 #pragma unroll
-    for (int j = 0; j < NKEY; ++j) cnt += (key[j] >= thr && key[j] != 0ull);
+    for (int j = 0; j < NE; ++j) cnt += (x[j] >= thr) && (scan_elem_index<VPT, VEC>(chunk, j) < V);
     int incl = cnt;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
@@ -156,14 +158,22 @@ __device__ __forceinline__ void block_topk_filtered(unsigned long long (&key)[NK
     if (base + total <= kCandCap) {
         int pos = base + incl - cnt;
 #pragma unroll
-        for (int j = 0; j < NKEY; ++j)
-            if (key[j] >= thr && key[j] != 0ull) scratch->cand[pos++] = key[j];
+        for (int j = 0; j < NE; ++j) {
+            const int e = scan_elem_index<VPT, VEC>(chunk, j);
+            if (x[j] >= thr && e < V) scratch->cand[pos++] = make_key(x[j], (uint32_t)e);
+        }
     } else if (lane == 0) {
         scratch->overflow = 1;
     }
     __syncthreads();
     if (scratch->overflow) {  // uniform over the block
-        block_topk<NKEY>(key, k, scratch->exact, out);
+        unsigned long long key[NE];
+#pragma unroll
+        for (int j = 0; j < NE; ++j) {
+            const int e = scan_elem_index<VPT, VEC>(chunk, j);
+            key[j] = e < V ? make_key(x[j], (uint32_t)e) : 0ull;
+        }
+        block_topk<NE>(key, k, scratch->exact, out);
         return;
     }
     if (warp == 0) {
