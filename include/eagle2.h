@@ -44,6 +44,7 @@ typedef struct CUstream_st* eagle2_stream_t; /* a cudaStream_t */
 #define EAGLE2_ERR_ALIGN (-3)       /* a base pointer or stride breaks the stated alignment */
 #define EAGLE2_ERR_WORKSPACE (-4)   /* workspace missing, misaligned or too small */
 #define EAGLE2_ERR_CUDA (-5)        /* the CUDA runtime refused the launch */
+#define EAGLE2_ERR_STATIC_LIMIT (-6) /* sizes need more scratch than the library's built-in buffer holds */
 
 /* device-side conditions (bits of *d_status) */
 #define EAGLE2_STATUS_NONFINITE_LOGIT 1 /* NaN or +Inf logit, or a row of only -Inf */
@@ -96,6 +97,29 @@ int eagle2_workspace_init(void* ws, size_t ws_bytes, eagle2_stream_t stream);
 int eagle2_expand(const float* draft_logits, long long batch_stride, int B, int V, int k, int D, int s,
                   int32_t* tree_token, int32_t* tree_parent, double* tree_value, int32_t* frontier,
                   void* ws, size_t ws_bytes, int32_t* d_status, eagle2_stream_t stream);
+
+/*
+ * Expansion without a caller workspace (the paper has no counterpart; this is a packaging variant of
+ * eagle2_expand, same arguments minus ws/ws_bytes, same kernels, same results).  It is meant for
+ * callers that cannot obtain device memory at the moment they need this step: a serving process
+ * that handed all of HBM to its KV-cache pool at start-up and has no allocator left to ask, or a
+ * host loop in which a cudaMalloc is unacceptable because it synchronises the whole device.  The
+ * scratch memory is a fixed array of EAGLE2_EXPAND_STATIC_BYTES that is part of the library image:
+ * every GPU context that loads the library holds it until the process exits.
+ *   - Sizes whose scratch need (what eagle2_workspace_bytes(EAGLE2_OP_EXPAND, ...) reports for the
+ *     step) exceeds EAGLE2_EXPAND_STATIC_BYTES are refused with EAGLE2_ERR_STATIC_LIMIT; nothing is
+ *     launched.  The call itself never allocates or frees device memory.
+ *   - The first call on a device looks up the array's device address (one runtime query, made with
+ *     that device current); make that first call outside any stream capture.
+ *   - All calls on a device share the one array.  Each call clears the few counters that must
+ *     start at zero, on `stream`, before its kernel.  Two calls that can run on the GPU at the same
+ *     time (different streams, no dependency) would overwrite each other's partial results: order
+ *     them, or give one of them eagle2_expand with its own workspace.
+ */
+#define EAGLE2_EXPAND_STATIC_BYTES (1 << 20)
+int eagle2_expand_static(const float* draft_logits, long long batch_stride, int B, int V, int k, int D,
+                         int s, int32_t* tree_token, int32_t* tree_parent, double* tree_value,
+                         int32_t* frontier, int32_t* d_status, eagle2_stream_t stream);
 
 /*
  * Step 2a -- reranking (paper Section 4.2): the n_sel = min(m, N) nodes with the highest value among

@@ -21,7 +21,7 @@ STATUS_TIMEOUT, STATUS_BOUNDS, STATUS_BAD_TREE = 8, 16, 32
 
 EXPORTS = ("eagle2_version", "eagle2_strerror", "eagle2_workspace_bytes", "eagle2_workspace_init",
            "eagle2_expand", "eagle2_rerank", "eagle2_tree_mask", "eagle2_tree_attention",
-           "eagle2_accept", "eagle2_kv_compact")
+           "eagle2_accept", "eagle2_kv_compact", "eagle2_expand_static")
 
 
 class Eagle2Error(RuntimeError):
@@ -53,6 +53,8 @@ def lib() -> C.CDLL:
         h.eagle2_workspace_bytes.argtypes = [i32] * 10
         h.eagle2_workspace_init.argtypes = [vp, sz, vp]
         h.eagle2_expand.argtypes = [vp, i64, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, sz, vp, vp]
+        h.eagle2_expand_static.argtypes = [vp, i64, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp]
+        h.eagle2_expand_static.restype = i32
         h.eagle2_rerank.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp]
         h.eagle2_tree_mask.argtypes = [vp, vp, vp, vp, i32, i32, vp, vp, vp, vp, vp]
         h.eagle2_tree_attention.argtypes = [vp, vp, vp, i64, vp, vp, vp, i32, i32, i32, i32, i32, i32,
@@ -117,6 +119,15 @@ def expand(draft_logits, batch_stride: int, B: int, V: int, k: int, D: int, s: i
     _check("eagle2_expand", lib().eagle2_expand(
         _ptr(draft_logits), batch_stride, B, V, k, D, s, _ptr(tree_token), _ptr(tree_parent),
         _ptr(tree_value), _ptr(frontier), p, n, _ptr(d_status), _stream(stream)))
+
+
+def expand_static(draft_logits, batch_stride: int, B: int, V: int, k: int, D: int, s: int, tree_token,
+                  tree_parent, tree_value, frontier, d_status, stream=None) -> None:
+    """``expand`` for callers that cannot allocate a workspace: the scratch is a fixed buffer inside
+    the library (see the header for its size limit and the rule against overlapping calls)."""
+    _check("eagle2_expand_static", lib().eagle2_expand_static(
+        _ptr(draft_logits), batch_stride, B, V, k, D, s, _ptr(tree_token), _ptr(tree_parent),
+        _ptr(tree_value), _ptr(frontier), _ptr(d_status), _stream(stream)))
 
 
 def rerank(tree_token, tree_parent, tree_value, B: int, k: int, D: int, m: int, sel_index, sel_parent,

@@ -17,6 +17,7 @@ extern "C" const char* eagle2_strerror(int code) {
         case EAGLE2_ERR_ALIGN: return "a pointer or stride is not aligned as required";
         case EAGLE2_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
         case EAGLE2_ERR_CUDA: return "the CUDA runtime refused the launch";
+        case EAGLE2_ERR_STATIC_LIMIT: return "sizes need more scratch than the library's built-in buffer holds";
         default: return "unknown error code";
     }
 }

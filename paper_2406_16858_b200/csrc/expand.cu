@@ -7,6 +7,8 @@
 // and ranks the new candidates by value to produce the next frontier.
 #include <math.h>
 
+#include <mutex>
+
 #include "vocab_scan.cuh"
 
 namespace eagle2 {
@@ -220,6 +222,33 @@ static int launch_expand(const float* draft_logits, long long batch_stride, int 
     return launch_result();
 }
 
+// Scratch of eagle2_expand_static: lives in every context that loads the library, until exit.
+static __device__ __align__(256) unsigned char g_expand_scratch[EAGLE2_EXPAND_STATIC_BYTES];
+
+// Device address of g_expand_scratch on the current device (looked up once per device; in host
+// code the array's name is only a handle for this query, never an address a kernel can use).
+static int expand_scratch_address(void** out) {
+    constexpr int kMaxDevices = 64;
+    static void* addr[kMaxDevices] = {nullptr};
+    static std::mutex mu;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+        cudaGetLastError();
+        return EAGLE2_ERR_CUDA;
+    }
+    std::lock_guard<std::mutex> lock(mu);
+    if (!addr[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_expand_scratch) != cudaSuccess || !p) {
+            cudaGetLastError();
+            return EAGLE2_ERR_CUDA;
+        }
+        addr[dev] = p;
+    }
+    *out = addr[dev];
+    return EAGLE2_OK;
+}
+
 }  // namespace eagle2
 
 using namespace eagle2;
@@ -244,6 +273,52 @@ extern "C" int eagle2_expand(const float* draft_logits, long long batch_stride, 
     if (expand_ws_layout(B, n_s, plan.chunks, k, ws, &w) > ws_bytes) return EAGLE2_ERR_WORKSPACE;
     const bool vec = aligned(draft_logits, 16) && V % 4 == 0 && batch_stride % 4 == 0;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+#define EAGLE2_EXPAND_CASE(VPT_)                                                                      \
+    case VPT_:                                                                                        \
+        return vec ? launch_expand<VPT_, true>(draft_logits, batch_stride, B, V, k, D, s, n_s,        \
+                                               plan.chunks, tree_token, tree_parent, tree_value,      \
+                                               frontier, w, d_status, st)                             \
+                   : launch_expand<VPT_, false>(draft_logits, batch_stride, B, V, k, D, s, n_s,       \
+                                                plan.chunks, tree_token, tree_parent, tree_value,     \
+                                                frontier, w, d_status, st);
+    switch (plan.vpt) {
+        EAGLE2_EXPAND_CASE(1)
+        EAGLE2_EXPAND_CASE(2)
+        EAGLE2_EXPAND_CASE(4)
+    }
+#undef EAGLE2_EXPAND_CASE
+    return EAGLE2_ERR_SHAPE;
+}
+
+extern "C" int eagle2_expand_static(const float* draft_logits, long long batch_stride, int B, int V, int k,
+                                    int D, int s, int32_t* tree_token, int32_t* tree_parent,
+                                    double* tree_value, int32_t* frontier, int32_t* d_status,
+                                    eagle2_stream_t stream) {
+    if (!draft_logits || !tree_token || !tree_parent || !tree_value || !frontier || !d_status)
+        return EAGLE2_ERR_NULL;
+    if (B < 0 || V < 1 || k < 1 || k > V || k > EAGLE2_MAX_K || D < 1 || D > EAGLE2_MAX_DEPTH || s < 0 ||
+        s >= D || nodes_of(k, D) > EAGLE2_MAX_NODES || batch_stride < 0)
+        return EAGLE2_ERR_SHAPE;
+    if (!aligned(draft_logits, 4) || !aligned(tree_value, 8)) return EAGLE2_ERR_ALIGN;
+    if (B == 0) return EAGLE2_OK;
+    const int n_s = s ? k : 1;
+    ExpandPlan plan;
+    if (!expand_plan((long long)B * n_s, V, k, &plan)) return EAGLE2_ERR_SHAPE;
+    if ((long long)B * n_s * plan.chunks > 0x7fffffffLL) return EAGLE2_ERR_SHAPE;
+    if (expand_ws_layout(B, n_s, plan.chunks, k, nullptr, nullptr) > (size_t)EAGLE2_EXPAND_STATIC_BYTES)
+        return EAGLE2_ERR_STATIC_LIMIT;
+    void* scratch = nullptr;
+    const int rc = expand_scratch_address(&scratch);
+    if (rc != EAGLE2_OK) return rc;
+    ExpandWs w;
+    expand_ws_layout(B, n_s, plan.chunks, k, scratch, &w);
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    // the array keeps whatever the last call left: the arrival counters must start at zero
+    if (cudaMemsetAsync(w.counters, 0, round_up(sizeof(int) * (size_t)B, kWsAlign), st) != cudaSuccess) {
+        cudaGetLastError();
+        return EAGLE2_ERR_CUDA;
+    }
+    const bool vec = aligned(draft_logits, 16) && V % 4 == 0 && batch_stride % 4 == 0;
 #define EAGLE2_EXPAND_CASE(VPT_)                                                                      \
     case VPT_:                                                                                        \
         return vec ? launch_expand<VPT_, true>(draft_logits, batch_stride, B, V, k, D, s, n_s,        \
