@@ -169,6 +169,69 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def max_over_ranks(value: float, world: int, device=None) -> float:
+    """The slowest rank's time: a single-element all-reduce (MAX) over the default process group."""
+    if world <= 1:
+        return float(value)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def replica_seed(rank: int) -> int:
+    """Every replica draws its own inputs."""
+    return 1000 * rank
+
+
+def batched_attention_extra(e2, dev, stream, hbm_peak, B=32, n_layers=3, reps=10):
+    """Tree attention alone at the batched, ragged LLaMA3-8B-shaped workload: the regime in which a
+    launch moves enough bytes (about 0.6 GB per layer) for the HBM fraction to be about the kernel
+    rather than about launch latency.  Attention-only, a few distinct layers larger than L2."""
+    import torch
+    cfg = get_config("llama3_8b_batched").with_(B=B)
+    kv_len_h = gen.kv_lengths(cfg, 0)
+    kv_off_h = gen.kv_offsets(kv_len_h, cfg.m)
+    rows = int(kv_off_h[-1] + kv_len_h[-1] + cfg.m)
+    max_len = int(kv_len_h.max())
+    g = torch.Generator(device=dev).manual_seed(99)
+    ks = [torch.randn((rows, cfg.Hkv, cfg.d), generator=g, device=dev).to(torch.bfloat16) for _ in range(n_layers)]
+    vs = [torch.randn((rows, cfg.Hkv, cfg.d), generator=g, device=dev).to(torch.bfloat16) for _ in range(n_layers)]
+    q = torch.randn((B, cfg.m, cfg.Hq, cfg.d), generator=g, device=dev).to(torch.bfloat16)
+    out = torch.zeros_like(q)
+    W = (cfg.m + 63) // 64
+    mask = torch.zeros((B, cfg.m, W), dtype=torch.int64, device=dev)
+    for i in range(cfg.m):  # a chain: token i sees tokens 0..i
+        mask[:, i, 0] = (1 << (i + 1)) - 1
+    kv_off, kv_len = torch.from_numpy(kv_off_h).to(dev), torch.from_numpy(kv_len_h).to(dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    ws = torch.empty(max(e2.workspace_bytes(e2.OP_TREE_ATTENTION, B=B, m=cfg.m, Hq=cfg.Hq, Hkv=cfg.Hkv, d=cfg.d,
+                                            max_kv_len=max_len), 256), dtype=torch.uint8, device=dev)
+    e2.workspace_init(ws)
+
+    def layers():
+        for kc, vc in zip(ks, vs):
+            e2.tree_attention(q, kc, vc, rows, kv_off, kv_len, mask, B, cfg.m, cfg.Hq, cfg.Hkv, cfg.d, max_len,
+                              1.0 / math.sqrt(cfg.d), out, None, ws, status)
+
+    with torch.cuda.stream(stream):
+        for _ in range(3):
+            layers()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev0.record(stream)
+        for _ in range(reps):
+            layers()
+        ev1.record(stream)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    us = ev0.elapsed_time(ev1) * 1e3 / (reps * n_layers)
+    nbytes = float(sum(2 * (int(L) + cfg.m) * cfg.Hkv * cfg.d * 2 for L in kv_len_h)) + 2.0 * B * cfg.m * cfg.Hq * cfg.d * 2
+    gbs = nbytes / (us * 1e-6) / 1e9
+    return {"workload": f"llama3_8b_batched B={B}, ragged kv_len {int(kv_len_h.min())}..{max_len}",
+            "us_per_layer": us, "algorithmic_bytes_per_layer": nbytes, "achieved_gbs": gbs, "frac_of_measured_hbm": gbs / hbm_peak}
+
+
 # ------------------------------------------------------------------------------------------------
 # the CUDA path
 
@@ -192,7 +255,7 @@ def run_ours(args):
     cfg = get_config(args.workload)
     if args.batch:
         cfg = cfg.with_(B=args.batch)
-    seed = 1000 * rank
+    seed = replica_seed(rank)
     kv_len_h = gen.kv_lengths(cfg, seed)
     kv_off_h = gen.kv_offsets(kv_len_h, cfg.m)
     rows = int(kv_off_h[-1] + kv_len_h[-1] + cfg.m)
@@ -259,6 +322,15 @@ def run_ours(args):
         with torch.cuda.graph(attn_graph, stream=stream):
             for qq, kc, vc, oo in zip(q_layers, k_layers, v_layers, out_layers):
                 buf.attention(qq, kc, vc, kv_off, kv_len0, oo, scale)
+        # the other steps on their own, for the per-step breakdown
+        step_graphs = {}
+        for name, fn in (("expand_x%d" % cfg.D, lambda: buf.expand_all(sets[0]["draft"])),
+                         ("rerank_mask", lambda: buf.rerank_and_mask(kv_len0)),
+                         ("accept", lambda: buf.accept(sets[0]["target"], sets[0]["draft"], sets[0]["ua"], sets[0]["ub"]))):
+            gr = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(gr, stream=stream):
+                fn()
+            step_graphs[name] = gr
     torch.cuda.synchronize()
 
     def barrier():
@@ -275,12 +347,7 @@ def run_ours(args):
                 fn(i)
             ev1.record(stream)
         barrier()
-        ms = ev0.elapsed_time(ev1)
-        if world > 1:
-            t = torch.tensor([ms], device=dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms
+        return max_over_ranks(ev0.elapsed_time(ev1), world, dev)
 
     K, W = args.steps, max(args.warmup, 3)
     with ClockSampler(local) as clocks:
@@ -289,6 +356,10 @@ def run_ours(args):
         attn_reps = max(20, min(K, 400))
         timed(lambda i: attn_graph.replay(), 3)
         ms_attn = timed(lambda i: attn_graph.replay(), attn_reps)
+        breakdown = {"tree_attention_x%d" % cfg.n_layers: ms_attn * 1e3 / attn_reps}
+        for name, gr in step_graphs.items():
+            timed(lambda i: gr.replay(), 3)
+            breakdown[name] = timed(lambda i: gr.replay(), 50) * 1e3 / 50
 
         # ---- end to end: inputs start in pinned host memory, results end in host memory -------------
         host_in = {
@@ -380,6 +451,9 @@ def run_ours(args):
         line["cpu_baseline"] = {"value": total * 1e6, "unit": "us", "cores": cores, "kind": "oracle",
                                 "sample": sample, "parts_us": {k: v * 1e6 for k, v in parts.items()}}
     line["roofline"]["traffic"] = NCU_DRAM_BYTES_PER_LAUNCH.get(cfg.name)
+    line["breakdown_us"] = breakdown  # each step replayed alone (warm logits for the small steps)
+    if world == 1 and not args.no_extras:
+        line["attention_batched"] = batched_attention_extra(e2, dev, stream, hbm_peak)
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
@@ -394,6 +468,7 @@ def main():
     ap.add_argument("--workload", default="llama3_8b")
     ap.add_argument("--batch", type=int, default=0, help="override the number of sequences")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extras", action="store_true", help="skip the batched attention side measurement")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -70,7 +70,8 @@ static size_t accept_ws_layout(int B, int m, int R, int gchunks, int bchunks, vo
 #define EAGLE2_WS_FIELD(field, type, count)                          \
     if (w) w->field = reinterpret_cast<type*>(p + off);              \
     off += round_up(sizeof(type) * (size_t)(count), kWsAlign);
-    EAGLE2_WS_FIELD(counters, int, B)
+    if (w) w->counters = reinterpret_cast<int*>(p);
+    off += counters_bytes(B);
     EAGLE2_WS_FIELD(keys, unsigned long long, (size_t)B * (m + 1) * gchunks)
     EAGLE2_WS_FIELD(thr, double, (size_t)B * m)
     EAGLE2_WS_FIELD(slots, ChainSlot, (size_t)B * R)

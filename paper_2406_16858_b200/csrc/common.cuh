@@ -16,6 +16,10 @@ __host__ __device__ inline long long nodes_of(int k, int D) {
     return (long long)k + (long long)(D - 1) * k * k;
 }
 
+// Every operation's workspace layout starts with the same arrival-counter region, zeroed once by
+// eagle2_workspace_init and left at zero by every kernel: one ticket per sequence.
+__host__ __device__ inline size_t counters_bytes(int B) { return round_up(sizeof(int) * (size_t)B, kWsAlign); }
+
 inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
 inline int launch_result() { return cudaGetLastError() == cudaSuccess ? EAGLE2_OK : EAGLE2_ERR_CUDA; }

@@ -2,9 +2,9 @@
 //
 // One launch per expansion step.  Block (chunk, row, sequence) holds a chunk of one logit row in
 // registers, reduces it to (max, sum exp) and its k best tokens, and writes that partial to the
-// workspace.  The last block of a sequence to arrive merges the partials of every row in fp64
-// (log-sum-exp, top-k), writes the new tree level (token, parent, value = parent value + log-prob)
-// and ranks the new candidates by value to produce the next frontier.
+// workspace.  The last block of a sequence to arrive merges the partials, a warp per row (fp64
+// log-sum-exp, top-k of the chunk winners), writes the new tree level (token, parent, value = parent
+// value + log-prob) and ranks the new candidates by value to produce the next frontier.
 #include <math.h>
 
 #include <mutex>
@@ -38,7 +38,7 @@ static size_t expand_ws_layout(int B, int n_s, int chunks, int k, void* base, Ex
     size_t off = 0;
     char* p = static_cast<char*>(base);
     if (w) w->counters = reinterpret_cast<int*>(p + off);
-    off += round_up(sizeof(int) * (size_t)B, kWsAlign);
+    off += counters_bytes(B);
     if (w) w->stats = reinterpret_cast<double2*>(p + off);
     off += round_up(sizeof(double2) * (size_t)B * n_s * chunks, kWsAlign);
     if (w) w->keys = reinterpret_cast<unsigned long long*>(p + off);
@@ -85,6 +85,18 @@ expand_kernel(const float* __restrict__ draft_logits, long long batch_stride, in
     // ---- scan this chunk: per-warp (max, sum of exponentials), block top-k -----------------------
     float x[NE];
     scan_load<VPT, VEC>(zrow, V, chunk, x);
+    // The block that arrives last merges every row and then needs the rows' parents and their
+    // values; whichever block that will be, the two dependent loads are already under way.
+    const long long N = nodes_of(k, D);
+    int my_parent = -1;
+    double my_parent_value = 0.0;
+    if (s && threadIdx.x < n_s) {
+        my_parent = frontier[(long long)b * k + threadIdx.x];
+        const long long prev_base = s >= 2 ? (long long)k + (long long)(s - 2) * k * k : 0;
+        const long long prev_count = s >= 2 ? (long long)k * k : k;
+        if (my_parent < prev_base || my_parent >= prev_base + prev_count) my_parent = -2;  // reported by the merger
+        else my_parent_value = tree_value[(long long)b * N + my_parent];
+    }
     if (threadIdx.x == 0) s_topk.count = 0, s_topk.overflow = 0;
     float tmax = -INFINITY;
     int bad = 0;
@@ -118,53 +130,55 @@ expand_kernel(const float* __restrict__ draft_logits, long long batch_stride, in
     }
     if (bad) raise_status(d_status, EAGLE2_STATUS_NONFINITE_LOGIT);
 
-    // ---- the last block of this sequence merges ---------------------------------------------
+    // ---- the last block of this sequence merges: a warp per row -------------------------------
     if (!last_block_arrives(ws.counters + b, chunks * n_s, &s_flag)) return;
 
-    const long long N = nodes_of(k, D);
+    __shared__ int s_parent[EAGLE2_MAX_K];
+    __shared__ double s_pvalue[EAGLE2_MAX_K];
     const long long base = s ? (long long)k + (long long)(s - 1) * k * k : 0;
-    const long long prev_base = s >= 2 ? (long long)k + (long long)(s - 2) * k * k : 0;
-    const long long prev_count = s >= 2 ? (long long)k * k : k;
     const int n_new = n_s * k;
-    const int keys_per_row = chunks * k;  // at most kMergeKeysMax = 32 per lane
+    const int keys_per_row = chunks * k;
     int32_t* tok = tree_token + (long long)b * N;
     int32_t* par = tree_parent + (long long)b * N;
     double* val = tree_value + (long long)b * N;
     int32_t* fr = frontier + (long long)b * k;
+    if (threadIdx.x < n_s) s_parent[threadIdx.x] = my_parent, s_pvalue[threadIdx.x] = my_parent_value;
+    __syncthreads();
     int status = 0;
 
-    // a warp per row; everything a row needs is fetched before any of it is used
     for (int r = warp; r < n_s; r += kScanWarps) {
         const size_t p0 = ((size_t)b * n_s + r) * chunks;
         constexpr int BATCH = 16;  // chunk winners per lane and pass
+        // everything the row needs is requested before any of it is used
         unsigned long long cand[BATCH + 1];
 #pragma unroll
         for (int t = 0; t < BATCH; ++t)
             cand[t] = lane + 32 * t < keys_per_row ? ws.keys[p0 * k + lane + 32 * t] : 0ull;
-        int parent = -1;
-        double parent_value = 0.0;
-        if (s) {
-            parent = fr[r];
-            if (parent < prev_base || parent >= prev_base + prev_count) {
-                status |= EAGLE2_STATUS_BAD_TREE;
-                parent = (int)prev_base;
-            }
-            parent_value = val[parent];
+        double2 st0 = make_double2(-INFINITY, 0.0);
+        if (lane < chunks) st0 = ws.stats[p0 + lane];
+        int parent = s ? s_parent[r] : -1;
+        const double parent_value = s ? s_pvalue[r] : 0.0;
+        if (parent < -1) {
+            status |= EAGLE2_STATUS_BAD_TREE;
+            parent = (int)(s >= 2 ? (long long)k + (long long)(s - 2) * k * k : 0);
         }
         // log-sum-exp of the row from the chunk partials, in double
-        double m = -INFINITY;
-        for (int c = lane; c < chunks; c += 32) m = fmax(m, ws.stats[p0 + c].x);
+        double m = st0.x;
+        for (int c = lane + 32; c < chunks; c += 32) m = fmax(m, ws.stats[p0 + c].x);
         m = warp_max_f64(m);
-        double sum = 0.0;
-        for (int c = lane; c < chunks; c += 32) {
+        double sum = st0.x > -INFINITY ? st0.y * exp(st0.x - m) : 0.0;
+        for (int c = lane + 32; c < chunks; c += 32) {
             const double2 st = ws.stats[p0 + c];
             if (st.x > -INFINITY) sum += st.y * exp(st.x - m);
         }
         sum = warp_sum_f64(sum);
         if (!(m > -INFINITY)) status |= EAGLE2_STATUS_NONFINITE_LOGIT;
         const double lse = m + log(sum);
-        // top-k of the chunk winners, 32*BATCH at a time together with the best so far: lane c
-        // ends up holding the c-th
+        // top-k of the chunk winners, 32*BATCH at a time together with the best so far; lane c ends
+        // up holding the c-th.  The k-th largest lane maximum is a threshold no winner can be below;
+        // when at most 32 keys reach it (the usual case) they are sorted across the lanes, otherwise
+        // k rounds of maximum extraction do the same job.
+        unsigned long long* s_pack = s_topk.cand + warp * 32;  // free: the chunk scan is over
         unsigned long long mine = 0;
         for (int e0 = 0; e0 < keys_per_row; e0 += 32 * BATCH) {
             if (e0) {
@@ -173,15 +187,40 @@ expand_kernel(const float* __restrict__ draft_logits, long long batch_stride, in
                     cand[t] = e0 + lane + 32 * t < keys_per_row ? ws.keys[p0 * k + e0 + lane + 32 * t] : 0ull;
             }
             cand[BATCH] = mine;
+            unsigned long long lane_best = 0;
+#pragma unroll
+            for (int t = 0; t <= BATCH; ++t) lane_best = cand[t] > lane_best ? cand[t] : lane_best;
+            const unsigned long long thr = __shfl_sync(0xffffffffu, warp_sort_desc_u64(lane_best), k - 1);
+            int cnt = 0;
+#pragma unroll
+            for (int t = 0; t <= BATCH; ++t) cnt += cand[t] >= thr && cand[t] != 0ull;
+            int incl = cnt;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int up = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += up;
+            }
+            const int total = __shfl_sync(0xffffffffu, incl, 31);
             unsigned long long next = 0;
-            for (int c = 0; c < k; ++c) {
-                unsigned long long best = 0;
+            if (total <= 32) {
+                int pos = incl - cnt;
 #pragma unroll
-                for (int t = 0; t <= BATCH; ++t) best = cand[t] > best ? cand[t] : best;
-                const unsigned long long top = warp_max_u64(best);
+                for (int t = 0; t <= BATCH; ++t)
+                    if (cand[t] >= thr && cand[t] != 0ull) s_pack[pos++] = cand[t];
+                __syncwarp();
+                next = warp_sort_desc_u64(lane < total ? s_pack[lane] : 0ull);
+                __syncwarp();
+                if (lane >= k) next = 0ull;
+            } else {
+                for (int c = 0; c < k; ++c) {
+                    unsigned long long best = 0;
 #pragma unroll
-                for (int t = 0; t <= BATCH; ++t) cand[t] = (cand[t] == top) ? 0ull : cand[t];
-                if (lane == c) next = top;
+                    for (int t = 0; t <= BATCH; ++t) best = cand[t] > best ? cand[t] : best;
+                    const unsigned long long top = warp_max_u64(best);
+#pragma unroll
+                    for (int t = 0; t <= BATCH; ++t) cand[t] = (cand[t] == top) ? 0ull : cand[t];
+                    if (lane == c) next = top;
+                }
             }
             mine = next;
         }
@@ -194,7 +233,7 @@ expand_kernel(const float* __restrict__ draft_logits, long long batch_stride, in
             s_rank[r * k + lane] = order_code_f64(v);
         }
     }
-    __syncthreads();  // all rows merged; every read of the old frontier is done
+    __syncthreads();  // all rows merged (the old frontier was read when the kernel started)
 
     // next frontier: rank the new candidates by (value desc, index asc); ranks < k are kept
     for (int i = threadIdx.x; i < n_new; i += kScanThreads) {
@@ -314,7 +353,7 @@ extern "C" int eagle2_expand_static(const float* draft_logits, long long batch_s
     expand_ws_layout(B, n_s, plan.chunks, k, scratch, &w);
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     // the array keeps whatever the last call left: the arrival counters must start at zero
-    if (cudaMemsetAsync(w.counters, 0, round_up(sizeof(int) * (size_t)B, kWsAlign), st) != cudaSuccess) {
+    if (cudaMemsetAsync(w.counters, 0, counters_bytes(B), st) != cudaSuccess) {
         cudaGetLastError();
         return EAGLE2_ERR_CUDA;
     }

@@ -803,7 +803,7 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
 
 // One warp per output row of a sequence that used several splits: combine their partials.  The
 // lanes first fetch the splits' (maximum, sum) pairs side by side, then every lane owns DH/32
-// columns and the partial rows are fetched eight splits at a time before any is used.
+// columns and the partial rows are fetched sixteen splits at a time before any is used.
 template <int DH>
 __global__ void __launch_bounds__(256)
 tree_attention_merge_kernel(const int64_t* __restrict__ kv_off, const int32_t* __restrict__ kv_len, int B, int m,
@@ -843,10 +843,10 @@ tree_attention_merge_kernel(const int64_t* __restrict__ kv_off, const int32_t* _
             if (ml.x != -INFINITY) w = exp2f(ml.x - mmax), l += ml.y * w;
         }
         const int n = min(32, S_b - s0);
-        for (int s1 = 0; s1 < n; s1 += 8) {
-            float v[8][PER];
+        for (int s1 = 0; s1 < n; s1 += 16) {
+            float v[16][PER];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) {
+            for (int u = 0; u < 16; ++u) {
                 const int sl = min(s1 + u, n - 1);  // clamped: a repeated row gets weight 0 below
                 const float* src = ws.o_part + (first + (size_t)(s0 + sl) * stride) * DH + lane * PER;
                 if (PER == 4) {
@@ -858,7 +858,7 @@ tree_attention_merge_kernel(const int64_t* __restrict__ kv_off, const int32_t* _
                 }
             }
 #pragma unroll
-            for (int u = 0; u < 8; ++u) {
+            for (int u = 0; u < 16; ++u) {
                 float wu = __shfl_sync(0xffffffffu, w, min(s1 + u, 31));
                 if (s1 + u >= n) wu = 0.f;
                 // a split without visible keys leaves its partial row unwritten: never multiply it

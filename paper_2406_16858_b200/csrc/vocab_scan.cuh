@@ -116,6 +116,22 @@ __device__ __forceinline__ float warp_sort_desc_f32(float v) {
     return v;
 }
 
+// The same for one 64-bit key per lane.
+__device__ __forceinline__ unsigned long long warp_sort_desc_u64(unsigned long long v) {
+    const int lane = threadIdx.x & 31;
+#pragma unroll
+    for (int size = 2; size <= 32; size <<= 1) {
+#pragma unroll
+        for (int stride = size >> 1; stride > 0; stride >>= 1) {
+            const unsigned long long other = __shfl_xor_sync(0xffffffffu, v, stride);
+            const bool desc = (lane & size) == 0, lower = (lane & stride) == 0;
+            const unsigned long long hi = v > other ? v : other, lo = v > other ? other : v;
+            v = (lower == desc) ? hi : lo;
+        }
+    }
+    return v;
+}
+
 constexpr int kCandCap = 512;  // candidate keys a block can stage for the filtered selection
 
 struct TopkScratch {
