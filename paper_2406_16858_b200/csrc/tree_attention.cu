@@ -33,7 +33,7 @@ constexpr int kMaxTilesPerSplit = 16; // a block never streams more than 2048 ke
 constexpr int kTmemCols = 512;
 constexpr int kSlots = 2;             // score slots in tensor memory
 constexpr long long kWaitCycles = 1LL << 31;  // ~1 s bound of a barrier wait
-constexpr uint32_t kSuspendNs = 20000;        // a waiting thread sleeps in hardware at most this long per try
+constexpr uint32_t kSuspendNs = 400;          // a waiting thread sleeps in hardware at most this long per try
 
 struct AttnPlan {
     int g, M;
@@ -45,6 +45,9 @@ struct AttnPlan {
     int splits;     // KV splits per sequence (blocks of the launch)
     int per_split;  // K/V tiles per split
     int stages;     // K/V ring depth
+    int pair;       // 1: two blocks (a cluster on one TPC) share every K/V tile through cta_group::2
+                    // MMAs: each holds 128 of the 256 query rows, half of each K tile's keys and
+                    // half of each V tile's columns
     size_t smem;
 };
 
@@ -56,9 +59,10 @@ static void attention_plan(int B, int m, int Hq, int Hkv, int d, int max_kv_len,
     p->per = p->per_tok * p->g;  // never above 256: n_rb >= m*g/256
     p->mt = p->per > kRowsPerTile ? 2 : 1;
     p->q_tma = (kRowsPerTile % p->g) == 0;
+    p->pair = 0 && (p->mt == 2 && p->q_tma && d == 128) ? 1 : 0;
     const long long items = (long long)B * Hkv * p->n_rb;
     const int tiles = (max_kv_len + m + kTK - 1) / kTK;
-    long long s = 148 / (items > 0 ? items : 1);
+    long long s = (p->pair ? 74 : 148) / (items > 0 ? items : 1);
     if (s < 1) s = 1;
     if (s > tiles) s = tiles;
     int per_split = (int)((tiles + s - 1) / s);
@@ -70,6 +74,10 @@ static void attention_plan(int B, int m, int Hq, int Hkv, int d, int max_kv_len,
     int stages = (int)((220 * 1024 - p->mt * unit) / (2 * unit));
     p->stages = stages > 4 ? 4 : (stages < 2 ? 2 : stages);
     p->smem = (p->mt + 2 * (size_t)p->stages) * unit + 1024;
+    if (p->pair) {  // per block: one 128-row query tile, half-size K and V stages
+        p->stages = 4;
+        p->smem = unit + 4 * unit + 1024;
+    }
 }
 
 struct AttnWs {
@@ -120,15 +128,16 @@ static EncodeTiledFn encode_tiled_fn() {
     return fn;
 }
 
-static bool make_cache_map(CUtensorMap* map, const void* base, long long rows, int Hkv, int d) {
+static bool make_cache_map(CUtensorMap* map, const void* base, long long rows, int Hkv, int d, int box_rows = kTK,
+                           CUtensorMapL2promotion promo = CU_TENSOR_MAP_L2_PROMOTION_L2_256B) {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return false;
     const cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)Hkv, (cuuint64_t)rows};
     const cuuint64_t strides[2] = {(cuuint64_t)d * 2, (cuuint64_t)Hkv * d * 2};
-    const cuuint32_t box[3] = {64, 1, (cuuint32_t)kTK};
+    const cuuint32_t box[3] = {64, 1, (cuuint32_t)box_rows};
     const cuuint32_t estr[3] = {1, 1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, promo,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -171,6 +180,30 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.b32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// The same bounded wait, polling without ever sleeping: for the single lanes whose reaction time
+// is on the critical path (MMA issue, producer).
+__device__ __forceinline__ bool mbar_wait_spin(uint32_t bar, uint32_t parity, volatile int* abort) {
+    if (mbar_test_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (int spin = 1;; ++spin) {
+        if (mbar_test_wait(bar, parity)) return true;
+        if ((spin & 1023) == 0 && (*abort || clock64() - t0 > kWaitCycles)) {
+            *abort = 1;
+            return false;
+        }
+    }
+}
 // Bounded wait for the phase of the given parity.  Returns false when the bound ran out or another
 // role of the block has already given up (*abort != 0).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort) {
@@ -193,7 +226,7 @@ __device__ __forceinline__ void fence_barrier_init() {
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2,
                                             uint32_t bar) {
     asm volatile(
-        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes "
+        "cp.async.bulk.tensor.3d.shared::cta.global.tile.mbarrier::complete_tx::bytes "
         "[%0], [%1, {%2, %3, %4}], [%5];"
         ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar)
         : "memory");
@@ -201,7 +234,7 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, int c3,
                                             uint32_t bar) {
     asm volatile(
-        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes "
+        "cp.async.bulk.tensor.4d.shared::cta.global.tile.mbarrier::complete_tx::bytes "
         "[%0], [%1, {%2, %3, %4, %5}], [%6];"
         ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar)
         : "memory");
@@ -263,6 +296,54 @@ __device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_
         ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
+// ---- the same for a pair of blocks (cta_group::2; issued by the pair's first block only) ----------
+__device__ __forceinline__ void tmem_alloc2(uint32_t dst_smem, uint32_t cols) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols)
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish2() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc2(uint32_t taddr, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+// arrives on the barrier at this shared-memory offset in both blocks of the pair
+__device__ __forceinline__ void tc_commit2(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"((uint16_t)3)
+                 : "memory");
+}
+__device__ __forceinline__ void mma2_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                        uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void mma2_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                        uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// arrive on the barrier at this shared-memory offset in block `rank` of the cluster
+__device__ __forceinline__ void mbar_arrive_in(uint32_t bar, uint32_t rank) {
+    uint32_t remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(bar), "r"(rank));
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(remote) : "memory");
+}
+
 // 32 consecutive 32-bit columns of this thread's tensor-memory lane
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
     asm volatile(
@@ -349,9 +430,9 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes)
            ((uint64_t)(1024u >> 4) << 32) | (1ull << 46) | (2ull << 61);
 }
 // Instruction descriptor: bf16 x bf16 -> fp32, M = 128, A K-major; B K-major or MN-major.
-__host__ __device__ constexpr uint32_t instr_desc(int n, bool b_mn_major) {
+__host__ __device__ constexpr uint32_t instr_desc(int n, bool b_mn_major, int m_rows = kRowsPerTile) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((uint32_t)(n >> 3) << 17) |
-           ((uint32_t)(kRowsPerTile >> 4) << 24);
+           ((uint32_t)(m_rows >> 4) << 24);
 }
 
 // A sequence is served only if its length is within the plan and its rows lie inside the cache.
@@ -367,6 +448,9 @@ struct AttnBarriers {
     // o_done[t][j & 1].  A waiter may skip phases (it only looks when it must rescale O, and at the
     // end); with two barriers the one it consults is never more than one phase ahead of it.
     unsigned long long o_done[2][2];
+    // pair mode, used in the pair's first block: the other block's query tile / K half / V half
+    // has landed (and its V tail is cleared)
+    unsigned long long q_peer, k_peer[4], v_peer[4];
 };
 
 // Visibility of the 128 keys of a tile that reaches past the committed cache, as four 32-bit words:
@@ -396,7 +480,7 @@ __device__ __forceinline__ void tile_visibility(unsigned long long mlo, unsigned
     vis[0] = (uint32_t)lo, vis[1] = (uint32_t)(lo >> 32), vis[2] = (uint32_t)hi, vis[3] = (uint32_t)(hi >> 32);
 }
 
-template <int DH, int MT>
+template <int DH, int MT, bool PAIR>
 __global__ void __launch_bounds__(MT * 128 + 64, 1)
 tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map,
                       const __grid_constant__ CUtensorMap q_map, const __nv_bfloat16* __restrict__ q, const int64_t* __restrict__ kv_off,
@@ -408,9 +492,13 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
     constexpr uint32_t kTile = HALVES * kPanel;
     constexpr int kSoftmaxThreads = MT * 128;
     constexpr int kTmaWarp = MT * 4, kMmaWarp = MT * 4 + 1;
-    constexpr uint32_t kIdescQK = instr_desc(kTK, false);
-    constexpr uint32_t kIdescPV = instr_desc(DH, true);
+    constexpr uint32_t kIdescQK = instr_desc(kTK, false, PAIR ? 256 : 128);
+    constexpr uint32_t kIdescPV = instr_desc(DH, true, PAIR ? 256 : 128);
     constexpr uint32_t kOCol = kSlots * kTK;           // first accumulator column of O
+    // bytes a block holds of one K tile and of one V tile (a pair splits K by keys, V by columns)
+    constexpr uint32_t kKPanel = PAIR ? kPanel / 2 : kPanel, kKTile = HALVES * kKPanel;
+    constexpr uint32_t kVTile = PAIR ? kPanel : kTile;
+    static_assert(!PAIR || (MT == 1 && DH == 128), "a pair block holds one 128-row tile, head_dim 128");
 
     extern __shared__ unsigned char smem_raw[];
     __shared__ AttnBarriers bars;
@@ -418,7 +506,8 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
     __shared__ int s_abort;
 
     const int g = plan.g, M = plan.M, S = plan.splits, NST = plan.stages;
-    int bid = blockIdx.x;
+    const uint32_t rank = PAIR ? cluster_ctarank() : 0u;  // 0: the block that issues the pair's MMAs
+    int bid = PAIR ? blockIdx.x >> 1 : blockIdx.x;
     const int split = bid % S;
     bid /= S;
     const int rb = bid % plan.n_rb;
@@ -438,17 +527,24 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
     const int nt = overflow ? 0 : min(plan.per_split, tiles - t_begin);
     const bool direct = S_b <= 1;  // a single split writes final rows
 
-    const int row0 = rb * plan.per;                      // first packed row of this block
-    const int rows_here = min(plan.per, M - row0);       // rows that exist
-    const size_t part_row0 = ((((size_t)b * Hkv + hk) * S + split) * plan.n_rb + rb) * (size_t)(MT * 128);
+    // first packed row of this block and the rows that exist in it (the second block of a pair may
+    // hold none: it still serves its halves of K and V)
+    const int rows_blk = min(plan.per, M - rb * plan.per);
+    const int row0 = rb * plan.per + (int)rank * 128;
+    const int rows_here = PAIR ? max(0, min(128, rows_blk - (int)rank * 128)) : rows_blk;
+    const size_t part_row0 = ((((size_t)b * Hkv + hk) * S + split) * plan.n_rb + rb) * (size_t)(plan.mt * 128) +
+                             (size_t)rank * 128;
 
-    if (overflow && tid == 0 && split == 0 && rb == 0 && hk == 0) raise_status(d_status, EAGLE2_STATUS_KV_OVERFLOW);
-    if (nt <= 0 || rows_here <= 0) return;  // a split past the sequence's last tile (never merged), or a rejected sequence
+    if (overflow && tid == 0 && split == 0 && rb == 0 && hk == 0 && rank == 0)
+        raise_status(d_status, EAGLE2_STATUS_KV_OVERFLOW);
+    // a split past the sequence's last tile (never merged), or a rejected sequence: both blocks of a
+    // pair take the same decision
+    if (nt <= 0 || rows_blk <= 0) return;
 
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t sQ = smem_base;
     const uint32_t sK = sQ + MT * kTile;
-    const uint32_t sV = sK + (uint32_t)NST * kTile;
+    const uint32_t sV = sK + (uint32_t)NST * kKTile;
     unsigned char* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
 
     // ---- set-up: barriers, tensor memory --------------------------------------------------------
@@ -463,24 +559,33 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
         }
         for (int s = 0; s < kSlots; ++s) {
             mbar_init(smem_u32(&bars.s_full[s]), 1);
-            mbar_init(smem_u32(&bars.p_full[s]), 128);
+            mbar_init(smem_u32(&bars.p_full[s]), PAIR ? 8 : 4);  // one arrival per softmax warp
+        }
+        mbar_init(smem_u32(&bars.q_peer), 1);
+        for (int s = 0; s < 4; ++s) {
+            mbar_init(smem_u32(&bars.k_peer[s]), 1);
+            mbar_init(smem_u32(&bars.v_peer[s]), 1);
         }
         for (int s = 0; s < 4; ++s) mbar_init(smem_u32(&bars.o_done[s >> 1][s & 1]), 1);
         fence_barrier_init();
     }
     if (warp == kMmaWarp) {
-        tmem_alloc(smem_u32(&s_tmem_base), kTmemCols);
-        tmem_relinquish();
+        if (PAIR) {
+            tmem_alloc2(smem_u32(&s_tmem_base), kTmemCols);
+            tmem_relinquish2();
+        } else {
+            tmem_alloc(smem_u32(&s_tmem_base), kTmemCols);
+            tmem_relinquish();
+        }
     }
     if (warp == kTmaWarp && lane == 0) {
         asm volatile("prefetch.tensormap [%0];" ::"l"(&k_map) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&v_map) : "memory");
         if (plan.q_tma) asm volatile("prefetch.tensormap [%0];" ::"l"(&q_map) : "memory");
     }
-    // the merge kernel of this call may be scheduled from here on (it waits for this grid to finish)
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     tc_fence_before();
-    __syncthreads();
+    if (PAIR) cluster_sync_all();  // both blocks' barriers exist before either signals the other
+    else __syncthreads();
     tc_fence_after();
     const uint32_t tmem = s_tmem_base;
     volatile int* abort_flag = &s_abort;
@@ -498,7 +603,8 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
 #pragma unroll
                     for (int h = 0; h < HALVES; ++h)
                         tma_load_4d(sQ + t * kTile + h * kPanel, &q_map, h * 64, 0,
-                                    b * m + rb * plan.per_tok + t * (kRowsPerTile / g), hk, smem_u32(&bars.q_full));
+                                    b * m + rb * plan.per_tok + (t + (int)rank) * (kRowsPerTile / g), hk,
+                                    smem_u32(&bars.q_full));
             }
             for (int j = 0; j < nt && ok; ++j) {
                 const int st = j % NST;
@@ -506,19 +612,24 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
                 const int row = (int)(row_base + (long long)(t_begin + j) * kTK);
                 if (j >= NST) ok = mbar_wait(smem_u32(&bars.k_empty[st]), ph ^ 1u, abort_flag);
                 if (!ok) break;
-                mbar_expect_tx(smem_u32(&bars.k_full[st]), kTile);
+                mbar_expect_tx(smem_u32(&bars.k_full[st]), kKTile);
 #pragma unroll
-                for (int h = 0; h < HALVES; ++h)
-                    tma_load_3d(sK + st * kTile + h * kPanel, &k_map, h * 64, hk, row, smem_u32(&bars.k_full[st]));
+                for (int h = 0; h < HALVES; ++h)  // a pair block takes its 64 of the tile's 128 keys
+                    tma_load_3d(sK + st * kKTile + h * kKPanel, &k_map, h * 64, hk, row + (int)rank * (kTK / 2),
+                                smem_u32(&bars.k_full[st]));
                 if (j >= NST) ok = mbar_wait(smem_u32(&bars.v_empty[st]), ph ^ 1u, abort_flag);
                 if (!ok) {  // K of this tile is in flight, V is not
                     mbar_wait(smem_u32(&bars.k_full[st]), ph, abort_flag);
                     break;
                 }
-                mbar_expect_tx(smem_u32(&bars.v_full[st]), kTile);
+                mbar_expect_tx(smem_u32(&bars.v_full[st]), kVTile);
+                if (PAIR) {  // all keys, this block's 64 of the 128 columns
+                    tma_load_3d(sV + st * kVTile, &v_map, (int)rank * 64, hk, row, smem_u32(&bars.v_full[st]));
+                } else {
 #pragma unroll
-                for (int h = 0; h < HALVES; ++h)
-                    tma_load_3d(sV + st * kTile + h * kPanel, &v_map, h * 64, hk, row, smem_u32(&bars.v_full[st]));
+                    for (int h = 0; h < HALVES; ++h)
+                        tma_load_3d(sV + st * kTile + h * kPanel, &v_map, h * 64, hk, row, smem_u32(&bars.v_full[st]));
+                }
                 issued = j + 1;
             }
             if (*abort_flag) {
@@ -541,69 +652,105 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
         // ===== MMA issuer (whole warp walks the loop, lane 0 waits and issues) =====================
         auto wait_all = [&](uint32_t bar, uint32_t parity) {  // lane 0 polls, the warp gets the outcome
             int r = 1;
-            if (lane == 0) r = mbar_wait(bar, parity, abort_flag) ? 1 : 0;
+            if (lane == 0) r = mbar_wait_spin(bar, parity, abort_flag) ? 1 : 0;
             r = __shfl_sync(0xffffffffu, r, 0);
             __syncwarp();
             return r != 0;
         };
+        // rows past the sequence's last key hold whatever follows it in the cache: clear them in
+        // this block's V tile so that a zero probability times a non-finite value cannot reach O
+        auto clear_v_tail = [&](int j, int st) {
+            const int valid = n_keys - (t_begin + j) * kTK;
+            if (valid < kTK) {
+                constexpr int PANELS = PAIR ? 1 : HALVES;
+                const int chunks = (kTK - valid) * 8;
+                for (int idx = lane; idx < chunks * PANELS; idx += 32) {
+                    const int h = idx / chunks, rem = idx % chunks;
+                    const int r = valid + rem / 8, c = rem % 8;
+                    *reinterpret_cast<uint4*>(smem_gen + (sV - smem_base) + st * kVTile + h * kPanel + r * 128 +
+                                              c * 16) = make_uint4(0, 0, 0, 0);
+                }
+                fence_proxy_async();
+                __syncwarp();
+            }
+        };
         bool ok = wait_all(smem_u32(&bars.q_full), 0);
-        auto issue_qk = [&](int i) {  // S[slot] = Q[row tile] . K[tile]^T
-            const int j = i / MT, t = i % MT, st = j % NST;
-            if (t == 0) ok = ok && wait_all(smem_u32(&bars.k_full[st]), (uint32_t)((j / NST) & 1));
-            if (!ok) return;
-            tc_fence_after();
-            if (lane == 0) {
-                const uint32_t d_tmem = tmem + (uint32_t)(i % kSlots) * kTK;
-#pragma unroll
-                for (int ks = 0; ks < DH / 16; ++ks) {
-                    const uint32_t koff = (uint32_t)(ks / 4) * kPanel + (uint32_t)(ks % 4) * 32u;
-                    mma_ss(d_tmem, smem_desc(sQ + t * kTile + koff, 16), smem_desc(sK + st * kTile + koff, 16),
-                           kIdescQK, ks > 0);
-                }
-                tc_commit(smem_u32(&bars.s_full[i % kSlots]));
-                if (t == MT - 1) tc_commit(smem_u32(&bars.k_empty[st]));
+        if (PAIR && rank != 0) {
+            // The second block of a pair issues no MMA: this warp tells the first block when this
+            // block's query tile, K half and V half are in place.
+            if (ok && lane == 0) mbar_arrive_in(smem_u32(&bars.q_peer), 0);
+            for (int j = 0; j < nt && ok; ++j) {
+                const int st = j % NST;
+                const uint32_t ph = (uint32_t)((j / NST) & 1);
+                ok = wait_all(smem_u32(&bars.k_full[st]), ph);
+                if (!ok) break;
+                if (lane == 0) mbar_arrive_in(smem_u32(&bars.k_peer[st]), 0);
+                ok = wait_all(smem_u32(&bars.v_full[st]), ph);
+                if (!ok) break;
+                clear_v_tail(j, st);
+                if (lane == 0) mbar_arrive_in(smem_u32(&bars.v_peer[st]), 0);
+                __syncwarp();
             }
-            __syncwarp();
-        };
-        auto issue_pv = [&](int i) {  // O[row tile] += P[slot] . V[tile]
-            const int j = i / MT, t = i % MT, st = j % NST;
-            if (t == 0) {
-                ok = ok && wait_all(smem_u32(&bars.v_full[st]), (uint32_t)((j / NST) & 1));
+        } else {
+            if (PAIR) ok = ok && wait_all(smem_u32(&bars.q_peer), 0);
+            auto commit = [&](uint32_t bar) {
+                if (PAIR) tc_commit2(bar);
+                else tc_commit(bar);
+            };
+            auto issue_qk = [&](int i) {  // S[slot] = Q[row tile] . K[tile]^T
+                const int j = i / MT, t = i % MT, st = j % NST;
+                if (t == 0) {
+                    ok = ok && wait_all(smem_u32(&bars.k_full[st]), (uint32_t)((j / NST) & 1));
+                    if (PAIR) ok = ok && wait_all(smem_u32(&bars.k_peer[st]), (uint32_t)((j / NST) & 1));
+                }
                 if (!ok) return;
-                const int valid = n_keys - (t_begin + j) * kTK;
-                if (valid < kTK) {
-                    // rows past the sequence's last key hold whatever follows it in the cache: clear
-                    // them so that a zero probability times a non-finite value cannot reach O
-                    const int chunks = (kTK - valid) * 8;
-                    for (int idx = lane; idx < chunks * HALVES; idx += 32) {
-                        const int h = idx / chunks, rem = idx % chunks;
-                        const int r = valid + rem / 8, c = rem % 8;
-                        *reinterpret_cast<uint4*>(smem_gen + (sV - smem_base) + st * kTile + h * kPanel + r * 128 +
-                                                  c * 16) = make_uint4(0, 0, 0, 0);
-                    }
-                    fence_proxy_async();
-                    __syncwarp();
-                }
-            }
-            ok = ok && wait_all(smem_u32(&bars.p_full[i % kSlots]), (uint32_t)((i / kSlots) & 1));
-            if (!ok) return;
-            tc_fence_after();
-            if (lane == 0) {
-                const uint32_t d_tmem = tmem + kOCol + (uint32_t)t * DH;
-                const uint32_t a_tmem = tmem + (uint32_t)(i % kSlots) * kTK;
+                tc_fence_after();
+                if (lane == 0) {
+                    const uint32_t d_tmem = tmem + (uint32_t)(i % kSlots) * kTK;
 #pragma unroll
-                for (int ks = 0; ks < kTK / 16; ++ks)
-                    mma_ts(d_tmem, a_tmem + ks * 8, smem_desc(sV + st * kTile + ks * 2048u, kPanel), kIdescPV,
-                           (j > 0 || ks > 0) ? 1u : 0u);
-                tc_commit(smem_u32(&bars.o_done[t][j & 1]));
-                if (t == MT - 1) tc_commit(smem_u32(&bars.v_empty[st]));
+                    for (int ks = 0; ks < DH / 16; ++ks) {
+                        const uint32_t qoff = (uint32_t)(ks / 4) * kPanel + (uint32_t)(ks % 4) * 32u;
+                        const uint32_t koff = (uint32_t)(ks / 4) * kKPanel + (uint32_t)(ks % 4) * 32u;
+                        const uint64_t qd = smem_desc(sQ + t * kTile + qoff, 16), kd = smem_desc(sK + st * kKTile + koff, 16);
+                        if (PAIR) mma2_ss(d_tmem, qd, kd, kIdescQK, ks > 0);
+                        else mma_ss(d_tmem, qd, kd, kIdescQK, ks > 0);
+                    }
+                    commit(smem_u32(&bars.s_full[i % kSlots]));
+                    if (t == MT - 1) commit(smem_u32(&bars.k_empty[st]));
+                }
+                __syncwarp();
+            };
+            auto issue_pv = [&](int i) {  // O[row tile] += P[slot] . V[tile]
+                const int j = i / MT, t = i % MT, st = j % NST;
+                if (t == 0) {
+                    ok = ok && wait_all(smem_u32(&bars.v_full[st]), (uint32_t)((j / NST) & 1));
+                    if (!ok) return;
+                    clear_v_tail(j, st);
+                    if (PAIR) ok = ok && wait_all(smem_u32(&bars.v_peer[st]), (uint32_t)((j / NST) & 1));
+                }
+                ok = ok && wait_all(smem_u32(&bars.p_full[i % kSlots]), (uint32_t)((i / kSlots) & 1));
+                if (!ok) return;
+                tc_fence_after();
+                if (lane == 0) {
+                    const uint32_t d_tmem = tmem + kOCol + (uint32_t)t * DH;
+                    const uint32_t a_tmem = tmem + (uint32_t)(i % kSlots) * kTK;
+#pragma unroll
+                    for (int ks = 0; ks < kTK / 16; ++ks) {
+                        const uint64_t vd = smem_desc(sV + st * kVTile + ks * 2048u, kPanel);
+                        const uint32_t acc = (j > 0 || ks > 0) ? 1u : 0u;
+                        if (PAIR) mma2_ts(d_tmem, a_tmem + ks * 8, vd, kIdescPV, acc);
+                        else mma_ts(d_tmem, a_tmem + ks * 8, vd, kIdescPV, acc);
+                    }
+                    commit(smem_u32(&bars.o_done[t][j & 1]));
+                    if (t == MT - 1) commit(smem_u32(&bars.v_empty[st]));
+                }
+                __syncwarp();
+            };
+            for (int i = 0; i < kSlots && i < n_items && ok; ++i) issue_qk(i);
+            for (int i = 0; i < n_items && ok; ++i) {
+                issue_pv(i);
+                if (ok && i + kSlots < n_items) issue_qk(i + kSlots);
             }
-            __syncwarp();
-        };
-        for (int i = 0; i < kSlots && i < n_items && ok; ++i) issue_qk(i);
-        for (int i = 0; i < n_items && ok; ++i) {
-            issue_pv(i);
-            if (ok && i + kSlots < n_items) issue_qk(i + kSlots);
         }
     } else {
         // ===== softmax warps: thread = packed query row ============================================
@@ -611,7 +758,7 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
         const int r_tile = ((warp & 3) << 5) | lane;      // row inside the tile = tensor-memory lane
         const int r_blk = wg * 128 + r_tile;              // row inside the block
         const bool row_ok = r_blk < rows_here;
-        const int pr = row0 + (row_ok ? r_blk : 0);       // packed row = token * g + head in group
+        const int pr = row_ok ? row0 + r_blk : rb * plan.per;  // packed row = token * g + head in group
         const int tok = pr / g, hq = hk * g + pr % g;
         const uint32_t lane_sel = (uint32_t)((warp & 3) << 5) << 16;
 
@@ -723,7 +870,11 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
             l_run += (sum_a.x + sum_a.y) + (sum_b.x + sum_b.y);
             tc_wait_st();
             tc_fence_before();
-            mbar_arrive(smem_u32(&bars.p_full[slot]));
+            __syncwarp();  // every lane's P is in tensor memory: one arrival speaks for the warp
+            if (lane == 0) {
+                if (PAIR) mbar_arrive_in(smem_u32(&bars.p_full[slot]), 0);  // the pair's first block issues P.V
+                else mbar_arrive(smem_u32(&bars.p_full[slot]));
+            }
         }
 
         // ---- epilogue: O rows leave tensor memory through shared memory, so that the global
@@ -794,11 +945,18 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
     }
 
     // ---- teardown ----------------------------------------------------------------------------------
+    // the merge kernel of this call may be scheduled from here on (it waits for this grid to finish)
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     tc_fence_before();
-    __syncthreads();
+    if (PAIR) cluster_sync_all();  // tensor memory is released by both blocks together
+    else __syncthreads();
     tc_fence_after();
-    if (warp == kMmaWarp) tmem_dealloc(tmem, kTmemCols);
+    if (warp == kMmaWarp) {
+        if (PAIR) tmem_dealloc2(tmem, kTmemCols);
+        else tmem_dealloc(tmem, kTmemCols);
+    }
     if (tid == 0 && s_abort) raise_status(d_status, EAGLE2_STATUS_TIMEOUT);
+    if (PAIR) cluster_sync_all();  // neither block leaves while the other may still signal it
 }
 
 // One warp per output row of a sequence that used several splits: combine their partials.  The
@@ -878,46 +1036,59 @@ tree_attention_merge_kernel(const int64_t* __restrict__ kv_off, const int32_t* _
         lse[((long long)b * Hq + hq) * m + tok] = (mmax + log2f(l)) * 0.69314718055994531f;
 }
 
-template <int DH, int MT>
+template <int DH, int MT, bool PAIR>
 static int launch_attention(const CUtensorMap& k_map, const CUtensorMap& v_map, const CUtensorMap& q_map,
                             const void* q,
                             const int64_t* kv_off, const int32_t* kv_len, const uint64_t* mask_bits, int B,
                             int m, int Hq, int Hkv, long long cache_rows, int max_kv_len, const AttnPlan& plan,
                             float scale, void* out, float* lse, const AttnWs& ws, int32_t* d_status,
                             cudaStream_t st) {
-    auto kern = tree_attention_kernel<DH, MT>;
+    auto kern = tree_attention_kernel<DH, MT, PAIR>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem) !=
         cudaSuccess) {
         cudaGetLastError();
         return EAGLE2_ERR_CUDA;
     }
-    const long long blocks = (long long)B * Hkv * plan.n_rb * plan.splits;
+    const long long blocks = (long long)B * Hkv * plan.n_rb * plan.splits * (PAIR ? 2 : 1);
     if (blocks > 0x7fffffffLL) return EAGLE2_ERR_SHAPE;
-    kern<<<(unsigned)blocks, MT * 128 + 64, plan.smem, st>>>(
-        k_map, v_map, q_map, static_cast<const __nv_bfloat16*>(q), kv_off, kv_len, mask_bits, m, Hq, Hkv, cache_rows,
-        max_kv_len, plan, scale * 1.4426950408889634f, static_cast<__nv_bfloat16*>(out), lse, ws, d_status);
-    if (launch_result() != EAGLE2_OK) return EAGLE2_ERR_CUDA;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)blocks, 1, 1);
+    cfg.blockDim = dim3(MT * 128 + 64, 1, 1);
+    cfg.dynamicSmemBytes = plan.smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = PAIR ? 2 : 1;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, kern, k_map, v_map, q_map, static_cast<const __nv_bfloat16*>(q), kv_off, kv_len,
+                           mask_bits, m, Hq, Hkv, cache_rows, max_kv_len, plan, scale * 1.4426950408889634f,
+                           static_cast<__nv_bfloat16*>(out), lse, ws, d_status) != cudaSuccess) {
+        cudaGetLastError();
+        return EAGLE2_ERR_CUDA;
+    }
     if (plan.splits > 1) {
         const long long warps = (long long)B * Hkv * plan.M;
         const long long mblocks = (warps + 7) / 8;
         if (mblocks > 0x7fffffffLL) return EAGLE2_ERR_SHAPE;
         // the merge kernel may be scheduled while the attention kernel still runs; it starts with
         // griddepcontrol.wait, which holds it until that kernel's writes are complete
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3((unsigned)mblocks, 1, 1);
-        cfg.blockDim = dim3(256, 1, 1);
-        cfg.stream = st;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[0].val.programmaticStreamSerializationAllowed = 1;
-        cfg.attrs = attr;
-        cfg.numAttrs = 1;
-        if (cudaLaunchKernelEx(&cfg, tree_attention_merge_kernel<DH>, kv_off, kv_len, B, m, Hq, Hkv, cache_rows,
+        cudaLaunchConfig_t mcfg = {};
+        mcfg.gridDim = dim3((unsigned)mblocks, 1, 1);
+        mcfg.blockDim = dim3(256, 1, 1);
+        mcfg.stream = st;
+        cudaLaunchAttribute mattr[1];
+        mattr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        mattr[0].val.programmaticStreamSerializationAllowed = 1;
+        mcfg.attrs = mattr;
+        mcfg.numAttrs = 1;
+        if (cudaLaunchKernelEx(&mcfg, tree_attention_merge_kernel<DH>, kv_off, kv_len, B, m, Hq, Hkv, cache_rows,
                                max_kv_len, plan, ws, static_cast<__nv_bfloat16*>(out), lse) != cudaSuccess) {
             cudaGetLastError();
             return EAGLE2_ERR_CUDA;
         }
-        return EAGLE2_OK;
     }
     return EAGLE2_OK;
 }
@@ -949,7 +1120,10 @@ extern "C" int eagle2_tree_attention(const void* q, const void* k_cache, const v
         if (attention_ws_layout(B, Hkv, d, plan, ws, &w) > ws_bytes) return EAGLE2_ERR_WORKSPACE;
     }
     CUtensorMap k_map, v_map, q_map;
-    if (!make_cache_map(&k_map, k_cache, cache_rows, Hkv, d) || !make_cache_map(&v_map, v_cache, cache_rows, Hkv, d))
+    // a pair block loads 64 keys of every K tile (and all 128 keys of 64 V columns)
+    if (!make_cache_map(&k_map, k_cache, cache_rows, Hkv, d, plan.pair ? kTK / 2 : kTK) ||
+        !make_cache_map(&v_map, v_cache, cache_rows, Hkv, d, kTK,
+                        plan.pair ? CU_TENSOR_MAP_L2_PROMOTION_L2_128B : CU_TENSOR_MAP_L2_PROMOTION_L2_256B))
         return EAGLE2_ERR_CUDA;
     if (plan.q_tma) {
         if (!make_query_map(&q_map, q, B, m, Hq, Hkv, d)) return EAGLE2_ERR_CUDA;
@@ -957,14 +1131,15 @@ extern "C" int eagle2_tree_attention(const void* q, const void* k_cache, const v
         q_map = k_map;  // unused by the kernel
     }
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-#define EAGLE2_ATTN_CASE(DH_, MT_)                                                                        \
-    return launch_attention<DH_, MT_>(k_map, v_map, q_map, q, kv_off, kv_len, mask_bits, B, m, Hq, Hkv, cache_rows, \
-                                      max_kv_len, plan, scale, out, lse, w, d_status, st)
+#define EAGLE2_ATTN_CASE(DH_, MT_, PAIR_)                                                                       \
+    return launch_attention<DH_, MT_, PAIR_>(k_map, v_map, q_map, q, kv_off, kv_len, mask_bits, B, m, Hq, Hkv,      \
+                                             cache_rows, max_kv_len, plan, scale, out, lse, w, d_status, st)
     if (d == 64) {
-        if (plan.mt == 1) EAGLE2_ATTN_CASE(64, 1);
-        EAGLE2_ATTN_CASE(64, 2);
+        if (plan.mt == 1) EAGLE2_ATTN_CASE(64, 1, false);
+        EAGLE2_ATTN_CASE(64, 2, false);
     }
-    if (plan.mt == 1) EAGLE2_ATTN_CASE(128, 1);
-    EAGLE2_ATTN_CASE(128, 2);
+    if (plan.pair) EAGLE2_ATTN_CASE(128, 1, true);
+    if (plan.mt == 1) EAGLE2_ATTN_CASE(128, 1, false);
+    EAGLE2_ATTN_CASE(128, 2, false);
 #undef EAGLE2_ATTN_CASE
 }
