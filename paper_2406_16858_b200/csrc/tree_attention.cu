@@ -32,6 +32,7 @@ constexpr int kRowsPerTile = 128;     // M of every tcgen05.mma
 constexpr int kMaxTilesPerSplit = 16; // a block never streams more than 2048 keys
 constexpr int kTmemCols = 512;
 constexpr int kSlots = 2;             // score slots in tensor memory
+constexpr int kAttnThreads = 320;     // 8 softmax warps, the TMA warp, the MMA warp
 constexpr long long kWaitCycles = 1LL << 31;  // ~1 s bound of a barrier wait
 constexpr uint32_t kSuspendNs = 400;          // a waiting thread sleeps in hardware at most this long per try
 
@@ -59,8 +60,11 @@ static void attention_plan(int B, int m, int Hq, int Hkv, int d, int max_kv_len,
     p->per = p->per_tok * p->g;  // never above 256: n_rb >= m*g/256
     p->mt = p->per > kRowsPerTile ? 2 : 1;
     p->q_tma = (kRowsPerTile % p->g) == 0;
-    p->pair = 0 && (p->mt == 2 && p->q_tma && d == 128) ? 1 : 0;
     const long long items = (long long)B * Hkv * p->n_rb;
+    // Pairs pay off while the launch is short of blocks and every sequence is cut into several
+    // splits (they halve the query and partial traffic); a launch that fills the device without
+    // splitting is better served by independent blocks.
+    p->pair = (p->mt == 2 && p->q_tma && d == 128 && items * 2 <= 74) ? 1 : 0;
     const int tiles = (max_kv_len + m + kTK - 1) / kTK;
     long long s = (p->pair ? 74 : 148) / (items > 0 ? items : 1);
     if (s < 1) s = 1;
@@ -379,6 +383,18 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return *reinterpret_cast<const uint32_t*>(&v);
 }
 
+// Barrier over `nthreads` threads (named barrier `id`) that also tells every one of them whether
+// all of them passed `pred`: threads about to part ways over a failed wait learn it here together.
+__device__ __forceinline__ bool named_barrier_and(int id, int nthreads, bool pred) {
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\tsetp.ne.b32 p, %3, 0;\n\t"
+        "bar.red.and.pred q, %1, %2, p;\n\tselp.b32 %0, 1, 0, q;\n\t}"
+        : "=r"(r)
+        : "r"(id), "r"(nthreads), "r"((uint32_t)pred)
+        : "memory");
+    return r != 0;
+}
 __device__ __forceinline__ float max3(float a, float b, float c) {
     float r;
     asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
@@ -481,7 +497,7 @@ __device__ __forceinline__ void tile_visibility(unsigned long long mlo, unsigned
 }
 
 template <int DH, int MT, bool PAIR>
-__global__ void __launch_bounds__(MT * 128 + 64, 1)
+__global__ void __launch_bounds__(kAttnThreads, 1)
 tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map,
                       const __grid_constant__ CUtensorMap q_map, const __nv_bfloat16* __restrict__ q, const int64_t* __restrict__ kv_off,
                       const int32_t* __restrict__ kv_len, const uint64_t* __restrict__ mask_bits, int m, int Hq,
@@ -490,8 +506,11 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
     constexpr int HALVES = DH / 64;                    // 64-column (128-byte) panels per operand tile
     constexpr uint32_t kPanel = kTK * 128;             // bytes of one panel: 128 rows x 128 bytes
     constexpr uint32_t kTile = HALVES * kPanel;
-    constexpr int kSoftmaxThreads = MT * 128;
-    constexpr int kTmaWarp = MT * 4, kMmaWarp = MT * 4 + 1;
+    // Two row tiles: a warp group (4 warps, thread = row) per tile.  One row tile: both warp groups
+    // serve it, each thread taking half of the columns of its row (SPLIT).
+    constexpr bool SPLIT = MT == 1;
+    constexpr int kSoftmaxThreads = 256;
+    constexpr int kTmaWarp = 8, kMmaWarp = 9;
     constexpr uint32_t kIdescQK = instr_desc(kTK, false, PAIR ? 256 : 128);
     constexpr uint32_t kIdescPV = instr_desc(DH, true, PAIR ? 256 : 128);
     constexpr uint32_t kOCol = kSlots * kTK;           // first accumulator column of O
@@ -559,7 +578,7 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
         }
         for (int s = 0; s < kSlots; ++s) {
             mbar_init(smem_u32(&bars.s_full[s]), 1);
-            mbar_init(smem_u32(&bars.p_full[s]), PAIR ? 8 : 4);  // one arrival per softmax warp
+            mbar_init(smem_u32(&bars.p_full[s]), PAIR ? 16 : (SPLIT ? 8 : 4));  // one arrival per softmax warp
         }
         mbar_init(smem_u32(&bars.q_peer), 1);
         for (int s = 0; s < 4; ++s) {
@@ -754,7 +773,10 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
         }
     } else {
         // ===== softmax warps: thread = packed query row ============================================
-        const int wg = warp >> 2;                         // row tile of this warp group
+        __shared__ float s_xmax[2][2][128];               // SPLIT: row maxima of the two column halves
+        __shared__ float s_xsum[2][128];                  // SPLIT: row sums of the two column halves
+        const int wg = SPLIT ? 0 : warp >> 2;             // row tile of this warp group
+        const int half = SPLIT ? warp >> 2 : 0;           // SPLIT: which half of the columns
         const int r_tile = ((warp & 3) << 5) | lane;      // row inside the tile = tensor-memory lane
         const int r_blk = wg * 128 + r_tile;              // row inside the block
         const bool row_ok = r_blk < rows_here;
@@ -769,7 +791,7 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
             // query rows into shared memory by hand, 128-byte swizzled (chunk c of row r at
             // c ^ (r & 7)); all copies of a thread are in flight together, absent rows zero-filled
 #pragma unroll
-            for (int it = 0; it < DH / 8; ++it) {
+            for (int it = 0; it < MT * 128 * (DH / 8) / kSoftmaxThreads; ++it) {
                 const int idx = tid + it * kSoftmaxThreads;
                 const int r = idx / (DH / 8), c = idx % (DH / 8);
                 const bool live = r < rows_here;
@@ -790,13 +812,78 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
             const int i = j * MT + wg, slot = i % kSlots;
             ok = mbar_wait(smem_u32(&bars.s_full[slot]), (uint32_t)((i / kSlots) & 1), abort_flag);
             ok = __all_sync(0xffffffffu, ok);  // the tensor-memory accesses below need the whole warp
-            if (!ok) break;
+            if (!SPLIT && !ok) break;          // SPLIT: all eight warps leave together, a few lines down
             tc_fence_after();
             const uint32_t s_addr = tmem + lane_sel + (uint32_t)slot * kTK;
             const int key0 = (t_begin + j) * kTK;
             const bool tail = key0 + kTK > L;  // the tile holds tree keys or runs past the last key
             uint32_t vis[4] = {~0u, ~0u, ~0u, ~0u};
             if (tail) tile_visibility(mlo, mhi, key0, L, n_keys, vis);
+
+            if constexpr (SPLIT) {
+                // This thread owns columns [64*half, 64*half+64) of its row; the thread of the other
+                // warp group owns the rest.  They exchange their maxima through shared memory; the
+                // barrier of that exchange also separates every read of S from the writes of P.
+                ok = named_barrier_and(2, kSoftmaxThreads, ok);
+                if (!ok) break;
+                uint32_t bufa[32], bufb[32];
+                tmem_ld32(s_addr + half * 64, bufa);
+                tmem_ld32(s_addr + half * 64 + 32, bufb);
+                tc_wait_ld(bufa);
+                tc_wait_ld(bufb);
+                float mx = -INFINITY;
+                mx = tail ? chunk_rowmax<true>(bufa, vis[half * 2], mx) : chunk_rowmax<false>(bufa, 0, mx);
+                mx = tail ? chunk_rowmax<true>(bufb, vis[half * 2 + 1], mx) : chunk_rowmax<false>(bufb, 0, mx);
+                s_xmax[j & 1][half][r_tile] = mx;
+                asm volatile("bar.sync 2, %0;" ::"n"(kSoftmaxThreads) : "memory");
+                mx = fmaxf(mx, s_xmax[j & 1][half ^ 1][r_tile]) * scale_log2;
+
+                const float m_new = fmaxf(m_ref, mx);
+                const bool grow = m_new > m_ref + 8.f;
+                if (__any_sync(0xffffffffu, grow)) {
+                    const float factor = !grow ? 1.f : (m_ref == -INFINITY ? 0.f : ex2(m_ref - m_new));
+                    if (grow) m_ref = m_new, l_run *= factor;
+                    bool waited = true;
+                    if (j > 0)
+                        waited = mbar_wait(smem_u32(&bars.o_done[0][(j - 1) & 1]), (uint32_t)(((j - 1) >> 1) & 1), abort_flag);
+                    waited = __all_sync(0xffffffffu, waited);
+                    if (!waited) ok = false;  // every warp learns it at the top of the next tile
+                    if (j > 0 && waited) {
+                        tc_fence_after();
+                        const uint32_t o_half = tmem + lane_sel + kOCol + (uint32_t)half * (DH / 2);
+                        uint32_t orow[32];
+#pragma unroll
+                        for (int c4 = 0; c4 < DH / 64; ++c4) {
+                            tmem_ld32(o_half + c4 * 32, orow);
+                            tc_wait_ld(orow);
+#pragma unroll
+                            for (int c = 0; c < 32; ++c) orow[c] = __float_as_uint(__uint_as_float(orow[c]) * factor);
+                            tmem_st32(o_half + c4 * 32, orow);
+                        }
+                    }
+                }
+                const float neg_ref = m_ref == -INFINITY ? 0.f : -m_ref;
+                const float2 scale2 = make_float2(scale_log2, scale_log2), neg_ref2 = make_float2(neg_ref, neg_ref);
+                float2 sum_a = make_float2(0.f, 0.f), sum_b = make_float2(0.f, 0.f);
+                uint32_t pk[32];
+                if (tail) {
+                    chunk_probs<true>(bufa, vis[half * 2], scale2, neg_ref2, sum_a, sum_b, pk);
+                    chunk_probs<true>(bufb, vis[half * 2 + 1], scale2, neg_ref2, sum_a, sum_b, pk + 16);
+                } else {
+                    chunk_probs<false>(bufa, 0, scale2, neg_ref2, sum_a, sum_b, pk);
+                    chunk_probs<false>(bufb, 0, scale2, neg_ref2, sum_a, sum_b, pk + 16);
+                }
+                tmem_st32(s_addr + half * 32, pk);  // keys [64*half, +64) as 32 packed columns
+                l_run += (sum_a.x + sum_a.y) + (sum_b.x + sum_b.y);
+                tc_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) {
+                    if (PAIR) mbar_arrive_in(smem_u32(&bars.p_full[slot]), 0);
+                    else mbar_arrive(smem_u32(&bars.p_full[slot]));
+                }
+                continue;
+            }
 
             // Both passes walk the row in four 32-column chunks through two register buffers: the
             // load of the next chunk is in flight while the current one is processed.  A tile that
@@ -878,14 +965,20 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
         }
 
         // ---- epilogue: O rows leave tensor memory through shared memory, so that the global
-        // stores are whole contiguous rows.  Row tile 0 stages in the query region (both row tiles'
-        // Q.K^T are complete once any last P.V is), the other one - and a single tile - in the K ring.
+        // stores are whole contiguous rows.  Row tile 0 of two stages in the query region (both row
+        // tiles' Q.K^T are complete once any last P.V is), the other one - and a single tile - in the
+        // K ring.  The threads that share a staging area first agree that none of them gave up.
         ok = ok && mbar_wait(smem_u32(&bars.o_done[wg][(nt - 1) & 1]), (uint32_t)(((nt - 1) >> 1) & 1), abort_flag);
-        ok = __all_sync(0xffffffffu, ok);
+        const int epi_id = SPLIT ? 2 : 1 + wg, epi_threads = SPLIT ? kSoftmaxThreads : 128;
+        if (SPLIT) s_xsum[half][r_tile] = l_run;
+        ok = named_barrier_and(epi_id, epi_threads, ok);
         if (ok) {
             tc_fence_after();
-            const uint32_t o_addr = tmem + lane_sel + kOCol + (uint32_t)wg * DH;
-            const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+            constexpr int NCOL = SPLIT ? DH / 2 : DH;          // columns of O this thread owns
+            const int col0 = half * NCOL;
+            const uint32_t o_addr = tmem + lane_sel + kOCol + (uint32_t)wg * DH + (uint32_t)col0;
+            const float l_tot = SPLIT ? l_run + s_xsum[half ^ 1][r_tile] : l_run;
+            const float inv = l_tot > 0.f ? 1.f / l_tot : 0.f;
             unsigned char* stage = smem_gen + ((MT == 2 && wg == 0) ? 0u : (sK - smem_base));
             // a staged row is DH fp32 (partial) or DH bf16 (final); 16-byte chunk c of row r sits at
             // chunk c ^ (r mod chunks-per-row), which keeps both the row-wise writes and the
@@ -893,7 +986,7 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
             const int row_bytes = direct ? DH * 2 : DH * 4;
             const int cmask = row_bytes / 16 - 1;
 #pragma unroll
-            for (int c4 = 0; c4 < DH / 32; ++c4) {
+            for (int c4 = 0; c4 < NCOL / 32; ++c4) {
                 uint32_t orow[32];
                 tmem_ld32(o_addr + c4 * 32, orow);
                 tc_wait_ld(orow);
@@ -906,31 +999,32 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
                         v.y = pack_bf16(__uint_as_float(orow[c + 2]) * inv, __uint_as_float(orow[c + 3]) * inv);
                         v.z = pack_bf16(__uint_as_float(orow[c + 4]) * inv, __uint_as_float(orow[c + 5]) * inv);
                         v.w = pack_bf16(__uint_as_float(orow[c + 6]) * inv, __uint_as_float(orow[c + 7]) * inv);
-                        const int chunk = c4 * 4 + (c >> 3);
+                        const int chunk = (col0 + c4 * 32 + c) >> 3;
                         *reinterpret_cast<uint4*>(srow + (((chunk ^ r_tile) & cmask) << 4)) = v;
                     }
                 } else {
 #pragma unroll
                     for (int c = 0; c < 32; c += 4) {
-                        const int chunk = c4 * 8 + (c >> 2);
+                        const int chunk = (col0 + c4 * 32 + c) >> 2;
                         *reinterpret_cast<uint4*>(srow + (((chunk ^ r_tile) & cmask) << 4)) =
                             make_uint4(orow[c], orow[c + 1], orow[c + 2], orow[c + 3]);
                     }
                 }
             }
-            if (row_ok) {
+            if (row_ok && half == 0) {
                 if (direct) {
-                    if (lse) lse[((long long)b * Hq + hq) * m + tok] = (m_ref + log2f(l_run)) * 0.69314718055994531f;
+                    if (lse) lse[((long long)b * Hq + hq) * m + tok] = (m_ref + log2f(l_tot)) * 0.69314718055994531f;
                 } else {
-                    ws.ml[part_row0 + r_blk] = make_float2(m_ref, l_run);
+                    ws.ml[part_row0 + r_blk] = make_float2(m_ref, l_tot);
                 }
             }
-            asm volatile("bar.sync %0, 128;" ::"r"(1 + wg) : "memory");  // the row tile's four warps
+            asm volatile("bar.sync %0, %1;" ::"r"(epi_id), "r"(epi_threads) : "memory");  // rows are staged
             const int rows_tile = min(128, rows_here - wg * 128);
             const int lanes_per_row = row_bytes / 16;       // 16 or 32 (8 for a 64-wide bf16 row)
             const int rows_per_pass = 32 / lanes_per_row;
             const int sub = lane / lanes_per_row, cl = lane % lanes_per_row;
-            for (int r = (warp & 3) * rows_per_pass + sub; r < rows_tile; r += 4 * rows_per_pass) {
+            const int cw = SPLIT ? warp : (warp & 3), ncw = SPLIT ? 8 : 4;  // copying warps of this tile
+            for (int r = cw * rows_per_pass + sub; r < rows_tile; r += ncw * rows_per_pass) {
                 const uint4 v = *reinterpret_cast<const uint4*>(stage + (size_t)r * row_bytes + (((cl ^ r) & cmask) << 4));
                 if (direct) {
                     const int p2 = row0 + wg * 128 + r;
@@ -1053,7 +1147,7 @@ static int launch_attention(const CUtensorMap& k_map, const CUtensorMap& v_map, 
     if (blocks > 0x7fffffffLL) return EAGLE2_ERR_SHAPE;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)blocks, 1, 1);
-    cfg.blockDim = dim3(MT * 128 + 64, 1, 1);
+    cfg.blockDim = dim3(kAttnThreads, 1, 1);
     cfg.dynamicSmemBytes = plan.smem;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
