@@ -106,6 +106,8 @@ accept_greedy_kernel(const float* __restrict__ target_logits, long long t_stride
     __shared__ int s_arg[EAGLE2_MAX_M + 1];
     __shared__ int s_par[EAGLE2_MAX_M], s_tok[EAGLE2_MAX_M];
 
+    chain_wait();
+    chain_release();
     const int chunk = blockIdx.x % chunks;
     const int row = (blockIdx.x / chunks) % (m + 1);
     const int b = blockIdx.x / (chunks * (m + 1));
@@ -233,6 +235,8 @@ accept_chain_kernel(const float* __restrict__ target_logits, long long t_stride,
                     const int32_t* __restrict__ sel_index, const int32_t* __restrict__ sel_parent,
                     const int32_t* __restrict__ sel_token, const int32_t* __restrict__ n_sel, int V,
                     int k, int m, int R, int slice, float inv_t, AcceptWs ws, int32_t* d_status) {
+    chain_wait();
+    chain_release();
     cg::cluster_group cluster = cg::this_cluster();
     const int cs = (int)cluster.num_blocks(), me = (int)cluster.block_rank();
     const int b = blockIdx.x / cs;
@@ -543,6 +547,8 @@ accept_bonus_kernel(const float* __restrict__ target_logits, long long t_stride,
     __shared__ double s_scan[kScanThreads];
     __shared__ int s_flag, s_pick;
 
+    chain_wait();
+    chain_release();
     const int chunk = blockIdx.x % chunks;
     const int b = blockIdx.x / chunks;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -807,22 +813,17 @@ extern "C" int eagle2_accept(const float* target_logits, long long t_stride,
         if (blocks > 0x7fffffffLL) return EAGLE2_ERR_SHAPE;
 #define EAGLE2_GREEDY_CASE(VPT_)                                                                         \
     case VPT_:                                                                                           \
-        if (vec_t)                                                                                       \
-            accept_greedy_kernel<VPT_, true><<<(unsigned)blocks, kScanThreads, 0, st>>>(                 \
-                target_logits, t_stride, sel_parent, sel_token, n_sel, V, D, m, gchunks, acc_len,        \
-                acc_path, bonus_token, w, d_status);                                                     \
-        else                                                                                             \
-            accept_greedy_kernel<VPT_, false><<<(unsigned)blocks, kScanThreads, 0, st>>>(                \
-                target_logits, t_stride, sel_parent, sel_token, n_sel, V, D, m, gchunks, acc_len,        \
-                acc_path, bonus_token, w, d_status);                                                     \
-        break;
+        return launch_chained(vec_t ? accept_greedy_kernel<VPT_, true> : accept_greedy_kernel<VPT_, false>,       \
+                              dim3((unsigned)blocks), dim3(kScanThreads), 0, st, 1, target_logits, t_stride,     \
+                              sel_parent, sel_token, n_sel, V, D, m, gchunks, acc_len, acc_path, bonus_token, w, \
+                              d_status);
         switch (gvpt) {
             EAGLE2_GREEDY_CASE(1)
             EAGLE2_GREEDY_CASE(2)
             EAGLE2_GREEDY_CASE(4)
         }
 #undef EAGLE2_GREEDY_CASE
-        return launch_result();
+        return EAGLE2_ERR_SHAPE;
     }
 
     // ---- temperature > 0 --------------------------------------------------------------------------
@@ -842,45 +843,25 @@ extern "C" int eagle2_accept(const float* target_logits, long long t_stride,
     if (dyn > 40 * 1024 &&
         cudaFuncSetAttribute(chain, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) != cudaSuccess)
         return EAGLE2_ERR_CUDA;
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)(B * cs), (unsigned)R, 1);
-    cfg.blockDim = dim3(kChainThreads, 1, 1);
-    cfg.dynamicSmemBytes = dyn;
-    cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = (unsigned)cs;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, chain, target_logits, t_stride, draft_logits_all, d_stride, sel_index,
-                           sel_parent, sel_token, n_sel, V, k, m, R, slice, inv_t, w,
-                           d_status) != cudaSuccess) {
-        cudaGetLastError();
+    if (launch_chained(chain, dim3((unsigned)(B * cs), (unsigned)R, 1), dim3(kChainThreads), dyn, st, (unsigned)cs,
+                       target_logits, t_stride, draft_logits_all, d_stride, sel_index, sel_parent, sel_token, n_sel, V,
+                       k, m, R, slice, inv_t, w, d_status) != EAGLE2_OK)
         return EAGLE2_ERR_CUDA;
-    }
 
     const long long blocks = (long long)B * bchunks;
     if (blocks > 0x7fffffffLL) return EAGLE2_ERR_SHAPE;
 #define EAGLE2_BONUS_CASE(VPT_)                                                                          \
     case VPT_:                                                                                           \
-        if (vec)                                                                                         \
-            accept_bonus_kernel<VPT_, true><<<(unsigned)blocks, kScanThreads, 0, st>>>(                  \
-                target_logits, t_stride, draft_logits_all, d_stride, sel_index, sel_parent, sel_token,   \
-                n_sel, u_accept, u_bonus, V, k, D, m, R, bchunks, inv_t, acc_len, acc_path, bonus_token, \
-                w, d_status);                                                                            \
-        else                                                                                             \
-            accept_bonus_kernel<VPT_, false><<<(unsigned)blocks, kScanThreads, 0, st>>>(                 \
-                target_logits, t_stride, draft_logits_all, d_stride, sel_index, sel_parent, sel_token,   \
-                n_sel, u_accept, u_bonus, V, k, D, m, R, bchunks, inv_t, acc_len, acc_path, bonus_token, \
-                w, d_status);                                                                            \
-        break;
+        return launch_chained(vec ? accept_bonus_kernel<VPT_, true> : accept_bonus_kernel<VPT_, false>,           \
+                              dim3((unsigned)blocks), dim3(kScanThreads), 0, st, 1, target_logits, t_stride,     \
+                              draft_logits_all, d_stride, sel_index, sel_parent, sel_token, n_sel, u_accept,     \
+                              u_bonus, V, k, D, m, R, bchunks, inv_t, acc_len, acc_path, bonus_token, w,         \
+                              d_status);
     switch (bvpt) {
         EAGLE2_BONUS_CASE(1)
         EAGLE2_BONUS_CASE(2)
         EAGLE2_BONUS_CASE(4)
     }
 #undef EAGLE2_BONUS_CASE
-    return launch_result();
+    return EAGLE2_ERR_SHAPE;
 }

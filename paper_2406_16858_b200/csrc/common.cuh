@@ -24,6 +24,40 @@ inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_
 
 inline int launch_result() { return cudaGetLastError() == cudaSuccess ? EAGLE2_OK : EAGLE2_ERR_CUDA; }
 
+// Every kernel of the library is launched with programmatic stream serialisation and begins with
+// chain_wait(): it may be scheduled while its predecessor in the stream is still draining, and it
+// touches no global memory before that predecessor (and, by induction, everything before it) has
+// completed.  chain_release() lets the successor be scheduled in turn.  After a kernel that never
+// releases, the successor simply starts when that kernel ends.
+#ifdef __CUDACC__
+__device__ __forceinline__ void chain_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void chain_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline int launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                          unsigned cluster_x, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = cluster_x;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = cluster_x > 1 ? 2 : 1;
+    if (cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...) != cudaSuccess) {
+        cudaGetLastError();
+        return EAGLE2_ERR_CUDA;
+    }
+    return EAGLE2_OK;
+}
+#endif
+
 #ifdef __CUDACC__
 
 __device__ __forceinline__ void raise_status(int32_t* d_status, int bits) {

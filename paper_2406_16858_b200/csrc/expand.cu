@@ -76,6 +76,8 @@ expand_kernel(const float* __restrict__ draft_logits, long long batch_stride, in
     __shared__ int s_flag;
     __shared__ unsigned long long s_rank[EAGLE2_MAX_K * EAGLE2_MAX_K];  // the new candidates' value codes
 
+    chain_wait();
+    chain_release();
     const int chunk = blockIdx.x % chunks;
     const int row = (blockIdx.x / chunks) % n_s;
     const int b = blockIdx.x / (chunks * n_s);
@@ -255,10 +257,8 @@ static int launch_expand(const float* draft_logits, long long batch_stride, int 
                          cudaStream_t stream) {
     auto kern = expand_kernel<VPT, VEC>;
     const long long blocks = (long long)B * n_s * chunks;
-    kern<<<(unsigned)blocks, kScanThreads, 0, stream>>>(draft_logits, batch_stride, V, k, D, s, n_s,
-                                                          chunks, tree_token, tree_parent, tree_value,
-                                                          frontier, ws, d_status);
-    return launch_result();
+    return launch_chained(kern, dim3((unsigned)blocks), dim3(kScanThreads), 0, stream, 1, draft_logits, batch_stride, V,
+                          k, D, s, n_s, chunks, tree_token, tree_parent, tree_value, frontier, ws, d_status);
 }
 
 // Scratch of eagle2_expand_static: lives in every context that loads the library, until exit.

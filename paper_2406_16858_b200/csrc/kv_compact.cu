@@ -27,6 +27,8 @@ kv_compact_kernel(void* const* __restrict__ k_layers, void* const* __restrict__ 
                   const int64_t* __restrict__ kv_off, const int32_t* __restrict__ kv_len,
                   const int32_t* __restrict__ acc_path, const int32_t* __restrict__ acc_len, int m,
                   int D, int segs, int seg_blocks) {
+    chain_wait();
+    chain_release();
     const int b = blockIdx.x / seg_blocks;
     const int seg = (blockIdx.x % seg_blocks) * kCompactThreads + threadIdx.x;
     const int layer = blockIdx.y >> 1, which = blockIdx.y & 1;
@@ -49,6 +51,8 @@ kv_compact_kernel(void* const* __restrict__ k_layers, void* const* __restrict__ 
 __global__ void kv_len_advance_kernel(int32_t* __restrict__ kv_len, const int32_t* __restrict__ acc_path,
                                       const int32_t* __restrict__ acc_len, int B, int m, int D,
                                       int32_t* d_status) {
+    chain_wait();
+    chain_release();
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
     if (b >= B) return;
     const int len = acc_len[b];
@@ -80,10 +84,10 @@ extern "C" int eagle2_kv_compact(void* const* k_layers, void* const* v_layers, i
     if (n_layers > 0) {
         if ((long long)B * seg_blocks > 0x7fffffffLL) return EAGLE2_ERR_SHAPE;
         dim3 grid((unsigned)(B * seg_blocks), (unsigned)(n_layers * 2));
-        kv_compact_kernel<<<grid, kCompactThreads, 0, st>>>(k_layers, v_layers, kv_off, kv_len, acc_path,
-                                                            acc_len, m, D, segs, seg_blocks);
-        if (launch_result() != EAGLE2_OK) return EAGLE2_ERR_CUDA;
+        if (launch_chained(kv_compact_kernel, grid, dim3(kCompactThreads), 0, st, 1, k_layers, v_layers, kv_off,
+                           kv_len, acc_path, acc_len, m, D, segs, seg_blocks) != EAGLE2_OK)
+            return EAGLE2_ERR_CUDA;
     }
-    kv_len_advance_kernel<<<(B + 127) / 128, 128, 0, st>>>(kv_len, acc_path, acc_len, B, m, D, d_status);
-    return launch_result();
+    return launch_chained(kv_len_advance_kernel, dim3((B + 127) / 128), dim3(128), 0, st, 1, kv_len, acc_path, acc_len,
+                          B, m, D, d_status);
 }

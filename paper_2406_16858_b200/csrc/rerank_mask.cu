@@ -33,6 +33,8 @@ rerank_kernel(const int32_t* __restrict__ tree_token, const int32_t* __restrict_
     int32_t* s_flat = s_par + N;                                                // [N] flat position or -1
     __shared__ int s_scan[kRerankThreads];
 
+    chain_wait();
+    chain_release();
     const int b = blockIdx.x, tid = threadIdx.x;
     const int32_t* tok = tree_token + (long long)b * N;
     const int32_t* par = tree_parent + (long long)b * N;
@@ -184,6 +186,8 @@ tree_mask_kernel(const int32_t* __restrict__ sel_parent, const int32_t* __restri
                  uint64_t* __restrict__ mask_bits, uint8_t* __restrict__ mask_dense,
                  int32_t* __restrict__ pos_ids, int32_t* d_status) {
     __shared__ int32_t s_par[EAGLE2_MAX_M];
+    chain_wait();
+    chain_release();
     const int b = blockIdx.x, i = threadIdx.x;
     const int W = (m + 63) / 64;
     const int ns = n_sel[b];
@@ -244,10 +248,9 @@ extern "C" int eagle2_rerank(const int32_t* tree_token, const int32_t* tree_pare
         cudaFuncSetAttribute(rerank_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) !=
             cudaSuccess)
         return EAGLE2_ERR_CUDA;
-    rerank_kernel<<<B, kRerankThreads, dyn, reinterpret_cast<cudaStream_t>(stream)>>>(
-        tree_token, tree_parent, tree_value, k, N, P, m, keep, sel_index, sel_parent, sel_token, sel_depth,
-        n_sel, d_status);
-    return launch_result();
+    return launch_chained(rerank_kernel, dim3(B), dim3(kRerankThreads), dyn, reinterpret_cast<cudaStream_t>(stream), 1,
+                          tree_token, tree_parent, tree_value, k, N, P, m, keep, sel_index, sel_parent, sel_token,
+                          sel_depth, n_sel, d_status);
 }
 
 extern "C" int eagle2_tree_mask(const int32_t* sel_parent, const int32_t* sel_depth,
@@ -259,7 +262,6 @@ extern "C" int eagle2_tree_mask(const int32_t* sel_parent, const int32_t* sel_de
     if (B < 0 || m < 1 || m > EAGLE2_MAX_M) return EAGLE2_ERR_SHAPE;
     if (!aligned(mask_bits, 8)) return EAGLE2_ERR_ALIGN;
     if (B == 0) return EAGLE2_OK;
-    tree_mask_kernel<<<B, EAGLE2_MAX_M, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
-        sel_parent, sel_depth, n_sel, kv_len, m, mask_bits, mask_dense, pos_ids, d_status);
-    return launch_result();
+    return launch_chained(tree_mask_kernel, dim3(B), dim3(EAGLE2_MAX_M), 0, reinterpret_cast<cudaStream_t>(stream), 1,
+                          sel_parent, sel_depth, n_sel, kv_len, m, mask_bits, mask_dense, pos_ids, d_status);
 }

@@ -524,6 +524,8 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_abort;
 
+    chain_wait();
+    chain_release();  // the merge kernel of this call (or whatever follows) may be scheduled from here on
     const int g = plan.g, M = plan.M, S = plan.splits, NST = plan.stages;
     const uint32_t rank = PAIR ? cluster_ctarank() : 0u;  // 0: the block that issues the pair's MMAs
     int bid = PAIR ? blockIdx.x >> 1 : blockIdx.x;
@@ -1039,8 +1041,6 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
     }
 
     // ---- teardown ----------------------------------------------------------------------------------
-    // the merge kernel of this call may be scheduled from here on (it waits for this grid to finish)
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     tc_fence_before();
     if (PAIR) cluster_sync_all();  // tensor memory is released by both blocks together
     else __syncthreads();
@@ -1061,8 +1061,8 @@ __global__ void __launch_bounds__(256)
 tree_attention_merge_kernel(const int64_t* __restrict__ kv_off, const int32_t* __restrict__ kv_len, int B, int m,
                             int Hq, int Hkv, long long cache_rows, int max_kv_len, AttnPlan plan, AttnWs ws, __nv_bfloat16* __restrict__ out,
                             float* __restrict__ lse) {
-    // launched with programmatic stream serialisation: wait for the attention kernel's writes
-    asm volatile("griddepcontrol.wait;" ::: "memory");
+    chain_wait();  // the attention kernel's partials are complete
+    chain_release();
     const int warp_global = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
     const int g = plan.g, S = plan.splits;
     const long long total = (long long)B * Hkv * plan.M;
@@ -1145,44 +1145,17 @@ static int launch_attention(const CUtensorMap& k_map, const CUtensorMap& v_map, 
     }
     const long long blocks = (long long)B * Hkv * plan.n_rb * plan.splits * (PAIR ? 2 : 1);
     if (blocks > 0x7fffffffLL) return EAGLE2_ERR_SHAPE;
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)blocks, 1, 1);
-    cfg.blockDim = dim3(kAttnThreads, 1, 1);
-    cfg.dynamicSmemBytes = plan.smem;
-    cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = PAIR ? 2 : 1;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, kern, k_map, v_map, q_map, static_cast<const __nv_bfloat16*>(q), kv_off, kv_len,
-                           mask_bits, m, Hq, Hkv, cache_rows, max_kv_len, plan, scale * 1.4426950408889634f,
-                           static_cast<__nv_bfloat16*>(out), lse, ws, d_status) != cudaSuccess) {
-        cudaGetLastError();
+    if (launch_chained(kern, dim3((unsigned)blocks), dim3(kAttnThreads), plan.smem, st, PAIR ? 2u : 1u, k_map, v_map, q_map,
+                       static_cast<const __nv_bfloat16*>(q), kv_off, kv_len, mask_bits, m, Hq, Hkv, cache_rows, max_kv_len,
+                       plan, scale * 1.4426950408889634f, static_cast<__nv_bfloat16*>(out), lse, ws, d_status) != EAGLE2_OK)
         return EAGLE2_ERR_CUDA;
-    }
     if (plan.splits > 1) {
         const long long warps = (long long)B * Hkv * plan.M;
         const long long mblocks = (warps + 7) / 8;
         if (mblocks > 0x7fffffffLL) return EAGLE2_ERR_SHAPE;
-        // the merge kernel may be scheduled while the attention kernel still runs; it starts with
-        // griddepcontrol.wait, which holds it until that kernel's writes are complete
-        cudaLaunchConfig_t mcfg = {};
-        mcfg.gridDim = dim3((unsigned)mblocks, 1, 1);
-        mcfg.blockDim = dim3(256, 1, 1);
-        mcfg.stream = st;
-        cudaLaunchAttribute mattr[1];
-        mattr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        mattr[0].val.programmaticStreamSerializationAllowed = 1;
-        mcfg.attrs = mattr;
-        mcfg.numAttrs = 1;
-        if (cudaLaunchKernelEx(&mcfg, tree_attention_merge_kernel<DH>, kv_off, kv_len, B, m, Hq, Hkv, cache_rows,
-                               max_kv_len, plan, ws, static_cast<__nv_bfloat16*>(out), lse) != cudaSuccess) {
-            cudaGetLastError();
+        if (launch_chained(tree_attention_merge_kernel<DH>, dim3((unsigned)mblocks), dim3(256), 0, st, 1, kv_off, kv_len, B, m,
+                           Hq, Hkv, cache_rows, max_kv_len, plan, ws, static_cast<__nv_bfloat16*>(out), lse) != EAGLE2_OK)
             return EAGLE2_ERR_CUDA;
-        }
     }
     return EAGLE2_OK;
 }
