@@ -46,6 +46,8 @@ struct AttnPlan {
     int splits;     // KV splits per sequence (blocks of the launch)
     int per_split;  // K/V tiles per split
     int stages;     // K/V ring depth
+    int setup_first;  // 1: blocks set up barriers and tensor memory before they wait for the preceding
+                      // kernel (worth it when no block of the launch is expected to be idle)
     int pair;       // 1: two blocks (a cluster on one TPC) share every K/V tile through cta_group::2
                     // MMAs: each holds 128 of the 256 query rows, half of each K tile's keys and
                     // half of each V tile's columns
@@ -78,6 +80,7 @@ static void attention_plan(int B, int m, int Hq, int Hkv, int d, int max_kv_len,
     int stages = (int)((220 * 1024 - p->mt * unit) / (2 * unit));
     p->stages = stages > 4 ? 4 : (stages < 2 ? 2 : stages);
     p->smem = (p->mt + 2 * (size_t)p->stages) * unit + 1024;
+    p->setup_first = B == 1;  // ragged batches leave many splits without tiles: those leave at once
     if (p->pair) {  // per block: one 128-row query tile, half-size K and V stages
         p->stages = 4;
         p->smem = unit + 4 * unit + 1024;
@@ -524,10 +527,61 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_abort;
 
-    chain_wait();
-    chain_release();  // the merge kernel of this call (or whatever follows) may be scheduled from here on
     const int g = plan.g, M = plan.M, S = plan.splits, NST = plan.stages;
     const uint32_t rank = PAIR ? cluster_ctarank() : 0u;  // 0: the block that issues the pair's MMAs
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t sQ = smem_base;
+    const uint32_t sK = sQ + MT * kTile;
+    const uint32_t sV = sK + (uint32_t)NST * kKTile;
+    unsigned char* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+
+    // ---- set-up: barriers, tensor memory (reads nothing an earlier kernel could have written) ----
+    auto set_up = [&]() {
+        if (tid == 0) {
+            s_abort = 0;
+            mbar_init(smem_u32(&bars.q_full), plan.q_tma ? 1 : kSoftmaxThreads);
+            for (int s = 0; s < 4; ++s) {
+                mbar_init(smem_u32(&bars.k_full[s]), 1);
+                mbar_init(smem_u32(&bars.k_empty[s]), 1);
+                mbar_init(smem_u32(&bars.v_full[s]), 1);
+                mbar_init(smem_u32(&bars.v_empty[s]), 1);
+            }
+            for (int s = 0; s < kSlots; ++s) {
+                mbar_init(smem_u32(&bars.s_full[s]), 1);
+                mbar_init(smem_u32(&bars.p_full[s]), PAIR ? 16 : (SPLIT ? 8 : 4));  // one arrival per softmax warp
+            }
+            mbar_init(smem_u32(&bars.q_peer), 1);
+            for (int s = 0; s < 4; ++s) {
+                mbar_init(smem_u32(&bars.k_peer[s]), 1);
+                mbar_init(smem_u32(&bars.v_peer[s]), 1);
+            }
+            for (int s = 0; s < 4; ++s) mbar_init(smem_u32(&bars.o_done[s >> 1][s & 1]), 1);
+            fence_barrier_init();
+        }
+        if (warp == kMmaWarp) {
+            if (PAIR) {
+                tmem_alloc2(smem_u32(&s_tmem_base), kTmemCols);
+                tmem_relinquish2();
+            } else {
+                tmem_alloc(smem_u32(&s_tmem_base), kTmemCols);
+                tmem_relinquish();
+            }
+        }
+        if (warp == kTmaWarp && lane == 0) {
+            asm volatile("prefetch.tensormap [%0];" ::"l"(&k_map) : "memory");
+            asm volatile("prefetch.tensormap [%0];" ::"l"(&v_map) : "memory");
+            if (plan.q_tma) asm volatile("prefetch.tensormap [%0];" ::"l"(&q_map) : "memory");
+        }
+        tc_fence_before();
+        if (PAIR) cluster_sync_all();  // both blocks' barriers exist before either signals the other
+        else __syncthreads();
+        tc_fence_after();
+    };
+    if (plan.setup_first) set_up();
+    chain_wait();
+    chain_release();  // the merge kernel of this call (or whatever follows) may be scheduled from here on
+
     int bid = PAIR ? blockIdx.x >> 1 : blockIdx.x;
     const int split = bid % S;
     bid /= S;
@@ -536,7 +590,6 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
     const int hk = bid % Hkv;
     const int b = bid / Hkv;
 
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int L_raw = kv_len[b];
     const long long row_base = kv_off[b];
     const bool overflow = !sequence_ok(L_raw, row_base, m, max_kv_len, cache_rows);
@@ -560,58 +613,16 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
         raise_status(d_status, EAGLE2_STATUS_KV_OVERFLOW);
     // a split past the sequence's last tile (never merged), or a rejected sequence: both blocks of a
     // pair take the same decision
-    if (nt <= 0 || rows_blk <= 0) return;
-
-    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t sQ = smem_base;
-    const uint32_t sK = sQ + MT * kTile;
-    const uint32_t sV = sK + (uint32_t)NST * kKTile;
-    unsigned char* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
-
-    // ---- set-up: barriers, tensor memory --------------------------------------------------------
-    if (tid == 0) {
-        s_abort = 0;
-        mbar_init(smem_u32(&bars.q_full), plan.q_tma ? 1 : kSoftmaxThreads);
-        for (int s = 0; s < 4; ++s) {
-            mbar_init(smem_u32(&bars.k_full[s]), 1);
-            mbar_init(smem_u32(&bars.k_empty[s]), 1);
-            mbar_init(smem_u32(&bars.v_full[s]), 1);
-            mbar_init(smem_u32(&bars.v_empty[s]), 1);
-        }
-        for (int s = 0; s < kSlots; ++s) {
-            mbar_init(smem_u32(&bars.s_full[s]), 1);
-            mbar_init(smem_u32(&bars.p_full[s]), PAIR ? 16 : (SPLIT ? 8 : 4));  // one arrival per softmax warp
-        }
-        mbar_init(smem_u32(&bars.q_peer), 1);
-        for (int s = 0; s < 4; ++s) {
-            mbar_init(smem_u32(&bars.k_peer[s]), 1);
-            mbar_init(smem_u32(&bars.v_peer[s]), 1);
-        }
-        for (int s = 0; s < 4; ++s) mbar_init(smem_u32(&bars.o_done[s >> 1][s & 1]), 1);
-        fence_barrier_init();
+    const bool active = nt > 0 && rows_blk > 0;
+    if (!plan.setup_first) {
+        if (!active) return;
+        set_up();
     }
-    if (warp == kMmaWarp) {
-        if (PAIR) {
-            tmem_alloc2(smem_u32(&s_tmem_base), kTmemCols);
-            tmem_relinquish2();
-        } else {
-            tmem_alloc(smem_u32(&s_tmem_base), kTmemCols);
-            tmem_relinquish();
-        }
-    }
-    if (warp == kTmaWarp && lane == 0) {
-        asm volatile("prefetch.tensormap [%0];" ::"l"(&k_map) : "memory");
-        asm volatile("prefetch.tensormap [%0];" ::"l"(&v_map) : "memory");
-        if (plan.q_tma) asm volatile("prefetch.tensormap [%0];" ::"l"(&q_map) : "memory");
-    }
-    tc_fence_before();
-    if (PAIR) cluster_sync_all();  // both blocks' barriers exist before either signals the other
-    else __syncthreads();
-    tc_fence_after();
     const uint32_t tmem = s_tmem_base;
     volatile int* abort_flag = &s_abort;
     const int n_items = nt * MT;  // item i = (tile i / MT, row tile i % MT), score slot i % 2
 
+    if (active) {
     if (warp == kTmaWarp) {
         // ===== TMA producer =======================================================================
         if (lane == 0) {
@@ -1039,6 +1050,8 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
             }
         }
     }
+
+    }  // active
 
     // ---- teardown ----------------------------------------------------------------------------------
     tc_fence_before();
