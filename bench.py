@@ -34,7 +34,7 @@ N_SETS = 4  # rotating logit sets: 4 x (draft + target rows) is larger than the 
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one tree-attention launch, from the ncu capture
 # summarised under profiles/ (None: not captured for that workload)
-NCU_DRAM_BYTES_PER_LAUNCH = {}
+NCU_DRAM_BYTES_PER_LAUNCH = {"llama3_8b": 17591808}
 
 
 def _peaks():
@@ -441,7 +441,7 @@ def run_ours(args):
         "e2e": {"value": ms_e2e * 1e3 / (e2e_steps * world), "unit": "us", "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h},
         "gpu_launches": buf.launches_per_cycle() * K,
-        "roofline": {"kernel": "tree_attention (+ split merge), one launch per layer", "bound": "hbm",
+        "roofline": {"kernel": "tree_attention_kernel + tree_attention_merge_kernel, one call per layer", "bound": "hbm",
                      "achieved": achieved, "peak": hbm_peak, "unit": "GB/s", "frac": achieved / hbm_peak,
                      "peak_kind": f"of {peak_kind}", "traffic": None, "us_per_launch": us_attn,
                      "algorithmic_bytes_per_launch": attn_bytes},
