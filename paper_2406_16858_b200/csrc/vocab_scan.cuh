@@ -137,8 +137,10 @@ constexpr int kCandCap = 512;  // candidate keys a block can stage for the filte
 struct TopkScratch {
     unsigned long long cand[kCandCap];
     unsigned long long exact[kScanWarps * EAGLE2_MAX_K];
+    unsigned long long win[EAGLE2_MAX_K];  // winners of an exact selection over one tile
     int count;
     int overflow;
+    float thr;  // value of the block's k-th best key so far (-inf: fewer than k keys yet)
 };
 
 // Block-level top-k (k <= 32) of the chunk elements x[] held in registers, written by warp 0 to

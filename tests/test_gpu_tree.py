@@ -98,6 +98,41 @@ def test_odd_shapes_scalar_and_vector_paths(V, k, D, B):
         _check_selection(want, k, D, m, kv_len=np.arange(B, dtype=np.int32) * 7)
 
 
+@pytest.mark.parametrize("kind", ["random", "ascending", "descending", "sawtooth", "plateaus", "late_spike"])
+def test_many_tiles_per_block_and_ordered_rows(kind):
+    """160 rows at the second step: each block streams several tiles of a row, keeps a running
+    k-th-best threshold and, on ordered input, overflows its candidate list and ranks tiles exactly."""
+    V, k, D, B = 70001, 5, 2, 32
+    R = ref.n_draft_rows(k, D)
+    rng = np.random.default_rng(len(kind))
+    idx = np.arange(V, dtype=np.float64)
+    slope = 1.0 + 0.1 * rng.random((B, R, 1))
+    noise = 1e-4 * rng.standard_normal((B, R, V))
+    if kind == "random":
+        draft = 2.0 * rng.standard_normal((B, R, V))
+    elif kind == "ascending":
+        draft = 1e-3 * idx * slope + noise
+    elif kind == "descending":
+        draft = -1e-3 * idx * slope + noise
+    elif kind == "sawtooth":
+        draft = 1e-3 * (idx % 6000) * slope + noise  # ramps that straddle the 4096-token tiles
+    elif kind == "plateaus":
+        draft = np.floor(1.5 * rng.standard_normal((B, R, V)))  # a handful of levels, thousands of ties
+    else:
+        draft = 0.1 * rng.standard_normal((B, R, V))
+        draft[:, :, V - 3:] += 9.0  # the winners sit in the ragged last tile
+        draft[:, :, 4096 * 7 + 5] += 8.0
+    draft = draft.astype(np.float32)
+    want = ref.build_tree(draft, V, k, D)
+    gpu = GpuTree(B, V, k, D).expand_all(dev(draft))
+    # with two steps every token choice compares raw fp32 logits of one row: exact, ties included
+    assert (host(gpu.token) == want.token).all()
+    assert (host(gpu.parent) == want.parent).all()
+    assert np.abs(host(gpu.value) - want.value).max() < 3e-6
+    cfg = get_config("tiny", B=B, V=V, k=k, D=D)
+    _check_tree(cfg, draft, gpu, want)
+
+
 def test_ties_and_negative_infinity_logits():
     V, k, D, B = 2048, 4, 2, 1
     draft = np.full((B, ref.n_draft_rows(k, D), V), -np.inf, np.float32)
