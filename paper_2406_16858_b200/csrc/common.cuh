@@ -119,9 +119,9 @@ __device__ __forceinline__ double warp_max_f64(double v) {
 // Arrival ticket: returns true in exactly one block, the last of `expected` to arrive, after every
 // other block's earlier global writes are visible to it.  The counter is left at zero.
 __device__ __forceinline__ bool last_block_arrives(int* counter, int expected, int* smem_flag) {
-    __threadfence();
     __syncthreads();
     if (threadIdx.x == 0) {
+        __threadfence();  // cumulative: covers the writes the barrier ordered before it
         const int t = atomicAdd(counter, 1);
         const int last = (t == expected - 1);
         if (last) *counter = 0;

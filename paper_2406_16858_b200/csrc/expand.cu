@@ -1,15 +1,16 @@
 // Step 1 of the hot path: draft-tree expansion (paper Section 4.1).
 //
 // One launch per expansion step.  Block (segment, row, sequence) streams its segment of one logit
-// row in tiles of 4096 tokens (next tile's loads in flight while the current one is processed),
-// keeps a per-thread running (max, sum exp) and a block list of top-k candidates filtered by the
-// value of the block's k-th best so far, and writes one partial per segment to the workspace.  The
+// row in tiles of 4096 tokens (two tiles of asynchronous copies in flight ahead of the one being processed); each
+// warp keeps per-thread running (max, sum exp) and its own short list of top-k candidates, and the
+// block writes one partial per segment to the workspace.  The
 // last block of a sequence to arrive merges the partials, a warp per row (fp64 log-sum-exp, top-k of
 // the segment winners), writes the new tree level (token, parent, value = parent value + log-prob)
 // and ranks the new candidates by value to produce the next frontier.
 #include <math.h>
 
 #include <mutex>
+#include <type_traits>
 
 #include "vocab_scan.cuh"
 
@@ -74,26 +75,7 @@ __device__ __forceinline__ unsigned long long order_code_f64(double x) {
     return (u >> 63) ? ~u : (u | 0x8000000000000000ull);
 }
 
-constexpr int kRing = 3;                                  // tiles in flight per block (vector path)
-constexpr long long kExpandWaitCycles = 1LL << 31;       // ~1 s bound of a wait for a tile
-
-__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-// one tile of a row, global -> shared, completion counted in bytes on an mbarrier
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-    asm volatile("cp.async.bulk.shared::cta.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
-                 : "memory");
-}
-__device__ __forceinline__ bool tile_landed(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.b32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
+constexpr int kWarpList = 64;  // candidate keys a warp holds between two tightenings of its threshold
 
 __device__ __forceinline__ float fast_ex2(float x) {
     float y;
@@ -101,6 +83,68 @@ __device__ __forceinline__ float fast_ex2(float x) {
     return y;
 }
 
+// The warp's candidate list (n <= 64 keys in shared memory, any order) is cut down to the entries
+// whose value reaches the k-th largest value in it: the 64 value codes (two per lane) are sorted
+// across the warp, the k-th gives the bar, ties at the bar stay.  Needs n >= k.  Returns the new n
+// (>= k) and the bar's code.
+__device__ __forceinline__ int warp_tighten(unsigned long long* list, int n, int k, uint32_t* bar_code) {
+    const int lane = threadIdx.x & 31;
+    const unsigned long long key0 = lane < n ? list[lane] : 0ull;
+    const unsigned long long key1 = lane + 32 < n ? list[lane + 32] : 0ull;
+    uint32_t c[2] = {(uint32_t)(key0 >> 32), (uint32_t)(key1 >> 32)};  // element r*32 + lane
+#pragma unroll
+    for (int size = 2; size <= 64; size <<= 1) {
+#pragma unroll
+        for (int stride = size >> 1; stride > 0; stride >>= 1) {
+            if (stride == 32) {  // partners sit in the same lane; descending overall
+                const uint32_t hi = max(c[0], c[1]), lo = min(c[0], c[1]);
+                c[0] = hi, c[1] = lo;
+            } else {
+#pragma unroll
+                for (int r = 0; r < 2; ++r) {
+                    const int g = r * 32 + lane;
+                    const uint32_t other = __shfl_xor_sync(0xffffffffu, c[r], stride);
+                    const bool desc = (g & size) == 0, lower = (g & stride) == 0;
+                    c[r] = (lower == desc) ? max(c[r], other) : min(c[r], other);
+                }
+            }
+        }
+    }
+    const uint32_t bar = __shfl_sync(0xffffffffu, c[0], k - 1);
+    const bool keep0 = key0 && (uint32_t)(key0 >> 32) >= bar, keep1 = key1 && (uint32_t)(key1 >> 32) >= bar;
+    const uint32_t m0 = __ballot_sync(0xffffffffu, keep0), m1 = __ballot_sync(0xffffffffu, keep1);
+    const uint32_t below = (1u << lane) - 1u;
+    if (keep0) list[__popc(m0 & below)] = key0;  // every lane read its two keys before the first ballot
+    if (keep1) list[__popc(m0) + __popc(m1 & below)] = key1;
+    __syncwarp();
+    *bar_code = bar;
+    return __popc(m0) + __popc(m1);
+}
+
+constexpr int kDepth = 3;  // tiles of a warp's ring: the one being read and two in flight
+
+__device__ __forceinline__ void async_copy16(float* dst_shared, const float* src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(dst_shared)),
+                 "l"(src)
+                 : "memory");
+}
+__device__ __forceinline__ void async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int PENDING>
+__device__ __forceinline__ void async_wait() {
+    asm volatile("cp.async.wait_group %0;" ::"n"(PENDING) : "memory");
+}
+
+// Phase 1 is warp-autonomous: no block-wide barrier inside the streaming loop.  Each warp keeps
+//   * per lane, a running (max, sum of exponentials) of the elements it has seen,
+//   * a bar: a value that its k-th best element so far reaches (-inf until k elements were seen);
+//     the largest bar of the block's warps is shared, since the block's k-th best reaches it too,
+//   * a list of up to 64 candidate keys, all at or above the bar when they were appended.
+// An element below the bar cannot be among the segment's k best.  When the list fills up the bar is
+// tightened to the k-th largest listed value; if a tile's candidates still do not fit (ordered
+// input, ties), the list and the tile's candidates are ranked exactly by k selection rounds.
+// With 16-byte aligned rows each lane copies its own four float4 of a tile asynchronously into the
+// warp's ring in shared memory, two tiles ahead, and reads back only what it copied itself; other
+// rows are prefetched one tile ahead into registers.
 template <bool VEC>
 __global__ void __launch_bounds__(kScanThreads, 3)
 expand_kernel(const float* __restrict__ draft_logits, long long batch_stride, int V, int k, int D,
@@ -109,42 +153,45 @@ expand_kernel(const float* __restrict__ draft_logits, long long batch_stride, in
               int32_t* __restrict__ frontier, ExpandWs ws, int32_t* d_status) {
     constexpr int VPT = 4, NE = 16;
     constexpr float kLog2e = 1.4426950408889634f;
-    __shared__ TopkScratch s_topk;
+    extern __shared__ __align__(16) float s_ring[];  // [kScanWarps][kDepth][512] (vector path)
+    __shared__ unsigned long long s_list[kScanWarps][kWarpList];
+    __shared__ int s_count[kScanWarps];
+    __shared__ uint32_t s_bar_code;  // largest bar of any warp, as a value code (0: none yet)
     __shared__ float s_wmax[kScanWarps], s_wsum[kScanWarps];
     __shared__ int s_flag;
     __shared__ unsigned long long s_rank[EAGLE2_MAX_K * EAGLE2_MAX_K];  // the new candidates' value codes
 
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) s_bar_code = 0u;
+    if (lane == 0) s_count[warp] = 0;
+    __syncthreads();  // the only block-wide barrier before the segment's end
     chain_wait();
     chain_release();
     const int chunk = blockIdx.x % chunks;
     const int row = (blockIdx.x / chunks) % n_s;
     const int b = blockIdx.x / (chunks * n_s);
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const float* zrow = draft_logits + (long long)b * batch_stride + (long long)row * V;
     const int tiles = (V + kTileTokens - 1) / kTileTokens;
     const int t0 = chunk * tpb, t1 = min(tiles, t0 + tpb);
 
-    // Vector path: tiles arrive by bulk copies into a ring in shared memory, kRing in flight.
-    // Scalar path (unaligned rows): the next tile is prefetched into registers.
-    extern __shared__ __align__(128) float s_ring[];  // [kRing][kTileTokens]
-    __shared__ unsigned long long s_bar[kRing];
-    auto issue_tile = [&](int t) {  // thread 0 only
-        const int first = t * kTileTokens;
-        const uint32_t bytes = (uint32_t)min(kTileTokens, V - first) * 4u;
-        bulk_load(smem_addr(s_ring + (size_t)((t - t0) % kRing) * kTileTokens), zrow + first, bytes,
-                  smem_addr(&s_bar[(t - t0) % kRing]));
-    };
-    if (VEC) {
-        if (threadIdx.x == 0) {
-            for (int i = 0; i < kRing; ++i)
-                asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr(&s_bar[i])) : "memory");
-            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-            for (int t = t0; t < t1 && t < t0 + kRing; ++t) issue_tile(t);
+    float* ring = s_ring + (size_t)warp * kDepth * (32 * NE);
+    auto issue_tile = [&](int t) {  // this lane's four float4 of tile t; pieces past the row are skipped
+        float* slot = ring + (size_t)((t - t0) % kDepth) * (32 * NE);
+#pragma unroll
+        for (int i = 0; i < VPT; ++i) {
+            const int e0 = scan_elem_index<VPT, true>(t, 4 * i);
+            if (e0 < V) async_copy16(slot + (i * 32 + lane) * 4, zrow + e0);
         }
-    }
+    };
     float cur[NE], nxt[NE];
-    if (!VEC) scan_load<VPT, false>(zrow, V, t0, cur);
-    int timed_out = 0;
+    if (VEC) {
+        issue_tile(t0);
+        async_commit();
+        if (t0 + 1 < t1) issue_tile(t0 + 1);
+        async_commit();
+    } else {
+        scan_load<VPT, false>(zrow, V, t0, cur);
+    }
     // The block that arrives last merges every row and then needs the rows' parents and their
     // values; whichever block that will be, the two dependent loads are already under way.
     const long long N = nodes_of(k, D);
@@ -157,158 +204,158 @@ expand_kernel(const float* __restrict__ draft_logits, long long batch_stride, in
         if (my_parent < prev_base || my_parent >= prev_base + prev_count) my_parent = -2;  // reported by the merger
         else my_parent_value = tree_value[(long long)b * N + my_parent];
     }
-    if (threadIdx.x == 0) s_topk.count = 0, s_topk.overflow = 0, s_topk.thr = -INFINITY;
-    for (int i = threadIdx.x; i < kCandCap; i += kScanThreads) s_topk.cand[i] = 0ull;  // empty list
-    __syncthreads();  // also: the ring's barriers are initialised for every thread
 
     // ---- stream the segment ------------------------------------------------------------------------
+    unsigned long long* list = s_list[warp];
+    int n = 0;                          // keys in the list (warp-uniform; s_count[warp] mirrors it between tiles)
+    float bar = -INFINITY;              // warp-uniform
     float m_t = -INFINITY, s_t = 0.f;  // this thread's running maximum and sum of exp(x - m_t)
-    for (int t = t0; t < t1; ++t) {
-        if (VEC) {
-            const int slot = (t - t0) % kRing;
-            const uint32_t parity = (uint32_t)(((t - t0) / kRing) & 1);
-            const long long w0 = clock64();
-            while (!tile_landed(smem_addr(&s_bar[slot]), parity)) {
-                if (clock64() - w0 > kExpandWaitCycles) {
-                    timed_out = 1;
-                    break;
-                }
-            }
-            const float* tile = s_ring + (size_t)slot * kTileTokens;
-#pragma unroll
-            for (int i = 0; i < VPT; ++i) {
-                const int off = (i * kScanThreads + (int)threadIdx.x) * 4;  // as scan_elem_index<VPT, true>
-                float4 v = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
-                if (!timed_out && t * kTileTokens + off < V) v = *reinterpret_cast<const float4*>(tile + off);
-                cur[4 * i + 0] = v.x, cur[4 * i + 1] = v.y, cur[4 * i + 2] = v.z, cur[4 * i + 3] = v.w;
-            }
-        } else if (t + 1 < t1) {
-            scan_load<VPT, false>(zrow, V, t + 1, nxt);
+
+    auto tighten = [&]() {  // needs n >= k
+        uint32_t code;
+        n = warp_tighten(list, n, k, &code);
+        bar = code ? order_decode(code) : -INFINITY;
+        if (lane == 0) {
+            s_count[warp] = n;
+            if (code) atomicMax(&s_bar_code, code);
         }
-        float tm = -INFINITY;
+        __syncwarp();
+    };
+    auto consume = [&](int t, auto ragged_tag) {
+        constexpr bool RAGGED = decltype(ragged_tag)::value;  // the tile reaches past the row's end
+        float gm[VPT];  // maxima of the four float4
 #pragma unroll
-        for (int j = 0; j < NE; ++j) tm = fmaxf(tm, cur[j]);
+        for (int i = 0; i < VPT; ++i)
+            gm[i] = fmaxf(fmaxf(cur[4 * i], cur[4 * i + 1]), fmaxf(cur[4 * i + 2], cur[4 * i + 3]));
+        const float tm = fmaxf(fmaxf(gm[0], gm[1]), fmaxf(gm[2], gm[3]));
         if (tm > m_t) {
             s_t *= fast_ex2((m_t - tm) * kLog2e);  // 0 when nothing was summed yet
             m_t = tm;
         }
         if (m_t > -INFINITY) {
             const float neg = -m_t * kLog2e;
+            float acc[4] = {0.f, 0.f, 0.f, 0.f};  // four chains instead of one of sixteen additions
 #pragma unroll
-            for (int j = 0; j < NE; ++j) s_t += fast_ex2(fmaf(cur[j], kLog2e, neg));
+            for (int j = 0; j < NE; ++j) acc[j & 3] += fast_ex2(fmaf(cur[j], kLog2e, neg));
+            s_t += (acc[0] + acc[1]) + (acc[2] + acc[3]);
         }
-        // candidates: elements at or above the value of the block's k-th best so far (it changes only
-        // in a compaction, between block-wide barriers); for the first tile each warp uses the k-th
-        // largest of its lanes' maxima (at least k elements reach it)
-        float thr = s_topk.thr;
-        const bool first = t == t0;
-        if (first) thr = __shfl_sync(0xffffffffu, warp_sort_desc_f32(tm), k - 1);
-        int cnt = 0;
+        const uint32_t block_code = *reinterpret_cast<volatile uint32_t*>(&s_bar_code);
+        float thr = block_code ? fmaxf(bar, order_decode(block_code)) : bar;
+        // Without a bar yet, the k-th largest of the lanes' maxima serves for this tile: at least k
+        // of the tile's elements reach it.
+        if (thr == -INFINITY) thr = __shfl_sync(0xffffffffu, warp_sort_desc_f32(tm), k - 1);
+        if (!__any_sync(0xffffffffu, tm >= thr)) return;
         if (tm >= thr) {
 #pragma unroll
-            for (int j = 0; j < NE; ++j) cnt += (cur[j] >= thr) && (scan_elem_index<VPT, VEC>(t, j) < V);
-        }
-        int crowded = 0;  // the list overflowed or passed half of its capacity
-        if (__ballot_sync(0xffffffffu, cnt > 0)) {
-            int incl = cnt;
+            for (int i = 0; i < VPT; ++i) {
+                if (gm[i] >= thr) {
 #pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const int up = __shfl_up_sync(0xffffffffu, incl, o);
-                if (lane >= o) incl += up;
-            }
-            const int total = __shfl_sync(0xffffffffu, incl, 31);
-            int base = 0;
-            if (lane == 0) base = atomicAdd(&s_topk.count, total);
-            base = __shfl_sync(0xffffffffu, base, 0);
-            if (base + total <= kCandCap) {
-                if (cnt) {
-                    int pos = base + incl - cnt;
-#pragma unroll
-                    for (int j = 0; j < NE; ++j) {
-                        const int e = scan_elem_index<VPT, VEC>(t, j);
-                        if (cur[j] >= thr && e < V) s_topk.cand[pos++] = make_key(cur[j], (uint32_t)e);
+                    for (int j = 4 * i; j < 4 * i + 4; ++j) {
+                        if (cur[j] >= thr) {
+                            const int e = scan_elem_index<VPT, VEC>(t, j);
+                            if (!RAGGED || e < V) {
+                                const int pos = atomicAdd(&s_count[warp], 1);
+                                if (pos < kWarpList) list[pos] = make_key(cur[j], (uint32_t)e);
+                            }
+                        }
                     }
                 }
-            } else if (lane == 0) {
-                s_topk.overflow = 1;  // this warp's range of the list stays empty (zero keys)
             }
-            crowded = base + total > kCandCap / 2;
         }
-        const bool last = t + 1 == t1;
-        // One barrier per tile: every thread has read its part of the ring slot, the appends are
-        // done, and all threads agree on whether the list needs compacting.
-        const bool compact = __syncthreads_or(crowded) || first || last;
-        if (VEC && threadIdx.x == 0 && t + kRing < t1) issue_tile(t + kRing);  // refill the slot just read
-        if (compact) {
-            const int overflow = s_topk.overflow;  // stable: the next appends come after this branch's barrier
-            if (overflow) {
-                // more candidates than the list holds (heavily ordered input): rank this tile exactly
-                unsigned long long key[NE];
+        __syncwarp();
+        const int n_new = *reinterpret_cast<volatile int*>(&s_count[warp]);
+        if (n_new <= kWarpList) {
+            n = n_new;
+        } else {
+            // exact: the k best of (the list as it was | this tile's candidates), lower index first
+            // among equal values
+            unsigned long long mine[NE + 2];
 #pragma unroll
-                for (int j = 0; j < NE; ++j) {
-                    const int e = scan_elem_index<VPT, VEC>(t, j);
-                    key[j] = e < V ? make_key(cur[j], (uint32_t)e) : 0ull;
-                }
-                block_topk<NE>(key, k, s_topk.exact, s_topk.win);
-                __syncthreads();
+            for (int j = 0; j < NE; ++j) {
+                const int e = scan_elem_index<VPT, VEC>(t, j);
+                mine[j] = (cur[j] >= thr && (!RAGGED || e < V)) ? make_key(cur[j], (uint32_t)e) : 0ull;
             }
-            if (warp == 0) {
-                // best k of the list; after an overflow, of (the list without this tile's entries | the
-                // tile's exact winners)
-                const int n = min(s_topk.count, kCandCap);
-                const uint32_t tile_first = (uint32_t)t * kTileTokens;
-                unsigned long long mine[kCandCap / 32 + 1];
-#pragma unroll
-                for (int u = 0; u < kCandCap / 32; ++u) {
-                    unsigned long long key = lane + 32 * u < n ? s_topk.cand[lane + 32 * u] : 0ull;
-                    if (overflow && key && key_index(key) - tile_first < (uint32_t)kTileTokens) key = 0ull;
-                    mine[u] = key;
-                }
-                mine[kCandCap / 32] = (overflow && lane < k) ? s_topk.win[lane] : 0ull;
-                __syncwarp();
-                warp_select<kCandCap / 32 + 1>(mine, k, s_topk.cand);
-                __syncwarp();
-                // past the k winners the list is empty again
-#pragma unroll
-                for (int u = 0; u < kCandCap / 32; ++u)
-                    if (lane + 32 * u >= k && lane + 32 * u < n) s_topk.cand[lane + 32 * u] = 0ull;
-                if (lane == 0) {
-                    s_topk.count = k;  // entries past the keys that exist are 0 and never win
-                    s_topk.overflow = 0;
-                    s_topk.thr = s_topk.cand[k - 1] ? key_value(s_topk.cand[k - 1]) : -INFINITY;
-                }
+            mine[NE] = lane < n ? list[lane] : 0ull;
+            mine[NE + 1] = lane + 32 < n ? list[lane + 32] : 0ull;
+            __syncwarp();
+            warp_select<NE + 2>(mine, k, list);
+            __syncwarp();
+            const unsigned long long kth = list[k - 1];
+            bar = kth ? key_value(kth) : -INFINITY;
+            n = __popc(__ballot_sync(0xffffffffu, lane < k && list[lane] != 0ull));  // the keys that exist
+            if (lane == 0) {
+                s_count[warp] = n;
+                if (kth) atomicMax(&s_bar_code, (uint32_t)(kth >> 32));
             }
-            __syncthreads();
+            __syncwarp();
         }
+        // a first bar as soon as k elements were seen; a tighter one when the list is three quarters full
+        if (t + 1 < t1 && n >= k && (bar == -INFINITY || n > kWarpList * 3 / 4)) tighten();
+    };
+
+    for (int t = t0; t < t1; ++t) {
+        if (VEC) {
+            if (t + 2 < t1) issue_tile(t + 2);
+            async_commit();
+            async_wait<2>();  // tile t has landed; t+1 and t+2 may still be in flight
+            const float* slot = ring + (size_t)((t - t0) % kDepth) * (32 * NE);
+#pragma unroll
+            for (int i = 0; i < VPT; ++i) {
+                float4 v = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+                if (scan_elem_index<VPT, true>(t, 4 * i) < V) v = *reinterpret_cast<const float4*>(slot + (i * 32 + lane) * 4);
+                cur[4 * i + 0] = v.x, cur[4 * i + 1] = v.y, cur[4 * i + 2] = v.z, cur[4 * i + 3] = v.w;
+            }
+        } else if (t + 1 < t1) {
+            scan_load<VPT, false>(zrow, V, t + 1, nxt);
+        }
+        if ((t + 1) * kTileTokens > V) consume(t, std::true_type{});
+        else consume(t, std::false_type{});
         if (!VEC) {
 #pragma unroll
             for (int j = 0; j < NE; ++j) cur[j] = nxt[j];
         }
     }
-    if (timed_out) raise_status(d_status, EAGLE2_STATUS_TIMEOUT);
 
-    // ---- the segment's partial: k best keys, (max, sum exp) ----------------------------------------
-    const size_t part = ((size_t)b * n_s + row) * chunks + chunk;
-    if (threadIdx.x < k) ws.keys[part * k + threadIdx.x] = s_topk.cand[threadIdx.x];
+    // ---- the warp's k best, then the block's ---------------------------------------------------------
+    if (n > 32) {
+        unsigned long long mine[2] = {list[lane], lane + 32 < n ? list[lane + 32] : 0ull};
+        __syncwarp();
+        warp_select<2>(mine, k, list);
+    } else {
+        const unsigned long long sorted = warp_sort_desc_u64(lane < n ? list[lane] : 0ull);
+        __syncwarp();
+        if (lane < k) list[lane] = sorted;  // zeros where fewer than k keys exist
+    }
     const float wmax = warp_max_f32(m_t);
     float scaled = m_t > -INFINITY ? s_t * fast_ex2((m_t - wmax) * kLog2e) : 0.f;
     scaled = warp_sum_f32(scaled);
     if (lane == 0) s_wmax[warp] = wmax, s_wsum[warp] = scaled;
-    int bad = !(scaled == scaled) || wmax == INFINITY;  // a NaN or +Inf logit poisons the sum / the max
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        float cmax = s_wmax[0];
-#pragma unroll
-        for (int w = 1; w < kScanWarps; ++w) cmax = fmaxf(cmax, s_wmax[w]);
-        double csum = 0.0;
-        if (cmax > -INFINITY) {
-#pragma unroll
-            for (int w = 0; w < kScanWarps; ++w)
-                if (s_wmax[w] > -INFINITY) csum += (double)s_wsum[w] * exp((double)s_wmax[w] - (double)cmax);
-        }
-        ws.stats[part] = make_double2((double)cmax, csum);
-    }
+    const int bad = !(scaled == scaled) || wmax == INFINITY;  // a NaN or +Inf logit poisons the sum / the max
     if (bad) raise_status(d_status, EAGLE2_STATUS_NONFINITE_LOGIT);
+    __syncthreads();
+    // The block's k best of the warps' k best: every thread ranks one of the 8k keys by counting the
+    // keys above it (keys differ, so ranks do), and the ranks below k are the winners' places.
+    const size_t part = ((size_t)b * n_s + row) * chunks + chunk;
+    {
+        const int n_keys = kScanWarps * k;  // <= 256 = threads
+        const unsigned long long mine = (int)threadIdx.x < n_keys ? s_list[threadIdx.x / k][threadIdx.x % k] : 0ull;
+        int rank = 0;
+        if (mine) {
+            for (int w = 0; w < kScanWarps; ++w)
+                for (int r = 0; r < k; ++r) rank += s_list[w][r] > mine;
+            if (rank < k) ws.keys[part * k + rank] = mine;
+        }
+        const int present = __syncthreads_count(mine != 0ull);
+        if ((int)threadIdx.x >= present && (int)threadIdx.x < k) ws.keys[part * k + threadIdx.x] = 0ull;
+    }
+    if (warp == 0) {
+        const float pm = lane < kScanWarps ? s_wmax[lane] : -INFINITY;
+        const float cmax = warp_max_f32(pm);
+        float term = 0.f;
+        if (lane < kScanWarps && pm > -INFINITY) term = s_wsum[lane] * fast_ex2((pm - cmax) * kLog2e);
+        const float csum = warp_sum_f32(term);
+        if (lane == 0) ws.stats[part] = make_double2((double)cmax, (double)csum);
+    }
 
     // ---- the last block of this sequence merges: a warp per row -------------------------------
     if (!last_block_arrives(ws.counters + b, chunks * n_s, &s_flag)) return;
@@ -358,7 +405,7 @@ expand_kernel(const float* __restrict__ draft_logits, long long batch_stride, in
         // up holding the c-th.  The k-th largest lane maximum is a threshold no winner can be below;
         // when at most 32 keys reach it (the usual case) they are sorted across the lanes, otherwise
         // k rounds of maximum extraction do the same job.
-        unsigned long long* s_pack = s_topk.cand + warp * 32;  // free: the chunk scan is over
+        unsigned long long* s_pack = s_list[warp];  // free: the segment scan is over
         unsigned long long mine = 0;
         for (int e0 = 0; e0 < keys_per_row; e0 += 32 * BATCH) {
             if (e0) {
@@ -434,9 +481,10 @@ static int launch_expand(const float* draft_logits, long long batch_stride, int 
                          double* tree_value, int32_t* frontier, const ExpandWs& ws, int32_t* d_status,
                          cudaStream_t stream) {
     const long long blocks = (long long)B * n_s * plan.chunks;
-    const size_t dyn = VEC ? sizeof(float) * (size_t)kRing * kTileTokens : 0;
-    if (dyn > 40 * 1024 && cudaFuncSetAttribute(expand_kernel<VEC>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                (int)dyn) != cudaSuccess) {
+    const size_t dyn = VEC ? sizeof(float) * (size_t)kScanWarps * kDepth * 512 : 0;
+    // the vector path's ring and the static arrays together exceed 48 KB
+    if (VEC && cudaFuncSetAttribute(expand_kernel<VEC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) !=
+                   cudaSuccess) {
         cudaGetLastError();
         return EAGLE2_ERR_CUDA;
     }
