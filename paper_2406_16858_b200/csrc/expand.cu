@@ -243,20 +243,28 @@ expand_kernel(const float* __restrict__ draft_logits, long long batch_stride, in
         float thr = block_code ? fmaxf(bar, order_decode(block_code)) : bar;
         // Without a bar yet, the k-th largest of the lanes' maxima serves for this tile: at least k
         // of the tile's elements reach it.
-        if (thr == -INFINITY) thr = __shfl_sync(0xffffffffu, warp_sort_desc_f32(tm), k - 1);
+        if (thr == -INFINITY) {
+            thr = __shfl_sync(0xffffffffu, warp_sort_desc_f32(tm), k - 1);
+            bar = thr;  // k lanes hold an element that reaches it: a valid first bar (still -inf if they do not)
+            if (lane == 0 && thr > -INFINITY) atomicMax(&s_bar_code, order_code(thr));
+        }
         if (!__any_sync(0xffffffffu, tm >= thr)) return;
         if (tm >= thr) {
 #pragma unroll
             for (int i = 0; i < VPT; ++i) {
-                if (gm[i] >= thr) {
+                if (gm[i] >= thr) {  // one reservation for the float4's candidates, then predicated stores
+                    bool pass[4];
+                    int c = 0;
 #pragma unroll
-                    for (int j = 4 * i; j < 4 * i + 4; ++j) {
-                        if (cur[j] >= thr) {
-                            const int e = scan_elem_index<VPT, VEC>(t, j);
-                            if (!RAGGED || e < V) {
-                                const int pos = atomicAdd(&s_count[warp], 1);
-                                if (pos < kWarpList) list[pos] = make_key(cur[j], (uint32_t)e);
-                            }
+                    for (int u = 0; u < 4; ++u) {
+                        pass[u] = cur[4 * i + u] >= thr && (!RAGGED || scan_elem_index<VPT, VEC>(t, 4 * i + u) < V);
+                        c += pass[u];
+                    }
+                    int pos = atomicAdd(&s_count[warp], c);
+                    if (pos + c <= kWarpList) {  // else the count says "overflow" and the exact path takes over
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            if (pass[u]) list[pos++] = make_key(cur[4 * i + u], (uint32_t)scan_elem_index<VPT, VEC>(t, 4 * i + u));
                         }
                     }
                 }
@@ -289,8 +297,8 @@ expand_kernel(const float* __restrict__ draft_logits, long long batch_stride, in
             }
             __syncwarp();
         }
-        // a first bar as soon as k elements were seen; a tighter one when the list is three quarters full
-        if (t + 1 < t1 && n >= k && (bar == -INFINITY || n > kWarpList * 3 / 4)) tighten();
+        // a tighter bar when the list is three quarters full
+        if (t + 1 < t1 && n >= k && n > kWarpList * 3 / 4) tighten();
     };
 
     for (int t = t0; t < t1; ++t) {
