@@ -232,6 +232,47 @@ def batched_attention_extra(e2, dev, stream, hbm_peak, B=32, n_layers=3, reps=10
             "us_per_layer": us, "algorithmic_bytes_per_layer": nbytes, "achieved_gbs": gbs, "frac_of_measured_hbm": gbs / hbm_peak}
 
 
+def batched_expand_extra(e2, dev, stream, hbm_peak, B=128, n_sets=4, reps=20):
+    """One expansion step (k rows per sequence) alone at a batch that gives a launch enough bytes
+    (B*k*V*4 = 0.66 GB) for the HBM fraction to be about the kernel; a few distinct logit sets
+    larger than L2."""
+    import torch
+    cfg = get_config("llama3_8b").with_(B=B)
+    k, V, D = cfg.k, cfg.V, cfg.D
+    g = torch.Generator(device=dev).manual_seed(7)
+    logits = [torch.randn((B, k, V), generator=g, device=dev) for _ in range(n_sets)]
+    N = k + (D - 1) * k * k
+    token = torch.zeros((B, N), dtype=torch.int32, device=dev)
+    parent = torch.zeros_like(token)
+    value = torch.zeros((B, N), dtype=torch.float64, device=dev)
+    frontier0 = torch.arange(k, dtype=torch.int32, device=dev).repeat(B, 1).contiguous()  # the step-0 nodes
+    frontier = frontier0.clone()
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    ws = torch.empty(e2.workspace_bytes(e2.OP_EXPAND, B=B, V=V, k=k, D=D), dtype=torch.uint8, device=dev)
+    e2.workspace_init(ws)
+
+    def steps():
+        for z in logits:
+            frontier.copy_(frontier0)  # every call expands the same level
+            e2.expand(z, k * V, B, V, k, D, 1, token, parent, value, frontier, ws, status)
+
+    with torch.cuda.stream(stream):
+        for _ in range(3):
+            steps()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev0.record(stream)
+        for _ in range(reps):
+            steps()
+        ev1.record(stream)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    us = ev0.elapsed_time(ev1) * 1e3 / (reps * n_sets)  # includes the 5 KB frontier reset per call
+    nbytes = float(B) * k * V * 4
+    gbs = nbytes / (us * 1e-6) / 1e9
+    return {"workload": f"llama3_8b expansion step 1, B={B} ({B * k} rows of {V} logits)", "us_per_call": us,
+            "algorithmic_bytes_per_call": nbytes, "achieved_gbs": gbs, "frac_of_measured_hbm": gbs / hbm_peak}
+
+
 # ------------------------------------------------------------------------------------------------
 # the CUDA path
 
@@ -454,6 +495,7 @@ def run_ours(args):
     line["breakdown_us"] = breakdown  # each step replayed alone (warm logits for the small steps)
     if world == 1 and not args.no_extras:
         line["attention_batched"] = batched_attention_extra(e2, dev, stream, hbm_peak)
+        line["expand_batched"] = batched_expand_extra(e2, dev, stream, hbm_peak)
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
@@ -468,7 +510,7 @@ def main():
     ap.add_argument("--workload", default="llama3_8b")
     ap.add_argument("--batch", type=int, default=0, help="override the number of sequences")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-extras", action="store_true", help="skip the batched attention side measurement")
+    ap.add_argument("--no-extras", action="store_true", help="skip the batched attention and expansion side measurements")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

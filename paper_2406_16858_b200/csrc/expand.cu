@@ -25,15 +25,27 @@ struct ExpandPlan {
 
 constexpr int kMergeKeysMax = 1024;  // segment winners per row that the merge handles (32 per lane, two passes of 16)
 
-// Enough blocks to fill the device three deep when the rows allow it, otherwise about 8 tiles per
-// block; never more segments per row than the merge can take, whole tiles per segment.
+// Segments per row.  A launch of up to three waves of one-tile blocks is about latency: one tile
+// per block.  Otherwise a block costs about kBlockFixed tile times of start-up and hand-over on top
+// of its tiles, blocks share an SM's issue slots, and the choice minimises (blocks per SM, rounded
+// up) x (cost of a block).  Never more segments per row than the merge can take, whole tiles per
+// segment.
 static bool expand_plan(long long rows, int V, int k, ExpandPlan* p) {
+    constexpr int kSMs = 148, kBlockFixed = 6;
     const int tiles = (V + kTileTokens - 1) / kTileTokens;
-    long long g = (3 * 148 + rows - 1) / (rows > 0 ? rows : 1);
-    if (g < (tiles + 7) / 8) g = (tiles + 7) / 8;  // at most 8 tiles per block: several waves balance out
-    if (g > tiles) g = tiles;
-    if (g * k > kMergeKeysMax) g = kMergeKeysMax / k;
-    if (g < 1) g = 1;
+    long long g_max = kMergeKeysMax / k;
+    if (g_max > tiles) g_max = tiles;
+    if (g_max < 1) g_max = 1;
+    if (rows < 1) rows = 1;
+    long long g = g_max;
+    if (rows * tiles > 9 * kSMs) {
+        long long best = -1;
+        for (long long c = 1; c <= g_max; ++c) {
+            const long long tpb = (tiles + c - 1) / c;
+            const long long cost = ((rows * c + kSMs - 1) / kSMs) * (kBlockFixed + tpb);
+            if (best < 0 || cost < best) best = cost, g = c;
+        }
+    }
     p->tpb = (int)((tiles + g - 1) / g);
     p->chunks = (tiles + p->tpb - 1) / p->tpb;
     return (long long)p->chunks * k <= kMergeKeysMax;
@@ -83,50 +95,16 @@ __device__ __forceinline__ float fast_ex2(float x) {
     return y;
 }
 
-// The warp's candidate list (n <= 64 keys in shared memory, any order) is cut down to the entries
-// whose value reaches the k-th largest value in it: the 64 value codes (two per lane) are sorted
-// across the warp, the k-th gives the bar, ties at the bar stay.  Needs n >= k.  Returns the new n
-// (>= k) and the bar's code.
-__device__ __forceinline__ int warp_tighten(unsigned long long* list, int n, int k, uint32_t* bar_code) {
-    const int lane = threadIdx.x & 31;
-    const unsigned long long key0 = lane < n ? list[lane] : 0ull;
-    const unsigned long long key1 = lane + 32 < n ? list[lane + 32] : 0ull;
-    uint32_t c[2] = {(uint32_t)(key0 >> 32), (uint32_t)(key1 >> 32)};  // element r*32 + lane
-#pragma unroll
-    for (int size = 2; size <= 64; size <<= 1) {
-#pragma unroll
-        for (int stride = size >> 1; stride > 0; stride >>= 1) {
-            if (stride == 32) {  // partners sit in the same lane; descending overall
-                const uint32_t hi = max(c[0], c[1]), lo = min(c[0], c[1]);
-                c[0] = hi, c[1] = lo;
-            } else {
-#pragma unroll
-                for (int r = 0; r < 2; ++r) {
-                    const int g = r * 32 + lane;
-                    const uint32_t other = __shfl_xor_sync(0xffffffffu, c[r], stride);
-                    const bool desc = (g & size) == 0, lower = (g & stride) == 0;
-                    c[r] = (lower == desc) ? max(c[r], other) : min(c[r], other);
-                }
-            }
-        }
-    }
-    const uint32_t bar = __shfl_sync(0xffffffffu, c[0], k - 1);
-    const bool keep0 = key0 && (uint32_t)(key0 >> 32) >= bar, keep1 = key1 && (uint32_t)(key1 >> 32) >= bar;
-    const uint32_t m0 = __ballot_sync(0xffffffffu, keep0), m1 = __ballot_sync(0xffffffffu, keep1);
-    const uint32_t below = (1u << lane) - 1u;
-    if (keep0) list[__popc(m0 & below)] = key0;  // every lane read its two keys before the first ballot
-    if (keep1) list[__popc(m0) + __popc(m1 & below)] = key1;
-    __syncwarp();
-    *bar_code = bar;
-    return __popc(m0) + __popc(m1);
-}
-
 constexpr int kDepth = 3;  // tiles of a warp's ring: the one being read and two in flight
 
-__device__ __forceinline__ void async_copy16(float* dst_shared, const float* src) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(dst_shared)),
-                 "l"(src)
-                 : "memory");
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void async_copy16(uint32_t dst_shared, const float* src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst_shared), "l"(src) : "memory");
+}
+__device__ __forceinline__ float4 load_shared16(uint32_t addr) {
+    float4 v;
+    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
+    return v;
 }
 __device__ __forceinline__ void async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int PENDING>
@@ -134,19 +112,42 @@ __device__ __forceinline__ void async_wait() {
     asm volatile("cp.async.wait_group %0;" ::"n"(PENDING) : "memory");
 }
 
-// Phase 1 is warp-autonomous: no block-wide barrier inside the streaming loop.  Each warp keeps
-//   * per lane, a running (max, sum of exponentials) of the elements it has seen,
-//   * a bar: a value that its k-th best element so far reaches (-inf until k elements were seen);
-//     the largest bar of the block's warps is shared, since the block's k-th best reaches it too,
-//   * a list of up to 64 candidate keys, all at or above the bar when they were appended.
-// An element below the bar cannot be among the segment's k best.  When the list fills up the bar is
-// tightened to the k-th largest listed value; if a tile's candidates still do not fit (ordered
-// input, ties), the list and the tile's candidates are ranked exactly by k selection rounds.
+constexpr int kQueue = 256;                              // candidate keys in flight to the selector warp
+constexpr long long kExpandWaitCycles = 1LL << 31;       // ~1 s bound of every wait below
+
+// Sorts a bitonic sequence of one key per lane (first rising then falling, or the reverse) into
+// descending order.
+__device__ __forceinline__ unsigned long long warp_bitonic_merge_desc(unsigned long long v) {
+    const int lane = threadIdx.x & 31;
+#pragma unroll
+    for (int stride = 16; stride > 0; stride >>= 1) {
+        const unsigned long long other = __shfl_xor_sync(0xffffffffu, v, stride);
+        const unsigned long long hi = v > other ? v : other, lo = v > other ? other : v;
+        v = (lane & stride) == 0 ? hi : lo;
+    }
+    return v;
+}
+
+// Phase 1 has no block-wide barrier inside the streaming loop.  Every streaming warp keeps, per
+// lane, a running (max, sum of exponentials) of the elements it has seen, and filters its elements
+// against a bar: a value that the k-th best element of the segment so far is known to reach, so that
+// an element below it cannot be among the segment's k best.  The bar is shared by the block (a value
+// code in shared memory that only rises).  Until there is one, a warp uses the k-th largest of its
+// lanes' maxima of the tile at hand (at least k elements reach it).
+//
+// STREAM = false (one tile per block, the latency case): each warp lists its candidates (at most 64;
+// more - ordered input, ties - are ranked exactly by k selection rounds), reduces them to its k best,
+// and the block ranks the warps' 8k keys by counting.
+// STREAM = true (several tiles per block): a ninth warp, the selector, owns the segment's k best.
+// The streaming warps push candidates into a ring in shared memory; the selector takes them 32 at a
+// time, merges them into its sorted 32 best (one key per lane) and raises the bar to the k-th.  How
+// far behind the selector is changes only how many needless candidates are pushed, never the result.
+//
 // With 16-byte aligned rows each lane copies its own four float4 of a tile asynchronously into the
 // warp's ring in shared memory, two tiles ahead, and reads back only what it copied itself; other
 // rows are prefetched one tile ahead into registers.
-template <bool VEC>
-__global__ void __launch_bounds__(kScanThreads, 3)
+template <bool VEC, bool STREAM>
+__global__ void __launch_bounds__(STREAM ? kScanThreads + 32 : kScanThreads, 3)
 expand_kernel(const float* __restrict__ draft_logits, long long batch_stride, int V, int k, int D,
               int s, int n_s, int chunks, int tpb, int32_t* __restrict__ tree_token,
               int32_t* __restrict__ tree_parent, double* __restrict__ tree_value,
@@ -154,16 +155,19 @@ expand_kernel(const float* __restrict__ draft_logits, long long batch_stride, in
     constexpr int VPT = 4, NE = 16;
     constexpr float kLog2e = 1.4426950408889634f;
     extern __shared__ __align__(16) float s_ring[];  // [kScanWarps][kDepth][512] (vector path)
-    __shared__ unsigned long long s_list[kScanWarps][kWarpList];
+    __shared__ unsigned long long s_list[kScanWarps][kWarpList];  // !STREAM: the warps' candidate lists
+    __shared__ unsigned long long s_queue[STREAM ? kQueue : 1];   // STREAM: keys on their way to the selector (0: empty)
     __shared__ int s_count[kScanWarps];
-    __shared__ uint32_t s_bar_code;  // largest bar of any warp, as a value code (0: none yet)
+    __shared__ int s_tail, s_head, s_done;  // STREAM: slots reserved / consumed, streaming warps finished
+    __shared__ uint32_t s_bar_code;         // the bar as a value code (0: none yet)
     __shared__ float s_wmax[kScanWarps], s_wsum[kScanWarps];
     __shared__ int s_flag;
     __shared__ unsigned long long s_rank[EAGLE2_MAX_K * EAGLE2_MAX_K];  // the new candidates' value codes
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    if (threadIdx.x == 0) s_bar_code = 0u;
-    if (lane == 0) s_count[warp] = 0;
+    if (threadIdx.x == 0) s_bar_code = 0u, s_tail = 0, s_head = 0, s_done = 0;
+    if (lane == 0 && warp < kScanWarps) s_count[warp] = 0;
+    if (STREAM && threadIdx.x < kQueue) s_queue[threadIdx.x] = 0ull;
     __syncthreads();  // the only block-wide barrier before the segment's end
     chain_wait();
     chain_release();
@@ -173,30 +177,45 @@ expand_kernel(const float* __restrict__ draft_logits, long long batch_stride, in
     const float* zrow = draft_logits + (long long)b * batch_stride + (long long)row * V;
     const int tiles = (V + kTileTokens - 1) / kTileTokens;
     const int t0 = chunk * tpb, t1 = min(tiles, t0 + tpb);
+    const size_t part = ((size_t)b * n_s + row) * chunks + chunk;
+    const long long N = nodes_of(k, D);
+    int my_parent = -1;
+    double my_parent_value = 0.0;
+    int timed_out = 0;
 
-    float* ring = s_ring + (size_t)warp * kDepth * (32 * NE);
-    auto issue_tile = [&](int t) {  // this lane's four float4 of tile t; pieces past the row are skipped
-        float* slot = ring + (size_t)((t - t0) % kDepth) * (32 * NE);
+    if (!STREAM || warp < kScanWarps) {
+    // ===== streaming warps ==============================================================================
+    // Vector path: float4 i of this lane sits 4096 bytes * i past the lane's first one in global
+    // memory and 512 bytes * i past it in the warp's ring slot.
+    const uint32_t ring_addr = smem_addr(s_ring + (size_t)warp * kDepth * (32 * NE)) + (uint32_t)lane * 16u;
+    const float* src_next = zrow + (size_t)t0 * kTileTokens + threadIdx.x * 4;  // of the next tile to request
+    int t_issue = t0, slot_issue = 0;
+    auto issue_next = [&]() {  // requests one more tile (nothing once the segment is exhausted); one group each
+        if (t_issue < t1) {
+            const uint32_t dst = ring_addr + (uint32_t)slot_issue * (32 * NE * 4);
+            if ((t_issue + 1) * kTileTokens <= V) {
 #pragma unroll
-        for (int i = 0; i < VPT; ++i) {
-            const int e0 = scan_elem_index<VPT, true>(t, 4 * i);
-            if (e0 < V) async_copy16(slot + (i * 32 + lane) * 4, zrow + e0);
+                for (int i = 0; i < VPT; ++i) async_copy16(dst + i * 512, src_next + i * (kScanThreads * 4));
+            } else {  // pieces past the row's end are skipped
+#pragma unroll
+                for (int i = 0; i < VPT; ++i)
+                    if (scan_elem_index<VPT, true>(t_issue, 4 * i) < V) async_copy16(dst + i * 512, src_next + i * (kScanThreads * 4));
+            }
         }
+        async_commit();
+        ++t_issue;
+        src_next += kTileTokens;
+        slot_issue = slot_issue == kDepth - 1 ? 0 : slot_issue + 1;
     };
     float cur[NE], nxt[NE];
     if (VEC) {
-        issue_tile(t0);
-        async_commit();
-        if (t0 + 1 < t1) issue_tile(t0 + 1);
-        async_commit();
+        issue_next();
+        issue_next();
     } else {
         scan_load<VPT, false>(zrow, V, t0, cur);
     }
     // The block that arrives last merges every row and then needs the rows' parents and their
     // values; whichever block that will be, the two dependent loads are already under way.
-    const long long N = nodes_of(k, D);
-    int my_parent = -1;
-    double my_parent_value = 0.0;
     if (s && threadIdx.x < n_s) {
         my_parent = frontier[(long long)b * k + threadIdx.x];
         const long long prev_base = s >= 2 ? (long long)k + (long long)(s - 2) * k * k : 0;
@@ -205,21 +224,21 @@ expand_kernel(const float* __restrict__ draft_logits, long long batch_stride, in
         else my_parent_value = tree_value[(long long)b * N + my_parent];
     }
 
-    // ---- stream the segment ------------------------------------------------------------------------
     unsigned long long* list = s_list[warp];
-    int n = 0;                          // keys in the list (warp-uniform; s_count[warp] mirrors it between tiles)
-    float bar = -INFINITY;              // warp-uniform
+    int n = 0;                          // !STREAM: keys in the list (warp-uniform; s_count[warp] mirrors it)
     float m_t = -INFINITY, s_t = 0.f;  // this thread's running maximum and sum of exp(x - m_t)
 
-    auto tighten = [&]() {  // needs n >= k
-        uint32_t code;
-        n = warp_tighten(list, n, k, &code);
-        bar = code ? order_decode(code) : -INFINITY;
-        if (lane == 0) {
-            s_count[warp] = n;
-            if (code) atomicMax(&s_bar_code, code);
+    auto push = [&](int pos, unsigned long long key) {  // STREAM: entry pos of the ring
+        if (pos - *reinterpret_cast<volatile int*>(&s_head) >= kQueue) {  // the slot still holds entry pos - kQueue
+            const long long w0 = clock64();
+            while (pos - *reinterpret_cast<volatile int*>(&s_head) >= kQueue) {
+                if (clock64() - w0 > kExpandWaitCycles) {
+                    timed_out = 1;
+                    return;
+                }
+            }
         }
-        __syncwarp();
+        *reinterpret_cast<volatile unsigned long long*>(&s_queue[pos & (kQueue - 1)]) = key;
     };
     auto consume = [&](int t, auto ragged_tag) {
         constexpr bool RAGGED = decltype(ragged_tag)::value;  // the tile reaches past the row's end
@@ -240,83 +259,98 @@ expand_kernel(const float* __restrict__ draft_logits, long long batch_stride, in
             s_t += (acc[0] + acc[1]) + (acc[2] + acc[3]);
         }
         const uint32_t block_code = *reinterpret_cast<volatile uint32_t*>(&s_bar_code);
-        float thr = block_code ? fmaxf(bar, order_decode(block_code)) : bar;
-        // Without a bar yet, the k-th largest of the lanes' maxima serves for this tile: at least k
-        // of the tile's elements reach it.
+        float thr = block_code ? order_decode(block_code) : -INFINITY;
         if (thr == -INFINITY) {
             thr = __shfl_sync(0xffffffffu, warp_sort_desc_f32(tm), k - 1);
-            bar = thr;  // k lanes hold an element that reaches it: a valid first bar (still -inf if they do not)
+            // k lanes hold an element that reaches it: a valid bar (if it is not -inf itself)
             if (lane == 0 && thr > -INFINITY) atomicMax(&s_bar_code, order_code(thr));
         }
         if (!__any_sync(0xffffffffu, tm >= thr)) return;
+        uint32_t pmask = 0;  // this lane's candidates
         if (tm >= thr) {
 #pragma unroll
-            for (int i = 0; i < VPT; ++i) {
-                if (gm[i] >= thr) {  // one reservation for the float4's candidates, then predicated stores
-                    bool pass[4];
-                    int c = 0;
+            for (int j = 0; j < NE; ++j)
+                if (cur[j] >= thr && (!RAGGED || scan_elem_index<VPT, VEC>(t, j) < V)) pmask |= 1u << j;
+        }
+        const int c = __popc(pmask);
+        if constexpr (STREAM) {
+            if (__any_sync(0xffffffffu, c >= NE / 2)) {
+                // ordered input or ties: the tile's k best of this warp, ranked exactly, are all it can
+                // contribute
+                unsigned long long mine[NE];
 #pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        pass[u] = cur[4 * i + u] >= thr && (!RAGGED || scan_elem_index<VPT, VEC>(t, 4 * i + u) < V);
-                        c += pass[u];
-                    }
-                    int pos = atomicAdd(&s_count[warp], c);
-                    if (pos + c <= kWarpList) {  // else the count says "overflow" and the exact path takes over
+                for (int j = 0; j < NE; ++j)
+                    mine[j] = (pmask >> j) & 1u ? make_key(cur[j], (uint32_t)scan_elem_index<VPT, VEC>(t, j)) : 0ull;
+                __syncwarp();
+                warp_select<NE>(mine, k, list);
+                __syncwarp();
+                const unsigned long long key = lane < k ? list[lane] : 0ull;
+                const uint32_t have = __ballot_sync(0xffffffffu, key != 0ull);
+                int pos = 0;
+                if (lane == 0) pos = atomicAdd(&s_tail, __popc(have));
+                pos = __shfl_sync(0xffffffffu, pos, 0);
+                if (key) push(pos + __popc(have & ((1u << lane) - 1u)), key);
+                __syncwarp();
+            } else if (c) {
+                int pos = atomicAdd(&s_tail, c);
 #pragma unroll
-                        for (int u = 0; u < 4; ++u) {
-                            if (pass[u]) list[pos++] = make_key(cur[4 * i + u], (uint32_t)scan_elem_index<VPT, VEC>(t, 4 * i + u));
-                        }
-                    }
+                for (int j = 0; j < NE; ++j)
+                    if ((pmask >> j) & 1u) push(pos++, make_key(cur[j], (uint32_t)scan_elem_index<VPT, VEC>(t, j)));
+            }
+        } else {
+            if (c) {
+                int pos = atomicAdd(&s_count[warp], c);
+                if (pos + c <= kWarpList) {  // else the count says "overflow" and the exact path takes over
+#pragma unroll
+                    for (int j = 0; j < NE; ++j)
+                        if ((pmask >> j) & 1u) list[pos++] = make_key(cur[j], (uint32_t)scan_elem_index<VPT, VEC>(t, j));
                 }
             }
-        }
-        __syncwarp();
-        const int n_new = *reinterpret_cast<volatile int*>(&s_count[warp]);
-        if (n_new <= kWarpList) {
-            n = n_new;
-        } else {
-            // exact: the k best of (the list as it was | this tile's candidates), lower index first
-            // among equal values
-            unsigned long long mine[NE + 2];
+            __syncwarp();
+            const int n_new = *reinterpret_cast<volatile int*>(&s_count[warp]);
+            if (n_new <= kWarpList) {
+                n = n_new;
+            } else {
+                // exact: the k best of (the list as it was | this tile's candidates), lower index first
+                // among equal values
+                unsigned long long mine[NE + 2];
 #pragma unroll
-            for (int j = 0; j < NE; ++j) {
-                const int e = scan_elem_index<VPT, VEC>(t, j);
-                mine[j] = (cur[j] >= thr && (!RAGGED || e < V)) ? make_key(cur[j], (uint32_t)e) : 0ull;
+                for (int j = 0; j < NE; ++j)
+                    mine[j] = (pmask >> j) & 1u ? make_key(cur[j], (uint32_t)scan_elem_index<VPT, VEC>(t, j)) : 0ull;
+                mine[NE] = lane < n ? list[lane] : 0ull;
+                mine[NE + 1] = lane + 32 < n ? list[lane + 32] : 0ull;
+                __syncwarp();
+                warp_select<NE + 2>(mine, k, list);
+                __syncwarp();
+                const unsigned long long kth = list[k - 1];
+                n = __popc(__ballot_sync(0xffffffffu, lane < k && list[lane] != 0ull));  // the keys that exist
+                if (lane == 0) {
+                    s_count[warp] = n;
+                    if (kth) atomicMax(&s_bar_code, (uint32_t)(kth >> 32));
+                }
+                __syncwarp();
             }
-            mine[NE] = lane < n ? list[lane] : 0ull;
-            mine[NE + 1] = lane + 32 < n ? list[lane + 32] : 0ull;
-            __syncwarp();
-            warp_select<NE + 2>(mine, k, list);
-            __syncwarp();
-            const unsigned long long kth = list[k - 1];
-            bar = kth ? key_value(kth) : -INFINITY;
-            n = __popc(__ballot_sync(0xffffffffu, lane < k && list[lane] != 0ull));  // the keys that exist
-            if (lane == 0) {
-                s_count[warp] = n;
-                if (kth) atomicMax(&s_bar_code, (uint32_t)(kth >> 32));
-            }
-            __syncwarp();
         }
-        // a tighter bar when the list is three quarters full
-        if (t + 1 < t1 && n >= k && n > kWarpList * 3 / 4) tighten();
     };
 
+    int slot_read = 0;
     for (int t = t0; t < t1; ++t) {
+        const bool ragged = (t + 1) * kTileTokens > V;
         if (VEC) {
-            if (t + 2 < t1) issue_tile(t + 2);
-            async_commit();
+            issue_next();
             async_wait<2>();  // tile t has landed; t+1 and t+2 may still be in flight
-            const float* slot = ring + (size_t)((t - t0) % kDepth) * (32 * NE);
+            const uint32_t slot = ring_addr + (uint32_t)slot_read * (32 * NE * 4);
+            slot_read = slot_read == kDepth - 1 ? 0 : slot_read + 1;
 #pragma unroll
             for (int i = 0; i < VPT; ++i) {
                 float4 v = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
-                if (scan_elem_index<VPT, true>(t, 4 * i) < V) v = *reinterpret_cast<const float4*>(slot + (i * 32 + lane) * 4);
+                if (!ragged || scan_elem_index<VPT, true>(t, 4 * i) < V) v = load_shared16(slot + i * 512);
                 cur[4 * i + 0] = v.x, cur[4 * i + 1] = v.y, cur[4 * i + 2] = v.z, cur[4 * i + 3] = v.w;
             }
         } else if (t + 1 < t1) {
             scan_load<VPT, false>(zrow, V, t + 1, nxt);
         }
-        if ((t + 1) * kTileTokens > V) consume(t, std::true_type{});
+        if (ragged) consume(t, std::true_type{});
         else consume(t, std::false_type{});
         if (!VEC) {
 #pragma unroll
@@ -324,27 +358,90 @@ expand_kernel(const float* __restrict__ draft_logits, long long batch_stride, in
         }
     }
 
-    // ---- the warp's k best, then the block's ---------------------------------------------------------
-    if (n > 32) {
-        unsigned long long mine[2] = {list[lane], lane + 32 < n ? list[lane + 32] : 0ull};
-        __syncwarp();
-        warp_select<2>(mine, k, list);
-    } else {
-        const unsigned long long sorted = warp_sort_desc_u64(lane < n ? list[lane] : 0ull);
-        __syncwarp();
-        if (lane < k) list[lane] = sorted;  // zeros where fewer than k keys exist
-    }
+    // ---- the warp's share of the segment's partial ---------------------------------------------------
     const float wmax = warp_max_f32(m_t);
     float scaled = m_t > -INFINITY ? s_t * fast_ex2((m_t - wmax) * kLog2e) : 0.f;
     scaled = warp_sum_f32(scaled);
     if (lane == 0) s_wmax[warp] = wmax, s_wsum[warp] = scaled;
     const int bad = !(scaled == scaled) || wmax == INFINITY;  // a NaN or +Inf logit poisons the sum / the max
     if (bad) raise_status(d_status, EAGLE2_STATUS_NONFINITE_LOGIT);
-    __syncthreads();
-    // The block's k best of the warps' k best: every thread ranks one of the 8k keys by counting the
-    // keys above it (keys differ, so ranks do), and the ranks below k are the winners' places.
-    const size_t part = ((size_t)b * n_s + row) * chunks + chunk;
-    {
+    if constexpr (STREAM) {
+        __threadfence_block();  // the pushes and the statistics come before the count below
+        __syncwarp();
+        if (lane == 0) atomicAdd(&s_done, 1);
+    } else {
+        if (n > 32) {
+            unsigned long long mine[2] = {list[lane], lane + 32 < n ? list[lane + 32] : 0ull};
+            __syncwarp();
+            warp_select<2>(mine, k, list);
+        } else {
+            const unsigned long long sorted = warp_sort_desc_u64(lane < n ? list[lane] : 0ull);
+            __syncwarp();
+            if (lane < k) list[lane] = sorted;  // zeros where fewer than k keys exist
+        }
+    }
+    } else {
+    // ===== selector warp (STREAM) ==========================================================================
+    unsigned long long top = 0ull;  // the segment's best keys so far, descending over the lanes
+    int head = 0;
+    const long long w0 = clock64();
+    for (;;) {
+        const int done = *reinterpret_cast<volatile int*>(&s_done);  // read before the tail
+        const int tail = *reinterpret_cast<volatile int*>(&s_tail);
+        const int take = min(tail - head, 32);
+        if (take <= 0) {
+            if (done == kScanWarps) break;  // every reservation was made before its warp counted itself
+            if (clock64() - w0 > 4 * kExpandWaitCycles) {
+                timed_out = 1;
+                break;
+            }
+            __nanosleep(32);
+            continue;
+        }
+        unsigned long long key = 0ull;
+        if (lane < take) {
+            volatile unsigned long long* slot = &s_queue[(head + lane) & (kQueue - 1)];
+            const long long w1 = clock64();
+            while ((key = *slot) == 0ull) {  // reserved, not yet written
+                if (clock64() - w1 > kExpandWaitCycles) {
+                    timed_out = 1;
+                    break;
+                }
+            }
+            *slot = 0ull;
+        }
+        __threadfence_block();  // the slots are empty before the head says so
+        __syncwarp();
+        head += take;
+        if (lane == 0) *reinterpret_cast<volatile int*>(&s_head) = head;
+        // keys pushed under an older bar may already be beaten by the current k-th: nothing to merge
+        const unsigned long long kth_now = __shfl_sync(0xffffffffu, top, k - 1);
+        if (key <= kth_now) key = 0ull;
+        if (!__any_sync(0xffffffffu, key != 0ull)) continue;
+        // the 32 best of (top | the new keys): sort the new keys, pair the two sorted runs end to
+        // end, keep the larger of each pair, sort the bitonic result
+        key = warp_sort_desc_u64(key);
+        const unsigned long long rev = __shfl_sync(0xffffffffu, key, 31 - lane);
+        top = warp_bitonic_merge_desc(top > rev ? top : rev);
+        const unsigned long long kth = __shfl_sync(0xffffffffu, top, k - 1);
+        if (lane == 0 && kth) atomicMax(&s_bar_code, (uint32_t)(kth >> 32));
+    }
+    if (lane < k) ws.keys[part * k + lane] = top;  // zeros where fewer than k keys exist
+    // the warps' statistics were written before they counted themselves done
+    const float pm = lane < kScanWarps ? *reinterpret_cast<volatile float*>(&s_wmax[lane]) : -INFINITY;
+    const float cmax = warp_max_f32(pm);
+    float term = 0.f;
+    if (lane < kScanWarps && pm > -INFINITY)
+        term = *reinterpret_cast<volatile float*>(&s_wsum[lane]) * fast_ex2((pm - cmax) * kLog2e);
+    const float csum = warp_sum_f32(term);
+    if (lane == 0) ws.stats[part] = make_double2((double)cmax, (double)csum);
+    }
+    if (timed_out) raise_status(d_status, EAGLE2_STATUS_TIMEOUT);
+
+    if constexpr (!STREAM) {
+        __syncthreads();
+        // The block's k best of the warps' k best: every thread ranks one of the 8k keys by counting
+        // the keys above it (keys differ, so ranks do), and the ranks below k are the winners' places.
         const int n_keys = kScanWarps * k;  // <= 256 = threads
         const unsigned long long mine = (int)threadIdx.x < n_keys ? s_list[threadIdx.x / k][threadIdx.x % k] : 0ull;
         int rank = 0;
@@ -355,14 +452,14 @@ expand_kernel(const float* __restrict__ draft_logits, long long batch_stride, in
         }
         const int present = __syncthreads_count(mine != 0ull);
         if ((int)threadIdx.x >= present && (int)threadIdx.x < k) ws.keys[part * k + threadIdx.x] = 0ull;
-    }
-    if (warp == 0) {
-        const float pm = lane < kScanWarps ? s_wmax[lane] : -INFINITY;
-        const float cmax = warp_max_f32(pm);
-        float term = 0.f;
-        if (lane < kScanWarps && pm > -INFINITY) term = s_wsum[lane] * fast_ex2((pm - cmax) * kLog2e);
-        const float csum = warp_sum_f32(term);
-        if (lane == 0) ws.stats[part] = make_double2((double)cmax, (double)csum);
+        if (warp == 0) {
+            const float pm = lane < kScanWarps ? s_wmax[lane] : -INFINITY;
+            const float cmax = warp_max_f32(pm);
+            float term = 0.f;
+            if (lane < kScanWarps && pm > -INFINITY) term = s_wsum[lane] * fast_ex2((pm - cmax) * kLog2e);
+            const float csum = warp_sum_f32(term);
+            if (lane == 0) ws.stats[part] = make_double2((double)cmax, (double)csum);
+        }
     }
 
     // ---- the last block of this sequence merges: a warp per row -------------------------------
@@ -381,7 +478,7 @@ expand_kernel(const float* __restrict__ draft_logits, long long batch_stride, in
     __syncthreads();
     int status = 0;
 
-    for (int r = warp; r < n_s; r += kScanWarps) {
+    for (int r = warp; r < n_s && warp < kScanWarps; r += kScanWarps) {
         const size_t p0 = ((size_t)b * n_s + r) * chunks;
         constexpr int BATCH = 16;  // chunk winners per lane and pass
         // everything the row needs is requested before any of it is used
@@ -471,7 +568,7 @@ expand_kernel(const float* __restrict__ draft_logits, long long batch_stride, in
     __syncthreads();  // all rows merged (the old frontier was read when the kernel started)
 
     // next frontier: rank the new candidates by (value desc, index asc); ranks < k are kept
-    for (int i = threadIdx.x; i < n_new; i += kScanThreads) {
+    for (int i = threadIdx.x; i < n_new && threadIdx.x < kScanThreads; i += kScanThreads) {
         const unsigned long long ci = s_rank[i];
         int rank = 0;
         for (int j = 0; j < n_new; ++j) {
@@ -483,22 +580,35 @@ expand_kernel(const float* __restrict__ draft_logits, long long batch_stride, in
     if (status && lane == 0) raise_status(d_status, status);
 }
 
+template <bool VEC, bool STREAM>
+static int launch_expand_as(const float* draft_logits, long long batch_stride, int B, int V, int k, int D,
+                            int s, int n_s, const ExpandPlan& plan, int32_t* tree_token, int32_t* tree_parent,
+                            double* tree_value, int32_t* frontier, const ExpandWs& ws, int32_t* d_status,
+                            cudaStream_t stream) {
+    const long long blocks = (long long)B * n_s * plan.chunks;
+    const size_t dyn = VEC ? sizeof(float) * (size_t)kScanWarps * kDepth * 512 : 0;
+    // the vector path's ring and the static arrays together exceed 48 KB
+    if (VEC && cudaFuncSetAttribute(expand_kernel<VEC, STREAM>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    (int)dyn) != cudaSuccess) {
+        cudaGetLastError();
+        return EAGLE2_ERR_CUDA;
+    }
+    return launch_chained(expand_kernel<VEC, STREAM>, dim3((unsigned)blocks),
+                          dim3(STREAM ? kScanThreads + 32 : kScanThreads), dyn, stream, 1, draft_logits, batch_stride, V,
+                          k, D, s, n_s, plan.chunks, plan.tpb, tree_token, tree_parent, tree_value, frontier, ws,
+                          d_status);
+}
+
+// Blocks that stream several tiles get the selector warp; one-tile blocks rank within the block.
 template <bool VEC>
 static int launch_expand(const float* draft_logits, long long batch_stride, int B, int V, int k, int D,
                          int s, int n_s, const ExpandPlan& plan, int32_t* tree_token, int32_t* tree_parent,
                          double* tree_value, int32_t* frontier, const ExpandWs& ws, int32_t* d_status,
                          cudaStream_t stream) {
-    const long long blocks = (long long)B * n_s * plan.chunks;
-    const size_t dyn = VEC ? sizeof(float) * (size_t)kScanWarps * kDepth * 512 : 0;
-    // the vector path's ring and the static arrays together exceed 48 KB
-    if (VEC && cudaFuncSetAttribute(expand_kernel<VEC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) !=
-                   cudaSuccess) {
-        cudaGetLastError();
-        return EAGLE2_ERR_CUDA;
-    }
-    return launch_chained(expand_kernel<VEC>, dim3((unsigned)blocks), dim3(kScanThreads), dyn, stream, 1, draft_logits,
-                          batch_stride, V, k, D, s, n_s, plan.chunks, plan.tpb, tree_token, tree_parent, tree_value,
-                          frontier, ws, d_status);
+    return plan.tpb > 1 ? launch_expand_as<VEC, true>(draft_logits, batch_stride, B, V, k, D, s, n_s, plan, tree_token,
+                                                      tree_parent, tree_value, frontier, ws, d_status, stream)
+                        : launch_expand_as<VEC, false>(draft_logits, batch_stride, B, V, k, D, s, n_s, plan, tree_token,
+                                                       tree_parent, tree_value, frontier, ws, d_status, stream);
 }
 
 // Scratch of eagle2_expand_static: lives in every context that loads the library, until exit.

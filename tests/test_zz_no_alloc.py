@@ -51,7 +51,7 @@ def test_static_scratch_expansion_matches_workspace_expansion(name, B):
 
 def test_sizes_beyond_the_built_in_buffer_are_refused():
     cfg = get_config("llama3_8b")
-    B = 512  # 512 sequences x 10 rows x 4 vocabulary segments x 10 keys exceed the 1 MiB buffer
+    B = 2048  # 2048 sequences x 10 rows x (10 keys + statistics) exceed the 1 MiB buffer
     assert e2.workspace_bytes(e2.OP_EXPAND, B=B, V=cfg.V, k=cfg.k, D=cfg.D) > (1 << 20)
     N = cfg.N
     token = torch.zeros((B, N), dtype=torch.int32, device=DEV)
