@@ -293,6 +293,12 @@ def run_ours(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
 
+    if args.extras_only:  # the two batched side measurements alone (one GPU; also what the ncu summaries capture)
+        stream = torch.cuda.Stream(device=dev)
+        hbm_peak = _peaks()[0]
+        print(json.dumps({"attention_batched": batched_attention_extra(e2, dev, stream, hbm_peak),
+                          "expand_batched": batched_expand_extra(e2, dev, stream, hbm_peak)}))
+        return
     cfg = get_config(args.workload)
     if args.batch:
         cfg = cfg.with_(B=args.batch)
@@ -511,6 +517,7 @@ def main():
     ap.add_argument("--batch", type=int, default=0, help="override the number of sequences")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="skip the batched attention and expansion side measurements")
+    ap.add_argument("--extras-only", action="store_true", help="run only those side measurements (no bench line)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -101,11 +101,6 @@ __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)
 __device__ __forceinline__ void async_copy16(uint32_t dst_shared, const float* src) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst_shared), "l"(src) : "memory");
 }
-__device__ __forceinline__ float4 load_shared16(uint32_t addr) {
-    float4 v;
-    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
-    return v;
-}
 __device__ __forceinline__ void async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int PENDING>
 __device__ __forceinline__ void async_wait() {
@@ -187,7 +182,8 @@ expand_kernel(const float* __restrict__ draft_logits, long long batch_stride, in
     // ===== streaming warps ==============================================================================
     // Vector path: float4 i of this lane sits 4096 bytes * i past the lane's first one in global
     // memory and 512 bytes * i past it in the warp's ring slot.
-    const uint32_t ring_addr = smem_addr(s_ring + (size_t)warp * kDepth * (32 * NE)) + (uint32_t)lane * 16u;
+    const float* ring_lane = s_ring + (size_t)warp * kDepth * (32 * NE) + lane * 4;
+    const uint32_t ring_addr = smem_addr(ring_lane);
     const float* src_next = zrow + (size_t)t0 * kTileTokens + threadIdx.x * 4;  // of the next tile to request
     int t_issue = t0, slot_issue = 0;
     auto issue_next = [&]() {  // requests one more tile (nothing once the segment is exhausted); one group each
@@ -252,11 +248,18 @@ expand_kernel(const float* __restrict__ draft_logits, long long batch_stride, in
             m_t = tm;
         }
         if (m_t > -INFINITY) {
-            const float neg = -m_t * kLog2e;
-            float acc[4] = {0.f, 0.f, 0.f, 0.f};  // four chains instead of one of sixteen additions
+            // packed pairs: two elements per multiply-add and per addition, four chains of additions
+            const float2 scale2 = make_float2(kLog2e, kLog2e), neg2 = make_float2(-m_t * kLog2e, -m_t * kLog2e);
+            float2 acc_a = make_float2(0.f, 0.f), acc_b = make_float2(0.f, 0.f);
 #pragma unroll
-            for (int j = 0; j < NE; ++j) acc[j & 3] += fast_ex2(fmaf(cur[j], kLog2e, neg));
-            s_t += (acc[0] + acc[1]) + (acc[2] + acc[3]);
+            for (int j = 0; j < NE; j += 4) {
+                float2 a = __ffma2_rn(make_float2(cur[j], cur[j + 1]), scale2, neg2);
+                float2 c2 = __ffma2_rn(make_float2(cur[j + 2], cur[j + 3]), scale2, neg2);
+                a.x = fast_ex2(a.x), a.y = fast_ex2(a.y), c2.x = fast_ex2(c2.x), c2.y = fast_ex2(c2.y);
+                acc_a = __fadd2_rn(acc_a, a);
+                acc_b = __fadd2_rn(acc_b, c2);
+            }
+            s_t += (acc_a.x + acc_a.y) + (acc_b.x + acc_b.y);
         }
         const uint32_t block_code = *reinterpret_cast<volatile uint32_t*>(&s_bar_code);
         float thr = block_code ? order_decode(block_code) : -INFINITY;
@@ -339,13 +342,21 @@ expand_kernel(const float* __restrict__ draft_logits, long long batch_stride, in
         if (VEC) {
             issue_next();
             async_wait<2>();  // tile t has landed; t+1 and t+2 may still be in flight
-            const uint32_t slot = ring_addr + (uint32_t)slot_read * (32 * NE * 4);
+            const float4* slot = reinterpret_cast<const float4*>(ring_lane + slot_read * (32 * NE));
             slot_read = slot_read == kDepth - 1 ? 0 : slot_read + 1;
+            if (!ragged) {
 #pragma unroll
-            for (int i = 0; i < VPT; ++i) {
-                float4 v = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
-                if (!ragged || scan_elem_index<VPT, true>(t, 4 * i) < V) v = load_shared16(slot + i * 512);
-                cur[4 * i + 0] = v.x, cur[4 * i + 1] = v.y, cur[4 * i + 2] = v.z, cur[4 * i + 3] = v.w;
+                for (int i = 0; i < VPT; ++i) {
+                    const float4 v = slot[i * 32];
+                    cur[4 * i + 0] = v.x, cur[4 * i + 1] = v.y, cur[4 * i + 2] = v.z, cur[4 * i + 3] = v.w;
+                }
+            } else {
+#pragma unroll
+                for (int i = 0; i < VPT; ++i) {
+                    float4 v = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+                    if (scan_elem_index<VPT, true>(t, 4 * i) < V) v = slot[i * 32];
+                    cur[4 * i + 0] = v.x, cur[4 * i + 1] = v.y, cur[4 * i + 2] = v.z, cur[4 * i + 3] = v.w;
+                }
             }
         } else if (t + 1 < t1) {
             scan_load<VPT, false>(zrow, V, t + 1, nxt);
