@@ -132,77 +132,6 @@ __device__ __forceinline__ unsigned long long warp_sort_desc_u64(unsigned long l
     return v;
 }
 
-constexpr int kCandCap = 512;  // candidate keys a block can stage for the filtered selection
-
-struct TopkScratch {
-    unsigned long long cand[kCandCap];
-    unsigned long long exact[kScanWarps * EAGLE2_MAX_K];
-    unsigned long long win[EAGLE2_MAX_K];  // winners of an exact selection over one tile
-    int count;
-    int overflow;
-    float thr;  // value of the block's k-th best key so far (-inf: fewer than k keys yet)
-};
-
-// Block-level top-k (k <= 32) of the chunk elements x[] held in registers, written by warp 0 to
-// out[0..k) as selection keys (descending; 0 = none).  Each warp takes the k-th largest of its lanes'
-// maxima as a threshold: at least k of its elements reach it and none below it can be among the
-// warp's k best, so only elements at or above it get a key and are staged and ranked.  If a block
-// stages more than kCandCap keys (possible for heavily ordered input) it falls back to k rounds of
-// exact warp selection over all keys.
-// The caller zeroes scratch->count and scratch->overflow and synchronises before the call.
-template <int VPT, bool VEC>
-__device__ __forceinline__ void block_topk_filtered(const float (&x)[4 * VPT], int chunk, int V, int k,
-                                                    TopkScratch* scratch, unsigned long long* out) {
-    constexpr int NE = 4 * VPT;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    float lane_max = -INFINITY;  // positions beyond V were loaded as -inf
-#pragma unroll
-    for (int j = 0; j < NE; ++j) lane_max = fmaxf(lane_max, x[j]);
-    const float sorted = warp_sort_desc_f32(lane_max);
-    const float thr = __shfl_sync(0xffffffffu, sorted, k - 1);
-    int cnt = 0;
-#pragma unroll
-    for (int j = 0; j < NE; ++j) cnt += (x[j] >= thr) && (scan_elem_index<VPT, VEC>(chunk, j) < V);
-    int incl = cnt;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const int up = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += up;
-    }
-    const int total = __shfl_sync(0xffffffffu, incl, 31);
-    int base = 0;
-    if (lane == 0) base = atomicAdd(&scratch->count, total);
-    base = __shfl_sync(0xffffffffu, base, 0);
-    if (base + total <= kCandCap) {
-        int pos = base + incl - cnt;
-#pragma unroll
-        for (int j = 0; j < NE; ++j) {
-            const int e = scan_elem_index<VPT, VEC>(chunk, j);
-            if (x[j] >= thr && e < V) scratch->cand[pos++] = make_key(x[j], (uint32_t)e);
-        }
-    } else if (lane == 0) {
-        scratch->overflow = 1;
-    }
-    __syncthreads();
-    if (scratch->overflow) {  // uniform over the block
-        unsigned long long key[NE];
-#pragma unroll
-        for (int j = 0; j < NE; ++j) {
-            const int e = scan_elem_index<VPT, VEC>(chunk, j);
-            key[j] = e < V ? make_key(x[j], (uint32_t)e) : 0ull;
-        }
-        block_topk<NE>(key, k, scratch->exact, out);
-        return;
-    }
-    if (warp == 0) {
-        const int n = scratch->count;
-        unsigned long long mine[kCandCap / 32];
-#pragma unroll
-        for (int t = 0; t < kCandCap / 32; ++t) mine[t] = lane + 32 * t < n ? scratch->cand[lane + 32 * t] : 0ull;
-        warp_select<kCandCap / 32>(mine, k, out);
-    }
-}
-
 // Choose elements per chunk (as float4 per thread: 1, 2 or 4) so that a launch fills the GPU when
 // it can and no row is cut into more pieces than the merge step can hold.
 inline int scan_pick_vpt(long long rows, int V) {
