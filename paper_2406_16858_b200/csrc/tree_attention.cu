@@ -29,7 +29,8 @@ namespace eagle2 {
 
 constexpr int kTK = 128;              // keys per K/V tile = N of the Q.K^T instruction
 constexpr int kRowsPerTile = 128;     // M of every tcgen05.mma
-constexpr int kMaxTilesPerSplit = 16; // a block never streams more than 2048 keys
+constexpr int kMaxTilesPerSplit = 16; // a block never streams more than 2048 keys ...
+constexpr int kMaxTilesPerSplitOrdered = 32;  // ... 4096 when the launch runs its longest blocks first
 constexpr int kTmemCols = 512;
 constexpr int kSlots = 2;             // score slots in tensor memory
 constexpr int kAttnThreads = 320;     // 8 softmax warps, the TMA warp, the MMA warp
@@ -51,6 +52,9 @@ struct AttnPlan {
     int pair;       // 1: two blocks (a cluster on one TPC) share every K/V tile through cta_group::2
                     // MMAs: each holds 128 of the 256 query rows, half of each K tile's keys and
                     // half of each V tile's columns
+    int ordered;    // 1: a small kernel first lists the (sequence, split) items that have tiles, longest
+                    // first, and blocks take their item from that list (ragged batches: the last wave
+                    // is then made of the shortest blocks, and idle splits cost nothing)
     size_t smem;
 };
 
@@ -72,7 +76,10 @@ static void attention_plan(int B, int m, int Hq, int Hkv, int d, int max_kv_len,
     if (s < 1) s = 1;
     if (s > tiles) s = tiles;
     int per_split = (int)((tiles + s - 1) / s);
-    if (per_split > kMaxTilesPerSplit) per_split = kMaxTilesPerSplit;
+    // a batch whose longest sequence needs several blocks anyway: order them, and let each stream more
+    p->ordered = (B > 1 && !p->pair && per_split > kMaxTilesPerSplit) ? 1 : 0;
+    const int cap = p->ordered ? kMaxTilesPerSplitOrdered : kMaxTilesPerSplit;
+    if (per_split > cap) per_split = cap;
     if (per_split < 1) per_split = 1;
     p->per_split = per_split;
     p->splits = (tiles + per_split - 1) / per_split;
@@ -90,19 +97,26 @@ static void attention_plan(int B, int m, int Hq, int Hkv, int d, int max_kv_len,
 struct AttnWs {
     float* o_part;  // [B][Hkv][splits][n_rb][mt*128][d]
     float2* ml;     // [B][Hkv][splits][n_rb][mt*128]  (reference maximum in log2 units, sum)
+    uint32_t* order;  // ordered launches: [0] = items with tiles, [1 + i] = sequence * splits + split of item i
 };
 
 static size_t attention_ws_layout(int B, int Hkv, int d, const AttnPlan& p, void* base, AttnWs* w) {
-    if (p.splits == 1) return 0;
-    const size_t rows = (size_t)B * Hkv * p.splits * p.n_rb * p.mt * kRowsPerTile;
+    if (p.splits == 1 && !p.ordered) return 0;
     // every operation keeps its arrival counters (B ints) at the start of the workspace and leaves
-    // them zero; the partials go behind that region so that a shared workspace stays valid
+    // them zero; everything else goes behind that region so that a shared workspace stays valid
     size_t off = round_up(sizeof(int) * (size_t)B, kWsAlign);
     char* c = static_cast<char*>(base);
-    if (w) w->o_part = reinterpret_cast<float*>(c + off);
-    off += round_up(rows * d * sizeof(float), kWsAlign);
-    if (w) w->ml = reinterpret_cast<float2*>(c + off);
-    off += round_up(rows * sizeof(float2), kWsAlign);
+    if (p.splits > 1) {
+        const size_t rows = (size_t)B * Hkv * p.splits * p.n_rb * p.mt * kRowsPerTile;
+        if (w) w->o_part = reinterpret_cast<float*>(c + off);
+        off += round_up(rows * d * sizeof(float), kWsAlign);
+        if (w) w->ml = reinterpret_cast<float2*>(c + off);
+        off += round_up(rows * sizeof(float2), kWsAlign);
+    }
+    if (p.ordered) {
+        if (w) w->order = reinterpret_cast<uint32_t*>(c + off);
+        off += round_up(sizeof(uint32_t) * ((size_t)B * p.splits + 1), kWsAlign);
+    }
     return off;
 }
 
@@ -583,12 +597,23 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
     chain_release();  // the merge kernel of this call (or whatever follows) may be scheduled from here on
 
     int bid = PAIR ? blockIdx.x >> 1 : blockIdx.x;
-    const int split = bid % S;
-    bid /= S;
-    const int rb = bid % plan.n_rb;
-    bid /= plan.n_rb;
-    const int hk = bid % Hkv;
-    const int b = bid / Hkv;
+    int split, rb, hk, b;
+    if (!PAIR && plan.ordered) {  // item-major: the list says which (sequence, split) this block serves
+        rb = bid % plan.n_rb;
+        bid /= plan.n_rb;
+        hk = bid % Hkv;
+        const int item = bid / Hkv;
+        if (item >= (int)ws.order[0]) return;  // (ordered launches set up after this point)
+        const uint32_t packed = ws.order[1 + item];
+        b = (int)(packed / (uint32_t)S), split = (int)(packed % (uint32_t)S);
+    } else {
+        split = bid % S;
+        bid /= S;
+        rb = bid % plan.n_rb;
+        bid /= plan.n_rb;
+        hk = bid % Hkv;
+        b = bid / Hkv;
+    }
 
     const int L_raw = kv_len[b];
     const long long row_base = kv_off[b];
@@ -1066,6 +1091,44 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
     if (PAIR) cluster_sync_all();  // neither block leaves while the other may still signal it
 }
 
+// Ordered launches: one block lists the (sequence, split) items that have tiles, most tiles first
+// (a counting sort over the tile counts; the order among equals is whatever the atomics give, which
+// changes nothing but the schedule).
+__global__ void __launch_bounds__(1024)
+tree_attention_schedule_kernel(const int64_t* __restrict__ kv_off, const int32_t* __restrict__ kv_len, int B, int m,
+                               long long cache_rows, int max_kv_len, AttnPlan plan, uint32_t* __restrict__ order) {
+    __shared__ int s_bin[kMaxTilesPerSplitOrdered + 1];  // per tile count: items, then the next free place
+    chain_wait();
+    chain_release();
+    const int S = plan.splits;
+    const long long n = (long long)B * S;
+    for (int i = threadIdx.x; i <= kMaxTilesPerSplitOrdered; i += blockDim.x) s_bin[i] = 0;
+    __syncthreads();
+    auto tiles_of = [&](long long item) {
+        const int b = (int)(item / S), split = (int)(item % S);
+        const int L = kv_len[b];
+        if (!sequence_ok(L, kv_off[b], m, max_kv_len, cache_rows)) return 0;
+        const int tiles = (L + m + kTK - 1) / kTK;
+        return max(0, min(plan.per_split, tiles - split * plan.per_split));
+    };
+    for (long long i = threadIdx.x; i < n; i += blockDim.x) atomicAdd(&s_bin[tiles_of(i)], 1);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int at = 0;
+        for (int t = kMaxTilesPerSplitOrdered; t >= 1; --t) {
+            const int c = s_bin[t];
+            s_bin[t] = at;
+            at += c;
+        }
+        order[0] = (uint32_t)at;
+    }
+    __syncthreads();
+    for (long long i = threadIdx.x; i < n; i += blockDim.x) {
+        const int t = tiles_of(i);
+        if (t > 0) order[1 + atomicAdd(&s_bin[t], 1)] = (uint32_t)i;
+    }
+}
+
 // One warp per output row of a sequence that used several splits: combine their partials.  The
 // lanes first fetch the splits' (maximum, sum) pairs side by side, then every lane owns DH/32
 // columns and the partial rows are fetched sixteen splits at a time before any is used.
@@ -1157,7 +1220,11 @@ static int launch_attention(const CUtensorMap& k_map, const CUtensorMap& v_map, 
         return EAGLE2_ERR_CUDA;
     }
     const long long blocks = (long long)B * Hkv * plan.n_rb * plan.splits * (PAIR ? 2 : 1);
-    if (blocks > 0x7fffffffLL) return EAGLE2_ERR_SHAPE;
+    if (blocks > 0x7fffffffLL || (long long)B * plan.splits > 0x7fffffffLL) return EAGLE2_ERR_SHAPE;
+    if (plan.ordered &&
+        launch_chained(tree_attention_schedule_kernel, dim3(1), dim3(1024), 0, st, 1, kv_off, kv_len, B, m, cache_rows,
+                       max_kv_len, plan, ws.order) != EAGLE2_OK)
+        return EAGLE2_ERR_CUDA;
     if (launch_chained(kern, dim3((unsigned)blocks), dim3(kAttnThreads), plan.smem, st, PAIR ? 2u : 1u, k_map, v_map, q_map,
                        static_cast<const __nv_bfloat16*>(q), kv_off, kv_len, mask_bits, m, Hq, Hkv, cache_rows, max_kv_len,
                        plan, scale * 1.4426950408889634f, static_cast<__nv_bfloat16*>(out), lse, ws, d_status) != EAGLE2_OK)
@@ -1194,10 +1261,11 @@ extern "C" int eagle2_tree_attention(const void* q, const void* k_cache, const v
     if (B == 0) return EAGLE2_OK;
     AttnPlan plan;
     attention_plan(B, m, Hq, Hkv, d, max_kv_len, &plan);
-    AttnWs w = {nullptr, nullptr};
-    if (plan.splits > 1) {
+    AttnWs w = {nullptr, nullptr, nullptr};
+    if (plan.splits > 1 || plan.ordered) {
         if (!ws || !aligned(ws, kWsAlign)) return EAGLE2_ERR_WORKSPACE;
         if (attention_ws_layout(B, Hkv, d, plan, ws, &w) > ws_bytes) return EAGLE2_ERR_WORKSPACE;
+        if (plan.ordered && !w.order) return EAGLE2_ERR_WORKSPACE;
     }
     CUtensorMap k_map, v_map, q_map;
     // a pair block loads 64 keys of every K tile (and all 128 keys of 64 V columns)

@@ -89,3 +89,11 @@ def test_null_and_shape_errors_are_found_on_the_host():
 def test_zero_batch_is_a_no_op():
     e2.rerank(FAKE, FAKE, FAKE, 0, 4, 3, 16, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE)
     e2.tree_mask(FAKE, FAKE, FAKE, FAKE, 0, 16, FAKE, None, FAKE, FAKE)
+
+
+def test_ordered_attention_launch_reports_its_list():
+    # 17 tiles per sequence and one block per (sequence, head): no partials, but the launch takes its
+    # blocks from a device-built list, which lives in the workspace
+    with_list = e2.workspace_bytes(e2.OP_TREE_ATTENTION, B=8, m=60, Hq=16, Hkv=16, d=128, max_kv_len=2100)
+    without = e2.workspace_bytes(e2.OP_TREE_ATTENTION, B=8, m=60, Hq=16, Hkv=16, d=128, max_kv_len=1900)
+    assert with_list >= 256 + 4 * 9 and without == 0
