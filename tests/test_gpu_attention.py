@@ -95,6 +95,21 @@ def test_many_tiles_per_block(m, Hq, Hkv, d, lens):
     _compare(q, kc, vc, off, kl, bits, 1.0 / np.sqrt(d), samples=samples)
 
 
+def test_ragged_batch_runs_longest_first_with_several_splits():
+    """192 (sequence, KV head) pairs and sequences of up to 71 tiles: the launch is ordered by a
+    device-built list, long sequences are cut into splits of 32 tiles and merged, short ones write
+    their rows directly, two sequences are empty."""
+    m, Hq, Hkv, d = 60, 32, 8, 128
+    lens = [9000, 300, 4500, 20, 70, 5200, 1300, 0, 4037, 4036, 8100, 64, 2500, 1, 700, 3100,
+            128, 4097, 0, 950, 6000, 33, 2047, 410]
+    q, kc, vc, off, kl, bits = _inputs(31, len(lens), m, Hq, Hkv, d, lens)
+    rng = np.random.default_rng(6)
+    n = 600
+    samples = np.stack([rng.integers(0, len(lens), n), rng.integers(0, Hq, n),
+                        rng.integers(0, m, n)], axis=1).astype(np.int32)
+    _compare(q, kc, vc, off, kl, bits, 1.0 / np.sqrt(d), samples=samples)
+
+
 def test_rows_after_a_sequence_may_hold_anything():
     """The kernel streams whole tiles, so it reads cache rows that follow a sequence's last key; their
     contents (here NaN and Inf bit patterns) must not reach the output."""
