@@ -22,6 +22,7 @@
 #include <math.h>
 
 #include <mutex>
+#include <type_traits>
 
 #include "common.cuh"
 
@@ -1139,18 +1140,20 @@ tree_attention_merge_kernel(const int64_t* __restrict__ kv_off, const int32_t* _
                             float* __restrict__ lse) {
     chain_wait();  // the attention kernel's partials are complete
     chain_release();
-    const int warp_global = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    const int lane = threadIdx.x & 31;
     const int g = plan.g, S = plan.splits;
     const long long total = (long long)B * Hkv * plan.M;
-    if (warp_global >= total) return;
-    const int pr = warp_global % plan.M;
-    const int hk = (warp_global / plan.M) % Hkv;
-    const int b = warp_global / (plan.M * Hkv);
+    const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
+    // a large batch is walked by a grid of a few blocks per SM: most rows need no merge
+    for (long long row = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; row < total; row += warps) {
+    const int pr = (int)(row % plan.M);
+    const int hk = (int)((row / plan.M) % Hkv);
+    const int b = (int)(row / ((long long)plan.M * Hkv));
     const int L = kv_len[b];
-    if (!sequence_ok(L, kv_off[b], m, max_kv_len, cache_rows)) return;
+    if (!sequence_ok(L, kv_off[b], m, max_kv_len, cache_rows)) continue;
     const int tiles = (L + m + kTK - 1) / kTK;
     const int S_b = (tiles + plan.per_split - 1) / plan.per_split;
-    if (S_b <= 1) return;  // the attention kernel wrote these rows itself
+    if (S_b <= 1) continue;  // the attention kernel wrote these rows itself
     const int rb = pr / plan.per, r = pr % plan.per;
     const size_t rows_per_block = (size_t)plan.mt * kRowsPerTile;
     const size_t stride = (size_t)plan.n_rb * rows_per_block;  // rows between consecutive splits
@@ -1171,29 +1174,38 @@ tree_attention_merge_kernel(const int64_t* __restrict__ kv_off, const int32_t* _
             if (ml.x != -INFINITY) w = exp2f(ml.x - mmax), l += ml.y * w;
         }
         const int n = min(32, S_b - s0);
-        for (int s1 = 0; s1 < n; s1 += 16) {
-            float v[16][PER];
+        // W partial rows are fetched before any is used: 16 when the sequence has many splits (one
+        // round trip for the batch-1 layer's nine), fewer when it has few, so that short lists do not
+        // fetch the same row over and over
+        auto take = [&](auto width_tag) {
+            constexpr int W = decltype(width_tag)::value;
+            for (int s1 = 0; s1 < n; s1 += W) {
+                float v[W][PER];
 #pragma unroll
-            for (int u = 0; u < 16; ++u) {
-                const int sl = min(s1 + u, n - 1);  // clamped: a repeated row gets weight 0 below
-                const float* src = ws.o_part + (first + (size_t)(s0 + sl) * stride) * DH + lane * PER;
-                if (PER == 4) {
-                    const float4 t = *reinterpret_cast<const float4*>(src);
-                    v[u][0] = t.x, v[u][1] = t.y, v[u][PER - 2] = t.z, v[u][PER - 1] = t.w;
-                } else {
-                    const float2 t = *reinterpret_cast<const float2*>(src);
-                    v[u][0] = t.x, v[u][1] = t.y;
+                for (int u = 0; u < W; ++u) {
+                    const int sl = min(s1 + u, n - 1);  // clamped: a repeated row gets weight 0 below
+                    const float* src = ws.o_part + (first + (size_t)(s0 + sl) * stride) * DH + lane * PER;
+                    if (PER == 4) {
+                        const float4 t = *reinterpret_cast<const float4*>(src);
+                        v[u][0] = t.x, v[u][1] = t.y, v[u][PER - 2] = t.z, v[u][PER - 1] = t.w;
+                    } else {
+                        const float2 t = *reinterpret_cast<const float2*>(src);
+                        v[u][0] = t.x, v[u][1] = t.y;
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < W; ++u) {
+                    float wu = __shfl_sync(0xffffffffu, w, min(s1 + u, 31));
+                    if (s1 + u >= n) wu = 0.f;
+                    // a split without visible keys leaves its partial row unwritten: never multiply it
+#pragma unroll
+                    for (int e = 0; e < PER; ++e) acc[e] += wu != 0.f ? v[u][e] * wu : 0.f;
                 }
             }
-#pragma unroll
-            for (int u = 0; u < 16; ++u) {
-                float wu = __shfl_sync(0xffffffffu, w, min(s1 + u, 31));
-                if (s1 + u >= n) wu = 0.f;
-                // a split without visible keys leaves its partial row unwritten: never multiply it
-#pragma unroll
-                for (int e = 0; e < PER; ++e) acc[e] += wu != 0.f ? v[u][e] * wu : 0.f;
-            }
-        }
+        };
+        if (n > 8) take(std::integral_constant<int, 16>{});
+        else if (n > 4) take(std::integral_constant<int, 8>{});
+        else take(std::integral_constant<int, 4>{});
     }
     l = warp_sum_f32(l);
     const float inv = l > 0.f ? 1.f / l : 0.f;
@@ -1204,6 +1216,7 @@ tree_attention_merge_kernel(const int64_t* __restrict__ kv_off, const int32_t* _
         *reinterpret_cast<uint32_t*>(dst + e) = pack_bf16(acc[e] * inv, acc[e + 1] * inv);
     if (lse && lane == 0)
         lse[((long long)b * Hq + hq) * m + tok] = (mmax + log2f(l)) * 0.69314718055994531f;
+    }
 }
 
 template <int DH, int MT, bool PAIR>
@@ -1231,8 +1244,8 @@ static int launch_attention(const CUtensorMap& k_map, const CUtensorMap& v_map, 
         return EAGLE2_ERR_CUDA;
     if (plan.splits > 1) {
         const long long warps = (long long)B * Hkv * plan.M;
-        const long long mblocks = (warps + 7) / 8;
-        if (mblocks > 0x7fffffffLL) return EAGLE2_ERR_SHAPE;
+        long long mblocks = (warps + 7) / 8;
+        if (mblocks > 8 * 148) mblocks = 8 * 148;
         if (launch_chained(tree_attention_merge_kernel<DH>, dim3((unsigned)mblocks), dim3(256), 0, st, 1, kv_off, kv_len, B, m,
                            Hq, Hkv, cache_rows, max_kv_len, plan, ws, static_cast<__nv_bfloat16*>(out), lse) != EAGLE2_OK)
             return EAGLE2_ERR_CUDA;
