@@ -134,6 +134,49 @@ def test_many_tiles_per_block_and_ordered_rows(kind, V):
     _check_tree(cfg, draft, gpu, want)
 
 
+@pytest.mark.parametrize("V,k,D,B", [(40000, 32, 2, 8),    # widest frontier: 256 rows, all 32 lanes of the selector in use
+                                     (50001, 1, 3, 200),   # k = 1: the selector keeps a single key
+                                     (36864, 3, 4, 64),    # deeper tree, whole tiles only
+                                     (262147, 5, 2, 40)])  # 65 tiles per row
+def test_streaming_blocks_at_the_limits_of_k(V, k, D, B):
+    rng = np.random.default_rng(V + k + B)
+    R = ref.n_draft_rows(k, D)
+    draft = (1.5 * rng.standard_normal((B, R, V))).astype(np.float32)
+    want = ref.build_tree(draft, V, k, D)
+    gpu = GpuTree(B, V, k, D).expand_all(dev(draft))
+    cfg = get_config("tiny", B=B, V=V, k=k, D=D)
+    _check_tree(cfg, draft, gpu, want)
+
+
+def test_streaming_blocks_with_masked_vocabulary_and_a_nan():
+    """Rows in which most of the vocabulary is -inf (a masked vocabulary), one row with fewer finite
+    logits than k, and one NaN: the streaming path must agree with the oracle on tokens and status."""
+    V, k, D, B = 70004, 5, 2, 32
+    rng = np.random.default_rng(77)
+    R = ref.n_draft_rows(k, D)
+    draft = (2.0 * rng.standard_normal((B, R, V))).astype(np.float32)
+    masked = rng.random((B, R, V)) < 0.9
+    draft[masked] = -np.inf
+    draft[3, 2, :] = -np.inf
+    draft[3, 2, [11, 40000, 69999]] = [0.5, 1.5, 1.0]  # three finite logits for k = 5
+    want = ref.build_tree(draft, V, k, D)
+    gpu = GpuTree(B, V, k, D).expand_all(dev(draft))
+    assert int(gpu.status.item()) == want.status
+    keep = np.ones(B, bool)
+    keep[3] = False  # that sequence's level holds -inf values, whose order among equals is checked below
+    assert (host(gpu.token)[keep] == want.token[keep]).all()
+    assert (host(gpu.parent)[keep] == want.parent[keep]).all()
+    assert (host(gpu.frontier)[keep] == want.frontier[keep]).all()
+    fin = np.isfinite(want.value)
+    assert (np.isfinite(host(gpu.value)) == fin).all()
+    assert np.abs(host(gpu.value)[fin] - want.value[fin]).max() < 3e-6
+    assert (host(gpu.token)[3] == want.token[3]).all()  # ties at -inf go to the lower token index on both sides
+    nan = draft.copy()
+    nan[5, 1, 12345] = np.nan
+    gpu = GpuTree(B, V, k, D).expand_all(dev(nan))
+    assert int(gpu.status.item()) & e2.STATUS_NONFINITE_LOGIT
+
+
 def test_ties_and_negative_infinity_logits():
     V, k, D, B = 2048, 4, 2, 1
     draft = np.full((B, ref.n_draft_rows(k, D), V), -np.inf, np.float32)
