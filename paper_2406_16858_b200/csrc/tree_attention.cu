@@ -1138,19 +1138,29 @@ __global__ void __launch_bounds__(256)
 tree_attention_merge_kernel(const int64_t* __restrict__ kv_off, const int32_t* __restrict__ kv_len, int B, int m,
                             int Hq, int Hkv, long long cache_rows, int max_kv_len, AttnPlan plan, AttnWs ws, __nv_bfloat16* __restrict__ out,
                             float* __restrict__ lse) {
-    chain_wait();  // the attention kernel's partials are complete
-    chain_release();
     const int lane = threadIdx.x & 31;
     const int g = plan.g, S = plan.splits;
     const long long total = (long long)B * Hkv * plan.M;
     const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
+    const long long row_first = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    // The sequence lengths are final before this kernel can start (the attention kernel lets its
+    // dependents in only after its own predecessors are complete, and does not write them): the
+    // first row's are read while the attention kernel is still running.
+    int len_first = 0;
+    long long off_first = 0;
+    if (row_first < total) {
+        const int b0 = (int)(row_first / ((long long)plan.M * Hkv));
+        len_first = kv_len[b0], off_first = kv_off[b0];
+    }
+    chain_wait();  // the attention kernel's partials are complete
+    chain_release();
     // a large batch is walked by a grid of a few blocks per SM: most rows need no merge
-    for (long long row = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; row < total; row += warps) {
+    for (long long row = row_first; row < total; row += warps) {
     const int pr = (int)(row % plan.M);
     const int hk = (int)((row / plan.M) % Hkv);
     const int b = (int)(row / ((long long)plan.M * Hkv));
-    const int L = kv_len[b];
-    if (!sequence_ok(L, kv_off[b], m, max_kv_len, cache_rows)) continue;
+    const int L = row == row_first ? len_first : kv_len[b];
+    if (!sequence_ok(L, row == row_first ? off_first : kv_off[b], m, max_kv_len, cache_rows)) continue;
     const int tiles = (L + m + kTK - 1) / kTK;
     const int S_b = (tiles + plan.per_split - 1) / plan.per_split;
     if (S_b <= 1) continue;  // the attention kernel wrote these rows itself
@@ -1158,41 +1168,47 @@ tree_attention_merge_kernel(const int64_t* __restrict__ kv_off, const int32_t* _
     const size_t rows_per_block = (size_t)plan.mt * kRowsPerTile;
     const size_t stride = (size_t)plan.n_rb * rows_per_block;  // rows between consecutive splits
     const size_t first = (((size_t)b * Hkv + hk) * S) * stride + rb * rows_per_block + r;
-    float mmax = -INFINITY;
-    for (int s0 = 0; s0 < S_b; s0 += 32)
-        if (s0 + lane < S_b) mmax = fmaxf(mmax, ws.ml[first + (size_t)(s0 + lane) * stride].x);
-    mmax = warp_max_f32(mmax);
     constexpr int PER = DH / 32;  // 4 or 2 consecutive columns per lane
     float acc[PER];
 #pragma unroll
     for (int e = 0; e < PER; ++e) acc[e] = 0.f;
-    float l = 0.f;
-    for (int s0 = 0; s0 < S_b; s0 += 32) {
-        float w = 0.f;  // weight of split s0 + lane
-        if (s0 + lane < S_b) {
-            const float2 ml = ws.ml[first + (size_t)(s0 + lane) * stride];
-            if (ml.x != -INFINITY) w = exp2f(ml.x - mmax), l += ml.y * w;
-        }
-        const int n = min(32, S_b - s0);
-        // W partial rows are fetched before any is used: 16 when the sequence has many splits (one
-        // round trip for the batch-1 layer's nine), fewer when it has few, so that short lists do not
-        // fetch the same row over and over
-        auto take = [&](auto width_tag) {
-            constexpr int W = decltype(width_tag)::value;
-            for (int s1 = 0; s1 < n; s1 += W) {
-                float v[W][PER];
+    float l = 0.f, mmax = -INFINITY;
+    // W partial rows are fetched before any is used: 16 when the sequence has many splits (one round
+    // trip for the batch-1 layer's nine), fewer when it has few, so that short lists do not fetch the
+    // same row over and over.  The first batch of rows is requested together with the splits'
+    // (maximum, sum) pairs: neither address depends on the other's data.
+    auto run = [&](auto width_tag) {
+        constexpr int W = decltype(width_tag)::value;
+        float v[W][PER];
+        auto fetch = [&](int s0, int s1, int n) {
 #pragma unroll
-                for (int u = 0; u < W; ++u) {
-                    const int sl = min(s1 + u, n - 1);  // clamped: a repeated row gets weight 0 below
-                    const float* src = ws.o_part + (first + (size_t)(s0 + sl) * stride) * DH + lane * PER;
-                    if (PER == 4) {
-                        const float4 t = *reinterpret_cast<const float4*>(src);
-                        v[u][0] = t.x, v[u][1] = t.y, v[u][PER - 2] = t.z, v[u][PER - 1] = t.w;
-                    } else {
-                        const float2 t = *reinterpret_cast<const float2*>(src);
-                        v[u][0] = t.x, v[u][1] = t.y;
-                    }
+            for (int u = 0; u < W; ++u) {
+                const int sl = min(s1 + u, n - 1);  // clamped: a repeated row gets weight 0 below
+                const float* src = ws.o_part + (first + (size_t)(s0 + sl) * stride) * DH + lane * PER;
+                if (PER == 4) {
+                    const float4 t = *reinterpret_cast<const float4*>(src);
+                    v[u][0] = t.x, v[u][1] = t.y, v[u][PER - 2] = t.z, v[u][PER - 1] = t.w;
+                } else {
+                    const float2 t = *reinterpret_cast<const float2*>(src);
+                    v[u][0] = t.x, v[u][1] = t.y;
                 }
+            }
+        };
+        const int n0 = min(32, S_b);
+        const float2 ml0 = lane < n0 ? ws.ml[first + (size_t)lane * stride] : make_float2(-INFINITY, 0.f);
+        fetch(0, 0, n0);
+        mmax = ml0.x;
+        for (int s0 = 32; s0 < S_b; s0 += 32)
+            if (s0 + lane < S_b) mmax = fmaxf(mmax, ws.ml[first + (size_t)(s0 + lane) * stride].x);
+        mmax = warp_max_f32(mmax);
+        for (int s0 = 0; s0 < S_b; s0 += 32) {
+            const int n = min(32, S_b - s0);
+            float2 ml = ml0;
+            if (s0) ml = lane < n ? ws.ml[first + (size_t)(s0 + lane) * stride] : make_float2(-INFINITY, 0.f);
+            float w = 0.f;  // weight of split s0 + lane
+            if (lane < n && ml.x != -INFINITY) w = exp2f(ml.x - mmax), l += ml.y * w;
+            for (int s1 = 0; s1 < n; s1 += W) {
+                if (s0 || s1) fetch(s0, s1, n);
 #pragma unroll
                 for (int u = 0; u < W; ++u) {
                     float wu = __shfl_sync(0xffffffffu, w, min(s1 + u, 31));
@@ -1202,11 +1218,11 @@ tree_attention_merge_kernel(const int64_t* __restrict__ kv_off, const int32_t* _
                     for (int e = 0; e < PER; ++e) acc[e] += wu != 0.f ? v[u][e] * wu : 0.f;
                 }
             }
-        };
-        if (n > 8) take(std::integral_constant<int, 16>{});
-        else if (n > 4) take(std::integral_constant<int, 8>{});
-        else take(std::integral_constant<int, 4>{});
-    }
+        }
+    };
+    if (S_b > 8) run(std::integral_constant<int, 16>{});
+    else if (S_b > 4) run(std::integral_constant<int, 8>{});
+    else run(std::integral_constant<int, 4>{});
     l = warp_sum_f32(l);
     const float inv = l > 0.f ? 1.f / l : 0.f;
     const int tok = pr / g, hq = hk * g + pr % g;
