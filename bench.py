@@ -273,6 +273,54 @@ def batched_expand_extra(e2, dev, stream, hbm_peak, B=128, n_sets=4, reps=20):
             "algorithmic_bytes_per_call": nbytes, "achieved_gbs": gbs, "frac_of_measured_hbm": gbs / hbm_peak}
 
 
+def batched_accept_extra(e2, dev, stream, hbm_peak, B=16, reps=10):
+    """Acceptance at temperature 1 alone for B sequences of the LLaMA3-8B-shaped tree: per sequence the
+    target and draft rows of every node that has selected children are read (once each), plus the
+    two rows of the stopping node for the extra token.  One input set (0.9 GB) is larger than L2."""
+    import torch
+    from paper_2406_16858_b200.cycle import CycleBuffers, CycleShape
+    cfg = get_config("llama3_8b").with_(B=B, temperature=1.0)
+    shape = CycleShape(cfg.B, cfg.V, cfg.k, cfg.D, cfg.m, 1, cfg.Hq, cfg.Hkv, cfg.d, 64, cfg.temperature)
+    buf = CycleBuffers(shape, dev)
+    g = torch.Generator(device=dev).manual_seed(11)
+    draft = torch.from_numpy(gen.draft_rows(cfg, 5)).to(dev)
+    kv_len = torch.zeros(B, dtype=torch.int32, device=dev)
+    with torch.cuda.stream(stream):
+        buf.expand_all(draft)
+        buf.rerank_and_mask(kv_len)
+    torch.cuda.synchronize()
+    nd = gen.node_draft_rows(buf.tree_parent.cpu().numpy(), cfg.k, cfg.D)
+    sel_index, sel_parent = buf.sel_index.cpu().numpy(), buf.sel_parent.cpu().numpy()
+    src_rows = np.zeros((B, cfg.m + 1), np.int64)
+    parents = 0  # nodes (the root included) with at least one selected child
+    for b in range(B):
+        for x in range(cfg.m):
+            r = nd[b, sel_index[b, x]] if sel_index[b, x] >= 0 else -1
+            src_rows[b, 1 + x] = r if r >= 0 else (x * 7 + 3) % cfg.R
+        parents += len(set(int(q) for q, i in zip(sel_parent[b], sel_index[b]) if i >= 0))
+    base = torch.gather(draft, 1, torch.from_numpy(src_rows).to(dev)[:, :, None].expand(-1, -1, cfg.V))
+    target = (base + 0.5 * torch.randn(base.shape, generator=g, device=dev)).contiguous()
+    del base
+    ua_h, ub_h = gen.uniforms(cfg, 5)
+    ua, ub = torch.from_numpy(ua_h).to(dev), torch.from_numpy(ub_h).to(dev)
+    with torch.cuda.stream(stream):
+        for _ in range(3):
+            buf.accept(target, draft, ua, ub)
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev0.record(stream)
+        for _ in range(reps):
+            buf.accept(target, draft, ua, ub)
+        ev1.record(stream)
+    torch.cuda.synchronize()
+    assert int(buf.status.item()) == 0
+    us = ev0.elapsed_time(ev1) * 1e3 / reps
+    nbytes = float(parents + B) * 2 * cfg.V * 4
+    gbs = nbytes / (us * 1e-6) / 1e9
+    return {"workload": f"llama3_8b acceptance at temperature 1, B={B} ({parents} nodes with selected children)",
+            "us_per_call": us, "algorithmic_bytes_per_call": nbytes, "achieved_gbs": gbs,
+            "frac_of_measured_hbm": gbs / hbm_peak}
+
+
 # ------------------------------------------------------------------------------------------------
 # the CUDA path
 
@@ -297,7 +345,8 @@ def run_ours(args):
         stream = torch.cuda.Stream(device=dev)
         hbm_peak = _peaks()[0]
         print(json.dumps({"attention_batched": batched_attention_extra(e2, dev, stream, hbm_peak),
-                          "expand_batched": batched_expand_extra(e2, dev, stream, hbm_peak)}))
+                          "expand_batched": batched_expand_extra(e2, dev, stream, hbm_peak),
+                          "accept_batched": batched_accept_extra(e2, dev, stream, hbm_peak)}))
         return
     cfg = get_config(args.workload)
     if args.batch:
@@ -502,6 +551,7 @@ def run_ours(args):
     if world == 1 and not args.no_extras:
         line["attention_batched"] = batched_attention_extra(e2, dev, stream, hbm_peak)
         line["expand_batched"] = batched_expand_extra(e2, dev, stream, hbm_peak)
+        line["accept_batched"] = batched_accept_extra(e2, dev, stream, hbm_peak)
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
@@ -516,7 +566,7 @@ def main():
     ap.add_argument("--workload", default="llama3_8b")
     ap.add_argument("--batch", type=int, default=0, help="override the number of sequences")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-extras", action="store_true", help="skip the batched attention and expansion side measurements")
+    ap.add_argument("--no-extras", action="store_true", help="skip the batched attention, expansion and acceptance side measurements")
     ap.add_argument("--extras-only", action="store_true", help="run only those side measurements (no bench line)")
     args = ap.parse_args()
     if args.impl == "reference":
