@@ -233,8 +233,9 @@ __global__ void __launch_bounds__(kChainThreads)
 accept_chain_kernel(const float* __restrict__ target_logits, long long t_stride,
                     const float* __restrict__ draft_logits_all, long long d_stride,
                     const int32_t* __restrict__ sel_index, const int32_t* __restrict__ sel_parent,
-                    const int32_t* __restrict__ sel_token, const int32_t* __restrict__ n_sel, int V,
-                    int k, int m, int R, int slice, float inv_t, AcceptWs ws, int32_t* d_status) {
+                    const int32_t* __restrict__ sel_token, const int32_t* __restrict__ n_sel,
+                    const float* __restrict__ u_accept, int V, int k, int m, int R, int slice, float inv_t,
+                    AcceptWs ws, int32_t* d_status) {
     chain_wait();
     chain_release();
     cg::cluster_group cluster = cg::this_cluster();
@@ -248,7 +249,7 @@ accept_chain_kernel(const float* __restrict__ target_logits, long long t_stride,
     __shared__ double s_redd[kChainWarps];
     __shared__ float s_redf[kChainWarps];
     __shared__ int s_child[EAGLE2_MAX_K], s_ctok[EAGLE2_MAX_K];
-    __shared__ float s_pf[EAGLE2_MAX_K], s_qf[EAGLE2_MAX_K];
+    __shared__ float s_pf[EAGLE2_MAX_K], s_qf[EAGLE2_MAX_K], s_uc[EAGLE2_MAX_K];  // children's p, q, uniform
     __shared__ double s_frozen[EAGLE2_MAX_K];
     __shared__ int s_nchild, s_parent;
 
@@ -259,6 +260,7 @@ accept_chain_kernel(const float* __restrict__ target_logits, long long t_stride,
     if (tid < EAGLE2_MAX_M) {
         const int x = tid;
         int tokx = 0, parx = -1;
+        float ux = 0.f;
         bool match = false;
         if (x < ns) {
             const int idx = sel_index[(long long)b * m + x];
@@ -266,6 +268,7 @@ accept_chain_kernel(const float* __restrict__ target_logits, long long t_stride,
             if (match) {
                 tokx = sel_token[(long long)b * m + x];
                 parx = sel_parent[(long long)b * m + x];
+                ux = u_accept[(long long)b * m + x];
             }
         }
         const unsigned bal = __ballot_sync(0xffffffffu, match);
@@ -280,6 +283,7 @@ accept_chain_kernel(const float* __restrict__ target_logits, long long t_stride,
         if (match && before < EAGLE2_MAX_K) {
             s_child[before] = x;
             s_ctok[before] = tokx;
+            s_uc[before] = ux;
             if (before == 0) s_parent = parx;
         }
         if (tid == 0) s_nchild = min(total, EAGLE2_MAX_K);
@@ -371,12 +375,6 @@ accept_chain_kernel(const float* __restrict__ target_logits, long long t_stride,
         for (int e = tid; e < n_local; e += kChainThreads)
             part_f1 += fmaxf(fmaf(-1.0f, prob_of(zq[lo + e], inv_t, gmax_q, c_q), prob_of(zp[lo + e], inv_t, gmax_p, c_p)), 0.f);
     }
-    double f_one = 0.0;
-    if (full_q && nc > 1) {
-        double unused = 0.0;
-        f_one = chain_block_sum((double)part_f1, s_redd);
-        cluster_allreduce2<false>(cluster, f_one, unused, s_xchg, parity);
-    }
     // the children's own probabilities, computed exactly like the resident values
     if (tid < nc) {
         const int t = s_ctok[tid];
@@ -428,6 +426,9 @@ accept_chain_kernel(const float* __restrict__ target_logits, long long t_stride,
         else
             a = pj > 0.0 ? 1.0 : 0.0;
         if (writer) thr[s_child[j]] = a;
+        // The walk takes the first child whose uniform is below its threshold and never looks at a
+        // later sibling: the chain of this node ends here (same decision in every thread and block).
+        if ((double)s_uc[j] < a) break;
 
         // residual after rejecting child j: alpha grows by beta * s for every token still in q
         const double alpha_new = alpha + beta * s;
@@ -440,8 +441,10 @@ accept_chain_kernel(const float* __restrict__ target_logits, long long t_stride,
             break;
         }
         double f_new;
-        if (j == 0) {
-            f_new = f_one;  // alpha_new == 1
+        if (j == 0) {  // alpha_new == 1: the sum was taken in the normalisation sweep
+            double unused = 0.0;
+            f_new = chain_block_sum((double)part_f1, s_redd);
+            cluster_allreduce2<false>(cluster, f_new, unused, s_xchg, parity);
         } else {
             float part = 0.f;
             for (int e = tid; e < n_local; e += kChainThreads) {
@@ -837,15 +840,15 @@ extern "C" int eagle2_accept(const float* target_logits, long long t_stride,
     if ((long long)B * cs > 0x7fffffffLL || R > 65535) return EAGLE2_ERR_SHAPE;
 
     void (*chain)(const float*, long long, const float*, long long, const int32_t*, const int32_t*,
-                  const int32_t*, const int32_t*, int, int, int, int, int, float, AcceptWs, int32_t*) =
+                  const int32_t*, const int32_t*, const float*, int, int, int, int, int, float, AcceptWs, int32_t*) =
         resident ? (vec ? accept_chain_kernel<true, true> : accept_chain_kernel<true, false>)
                  : (vec ? accept_chain_kernel<false, true> : accept_chain_kernel<false, false>);
     if (dyn > 40 * 1024 &&
         cudaFuncSetAttribute(chain, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) != cudaSuccess)
         return EAGLE2_ERR_CUDA;
     if (launch_chained(chain, dim3((unsigned)(B * cs), (unsigned)R, 1), dim3(kChainThreads), dyn, st, (unsigned)cs,
-                       target_logits, t_stride, draft_logits_all, d_stride, sel_index, sel_parent, sel_token, n_sel, V,
-                       k, m, R, slice, inv_t, w, d_status) != EAGLE2_OK)
+                       target_logits, t_stride, draft_logits_all, d_stride, sel_index, sel_parent, sel_token, n_sel,
+                       u_accept, V, k, m, R, slice, inv_t, w, d_status) != EAGLE2_OK)
         return EAGLE2_ERR_CUDA;
 
     const long long blocks = (long long)B * bchunks;
