@@ -56,6 +56,8 @@ struct AttnPlan {
     int ordered;    // 1: a small kernel first lists the (sequence, split) items that have tiles, longest
                     // first, and blocks take their item from that list (ragged batches: the last wave
                     // is then made of the shortest blocks, and idle splits cost nothing)
+    int fused_merge;  // 1 (ordered launches with several splits): the last block of a (sequence, KV head, row
+                      // block) to finish combines the splits' partials itself, while other blocks still run
     size_t smem;
 };
 
@@ -84,6 +86,7 @@ static void attention_plan(int B, int m, int Hq, int Hkv, int d, int max_kv_len,
     if (per_split < 1) per_split = 1;
     p->per_split = per_split;
     p->splits = (tiles + per_split - 1) / per_split;
+    p->fused_merge = (p->ordered && p->splits > 1) ? 1 : 0;
     const size_t unit = (size_t)(d / 64) * kTK * 128;  // one 128-row operand tile
     int stages = (int)((220 * 1024 - p->mt * unit) / (2 * unit));
     p->stages = stages > 4 ? 4 : (stages < 2 ? 2 : stages);
@@ -99,6 +102,7 @@ struct AttnWs {
     float* o_part;  // [B][Hkv][splits][n_rb][mt*128][d]
     float2* ml;     // [B][Hkv][splits][n_rb][mt*128]  (reference maximum in log2 units, sum)
     uint32_t* order;  // ordered launches: [0] = items with tiles, [1 + i] = sequence * splits + split of item i
+    int* tickets;     // merging launches: [B][Hkv][n_rb] arrival counters, left at zero
 };
 
 static size_t attention_ws_layout(int B, int Hkv, int d, const AttnPlan& p, void* base, AttnWs* w) {
@@ -117,6 +121,10 @@ static size_t attention_ws_layout(int B, int Hkv, int d, const AttnPlan& p, void
     if (p.ordered) {
         if (w) w->order = reinterpret_cast<uint32_t*>(c + off);
         off += round_up(sizeof(uint32_t) * ((size_t)B * p.splits + 1), kWsAlign);
+    }
+    if (p.fused_merge) {
+        if (w) w->tickets = reinterpret_cast<int*>(c + off);
+        off += round_up(sizeof(int) * (size_t)B * Hkv * p.n_rb, kWsAlign);
     }
     return off;
 }
@@ -512,6 +520,85 @@ __device__ __forceinline__ void tile_visibility(unsigned long long mlo, unsigned
         else hi = 0;
     }
     vis[0] = (uint32_t)lo, vis[1] = (uint32_t)(lo >> 32), vis[2] = (uint32_t)hi, vis[3] = (uint32_t)(hi >> 32);
+}
+
+// One warp combines the partials of one packed query row `pr` of (sequence b, KV head hk) that was
+// computed in S_b > 1 splits: the lanes fetch the splits' (maximum, sum) pairs side by side, then
+// every lane owns DH/32 columns of the row.
+template <int DH>
+__device__ __forceinline__ void merge_row(const AttnPlan& plan, const AttnWs& ws, int b, int hk, int pr, int S_b,
+                                          int m, int Hq, int Hkv, __nv_bfloat16* __restrict__ out,
+                                          float* __restrict__ lse) {
+    const int lane = threadIdx.x & 31;
+    const int g = plan.g, S = plan.splits;
+    const int rb = pr / plan.per, r = pr % plan.per;
+    const size_t rows_per_block = (size_t)plan.mt * kRowsPerTile;
+    const size_t stride = (size_t)plan.n_rb * rows_per_block;  // rows between consecutive splits
+    const size_t first = (((size_t)b * Hkv + hk) * S) * stride + rb * rows_per_block + r;
+    constexpr int PER = DH / 32;  // 4 or 2 consecutive columns per lane
+    float acc[PER];
+#pragma unroll
+    for (int e = 0; e < PER; ++e) acc[e] = 0.f;
+    float l = 0.f, mmax = -INFINITY;
+    // W partial rows are fetched before any is used: 16 when the sequence has many splits (one round
+    // trip for the batch-1 layer's nine), fewer when it has few, so that short lists do not fetch the
+    // same row over and over.  The first batch of rows is requested together with the splits'
+    // (maximum, sum) pairs: neither address depends on the other's data.
+    auto run = [&](auto width_tag) {
+        constexpr int W = decltype(width_tag)::value;
+        float v[W][PER];
+        auto fetch = [&](int s0, int s1, int n) {
+#pragma unroll
+            for (int u = 0; u < W; ++u) {
+                const int sl = min(s1 + u, n - 1);  // clamped: a repeated row gets weight 0 below
+                const float* src = ws.o_part + (first + (size_t)(s0 + sl) * stride) * DH + lane * PER;
+                if (PER == 4) {
+                    const float4 t = *reinterpret_cast<const float4*>(src);
+                    v[u][0] = t.x, v[u][1] = t.y, v[u][PER - 2] = t.z, v[u][PER - 1] = t.w;
+                } else {
+                    const float2 t = *reinterpret_cast<const float2*>(src);
+                    v[u][0] = t.x, v[u][1] = t.y;
+                }
+            }
+        };
+        const int n0 = min(32, S_b);
+        const float2 ml0 = lane < n0 ? ws.ml[first + (size_t)lane * stride] : make_float2(-INFINITY, 0.f);
+        fetch(0, 0, n0);
+        mmax = ml0.x;
+        for (int s0 = 32; s0 < S_b; s0 += 32)
+            if (s0 + lane < S_b) mmax = fmaxf(mmax, ws.ml[first + (size_t)(s0 + lane) * stride].x);
+        mmax = warp_max_f32(mmax);
+        for (int s0 = 0; s0 < S_b; s0 += 32) {
+            const int n = min(32, S_b - s0);
+            float2 ml = ml0;
+            if (s0) ml = lane < n ? ws.ml[first + (size_t)(s0 + lane) * stride] : make_float2(-INFINITY, 0.f);
+            float w = 0.f;  // weight of split s0 + lane
+            if (lane < n && ml.x != -INFINITY) w = exp2f(ml.x - mmax), l += ml.y * w;
+            for (int s1 = 0; s1 < n; s1 += W) {
+                if (s0 || s1) fetch(s0, s1, n);
+#pragma unroll
+                for (int u = 0; u < W; ++u) {
+                    float wu = __shfl_sync(0xffffffffu, w, min(s1 + u, 31));
+                    if (s1 + u >= n) wu = 0.f;
+                    // a split without visible keys leaves its partial row unwritten: never multiply it
+#pragma unroll
+                    for (int e = 0; e < PER; ++e) acc[e] += wu != 0.f ? v[u][e] * wu : 0.f;
+                }
+            }
+        }
+    };
+    if (S_b > 8) run(std::integral_constant<int, 16>{});
+    else if (S_b > 4) run(std::integral_constant<int, 8>{});
+    else run(std::integral_constant<int, 4>{});
+    l = warp_sum_f32(l);
+    const float inv = l > 0.f ? 1.f / l : 0.f;
+    const int tok = pr / g, hq = hk * g + pr % g;
+    __nv_bfloat16* dst = out + (((long long)b * m + tok) * Hq + hq) * DH + lane * PER;
+#pragma unroll
+    for (int e = 0; e < PER; e += 2)
+        *reinterpret_cast<uint32_t*>(dst + e) = pack_bf16(acc[e] * inv, acc[e + 1] * inv);
+    if (lse && lane == 0)
+        lse[((long long)b * Hq + hq) * m + tok] = (mmax + log2f(l)) * 0.69314718055994531f;
 }
 
 template <int DH, int MT, bool PAIR>
@@ -1079,6 +1166,15 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
 
     }  // active
 
+    // ---- merging launches: whoever finishes a (sequence, KV head, row block) last combines its splits
+    if (!PAIR && plan.fused_merge && !direct) {  // uniform over the block; blocks without tiles left long ago
+        __shared__ int s_last;
+        if (last_block_arrives(ws.tickets + ((size_t)b * Hkv + hk) * plan.n_rb + rb, S_b, &s_last)) {
+            for (int r = warp; r < rows_blk; r += kAttnThreads / 32)
+                merge_row<DH>(plan, ws, b, hk, rb * plan.per + r, S_b, m, Hq, Hkv, out, lse);
+        }
+    }
+
     // ---- teardown ----------------------------------------------------------------------------------
     tc_fence_before();
     if (PAIR) cluster_sync_all();  // tensor memory is released by both blocks together
@@ -1130,16 +1226,13 @@ tree_attention_schedule_kernel(const int64_t* __restrict__ kv_off, const int32_t
     }
 }
 
-// One warp per output row of a sequence that used several splits: combine their partials.  The
-// lanes first fetch the splits' (maximum, sum) pairs side by side, then every lane owns DH/32
-// columns and the partial rows are fetched sixteen splits at a time before any is used.
+// One warp per output row of a sequence that used several splits (launches that do not merge inside
+// the attention kernel).
 template <int DH>
 __global__ void __launch_bounds__(256)
 tree_attention_merge_kernel(const int64_t* __restrict__ kv_off, const int32_t* __restrict__ kv_len, int B, int m,
                             int Hq, int Hkv, long long cache_rows, int max_kv_len, AttnPlan plan, AttnWs ws, __nv_bfloat16* __restrict__ out,
                             float* __restrict__ lse) {
-    const int lane = threadIdx.x & 31;
-    const int g = plan.g, S = plan.splits;
     const long long total = (long long)B * Hkv * plan.M;
     const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
     const long long row_first = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -1156,82 +1249,15 @@ tree_attention_merge_kernel(const int64_t* __restrict__ kv_off, const int32_t* _
     chain_release();
     // a large batch is walked by a grid of a few blocks per SM: most rows need no merge
     for (long long row = row_first; row < total; row += warps) {
-    const int pr = (int)(row % plan.M);
-    const int hk = (int)((row / plan.M) % Hkv);
-    const int b = (int)(row / ((long long)plan.M * Hkv));
-    const int L = row == row_first ? len_first : kv_len[b];
-    if (!sequence_ok(L, row == row_first ? off_first : kv_off[b], m, max_kv_len, cache_rows)) continue;
-    const int tiles = (L + m + kTK - 1) / kTK;
-    const int S_b = (tiles + plan.per_split - 1) / plan.per_split;
-    if (S_b <= 1) continue;  // the attention kernel wrote these rows itself
-    const int rb = pr / plan.per, r = pr % plan.per;
-    const size_t rows_per_block = (size_t)plan.mt * kRowsPerTile;
-    const size_t stride = (size_t)plan.n_rb * rows_per_block;  // rows between consecutive splits
-    const size_t first = (((size_t)b * Hkv + hk) * S) * stride + rb * rows_per_block + r;
-    constexpr int PER = DH / 32;  // 4 or 2 consecutive columns per lane
-    float acc[PER];
-#pragma unroll
-    for (int e = 0; e < PER; ++e) acc[e] = 0.f;
-    float l = 0.f, mmax = -INFINITY;
-    // W partial rows are fetched before any is used: 16 when the sequence has many splits (one round
-    // trip for the batch-1 layer's nine), fewer when it has few, so that short lists do not fetch the
-    // same row over and over.  The first batch of rows is requested together with the splits'
-    // (maximum, sum) pairs: neither address depends on the other's data.
-    auto run = [&](auto width_tag) {
-        constexpr int W = decltype(width_tag)::value;
-        float v[W][PER];
-        auto fetch = [&](int s0, int s1, int n) {
-#pragma unroll
-            for (int u = 0; u < W; ++u) {
-                const int sl = min(s1 + u, n - 1);  // clamped: a repeated row gets weight 0 below
-                const float* src = ws.o_part + (first + (size_t)(s0 + sl) * stride) * DH + lane * PER;
-                if (PER == 4) {
-                    const float4 t = *reinterpret_cast<const float4*>(src);
-                    v[u][0] = t.x, v[u][1] = t.y, v[u][PER - 2] = t.z, v[u][PER - 1] = t.w;
-                } else {
-                    const float2 t = *reinterpret_cast<const float2*>(src);
-                    v[u][0] = t.x, v[u][1] = t.y;
-                }
-            }
-        };
-        const int n0 = min(32, S_b);
-        const float2 ml0 = lane < n0 ? ws.ml[first + (size_t)lane * stride] : make_float2(-INFINITY, 0.f);
-        fetch(0, 0, n0);
-        mmax = ml0.x;
-        for (int s0 = 32; s0 < S_b; s0 += 32)
-            if (s0 + lane < S_b) mmax = fmaxf(mmax, ws.ml[first + (size_t)(s0 + lane) * stride].x);
-        mmax = warp_max_f32(mmax);
-        for (int s0 = 0; s0 < S_b; s0 += 32) {
-            const int n = min(32, S_b - s0);
-            float2 ml = ml0;
-            if (s0) ml = lane < n ? ws.ml[first + (size_t)(s0 + lane) * stride] : make_float2(-INFINITY, 0.f);
-            float w = 0.f;  // weight of split s0 + lane
-            if (lane < n && ml.x != -INFINITY) w = exp2f(ml.x - mmax), l += ml.y * w;
-            for (int s1 = 0; s1 < n; s1 += W) {
-                if (s0 || s1) fetch(s0, s1, n);
-#pragma unroll
-                for (int u = 0; u < W; ++u) {
-                    float wu = __shfl_sync(0xffffffffu, w, min(s1 + u, 31));
-                    if (s1 + u >= n) wu = 0.f;
-                    // a split without visible keys leaves its partial row unwritten: never multiply it
-#pragma unroll
-                    for (int e = 0; e < PER; ++e) acc[e] += wu != 0.f ? v[u][e] * wu : 0.f;
-                }
-            }
-        }
-    };
-    if (S_b > 8) run(std::integral_constant<int, 16>{});
-    else if (S_b > 4) run(std::integral_constant<int, 8>{});
-    else run(std::integral_constant<int, 4>{});
-    l = warp_sum_f32(l);
-    const float inv = l > 0.f ? 1.f / l : 0.f;
-    const int tok = pr / g, hq = hk * g + pr % g;
-    __nv_bfloat16* dst = out + (((long long)b * m + tok) * Hq + hq) * DH + lane * PER;
-#pragma unroll
-    for (int e = 0; e < PER; e += 2)
-        *reinterpret_cast<uint32_t*>(dst + e) = pack_bf16(acc[e] * inv, acc[e + 1] * inv);
-    if (lse && lane == 0)
-        lse[((long long)b * Hq + hq) * m + tok] = (mmax + log2f(l)) * 0.69314718055994531f;
+        const int pr = (int)(row % plan.M);
+        const int hk = (int)((row / plan.M) % Hkv);
+        const int b = (int)(row / ((long long)plan.M * Hkv));
+        const int L = row == row_first ? len_first : kv_len[b];
+        if (!sequence_ok(L, row == row_first ? off_first : kv_off[b], m, max_kv_len, cache_rows)) continue;
+        const int tiles = (L + m + kTK - 1) / kTK;
+        const int S_b = (tiles + plan.per_split - 1) / plan.per_split;
+        if (S_b <= 1) continue;  // the attention kernel wrote these rows itself
+        merge_row<DH>(plan, ws, b, hk, pr, S_b, m, Hq, Hkv, out, lse);
     }
 }
 
@@ -1258,7 +1284,7 @@ static int launch_attention(const CUtensorMap& k_map, const CUtensorMap& v_map, 
                        static_cast<const __nv_bfloat16*>(q), kv_off, kv_len, mask_bits, m, Hq, Hkv, cache_rows, max_kv_len,
                        plan, scale * 1.4426950408889634f, static_cast<__nv_bfloat16*>(out), lse, ws, d_status) != EAGLE2_OK)
         return EAGLE2_ERR_CUDA;
-    if (plan.splits > 1) {
+    if (plan.splits > 1 && !plan.fused_merge) {
         const long long warps = (long long)B * Hkv * plan.M;
         long long mblocks = (warps + 7) / 8;
         if (mblocks > 8 * 148) mblocks = 8 * 148;
@@ -1290,11 +1316,11 @@ extern "C" int eagle2_tree_attention(const void* q, const void* k_cache, const v
     if (B == 0) return EAGLE2_OK;
     AttnPlan plan;
     attention_plan(B, m, Hq, Hkv, d, max_kv_len, &plan);
-    AttnWs w = {nullptr, nullptr, nullptr};
+    AttnWs w = {nullptr, nullptr, nullptr, nullptr};
     if (plan.splits > 1 || plan.ordered) {
         if (!ws || !aligned(ws, kWsAlign)) return EAGLE2_ERR_WORKSPACE;
         if (attention_ws_layout(B, Hkv, d, plan, ws, &w) > ws_bytes) return EAGLE2_ERR_WORKSPACE;
-        if (plan.ordered && !w.order) return EAGLE2_ERR_WORKSPACE;
+        if ((plan.ordered && !w.order) || (plan.fused_merge && !w.tickets)) return EAGLE2_ERR_WORKSPACE;
     }
     CUtensorMap k_map, v_map, q_map;
     // a pair block loads 64 keys of every K tile (and all 128 keys of 64 V columns)
