@@ -151,9 +151,11 @@ expand_kernel(const float* __restrict__ draft_logits, long long batch_stride, in
     constexpr float kLog2e = 1.4426950408889634f;
     extern __shared__ __align__(16) float s_ring[];  // [kScanWarps][kDepth][512] (vector path)
     __shared__ unsigned long long s_list[kScanWarps][kWarpList];  // !STREAM: the warps' candidate lists
-    __shared__ unsigned long long s_queue[STREAM ? kQueue : 1];   // STREAM: keys on their way to the selector (0: empty)
+    __shared__ unsigned long long s_queue[kQueue];  // STREAM: keys on their way to the selector (0: empty);
+                                                     // otherwise: the block's surviving candidates at the end
     __shared__ int s_count[kScanWarps];
     __shared__ int s_tail, s_head, s_done;  // STREAM: slots reserved / consumed, streaming warps finished
+                                            // (otherwise s_tail counts the surviving candidates)
     __shared__ uint32_t s_bar_code;         // the bar as a value code (0: none yet)
     __shared__ float s_wmax[kScanWarps], s_wsum[kScanWarps];
     __shared__ int s_flag;
@@ -381,15 +383,7 @@ expand_kernel(const float* __restrict__ draft_logits, long long batch_stride, in
         __syncwarp();
         if (lane == 0) atomicAdd(&s_done, 1);
     } else {
-        if (n > 32) {
-            unsigned long long mine[2] = {list[lane], lane + 32 < n ? list[lane + 32] : 0ull};
-            __syncwarp();
-            warp_select<2>(mine, k, list);
-        } else {
-            const unsigned long long sorted = warp_sort_desc_u64(lane < n ? list[lane] : 0ull);
-            __syncwarp();
-            if (lane < k) list[lane] = sorted;  // zeros where fewer than k keys exist
-        }
+        if (lane == 0) s_count[warp] = n;
     }
     } else {
     // ===== selector warp (STREAM) ==========================================================================
@@ -451,18 +445,55 @@ expand_kernel(const float* __restrict__ draft_logits, long long batch_stride, in
 
     if constexpr (!STREAM) {
         __syncthreads();
-        // The block's k best of the warps' k best: every thread ranks one of the 8k keys by counting
-        // the keys above it (keys differ, so ranks do), and the ranks below k are the winners' places.
-        const int n_keys = kScanWarps * k;  // <= 256 = threads
-        const unsigned long long mine = (int)threadIdx.x < n_keys ? s_list[threadIdx.x / k][threadIdx.x % k] : 0ull;
-        int rank = 0;
-        if (mine) {
-            for (int w = 0; w < kScanWarps; ++w)
-                for (int r = 0; r < k; ++r) rank += s_list[w][r] > mine;
-            if (rank < k) ws.keys[part * k + rank] = mine;
+        // The block's k-th best reaches the largest of the warps' bars, so only the listed candidates
+        // at or above it can be among the block's k best: usually a couple of dozen.  They are
+        // gathered and every one is ranked by counting the ones above it (keys differ, so ranks do);
+        // the ranks below k are the winners' places.
+        const uint32_t bar_code = s_bar_code;
+        const int n_w = s_count[warp];
+#pragma unroll
+        for (int u = 0; u < kWarpList / 32; ++u) {
+            const unsigned long long key = lane + 32 * u < n_w ? s_list[warp][lane + 32 * u] : 0ull;
+            if (key && (uint32_t)(key >> 32) >= bar_code) {
+                const int pos = atomicAdd(&s_tail, 1);
+                if (pos < kQueue) s_queue[pos] = key;
+            }
         }
-        const int present = __syncthreads_count(mine != 0ull);
-        if ((int)threadIdx.x >= present && (int)threadIdx.x < k) ws.keys[part * k + threadIdx.x] = 0ull;
+        __syncthreads();
+        const int n_final = s_tail;
+        if (n_final <= kQueue) {
+            const unsigned long long mine = (int)threadIdx.x < n_final ? s_queue[threadIdx.x] : 0ull;
+            if (mine) {
+                int rank = 0;
+                for (int j = 0; j < n_final; ++j) rank += s_queue[j] > mine;
+                if (rank < k) ws.keys[part * k + rank] = mine;
+            }
+            if ((int)threadIdx.x >= n_final && (int)threadIdx.x < k) ws.keys[part * k + threadIdx.x] = 0ull;
+        } else {
+            // no useful bar (ties, rows of -inf): every warp reduces its list to its k best, then the
+            // 8k keys are ranked in the same way
+            unsigned long long* list = s_list[warp];
+            if (n_w > 32) {
+                unsigned long long two[2] = {list[lane], lane + 32 < n_w ? list[lane + 32] : 0ull};
+                __syncwarp();
+                warp_select<2>(two, k, list);
+            } else {
+                const unsigned long long sorted = warp_sort_desc_u64(lane < n_w ? list[lane] : 0ull);
+                __syncwarp();
+                if (lane < k) list[lane] = sorted;  // zeros where fewer than k keys exist
+            }
+            __syncthreads();
+            const int n_keys = kScanWarps * k;  // <= 256 = threads
+            const unsigned long long mine = (int)threadIdx.x < n_keys ? s_list[threadIdx.x / k][threadIdx.x % k] : 0ull;
+            int rank = 0;
+            if (mine) {
+                for (int w = 0; w < kScanWarps; ++w)
+                    for (int r = 0; r < k; ++r) rank += s_list[w][r] > mine;
+                if (rank < k) ws.keys[part * k + rank] = mine;
+            }
+            const int present = __syncthreads_count(mine != 0ull);
+            if ((int)threadIdx.x >= present && (int)threadIdx.x < k) ws.keys[part * k + threadIdx.x] = 0ull;
+        }
         if (warp == 0) {
             const float pm = lane < kScanWarps ? s_wmax[lane] : -INFINITY;
             const float cmax = warp_max_f32(pm);
