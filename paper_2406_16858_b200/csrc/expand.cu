@@ -107,6 +107,26 @@ __device__ __forceinline__ void async_wait() {
     asm volatile("cp.async.wait_group %0;" ::"n"(PENDING) : "memory");
 }
 
+// warp_sort_desc_u64 for N independent keys per lane (key n of all lanes is one sequence): the N
+// chains of dependent shuffles advance side by side.
+template <int N>
+__device__ __forceinline__ void warp_sort_desc_u64_n(unsigned long long (&v)[N]) {
+    const int lane = threadIdx.x & 31;
+#pragma unroll
+    for (int size = 2; size <= 32; size <<= 1) {
+#pragma unroll
+        for (int stride = size >> 1; stride > 0; stride >>= 1) {
+            const bool desc = (lane & size) == 0, lower = (lane & stride) == 0;
+#pragma unroll
+            for (int n = 0; n < N; ++n) {
+                const unsigned long long other = __shfl_xor_sync(0xffffffffu, v[n], stride);
+                const unsigned long long hi = v[n] > other ? v[n] : other, lo = v[n] > other ? other : v[n];
+                v[n] = (lower == desc) ? hi : lo;
+            }
+        }
+    }
+}
+
 constexpr int kQueue = 256;                              // candidate keys in flight to the selector warp
 constexpr long long kExpandWaitCycles = 1LL << 31;       // ~1 s bound of every wait below
 
@@ -520,92 +540,161 @@ expand_kernel(const float* __restrict__ draft_logits, long long batch_stride, in
     __syncthreads();
     int status = 0;
 
-    for (int r = warp; r < n_s && warp < kScanWarps; r += kScanWarps) {
-        const size_t p0 = ((size_t)b * n_s + r) * chunks;
-        constexpr int BATCH = 16;  // chunk winners per lane and pass
-        // everything the row needs is requested before any of it is used
-        unsigned long long cand[BATCH + 1];
+    // A warp merges NR rows at a time, r and r + 8: the work of a row is a chain of dependent
+    // shuffles, so when there are more rows than warps (the ten rows of a step on eight warps) the
+    // second row rides along in the first one's latency instead of taking a second pass.
+    auto merge_rows = [&](auto nr_tag, auto batch_tag) {
+        constexpr int NR = decltype(nr_tag)::value;
+        constexpr int BATCH = decltype(batch_tag)::value;  // chunk winners per lane and pass
+        for (int r_base = warp; r_base < n_s; r_base += kScanWarps * NR) {
+            int r[NR];
+            bool valid[NR];
+            size_t p0[NR];
+            unsigned long long cand[NR][BATCH + 1];
+            double2 st0[NR];
+            int parent[NR];
+            double parent_value[NR], lse[NR];
+            // everything the rows need is requested before any of it is used
 #pragma unroll
-        for (int t = 0; t < BATCH; ++t)
-            cand[t] = lane + 32 * t < keys_per_row ? ws.keys[p0 * k + lane + 32 * t] : 0ull;
-        double2 st0 = make_double2(-INFINITY, 0.0);
-        if (lane < chunks) st0 = ws.stats[p0 + lane];
-        int parent = s ? s_parent[r] : -1;
-        const double parent_value = s ? s_pvalue[r] : 0.0;
-        if (parent < -1) {
-            status |= EAGLE2_STATUS_BAD_TREE;
-            parent = (int)(s >= 2 ? (long long)k + (long long)(s - 2) * k * k : 0);
-        }
-        // log-sum-exp of the row from the chunk partials, in double
-        double m = st0.x;
-        for (int c = lane + 32; c < chunks; c += 32) m = fmax(m, ws.stats[p0 + c].x);
-        m = warp_max_f64(m);
-        double sum = st0.x > -INFINITY ? st0.y * exp(st0.x - m) : 0.0;
-        for (int c = lane + 32; c < chunks; c += 32) {
-            const double2 st = ws.stats[p0 + c];
-            if (st.x > -INFINITY) sum += st.y * exp(st.x - m);
-        }
-        sum = warp_sum_f64(sum);
-        if (!(m > -INFINITY)) status |= EAGLE2_STATUS_NONFINITE_LOGIT;
-        const double lse = m + log(sum);
-        // top-k of the chunk winners, 32*BATCH at a time together with the best so far; lane c ends
-        // up holding the c-th.  The k-th largest lane maximum is a threshold no winner can be below;
-        // when at most 32 keys reach it (the usual case) they are sorted across the lanes, otherwise
-        // k rounds of maximum extraction do the same job.
-        unsigned long long* s_pack = s_list[warp];  // free: the segment scan is over
-        unsigned long long mine = 0;
-        for (int e0 = 0; e0 < keys_per_row; e0 += 32 * BATCH) {
-            if (e0) {
+            for (int q = 0; q < NR; ++q) {
+                r[q] = r_base + q * kScanWarps;
+                valid[q] = r[q] < n_s;
+                p0[q] = ((size_t)b * n_s + (valid[q] ? r[q] : 0)) * chunks;
 #pragma unroll
                 for (int t = 0; t < BATCH; ++t)
-                    cand[t] = e0 + lane + 32 * t < keys_per_row ? ws.keys[p0 * k + e0 + lane + 32 * t] : 0ull;
-            }
-            cand[BATCH] = mine;
-            unsigned long long lane_best = 0;
-#pragma unroll
-            for (int t = 0; t <= BATCH; ++t) lane_best = cand[t] > lane_best ? cand[t] : lane_best;
-            const unsigned long long thr = __shfl_sync(0xffffffffu, warp_sort_desc_u64(lane_best), k - 1);
-            int cnt = 0;
-#pragma unroll
-            for (int t = 0; t <= BATCH; ++t) cnt += cand[t] >= thr && cand[t] != 0ull;
-            int incl = cnt;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const int up = __shfl_up_sync(0xffffffffu, incl, o);
-                if (lane >= o) incl += up;
-            }
-            const int total = __shfl_sync(0xffffffffu, incl, 31);
-            unsigned long long next = 0;
-            if (total <= 32) {
-                int pos = incl - cnt;
-#pragma unroll
-                for (int t = 0; t <= BATCH; ++t)
-                    if (cand[t] >= thr && cand[t] != 0ull) s_pack[pos++] = cand[t];
-                __syncwarp();
-                next = warp_sort_desc_u64(lane < total ? s_pack[lane] : 0ull);
-                __syncwarp();
-                if (lane >= k) next = 0ull;
-            } else {
-                for (int c = 0; c < k; ++c) {
-                    unsigned long long best = 0;
-#pragma unroll
-                    for (int t = 0; t <= BATCH; ++t) best = cand[t] > best ? cand[t] : best;
-                    const unsigned long long top = warp_max_u64(best);
-#pragma unroll
-                    for (int t = 0; t <= BATCH; ++t) cand[t] = (cand[t] == top) ? 0ull : cand[t];
-                    if (lane == c) next = top;
+                    cand[q][t] = (valid[q] && lane + 32 * t < keys_per_row) ? ws.keys[p0[q] * k + lane + 32 * t] : 0ull;
+                st0[q] = make_double2(-INFINITY, 0.0);
+                if (valid[q] && lane < chunks) st0[q] = ws.stats[p0[q] + lane];
+                parent[q] = (s && valid[q]) ? s_parent[r[q]] : -1;
+                parent_value[q] = (s && valid[q]) ? s_pvalue[r[q]] : 0.0;
+                if (parent[q] < -1) {
+                    status |= EAGLE2_STATUS_BAD_TREE;
+                    parent[q] = (int)(s >= 2 ? (long long)k + (long long)(s - 2) * k * k : 0);
                 }
             }
-            mine = next;
+            // log-sum-exp of the rows from the chunk partials, in double
+#pragma unroll
+            for (int q = 0; q < NR; ++q) {
+                double m = st0[q].x;
+                if (valid[q])
+                    for (int c = lane + 32; c < chunks; c += 32) m = fmax(m, ws.stats[p0[q] + c].x);
+                m = warp_max_f64(m);
+                double sum = st0[q].x > -INFINITY ? st0[q].y * exp(st0[q].x - m) : 0.0;
+                if (valid[q])
+                    for (int c = lane + 32; c < chunks; c += 32) {
+                        const double2 st = ws.stats[p0[q] + c];
+                        if (st.x > -INFINITY) sum += st.y * exp(st.x - m);
+                    }
+                sum = warp_sum_f64(sum);
+                if (valid[q] && !(m > -INFINITY)) status |= EAGLE2_STATUS_NONFINITE_LOGIT;
+                lse[q] = m + log(sum);
+            }
+            // top-k of the chunk winners, 32*BATCH at a time together with the best so far; lane c ends
+            // up holding the c-th.  The k-th largest lane maximum is a threshold no winner can be below;
+            // when at most 32 keys reach it (the usual case) they are sorted across the lanes, otherwise
+            // k rounds of maximum extraction do the same job.
+            unsigned long long mine[NR];
+#pragma unroll
+            for (int q = 0; q < NR; ++q) mine[q] = 0ull;
+            for (int e0 = 0; e0 < keys_per_row; e0 += 32 * BATCH) {
+                unsigned long long thr[NR];
+                int cnt[NR], incl[NR], total[NR];
+#pragma unroll
+                for (int q = 0; q < NR; ++q) {
+                    if (e0) {
+#pragma unroll
+                        for (int t = 0; t < BATCH; ++t)
+                            cand[q][t] = (valid[q] && e0 + lane + 32 * t < keys_per_row)
+                                             ? ws.keys[p0[q] * k + e0 + lane + 32 * t]
+                                             : 0ull;
+                    }
+                    cand[q][BATCH] = mine[q];
+                }
+                unsigned long long lane_best[NR];
+#pragma unroll
+                for (int q = 0; q < NR; ++q) {
+                    lane_best[q] = 0;
+#pragma unroll
+                    for (int t = 0; t <= BATCH; ++t) lane_best[q] = cand[q][t] > lane_best[q] ? cand[q][t] : lane_best[q];
+                }
+                warp_sort_desc_u64_n<NR>(lane_best);
+#pragma unroll
+                for (int q = 0; q < NR; ++q) {
+                    thr[q] = __shfl_sync(0xffffffffu, lane_best[q], k - 1);
+                    cnt[q] = 0;
+#pragma unroll
+                    for (int t = 0; t <= BATCH; ++t) cnt[q] += cand[q][t] >= thr[q] && cand[q][t] != 0ull;
+                    incl[q] = cnt[q];
+                }
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+#pragma unroll
+                    for (int q = 0; q < NR; ++q) {
+                        const int up = __shfl_up_sync(0xffffffffu, incl[q], o);
+                        if (lane >= o) incl[q] += up;
+                    }
+                }
+                bool packed = true;
+                unsigned long long next[NR];
+#pragma unroll
+                for (int q = 0; q < NR; ++q) {
+                    total[q] = __shfl_sync(0xffffffffu, incl[q], 31);
+                    packed = packed && total[q] <= 32;
+                    next[q] = 0ull;
+                }
+                if (packed) {  // every row of the warp: pack, then sort the rows side by side
+#pragma unroll
+                    for (int q = 0; q < NR; ++q) {
+                        unsigned long long* s_pack = s_list[warp] + q * 32;  // free: the segment scan is over
+                        int pos = incl[q] - cnt[q];
+#pragma unroll
+                        for (int t = 0; t <= BATCH; ++t)
+                            if (cand[q][t] >= thr[q] && cand[q][t] != 0ull) s_pack[pos++] = cand[q][t];
+                    }
+                    __syncwarp();
+#pragma unroll
+                    for (int q = 0; q < NR; ++q) next[q] = lane < total[q] ? s_list[warp][q * 32 + lane] : 0ull;
+                    warp_sort_desc_u64_n<NR>(next);
+                    __syncwarp();
+#pragma unroll
+                    for (int q = 0; q < NR; ++q)
+                        if (lane >= k) next[q] = 0ull;
+                } else {
+#pragma unroll
+                    for (int q = 0; q < NR; ++q) {
+                        for (int c = 0; c < k; ++c) {
+                            unsigned long long best = 0;
+#pragma unroll
+                            for (int t = 0; t <= BATCH; ++t) best = cand[q][t] > best ? cand[q][t] : best;
+                            const unsigned long long top = warp_max_u64(best);
+#pragma unroll
+                            for (int t = 0; t <= BATCH; ++t) cand[q][t] = (cand[q][t] == top) ? 0ull : cand[q][t];
+                            if (lane == c) next[q] = top;
+                        }
+                    }
+                }
+#pragma unroll
+                for (int q = 0; q < NR; ++q) mine[q] = next[q];
+            }
+#pragma unroll
+            for (int q = 0; q < NR; ++q) {
+                if (valid[q] && lane < k) {
+                    const long long node = base + (long long)r[q] * k + lane;
+                    const double v = parent_value[q] + ((double)key_value(mine[q]) - lse[q]);
+                    tok[node] = (int32_t)key_index(mine[q]);
+                    par[node] = parent[q];
+                    val[node] = v;
+                    s_rank[r[q] * k + lane] = order_code_f64(v);
+                }
+            }
         }
-        if (lane < k) {
-            const long long node = base + (long long)r * k + lane;
-            const double v = parent_value + ((double)key_value(mine) - lse);
-            tok[node] = (int32_t)key_index(mine);
-            par[node] = parent;
-            val[node] = v;
-            s_rank[r * k + lane] = order_code_f64(v);
-        }
+    };
+    if (warp < kScanWarps) {
+        using std::integral_constant;
+        if (n_s > kScanWarps && n_s <= 2 * kScanWarps && keys_per_row <= 32 * 10)
+            merge_rows(integral_constant<int, 2>{}, integral_constant<int, 10>{});
+        else
+            merge_rows(integral_constant<int, 1>{}, integral_constant<int, 16>{});
     }
     __syncthreads();  // all rows merged (the old frontier was read when the kernel started)
 
