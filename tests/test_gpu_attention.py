@@ -110,6 +110,21 @@ def test_ragged_batch_runs_longest_first_with_several_splits():
     _compare(q, kc, vc, off, kl, bits, 1.0 / np.sqrt(d), samples=samples)
 
 
+@pytest.mark.parametrize("m,Hq,Hkv,d,B,longest", [
+    (33, 8, 8, 64, 20, 6000),    # head_dim 64: deeper K/V ring, two splits for the longest sequences
+    (40, 6, 2, 128, 80, 5000),   # three query heads per KV head: query rows copied by hand, not by TMA
+])
+def test_ordered_launch_other_shapes(m, Hq, Hkv, d, B, longest):
+    rng = np.random.default_rng(B + d)
+    lens = rng.integers(0, 900, B)
+    lens[[1, B // 2, B - 2]] = [longest, longest - 1700, longest - 300]
+    q, kc, vc, off, kl, bits = _inputs(41, B, m, Hq, Hkv, d, [int(x) for x in lens])
+    n = 500
+    samples = np.stack([rng.integers(0, B, n), rng.integers(0, Hq, n), rng.integers(0, m, n)], axis=1).astype(np.int32)
+    samples[:60, 0] = np.array([1, B // 2, B - 2])[rng.integers(0, 3, 60)]  # the split sequences for sure
+    _compare(q, kc, vc, off, kl, bits, 1.0 / np.sqrt(d), samples=samples)
+
+
 def test_rows_after_a_sequence_may_hold_anything():
     """The kernel streams whole tiles, so it reads cache rows that follow a sequence's last key; their
     contents (here NaN and Inf bit patterns) must not reach the output."""
