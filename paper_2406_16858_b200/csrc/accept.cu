@@ -223,7 +223,13 @@ __device__ __forceinline__ void cluster_allreduce2(cg::cluster_group& cluster, d
 // Probability of one token.  Explicit round-to-nearest operations (never contracted into an FMA)
 // so that a token looked up on its own gets bit for bit the value its resident copy has.
 __device__ __forceinline__ float scale_logit(float z, float inv_t) { return __fmul_rn(z, inv_t); }
-__device__ __forceinline__ float exp_scaled(float zs, float gmax) { return expf(__fsub_rn(zs, gmax)); }
+// exp(zs - gmax) as 2^((zs - gmax) * log2 e) with the hardware's approximate 2^x (2 ulp); the
+// difference and the product are separately rounded, so every caller gets the same bits for the same token
+__device__ __forceinline__ float exp_scaled(float zs, float gmax) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(__fmul_rn(__fsub_rn(zs, gmax), 1.4426950408889634f)));
+    return y;
+}
 __device__ __forceinline__ float prob_of(float z, float inv_t, float gmax, float c) {
     return __fmul_rn(exp_scaled(scale_logit(z, inv_t), gmax), c);
 }
@@ -308,20 +314,35 @@ accept_chain_kernel(const float* __restrict__ target_logits, long long t_stride,
     // ---- pass 1: scaled logits -> shared memory, maxima ---------------------------------------
     float mp = -INFINITY, mq = -INFINITY;
     if (VEC) {
-        for (int e = tid * 4; e < n_local; e += kChainThreads * 4) {
-            float4 a = __ldcs(reinterpret_cast<const float4*>(zp + lo + e));
-            a.x = scale_logit(a.x, inv_t), a.y = scale_logit(a.y, inv_t);
-            a.z = scale_logit(a.z, inv_t), a.w = scale_logit(a.w, inv_t);
-            bad |= !(a.x < INFINITY) | !(a.y < INFINITY) | !(a.z < INFINITY) | !(a.w < INFINITY);
-            mp = fmaxf(fmaxf(mp, fmaxf(a.x, a.y)), fmaxf(a.z, a.w));
-            if (RESIDENT) *reinterpret_cast<float4*>(sp + e) = a;
-            if (full_q) {
-                float4 c = __ldcs(reinterpret_cast<const float4*>(zq + lo + e));
-                c.x = scale_logit(c.x, inv_t), c.y = scale_logit(c.y, inv_t);
-                c.z = scale_logit(c.z, inv_t), c.w = scale_logit(c.w, inv_t);
-                bad |= !(c.x < INFINITY) | !(c.y < INFINITY) | !(c.z < INFINITY) | !(c.w < INFINITY);
-                mq = fmaxf(fmaxf(mq, fmaxf(c.x, c.y)), fmaxf(c.z, c.w));
-                if (RESIDENT) *reinterpret_cast<float4*>(sq + e) = c;
+        constexpr int kPre = 4;  // float4 per row requested before any is used
+        for (int e0 = tid * 4; e0 < n_local; e0 += kChainThreads * 4 * kPre) {
+            float4 a[kPre], c[kPre];
+#pragma unroll
+            for (int u = 0; u < kPre; ++u) {
+                const int e = e0 + u * kChainThreads * 4;
+                if (e < n_local) {
+                    a[u] = __ldcs(reinterpret_cast<const float4*>(zp + lo + e));
+                    if (full_q) c[u] = __ldcs(reinterpret_cast<const float4*>(zq + lo + e));
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < kPre; ++u) {
+                const int e = e0 + u * kChainThreads * 4;
+                if (e >= n_local) continue;
+                float4 x = a[u];
+                x.x = scale_logit(x.x, inv_t), x.y = scale_logit(x.y, inv_t);
+                x.z = scale_logit(x.z, inv_t), x.w = scale_logit(x.w, inv_t);
+                bad |= !(x.x < INFINITY) | !(x.y < INFINITY) | !(x.z < INFINITY) | !(x.w < INFINITY);
+                mp = fmaxf(fmaxf(mp, fmaxf(x.x, x.y)), fmaxf(x.z, x.w));
+                if (RESIDENT) *reinterpret_cast<float4*>(sp + e) = x;
+                if (full_q) {
+                    float4 y = c[u];
+                    y.x = scale_logit(y.x, inv_t), y.y = scale_logit(y.y, inv_t);
+                    y.z = scale_logit(y.z, inv_t), y.w = scale_logit(y.w, inv_t);
+                    bad |= !(y.x < INFINITY) | !(y.y < INFINITY) | !(y.z < INFINITY) | !(y.w < INFINITY);
+                    mq = fmaxf(fmaxf(mq, fmaxf(y.x, y.y)), fmaxf(y.z, y.w));
+                    if (RESIDENT) *reinterpret_cast<float4*>(sq + e) = y;
+                }
             }
         }
     } else {
@@ -343,38 +364,61 @@ accept_chain_kernel(const float* __restrict__ target_logits, long long t_stride,
     const float gmax_p = (float)gp, gmax_q = (float)gq;
     if (!(gmax_p > -INFINITY) || (full_q && !(gmax_q > -INFINITY))) bad = 1;
 
-    // ---- pass 2: exponentials (kept in place), sums ---------------------------------------------
+    // ---- pass 2: exponentials (kept in place, unnormalised), sums -----------------------------------
     float tp = 0.f, tq = 0.f;
-    for (int e = tid; e < n_local; e += kChainThreads) {
-        const float a = exp_scaled(RESIDENT ? sp[e] : scale_logit(zp[lo + e], inv_t), gmax_p);
-        tp += a;
-        if (RESIDENT) sp[e] = a;
-        if (full_q) {
-            const float c = exp_scaled(RESIDENT ? sq[e] : scale_logit(zq[lo + e], inv_t), gmax_q);
-            tq += c;
-            if (RESIDENT) sq[e] = c;
+    if (RESIDENT && VEC) {
+        for (int e = tid * 4; e < n_local; e += kChainThreads * 4) {
+            float4 a = *reinterpret_cast<const float4*>(sp + e);
+            a.x = exp_scaled(a.x, gmax_p), a.y = exp_scaled(a.y, gmax_p);
+            a.z = exp_scaled(a.z, gmax_p), a.w = exp_scaled(a.w, gmax_p);
+            tp += (a.x + a.y) + (a.z + a.w);
+            *reinterpret_cast<float4*>(sp + e) = a;
+            if (full_q) {
+                float4 c = *reinterpret_cast<const float4*>(sq + e);
+                c.x = exp_scaled(c.x, gmax_q), c.y = exp_scaled(c.y, gmax_q);
+                c.z = exp_scaled(c.z, gmax_q), c.w = exp_scaled(c.w, gmax_q);
+                tq += (c.x + c.y) + (c.z + c.w);
+                *reinterpret_cast<float4*>(sq + e) = c;
+            }
+        }
+    } else {
+        for (int e = tid; e < n_local; e += kChainThreads) {
+            const float a = exp_scaled(RESIDENT ? sp[e] : scale_logit(zp[lo + e], inv_t), gmax_p);
+            tp += a;
+            if (RESIDENT) sp[e] = a;
+            if (full_q) {
+                const float c = exp_scaled(RESIDENT ? sq[e] : scale_logit(zq[lo + e], inv_t), gmax_q);
+                tq += c;
+                if (RESIDENT) sq[e] = c;
+            }
         }
     }
     double sum_p = chain_block_sum((double)tp, s_redd), sum_q = chain_block_sum((double)tq, s_redd);
     cluster_allreduce2<false>(cluster, sum_p, sum_q, s_xchg, parity);
     const float c_p = (float)(1.0 / sum_p), c_q = full_q ? (float)(1.0 / sum_q) : 0.f;
-    // The first rejection always leads to alpha = 1 (alpha_0 = 0, beta_0 = 1, nothing removed from
-    // q yet), so its residual mass F(1) = sum max(p_0 - q_0, 0) is taken in this same sweep.
-    float part_f1 = 0.f;
-    if (RESIDENT) {
-        for (int e = tid; e < n_local; e += kChainThreads) {
-            const float pe = __fmul_rn(sp[e], c_p);
-            sp[e] = pe;
-            if (full_q) {
-                const float qe = __fmul_rn(sq[e], c_q);
-                sq[e] = qe;
-                part_f1 += fmaxf(fmaf(-1.0f, qe, pe), 0.f);
+    // Residual mass sum_v max(p_0(v) - alpha q_0(v), 0) over this block's slice.  The resident copies
+    // hold the unnormalised exponentials; p and q are formed on the fly with the same two roundings
+    // as prob_of(), so a token looked up on its own has bit for bit the value used here.
+    auto residual_mass = [&](float an) {
+        float part = 0.f;
+        if (RESIDENT && VEC) {
+            for (int e = tid * 4; e < n_local; e += kChainThreads * 4) {
+                const float4 a = *reinterpret_cast<const float4*>(sp + e);
+                const float4 c = *reinterpret_cast<const float4*>(sq + e);
+                part += fmaxf(fmaf(-an, __fmul_rn(c.x, c_q), __fmul_rn(a.x, c_p)), 0.f);
+                part += fmaxf(fmaf(-an, __fmul_rn(c.y, c_q), __fmul_rn(a.y, c_p)), 0.f);
+                part += fmaxf(fmaf(-an, __fmul_rn(c.z, c_q), __fmul_rn(a.z, c_p)), 0.f);
+                part += fmaxf(fmaf(-an, __fmul_rn(c.w, c_q), __fmul_rn(a.w, c_p)), 0.f);
+            }
+        } else {
+            for (int e = tid; e < n_local; e += kChainThreads) {
+                const float pe = RESIDENT ? __fmul_rn(sp[e], c_p) : prob_of(zp[lo + e], inv_t, gmax_p, c_p);
+                const float qe = RESIDENT ? __fmul_rn(sq[e], c_q) : prob_of(zq[lo + e], inv_t, gmax_q, c_q);
+                part += fmaxf(fmaf(-an, qe, pe), 0.f);
             }
         }
-    } else if (full_q && nc > 1) {
-        for (int e = tid; e < n_local; e += kChainThreads)
-            part_f1 += fmaxf(fmaf(-1.0f, prob_of(zq[lo + e], inv_t, gmax_q, c_q), prob_of(zp[lo + e], inv_t, gmax_p, c_p)), 0.f);
-    }
+        return part;
+    };
     // the children's own probabilities, computed exactly like the resident values
     if (tid < nc) {
         const int t = s_ctok[tid];
@@ -440,22 +484,9 @@ accept_chain_kernel(const float* __restrict__ target_logits, long long t_stride,
             if (tid == 0) s_frozen[j] = alpha;
             break;
         }
-        double f_new;
-        if (j == 0) {  // alpha_new == 1: the sum was taken in the normalisation sweep
-            double unused = 0.0;
-            f_new = chain_block_sum((double)part_f1, s_redd);
-            cluster_allreduce2<false>(cluster, f_new, unused, s_xchg, parity);
-        } else {
-            float part = 0.f;
-            for (int e = tid; e < n_local; e += kChainThreads) {
-                const float pe = RESIDENT ? sp[e] : prob_of(zp[lo + e], inv_t, gmax_p, c_p);
-                const float qe = RESIDENT ? sq[e] : prob_of(zq[lo + e], inv_t, gmax_q, c_q);
-                part += fmaxf(fmaf(-an, qe, pe), 0.f);
-            }
-            double unused = 0.0;
-            f_new = chain_block_sum((double)part, s_redd);
-            cluster_allreduce2<false>(cluster, f_new, unused, s_xchg, parity);
-        }
+        double f_new, unused = 0.0;
+        f_new = chain_block_sum((double)residual_mass(an), s_redd);
+        cluster_allreduce2<false>(cluster, f_new, unused, s_xchg, parity);
         // tokens removed in earlier rounds keep the alpha in force when they were removed
         for (int i = 0; i < j; ++i) {
             const float pi = s_pf[i], qi = s_qf[i];
