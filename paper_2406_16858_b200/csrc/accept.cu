@@ -185,15 +185,26 @@ __device__ __forceinline__ double chain_block_sum(double v, double* s_red) {
     for (int w = 0; w < kChainWarps; ++w) r += s_red[w];
     return r;
 }
-__device__ __forceinline__ float chain_block_max(float v, float* s_red) {
-    v = warp_max_f32(v);
+// Two block-wide sums (or maxima) behind one pair of barriers.  s_red: 2 * kChainWarps entries.
+__device__ __forceinline__ void chain_block_sum2(double& a, double& b, double* s_red) {
+    a = warp_sum_f64(a), b = warp_sum_f64(b);
     __syncthreads();
-    if ((threadIdx.x & 31) == 0) s_red[threadIdx.x >> 5] = v;
+    if ((threadIdx.x & 31) == 0) s_red[threadIdx.x >> 5] = a, s_red[kChainWarps + (threadIdx.x >> 5)] = b;
     __syncthreads();
-    float r = s_red[0];
+    double ra = 0.0, rb = 0.0;
 #pragma unroll
-    for (int w = 1; w < kChainWarps; ++w) r = fmaxf(r, s_red[w]);
-    return r;
+    for (int w = 0; w < kChainWarps; ++w) ra += s_red[w], rb += s_red[kChainWarps + w];
+    a = ra, b = rb;
+}
+__device__ __forceinline__ void chain_block_max2(float& a, float& b, float* s_red) {
+    a = warp_max_f32(a), b = warp_max_f32(b);
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) s_red[threadIdx.x >> 5] = a, s_red[kChainWarps + (threadIdx.x >> 5)] = b;
+    __syncthreads();
+    float ra = s_red[0], rb = s_red[kChainWarps];
+#pragma unroll
+    for (int w = 1; w < kChainWarps; ++w) ra = fmaxf(ra, s_red[w]), rb = fmaxf(rb, s_red[kChainWarps + w]);
+    a = ra, b = rb;
 }
 
 // All-reduce of two doubles across the blocks of the cluster through distributed shared memory.
@@ -252,8 +263,8 @@ accept_chain_kernel(const float* __restrict__ target_logits, long long t_stride,
 
     extern __shared__ __align__(16) float s_rows[];  // RESIDENT: p slice then q slice
     __shared__ double s_xchg[2 * kMaxCluster * 2];
-    __shared__ double s_redd[kChainWarps];
-    __shared__ float s_redf[kChainWarps];
+    __shared__ double s_redd[2 * kChainWarps];
+    __shared__ float s_redf[2 * kChainWarps];
     __shared__ int s_child[EAGLE2_MAX_K], s_ctok[EAGLE2_MAX_K];
     __shared__ float s_pf[EAGLE2_MAX_K], s_qf[EAGLE2_MAX_K], s_uc[EAGLE2_MAX_K];  // children's p, q, uniform
     __shared__ double s_frozen[EAGLE2_MAX_K];
@@ -359,7 +370,8 @@ accept_chain_kernel(const float* __restrict__ target_logits, long long t_stride,
             }
         }
     }
-    double gp = (double)chain_block_max(mp, s_redf), gq = (double)chain_block_max(mq, s_redf);
+    chain_block_max2(mp, mq, s_redf);
+    double gp = (double)mp, gq = (double)mq;
     cluster_allreduce2<true>(cluster, gp, gq, s_xchg, parity);
     const float gmax_p = (float)gp, gmax_q = (float)gq;
     if (!(gmax_p > -INFINITY) || (full_q && !(gmax_q > -INFINITY))) bad = 1;
@@ -393,7 +405,8 @@ accept_chain_kernel(const float* __restrict__ target_logits, long long t_stride,
             }
         }
     }
-    double sum_p = chain_block_sum((double)tp, s_redd), sum_q = chain_block_sum((double)tq, s_redd);
+    double sum_p = (double)tp, sum_q = (double)tq;
+    chain_block_sum2(sum_p, sum_q, s_redd);
     cluster_allreduce2<false>(cluster, sum_p, sum_q, s_xchg, parity);
     const float c_p = (float)(1.0 / sum_p), c_q = full_q ? (float)(1.0 / sum_q) : 0.f;
     // Residual mass sum_v max(p_0(v) - alpha q_0(v), 0) over this block's slice.  The resident copies
