@@ -471,6 +471,11 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes)
     return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) |
            ((uint64_t)(1024u >> 4) << 32) | (1ull << 46) | (2ull << 61);
 }
+// The descriptor of the same tile `bytes` further on (a multiple of 16 that keeps the address below
+// 256 KB): one addition on the low word, so the lane that issues the MMAs spends few instructions.
+__device__ __forceinline__ uint64_t desc_advance(uint64_t desc, uint32_t bytes) {
+    return (desc & 0xFFFFFFFF00000000ull) | (uint64_t)((uint32_t)desc + (bytes >> 4));
+}
 // Instruction descriptor: bf16 x bf16 -> fp32, M = 128, A K-major; B K-major or MN-major.
 __host__ __device__ constexpr uint32_t instr_desc(int n, bool b_mn_major, int m_rows = kRowsPerTile) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((uint32_t)(n >> 3) << 17) |
@@ -852,11 +857,11 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
                 tc_fence_after();
                 if (lane == 0) {
                     const uint32_t d_tmem = tmem + (uint32_t)(i % kSlots) * kTK;
+                    const uint64_t qd0 = smem_desc(sQ + t * kTile, 16), kd0 = smem_desc(sK + st * kKTile, 16);
 #pragma unroll
                     for (int ks = 0; ks < DH / 16; ++ks) {
-                        const uint32_t qoff = (uint32_t)(ks / 4) * kPanel + (uint32_t)(ks % 4) * 32u;
-                        const uint32_t koff = (uint32_t)(ks / 4) * kKPanel + (uint32_t)(ks % 4) * 32u;
-                        const uint64_t qd = smem_desc(sQ + t * kTile + qoff, 16), kd = smem_desc(sK + st * kKTile + koff, 16);
+                        const uint64_t qd = desc_advance(qd0, (uint32_t)(ks / 4) * kPanel + (uint32_t)(ks % 4) * 32u);
+                        const uint64_t kd = desc_advance(kd0, (uint32_t)(ks / 4) * kKPanel + (uint32_t)(ks % 4) * 32u);
                         if (PAIR) mma2_ss(d_tmem, qd, kd, kIdescQK, ks > 0);
                         else mma_ss(d_tmem, qd, kd, kIdescQK, ks > 0);
                     }
@@ -879,9 +884,10 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
                 if (lane == 0) {
                     const uint32_t d_tmem = tmem + kOCol + (uint32_t)t * DH;
                     const uint32_t a_tmem = tmem + (uint32_t)(i % kSlots) * kTK;
+                    const uint64_t vd0 = smem_desc(sV + st * kVTile, kPanel);
 #pragma unroll
                     for (int ks = 0; ks < kTK / 16; ++ks) {
-                        const uint64_t vd = smem_desc(sV + st * kVTile + ks * 2048u, kPanel);
+                        const uint64_t vd = desc_advance(vd0, ks * 2048u);
                         const uint32_t acc = (j > 0 || ks > 0) ? 1u : 0u;
                         if (PAIR) mma2_ts(d_tmem, a_tmem + ks * 8, vd, kIdescPV, acc);
                         else mma_ts(d_tmem, a_tmem + ks * 8, vd, kIdescPV, acc);
