@@ -34,7 +34,7 @@ def _static_tree(draft_dev, B, V, k, D):
     return token, parent, value, frontier, status
 
 
-@pytest.mark.parametrize("name,B", [("tiny", 1), ("tiny", 3), ("vicuna7b", 2)])
+@pytest.mark.parametrize("name,B", [("tiny", 1), ("tiny", 3), ("vicuna7b", 2), ("vicuna7b", 24)])  # the last: several tiles per block
 def test_static_scratch_expansion_matches_workspace_expansion(name, B):
     cfg = get_config(name).with_(B=B)
     for seed in (3, 4):  # two trees back to back through the one shared buffer
