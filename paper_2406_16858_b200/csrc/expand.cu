@@ -290,6 +290,14 @@ expand_kernel(const float* __restrict__ draft_logits, long long batch_stride, in
             // k lanes hold an element that reaches it: a valid bar (if it is not -inf itself)
             if (lane == 0 && thr > -INFINITY) atomicMax(&s_bar_code, order_code(thr));
         }
+        if (STREAM && t == t0) {
+            // Once per block the streaming warps wait for each other's first bars: the largest of them
+            // lets a handful of the first tile's elements through instead of a dozen per warp, which
+            // is what the selector would otherwise spend the block's first microseconds on.
+            asm volatile("bar.sync 1, %0;" ::"n"(kScanThreads) : "memory");
+            const uint32_t code = *reinterpret_cast<volatile uint32_t*>(&s_bar_code);
+            if (code) thr = fmaxf(thr, order_decode(code));
+        }
         if (!__any_sync(0xffffffffu, tm >= thr)) return;
         uint32_t pmask = 0;  // this lane's candidates
         if (tm >= thr) {
