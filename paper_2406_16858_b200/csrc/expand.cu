@@ -451,11 +451,22 @@ expand_kernel(const float* __restrict__ draft_logits, long long batch_stride, in
         const unsigned long long kth_now = __shfl_sync(0xffffffffu, top, k - 1);
         if (key <= kth_now) key = 0ull;
         if (!__any_sync(0xffffffffu, key != 0ull)) continue;
-        // the 32 best of (top | the new keys): sort the new keys, pair the two sorted runs end to
-        // end, keep the larger of each pair, sort the bitonic result
-        key = warp_sort_desc_u64(key);
-        const unsigned long long rev = __shfl_sync(0xffffffffu, key, 31 - lane);
-        top = warp_bitonic_merge_desc(top > rev ? top : rev);
+        const uint32_t fresh = __ballot_sync(0xffffffffu, key != 0ull);
+        if (__popc(fresh) <= 6) {
+            // a few keys: each is inserted at its place among the sorted 32 (the last one drops out)
+            for (uint32_t left = fresh; left; left &= left - 1) {
+                const unsigned long long x = __shfl_sync(0xffffffffu, key, __ffs(left) - 1);
+                const int at = __popc(__ballot_sync(0xffffffffu, top > x));  // keys that stay ahead of x
+                const unsigned long long up = __shfl_up_sync(0xffffffffu, top, 1);
+                top = lane < at ? top : (lane == at ? x : up);
+            }
+        } else {
+            // the 32 best of (top | the new keys): sort the new keys, pair the two sorted runs end to
+            // end, keep the larger of each pair, sort the bitonic result
+            key = warp_sort_desc_u64(key);
+            const unsigned long long rev = __shfl_sync(0xffffffffu, key, 31 - lane);
+            top = warp_bitonic_merge_desc(top > rev ? top : rev);
+        }
         const unsigned long long kth = __shfl_sync(0xffffffffu, top, k - 1);
         if (lane == 0 && kth) atomicMax(&s_bar_code, (uint32_t)(kth >> 32));
     }
