@@ -177,7 +177,7 @@ def test_large_scores_do_not_overflow():
 
 @pytest.mark.parametrize("name", ["vicuna7b", "llama3_8b", "llama2_70b"])
 def test_full_size_one_layer_sampled(name):
-    """BASELINE sizes, the launch configuration the benchmark times; the oracle computes sampled
+    """Full model-shaped sizes, the launch configuration the benchmark times; the oracle computes sampled
     (sequence, head, query) rows one by one."""
     cfg = get_config(name)
     g = torch.Generator(device=DEV).manual_seed(1234)
