@@ -321,6 +321,68 @@ def batched_accept_extra(e2, dev, stream, hbm_peak, B=16, reps=10):
             "frac_of_measured_hbm": gbs / hbm_peak}
 
 
+def draft_attention_extra(e2, dev, stream, hbm_peak, reps=200):
+    """The draft model's own attention during expansion (one decoder layer with the target's head
+    geometry): at step s its s*k tokens fed so far are the tree rows, the k newest are the step's
+    queries.  Same entry point as the verification pass, m = s*k; a chain-shaped mask stands in for
+    the tree's; 8 rotating caches (136 MB) are larger than L2."""
+    import torch
+    cfg = get_config("llama3_8b")
+    L, k, D = int(cfg.kv_len), cfg.k, cfg.D
+    g = torch.Generator(device=dev).manual_seed(3)
+    m_max = (D - 1) * k
+    rows = L + m_max
+    n_sets = 8
+    ks = [torch.randn((rows, cfg.Hkv, cfg.d), generator=g, device=dev).to(torch.bfloat16) for _ in range(n_sets)]
+    vs = [torch.randn((rows, cfg.Hkv, cfg.d), generator=g, device=dev).to(torch.bfloat16) for _ in range(n_sets)]
+    kv_off = torch.zeros(1, dtype=torch.int64, device=dev)
+    kv_len = torch.full((1,), L, dtype=torch.int32, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    scale = 1.0 / math.sqrt(cfg.d)
+    per_step = []
+    for s in range(1, D):
+        m = s * k
+        q = torch.randn((1, m, cfg.Hq, cfg.d), generator=g, device=dev).to(torch.bfloat16)
+        out = torch.zeros_like(q)
+        mask = torch.zeros((1, m, 1), dtype=torch.int64, device=dev)
+        for i in range(m):  # token i sees itself and the tokens k, 2k, ... before it
+            bits = 0
+            j = i
+            while j >= 0:
+                bits |= 1 << j
+                j -= k
+            mask[0, i, 0] = bits
+        ws = torch.empty(max(e2.workspace_bytes(e2.OP_TREE_ATTENTION, B=1, m=m, Hq=cfg.Hq, Hkv=cfg.Hkv, d=cfg.d,
+                                                max_kv_len=L), 256), dtype=torch.uint8, device=dev)
+        e2.workspace_init(ws)
+
+        def calls():
+            for kc, vc in zip(ks, vs):
+                e2.tree_attention(q, kc, vc, rows, kv_off, kv_len, mask, 1, m, cfg.Hq, cfg.Hkv, cfg.d, L, scale, out,
+                                  None, ws, status)
+
+        with torch.cuda.stream(stream):
+            calls()
+            stream.synchronize()
+            gr = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(gr, stream=stream):
+                calls()
+            for _ in range(3):
+                gr.replay()
+            ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            ev0.record(stream)
+            for _ in range(reps // n_sets):
+                gr.replay()
+            ev1.record(stream)
+        torch.cuda.synchronize()
+        per_step.append(ev0.elapsed_time(ev1) * 1e3 / ((reps // n_sets) * n_sets))
+    assert int(status.item()) == 0
+    nbytes = 2.0 * (L + m_max) * cfg.Hkv * cfg.d * 2
+    return {"workload": f"llama3_8b-shaped draft layer, kv_len {L}, steps 1..{D - 1} with m = {k}..{m_max}",
+            "us_per_step": per_step, "us_all_steps": float(sum(per_step)),
+            "frac_of_measured_hbm_last_step": nbytes / (per_step[-1] * 1e-6) / 1e9 / hbm_peak}
+
+
 # ------------------------------------------------------------------------------------------------
 # the CUDA path
 
@@ -346,7 +408,8 @@ def run_ours(args):
         hbm_peak = _peaks()[0]
         print(json.dumps({"attention_batched": batched_attention_extra(e2, dev, stream, hbm_peak),
                           "expand_batched": batched_expand_extra(e2, dev, stream, hbm_peak),
-                          "accept_batched": batched_accept_extra(e2, dev, stream, hbm_peak)}))
+                          "accept_batched": batched_accept_extra(e2, dev, stream, hbm_peak),
+                          "draft_attention": draft_attention_extra(e2, dev, stream, hbm_peak)}))
         return
     cfg = get_config(args.workload)
     if args.batch:
@@ -568,6 +631,7 @@ def run_ours(args):
         line["attention_batched"] = batched_attention_extra(e2, dev, stream, hbm_peak)
         line["expand_batched"] = batched_expand_extra(e2, dev, stream, hbm_peak)
         line["accept_batched"] = batched_accept_extra(e2, dev, stream, hbm_peak)
+        line["draft_attention"] = draft_attention_extra(e2, dev, stream, hbm_peak)
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

@@ -125,6 +125,47 @@ def test_ordered_launch_other_shapes(m, Hq, Hkv, d, B, longest):
     _compare(q, kc, vc, off, kl, bits, 1.0 / np.sqrt(d), samples=samples)
 
 
+def test_draft_side_attention_over_the_growing_tree():
+    """The draft model's own attention while it expands the tree (Section 4.1): at step s the k
+    frontier tokens attend to the committed cache and to their ancestors among the tokens expanded
+    so far.  The tokens fed so far - k per step, in feeding order - are the tree rows of the call, so
+    the same entry point serves it at m = s*k; the tree is the one the oracle's expansion builds."""
+    V, k, D, B = 500, 10, 6, 2
+    Hq, Hkv, d = 32, 8, 128
+    rng = np.random.default_rng(12)
+    draft = (2.0 * rng.standard_normal((B, ref.n_draft_rows(k, D), V))).astype(np.float32)
+    tree = ref.new_tree(B, k, D)
+    fed = [[] for _ in range(B)]  # candidate indices of the tokens fed to the draft model so far
+    kv_len = np.array([700, 129], np.int32)
+    for s in range(D):
+        lo = 0 if s == 0 else 1 + (s - 1) * k
+        ref.expand(tree, draft.reshape(-1)[lo * V:], V, k, D, s, batch_stride=draft.shape[1] * V)
+        if s == D - 1:
+            break  # the last level is never fed back
+        for b in range(B):
+            fed[b] += [int(x) for x in tree.frontier[b]]
+        m = (s + 1) * k
+        parent = np.full((B, m), -1, np.int32)
+        depth = np.zeros((B, m), np.int32)
+        for b in range(B):
+            where = {c: i for i, c in enumerate(fed[b])}
+            for i, c in enumerate(fed[b]):
+                pc = int(tree.parent[b, c])
+                if pc >= 0:  # an ancestor of a frontier token was itself a frontier token earlier
+                    parent[b, i] = where[pc]
+                    depth[b, i] = depth[b, where[pc]] + 1
+        bits, _, _, st = ref.tree_mask(parent, depth, np.full(B, m, np.int32), kv_len, m)
+        assert st == 0
+        kv_off = gen.kv_offsets(kv_len, m)
+        rows = int(kv_off[-1] + kv_len[-1] + m)
+        q = gen.f32_to_bf16_bits(rng.standard_normal((B, m, Hq, d)).astype(np.float32))
+        kc = gen.f32_to_bf16_bits(rng.standard_normal((rows, Hkv, d)).astype(np.float32))
+        vc = gen.f32_to_bf16_bits(rng.standard_normal((rows, Hkv, d)).astype(np.float32))
+        new = np.arange(m - k, m)  # the step's own queries: every head of the k newest tokens
+        samples = np.array([(b, h, i) for b in range(B) for h in (0, 5, Hq - 1) for i in new], np.int32)
+        _compare(q, kc, vc, kv_off, kv_len, bits, 1.0 / np.sqrt(d), samples=samples)
+
+
 def test_rows_after_a_sequence_may_hold_anything():
     """The kernel streams whole tiles, so it reads cache rows that follow a sequence's last key; their
     contents (here NaN and Inf bit patterns) must not reach the output."""
