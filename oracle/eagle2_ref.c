@@ -100,9 +100,9 @@ static int log_sum_exp(const float* z, int V, double inv_t, double* out) {
  * contributes a factor 1).  Then the k best new candidates by value (ties:
  * lower candidate index) become the next frontier.
  */
-int eagle2_expand_ref(const float* draft_logits, long long batch_stride, int B, int V, int k, int D,
-                      int s, int32_t* tree_token, int32_t* tree_parent, double* tree_value,
-                      int32_t* frontier, int32_t* status) {
+static int expand_impl(const float* draft_logits, long long batch_stride, int B, int V, int k, int D,
+                       int s, int by_confidence, int32_t* tree_token, int32_t* tree_parent,
+                       double* tree_value, int32_t* frontier, int32_t* status) {
     if (!draft_logits || !tree_token || !tree_parent || !tree_value || !frontier || !status)
         return ERR_NULL;
     if (B < 0 || V < 1 || k < 1 || k > V || D < 1 || s < 0 || s >= D) return ERR_SHAPE;
@@ -138,7 +138,7 @@ int eagle2_expand_ref(const float* draft_logits, long long batch_stride, int B, 
                 const long long node = base + (long long)r * k + c;
                 tok[node] = order[c].idx;
                 par[node] = parent;
-                val[node] = parent_value + (order[c].key - lse);
+                val[node] = (by_confidence ? 0.0 : parent_value) + (order[c].key - lse);
             }
         }
         free(order);
@@ -159,6 +159,28 @@ int eagle2_expand_ref(const float* draft_logits, long long batch_stride, int B, 
         }
     }
     return 0;
+}
+
+int eagle2_expand_ref(const float* draft_logits, long long batch_stride, int B, int V, int k, int D,
+                      int s, int32_t* tree_token, int32_t* tree_parent, double* tree_value,
+                      int32_t* frontier, int32_t* status) {
+    return expand_impl(draft_logits, batch_stride, B, V, k, D, s, 0, tree_token, tree_parent, tree_value,
+                       frontier, status);
+}
+
+/*
+ * The ablation of Section 5.2 "w/o value": nodes are ranked by their own confidence c_i (the draft
+ * model's probability of the token given its path) instead of the value V_i, the product of the
+ * confidences along the path.  With by_confidence != 0 a node's stored value is log c_i alone; the
+ * frontier and, later, the reranking then order by it (the reranking's ancestor clamp keeps the
+ * selection closed).  by_confidence == 0 is eagle2_expand_ref.
+ */
+int eagle2_expand_variant_ref(const float* draft_logits, long long batch_stride, int B, int V, int k,
+                              int D, int s, int by_confidence, int32_t* tree_token,
+                              int32_t* tree_parent, double* tree_value, int32_t* frontier,
+                              int32_t* status) {
+    return expand_impl(draft_logits, batch_stride, B, V, k, D, s, by_confidence != 0, tree_token, tree_parent,
+                       tree_value, frontier, status);
 }
 
 /* ---------- step 2a: reranking (Section 4.2) ----------------------------- */

@@ -85,7 +85,7 @@ def new_tree(B: int, k: int, D: int) -> Tree:
 
 
 def expand(tree: Tree, draft_logits: np.ndarray, V: int, k: int, D: int, s: int,
-           batch_stride: int | None = None) -> None:
+           batch_stride: int | None = None, by_confidence: bool = False) -> None:
     """draft_logits: fp32 [B, n_s, V] (n_s = 1 at s == 0, else k), or any buffer with batch_stride."""
     B = tree.token.shape[0]
     assert draft_logits.dtype == np.float32
@@ -94,14 +94,14 @@ def expand(tree: Tree, draft_logits: np.ndarray, V: int, k: int, D: int, s: int,
         assert draft_logits.size == B * n_s * V
         batch_stride = n_s * V
     st = np.zeros(1, np.int32)
-    _check(lib().eagle2_expand_ref(
-        _p(draft_logits, C.c_float), C.c_longlong(batch_stride), B, V, k, D, s,
+    _check(lib().eagle2_expand_variant_ref(
+        _p(draft_logits, C.c_float), C.c_longlong(batch_stride), B, V, k, D, s, int(by_confidence),
         _p(tree.token, C.c_int32), _p(tree.parent, C.c_int32), _p(tree.value, C.c_double),
-        _p(tree.frontier, C.c_int32), _p(st, C.c_int32)), "eagle2_expand_ref")
+        _p(tree.frontier, C.c_int32), _p(st, C.c_int32)), "eagle2_expand_variant_ref")
     tree.status |= int(st[0])
 
 
-def build_tree(draft_rows: np.ndarray, V: int, k: int, D: int) -> Tree:
+def build_tree(draft_rows: np.ndarray, V: int, k: int, D: int, by_confidence: bool = False) -> Tree:
     """Run all D expansion steps.  draft_rows: fp32 [B, R, V]; row 0 feeds step 0 and rows
     1+(s-1)k .. 1+sk-1 feed step s."""
     B = draft_rows.shape[0]
@@ -112,10 +112,16 @@ def build_tree(draft_rows: np.ndarray, V: int, k: int, D: int) -> Tree:
         lo = 0 if s == 0 else 1 + (s - 1) * k
         flat = draft_rows.reshape(-1)[lo * V:]
         st = np.zeros(1, np.int32)
-        _check(lib().eagle2_expand_ref(
-            _p(flat, C.c_float), C.c_longlong(R * V), B, V, k, D, s,
-            _p(tree.token, C.c_int32), _p(tree.parent, C.c_int32), _p(tree.value, C.c_double),
-            _p(tree.frontier, C.c_int32), _p(st, C.c_int32)), "eagle2_expand_ref")
+        if by_confidence:
+            _check(lib().eagle2_expand_variant_ref(
+                _p(flat, C.c_float), C.c_longlong(R * V), B, V, k, D, s, 1,
+                _p(tree.token, C.c_int32), _p(tree.parent, C.c_int32), _p(tree.value, C.c_double),
+                _p(tree.frontier, C.c_int32), _p(st, C.c_int32)), "eagle2_expand_variant_ref")
+        else:
+            _check(lib().eagle2_expand_ref(
+                _p(flat, C.c_float), C.c_longlong(R * V), B, V, k, D, s,
+                _p(tree.token, C.c_int32), _p(tree.parent, C.c_int32), _p(tree.value, C.c_double),
+                _p(tree.frontier, C.c_int32), _p(st, C.c_int32)), "eagle2_expand_ref")
         tree.status |= int(st[0])
     return tree
 
