@@ -99,6 +99,22 @@ int eagle2_expand(const float* draft_logits, long long batch_stride, int B, int 
                   void* ws, size_t ws_bytes, int32_t* d_status, eagle2_stream_t stream);
 
 /*
+ * Expansion with a choice of ranking score (paper Section 5.2, the ablation "without value").
+ * flags = 0 is eagle2_expand.  With EAGLE2_EXPAND_BY_CONFIDENCE a new node's stored score is its own
+ * confidence alone, the log-probability the draft model gives the token after its path, instead of
+ * the sum along the path; the children, their order and the tie rules are unchanged, and the next
+ * frontier is the k best of the step by that score.  Scores are then no longer monotone along a
+ * path: eagle2_rerank's ancestor rule is what keeps the selected set a connected tree.  Every other
+ * argument, the workspace and the errors are those of eagle2_expand; an unknown flag bit is
+ * EAGLE2_ERR_SHAPE.  All steps of one tree must use the same flags.
+ */
+#define EAGLE2_EXPAND_BY_CONFIDENCE 1u
+int eagle2_expand_variant(const float* draft_logits, long long batch_stride, int B, int V, int k, int D,
+                          int s, unsigned flags, int32_t* tree_token, int32_t* tree_parent,
+                          double* tree_value, int32_t* frontier, void* ws, size_t ws_bytes,
+                          int32_t* d_status, eagle2_stream_t stream);
+
+/*
  * Expansion without a caller workspace (the paper has no counterpart; this is a packaging variant of
  * eagle2_expand, same arguments minus ws/ws_bytes, same kernels, same results).  It is meant for
  * callers that cannot obtain device memory at the moment they need this step: a serving process

@@ -21,7 +21,8 @@ STATUS_TIMEOUT, STATUS_BOUNDS, STATUS_BAD_TREE = 8, 16, 32
 
 EXPORTS = ("eagle2_version", "eagle2_strerror", "eagle2_workspace_bytes", "eagle2_workspace_init",
            "eagle2_expand", "eagle2_rerank", "eagle2_tree_mask", "eagle2_tree_attention",
-           "eagle2_accept", "eagle2_kv_compact", "eagle2_expand_static")
+           "eagle2_accept", "eagle2_kv_compact", "eagle2_expand_static", "eagle2_expand_variant")
+EXPAND_BY_CONFIDENCE = 1
 
 
 class Eagle2Error(RuntimeError):
@@ -55,6 +56,9 @@ def lib() -> C.CDLL:
         h.eagle2_expand.argtypes = [vp, i64, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, sz, vp, vp]
         h.eagle2_expand_static.argtypes = [vp, i64, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp]
         h.eagle2_expand_static.restype = i32
+        h.eagle2_expand_variant.argtypes = [vp, i64, i32, i32, i32, i32, i32, C.c_uint, vp, vp, vp, vp, vp, sz,
+                                            vp, vp]
+        h.eagle2_expand_variant.restype = i32
         h.eagle2_rerank.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp]
         h.eagle2_tree_mask.argtypes = [vp, vp, vp, vp, i32, i32, vp, vp, vp, vp, vp]
         h.eagle2_tree_attention.argtypes = [vp, vp, vp, i64, vp, vp, vp, i32, i32, i32, i32, i32, i32,
@@ -118,6 +122,16 @@ def expand(draft_logits, batch_stride: int, B: int, V: int, k: int, D: int, s: i
     p, n = _ws(ws)
     _check("eagle2_expand", lib().eagle2_expand(
         _ptr(draft_logits), batch_stride, B, V, k, D, s, _ptr(tree_token), _ptr(tree_parent),
+        _ptr(tree_value), _ptr(frontier), p, n, _ptr(d_status), _stream(stream)))
+
+
+def expand_variant(draft_logits, batch_stride: int, B: int, V: int, k: int, D: int, s: int, flags: int,
+                   tree_token, tree_parent, tree_value, frontier, ws, d_status, stream=None) -> None:
+    """``expand`` with a choice of ranking score (``EXPAND_BY_CONFIDENCE``: a node's own
+    log-probability instead of the sum along its path)."""
+    p, n = _ws(ws)
+    _check("eagle2_expand_variant", lib().eagle2_expand_variant(
+        _ptr(draft_logits), batch_stride, B, V, k, D, s, flags, _ptr(tree_token), _ptr(tree_parent),
         _ptr(tree_value), _ptr(frontier), p, n, _ptr(d_status), _stream(stream)))
 
 

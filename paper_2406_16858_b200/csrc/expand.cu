@@ -164,7 +164,7 @@ __device__ __forceinline__ unsigned long long warp_bitonic_merge_desc(unsigned l
 template <bool VEC, bool STREAM>
 __global__ void __launch_bounds__(STREAM ? kScanThreads + 32 : kScanThreads, 3)
 expand_kernel(const float* __restrict__ draft_logits, long long batch_stride, int V, int k, int D,
-              int s, int n_s, int chunks, int tpb, int32_t* __restrict__ tree_token,
+              int s, int n_s, int chunks, int tpb, int by_confidence, int32_t* __restrict__ tree_token,
               int32_t* __restrict__ tree_parent, double* __restrict__ tree_value,
               int32_t* __restrict__ frontier, ExpandWs ws, int32_t* d_status) {
     constexpr int VPT = 4, NE = 16;
@@ -239,7 +239,7 @@ expand_kernel(const float* __restrict__ draft_logits, long long batch_stride, in
         const long long prev_base = s >= 2 ? (long long)k + (long long)(s - 2) * k * k : 0;
         const long long prev_count = s >= 2 ? (long long)k * k : k;
         if (my_parent < prev_base || my_parent >= prev_base + prev_count) my_parent = -2;  // reported by the merger
-        else my_parent_value = tree_value[(long long)b * N + my_parent];
+        else if (!by_confidence) my_parent_value = tree_value[(long long)b * N + my_parent];  // else log 1
     }
 
     unsigned long long* list = s_list[warp];
@@ -732,7 +732,8 @@ expand_kernel(const float* __restrict__ draft_logits, long long batch_stride, in
 
 template <bool VEC, bool STREAM>
 static int launch_expand_as(const float* draft_logits, long long batch_stride, int B, int V, int k, int D,
-                            int s, int n_s, const ExpandPlan& plan, int32_t* tree_token, int32_t* tree_parent,
+                            int s, int n_s, int by_confidence, const ExpandPlan& plan, int32_t* tree_token,
+                            int32_t* tree_parent,
                             double* tree_value, int32_t* frontier, const ExpandWs& ws, int32_t* d_status,
                             cudaStream_t stream) {
     const long long blocks = (long long)B * n_s * plan.chunks;
@@ -745,20 +746,22 @@ static int launch_expand_as(const float* draft_logits, long long batch_stride, i
     }
     return launch_chained(expand_kernel<VEC, STREAM>, dim3((unsigned)blocks),
                           dim3(STREAM ? kScanThreads + 32 : kScanThreads), dyn, stream, 1, draft_logits, batch_stride, V,
-                          k, D, s, n_s, plan.chunks, plan.tpb, tree_token, tree_parent, tree_value, frontier, ws,
-                          d_status);
+                          k, D, s, n_s, plan.chunks, plan.tpb, by_confidence, tree_token, tree_parent, tree_value,
+                          frontier, ws, d_status);
 }
 
 // Blocks that stream several tiles get the selector warp; one-tile blocks rank within the block.
 template <bool VEC>
 static int launch_expand(const float* draft_logits, long long batch_stride, int B, int V, int k, int D,
-                         int s, int n_s, const ExpandPlan& plan, int32_t* tree_token, int32_t* tree_parent,
-                         double* tree_value, int32_t* frontier, const ExpandWs& ws, int32_t* d_status,
-                         cudaStream_t stream) {
-    return plan.tpb > 1 ? launch_expand_as<VEC, true>(draft_logits, batch_stride, B, V, k, D, s, n_s, plan, tree_token,
-                                                      tree_parent, tree_value, frontier, ws, d_status, stream)
-                        : launch_expand_as<VEC, false>(draft_logits, batch_stride, B, V, k, D, s, n_s, plan, tree_token,
-                                                       tree_parent, tree_value, frontier, ws, d_status, stream);
+                         int s, int n_s, int by_confidence, const ExpandPlan& plan, int32_t* tree_token,
+                         int32_t* tree_parent, double* tree_value, int32_t* frontier, const ExpandWs& ws,
+                         int32_t* d_status, cudaStream_t stream) {
+    return plan.tpb > 1 ? launch_expand_as<VEC, true>(draft_logits, batch_stride, B, V, k, D, s, n_s, by_confidence,
+                                                      plan, tree_token, tree_parent, tree_value, frontier, ws,
+                                                      d_status, stream)
+                        : launch_expand_as<VEC, false>(draft_logits, batch_stride, B, V, k, D, s, n_s, by_confidence,
+                                                       plan, tree_token, tree_parent, tree_value, frontier, ws,
+                                                       d_status, stream);
 }
 
 // Scratch of eagle2_expand_static: lives in every context that loads the library, until exit.
@@ -792,10 +795,11 @@ static int expand_scratch_address(void** out) {
 
 using namespace eagle2;
 
-extern "C" int eagle2_expand(const float* draft_logits, long long batch_stride, int B, int V, int k,
-                             int D, int s, int32_t* tree_token, int32_t* tree_parent,
-                             double* tree_value, int32_t* frontier, void* ws, size_t ws_bytes,
-                             int32_t* d_status, eagle2_stream_t stream) {
+// Expansion with a caller workspace; by_confidence selects the ablation's ranking score.
+static int expand_with_workspace(const float* draft_logits, long long batch_stride, int B, int V, int k,
+                                 int D, int s, int by_confidence, int32_t* tree_token,
+                                 int32_t* tree_parent, double* tree_value, int32_t* frontier, void* ws,
+                                 size_t ws_bytes, int32_t* d_status, eagle2_stream_t stream) {
     if (!draft_logits || !tree_token || !tree_parent || !tree_value || !frontier || !d_status)
         return EAGLE2_ERR_NULL;
     if (B < 0 || V < 1 || k < 1 || k > V || k > EAGLE2_MAX_K || D < 1 || D > EAGLE2_MAX_DEPTH || s < 0 ||
@@ -812,10 +816,28 @@ extern "C" int eagle2_expand(const float* draft_logits, long long batch_stride, 
     if (expand_ws_layout(B, n_s, plan.chunks, k, ws, &w) > ws_bytes) return EAGLE2_ERR_WORKSPACE;
     const bool vec = aligned(draft_logits, 16) && V % 4 == 0 && batch_stride % 4 == 0;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-    return vec ? launch_expand<true>(draft_logits, batch_stride, B, V, k, D, s, n_s, plan, tree_token, tree_parent,
-                                     tree_value, frontier, w, d_status, st)
-               : launch_expand<false>(draft_logits, batch_stride, B, V, k, D, s, n_s, plan, tree_token, tree_parent,
-                                      tree_value, frontier, w, d_status, st);
+    return vec ? launch_expand<true>(draft_logits, batch_stride, B, V, k, D, s, n_s, by_confidence, plan, tree_token,
+                                     tree_parent, tree_value, frontier, w, d_status, st)
+               : launch_expand<false>(draft_logits, batch_stride, B, V, k, D, s, n_s, by_confidence, plan, tree_token,
+                                      tree_parent, tree_value, frontier, w, d_status, st);
+}
+
+extern "C" int eagle2_expand(const float* draft_logits, long long batch_stride, int B, int V, int k,
+                             int D, int s, int32_t* tree_token, int32_t* tree_parent,
+                             double* tree_value, int32_t* frontier, void* ws, size_t ws_bytes,
+                             int32_t* d_status, eagle2_stream_t stream) {
+    return expand_with_workspace(draft_logits, batch_stride, B, V, k, D, s, 0, tree_token, tree_parent, tree_value,
+                                 frontier, ws, ws_bytes, d_status, stream);
+}
+
+extern "C" int eagle2_expand_variant(const float* draft_logits, long long batch_stride, int B, int V, int k,
+                                     int D, int s, unsigned flags, int32_t* tree_token,
+                                     int32_t* tree_parent, double* tree_value, int32_t* frontier, void* ws,
+                                     size_t ws_bytes, int32_t* d_status, eagle2_stream_t stream) {
+    if (flags & ~(unsigned)EAGLE2_EXPAND_BY_CONFIDENCE) return EAGLE2_ERR_SHAPE;
+    return expand_with_workspace(draft_logits, batch_stride, B, V, k, D, s,
+                                 (flags & EAGLE2_EXPAND_BY_CONFIDENCE) ? 1 : 0, tree_token, tree_parent,
+                                 tree_value, frontier, ws, ws_bytes, d_status, stream);
 }
 
 extern "C" int eagle2_expand_static(const float* draft_logits, long long batch_stride, int B, int V, int k,
@@ -847,8 +869,8 @@ extern "C" int eagle2_expand_static(const float* draft_logits, long long batch_s
         return EAGLE2_ERR_CUDA;
     }
     const bool vec = aligned(draft_logits, 16) && V % 4 == 0 && batch_stride % 4 == 0;
-    return vec ? launch_expand<true>(draft_logits, batch_stride, B, V, k, D, s, n_s, plan, tree_token, tree_parent,
+    return vec ? launch_expand<true>(draft_logits, batch_stride, B, V, k, D, s, n_s, 0, plan, tree_token, tree_parent,
                                      tree_value, frontier, w, d_status, st)
-               : launch_expand<false>(draft_logits, batch_stride, B, V, k, D, s, n_s, plan, tree_token, tree_parent,
-                                      tree_value, frontier, w, d_status, st);
+               : launch_expand<false>(draft_logits, batch_stride, B, V, k, D, s, n_s, 0, plan, tree_token,
+                                      tree_parent, tree_value, frontier, w, d_status, st);
 }

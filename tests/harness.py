@@ -45,16 +45,20 @@ class GpuTree:
         self.status = new_status()
         self.ws = make_ws(e2.workspace_bytes(e2.OP_EXPAND, B=B, V=V, k=k, D=D))
 
-    def expand_all(self, draft_rows_dev: torch.Tensor):
-        """draft_rows_dev: fp32 [B, R, V] on the device."""
+    def expand_all(self, draft_rows_dev: torch.Tensor, flags: int = 0):
+        """draft_rows_dev: fp32 [B, R, V] on the device.  flags != 0 goes through the variant entry."""
         B, V, k, D = self.B, self.V, self.k, self.D
         R = 1 + (D - 1) * k
         assert draft_rows_dev.shape == (B, R, V) and draft_rows_dev.is_contiguous()
         for s in range(D):
             lo = 0 if s == 0 else 1 + (s - 1) * k
             ptr = draft_rows_dev.data_ptr() + lo * V * 4
-            e2.expand(ptr, R * V, B, V, k, D, s, self.token, self.parent, self.value, self.frontier,
-                      self.ws, self.status)
+            if flags:
+                e2.expand_variant(ptr, R * V, B, V, k, D, s, flags, self.token, self.parent, self.value,
+                                  self.frontier, self.ws, self.status)
+            else:
+                e2.expand(ptr, R * V, B, V, k, D, s, self.token, self.parent, self.value, self.frontier,
+                          self.ws, self.status)
         torch.cuda.synchronize()
         return self
 
