@@ -192,19 +192,20 @@ int eagle2_expand_variant_ref(const float* draft_logits, long long batch_stride,
  * makes the closure property hold for arbitrary caller-supplied values.
  * The selection is emitted in ascending candidate index, a topological order.
  */
-int eagle2_rerank_ref(const int32_t* tree_token, const int32_t* tree_parent,
-                      const double* tree_value, int B, int k, int D, int m, int32_t* sel_index,
-                      int32_t* sel_parent, int32_t* sel_token, int32_t* sel_depth, int32_t* n_sel,
-                      int32_t* status) {
+static int rerank_impl(const int32_t* tree_token, const int32_t* tree_parent,
+                       const double* tree_value, const int32_t* frontier, int B, int k, int D, int m,
+                       int32_t* sel_index, int32_t* sel_parent, int32_t* sel_token,
+                       int32_t* sel_depth, int32_t* n_sel, int32_t* status) {
     if (!tree_token || !tree_parent || !tree_value || !sel_index || !sel_parent || !sel_token ||
         !sel_depth || !n_sel || !status)
         return ERR_NULL;
     if (B < 0 || k < 1 || D < 1 || m < 1) return ERR_SHAPE;
     const long long N = n_nodes(k, D);
-    const int keep = (long long)m < N ? m : (int)N;
+    const int most = (long long)m < N ? m : (int)N;
 
 #pragma omp parallel for schedule(dynamic)
     for (int b = 0; b < B; ++b) {
+        int keep = most;
         const int32_t* tok = tree_token + (long long)b * N;
         const int32_t* par = tree_parent + (long long)b * N;
         const double* val = tree_value + (long long)b * N;
@@ -212,7 +213,7 @@ int eagle2_rerank_ref(const int32_t* tree_token, const int32_t* tree_parent,
         double* v_eff = (double*)malloc(sizeof(double) * (size_t)N);
         keyed_t* order = (keyed_t*)malloc(sizeof(keyed_t) * (size_t)N);
         int* flat_of = (int*)malloc(sizeof(int) * (size_t)N);
-        int* chosen = (int*)malloc(sizeof(int) * (size_t)keep);
+        int* chosen = (int*)malloc(sizeof(int) * (size_t)most);
 
         for (int i = 0; i < N; ++i) {
             int p = par[i];
@@ -230,9 +231,30 @@ int eagle2_rerank_ref(const int32_t* tree_token, const int32_t* tree_parent,
             order[i].idx = i;
             flat_of[i] = -1;
         }
-        qsort(order, (size_t)N, sizeof(keyed_t), cmp_desc_key_asc_idx);
-        for (int j = 0; j < keep; ++j) chosen[j] = order[j].idx;
-        qsort(chosen, (size_t)keep, sizeof(int), cmp_int_asc);
+        if (!frontier) {
+            qsort(order, (size_t)N, sizeof(keyed_t), cmp_desc_key_asc_idx);
+            for (int j = 0; j < keep; ++j) chosen[j] = order[j].idx;
+            qsort(chosen, (size_t)keep, sizeof(int), cmp_int_asc);
+        } else {
+            /* No reranking: the draft is what the expansion phase itself selected, the frontier of
+             * every step.  A frontier node of an earlier step is one that was expanded, i.e. one
+             * that some node names as its parent; the last step's frontier is passed in.  Lowest
+             * indices (shallowest) first if there are more than m. */
+            char* picked = (char*)calloc((size_t)N, 1);
+            for (int i = 0; i < N; ++i) {
+                const int p = par[i];
+                if (p >= 0 && p < i) picked[p] = 1;
+            }
+            for (int j = 0; j < k; ++j) {
+                const int f = frontier[(long long)b * k + j];
+                if (f < 0 || f >= N) st |= ST_BAD_TREE;
+                else picked[f] = 1;
+            }
+            keep = 0;
+            for (int i = 0; i < N && keep < most; ++i)
+                if (picked[i]) chosen[keep++] = i;
+            free(picked);
+        }
         for (int j = 0; j < keep; ++j) flat_of[chosen[j]] = j;
 
         int32_t* o_idx = sel_index + (long long)b * m;
@@ -273,6 +295,28 @@ int eagle2_rerank_ref(const int32_t* tree_token, const int32_t* tree_parent,
         }
     }
     return 0;
+}
+
+int eagle2_rerank_ref(const int32_t* tree_token, const int32_t* tree_parent,
+                      const double* tree_value, int B, int k, int D, int m, int32_t* sel_index,
+                      int32_t* sel_parent, int32_t* sel_token, int32_t* sel_depth, int32_t* n_sel,
+                      int32_t* status) {
+    return rerank_impl(tree_token, tree_parent, tree_value, NULL, B, k, D, m, sel_index, sel_parent,
+                       sel_token, sel_depth, n_sel, status);
+}
+
+/*
+ * The ablation of Section 5.2 "w/o reranking": the tree sent to verification is the set of nodes the
+ * expansion phase selected (k per step, at most kD), flattened exactly as above.  `frontier` is the
+ * last step's frontier [B][k].  The paper does not spell this set out; this is the reading taken.
+ */
+int eagle2_rerank_skipped_ref(const int32_t* tree_token, const int32_t* tree_parent,
+                              const double* tree_value, const int32_t* frontier, int B, int k, int D,
+                              int m, int32_t* sel_index, int32_t* sel_parent, int32_t* sel_token,
+                              int32_t* sel_depth, int32_t* n_sel, int32_t* status) {
+    if (!frontier) return ERR_NULL;
+    return rerank_impl(tree_token, tree_parent, tree_value, frontier, B, k, D, m, sel_index, sel_parent,
+                       sel_token, sel_depth, n_sel, status);
 }
 
 /* ---------- step 2b: tree mask and position ids (Section 4.2) ------------ */

@@ -150,6 +150,23 @@ def rerank(token, parent, value, k: int, D: int, m: int) -> Selection:
     return sel
 
 
+def rerank_skipped(token, parent, value, frontier, k: int, D: int, m: int) -> Selection:
+    """Section 5.2, the ablation without reranking: the expansion phase's own selection, flattened."""
+    B = token.shape[0]
+    sel = Selection(*(np.zeros((B, m), np.int32) for _ in range(4)), np.zeros(B, np.int32))
+    st = np.zeros(1, np.int32)
+    _check(lib().eagle2_rerank_skipped_ref(
+        _p(np.ascontiguousarray(token, np.int32), C.c_int32),
+        _p(np.ascontiguousarray(parent, np.int32), C.c_int32),
+        _p(np.ascontiguousarray(value, np.float64), C.c_double),
+        _p(np.ascontiguousarray(frontier, np.int32), C.c_int32), B, k, D, m,
+        _p(sel.index, C.c_int32), _p(sel.parent, C.c_int32), _p(sel.token, C.c_int32),
+        _p(sel.depth, C.c_int32), _p(sel.n_sel, C.c_int32), _p(st, C.c_int32)),
+        "eagle2_rerank_skipped_ref")
+    sel.status = int(st[0])
+    return sel
+
+
 def tree_mask(sel_parent, sel_depth, n_sel, kv_len, m: int, dense: bool = False):
     """Returns (mask_bits u64 [B,m,W], mask_dense u8 [B,m,m] or None, pos_ids i32 [B,m], status)."""
     B = sel_parent.shape[0]

@@ -143,3 +143,51 @@ def test_bad_parent_sets_status():
     _, _, _, st = ref.tree_mask(sel_parent, sel_depth, np.array([4], np.int32),
                                 np.array([0], np.int32), 4)
     assert st & ref.ST_BAD_TREE
+
+
+@pytest.mark.parametrize("by_confidence", [False, True])
+@pytest.mark.parametrize("m", [3, 12, 20, 50])
+def test_without_reranking_the_draft_is_the_frontiers_of_all_steps(m, by_confidence):
+    """Section 5.2, the ablation without reranking.  The frontier after every step is recorded while the
+    tree is grown one step at a time (those frontiers are themselves pinned against a brute force); the
+    selection must be their union, lowest indices first when it exceeds m, flattened like any other."""
+    V, k, D = 60, 4, 5
+    for seed in range(5):
+        rng = np.random.default_rng(500 + seed)
+        rows = (2.0 * rng.standard_normal((1, ref.n_draft_rows(k, D), V))).astype(np.float32)
+        tree = ref.new_tree(1, k, D)
+        union = set()
+        for s in range(D):
+            lo = 0 if s == 0 else 1 + (s - 1) * k
+            n_s = 1 if s == 0 else k
+            ref.expand(tree, np.ascontiguousarray(rows[:, lo:lo + n_s]), V, k, D, s, by_confidence=by_confidence)
+            union |= set(tree.frontier[0].tolist())
+        assert len(union) == k * D
+        want = sorted(union)[:m]
+        sel = ref.rerank_skipped(tree.token, tree.parent, tree.value, tree.frontier, k, D, m)
+        assert sel.status == 0
+        assert sel.n_sel[0] == len(want)
+        assert sel.index[0, :len(want)].tolist() == want
+        assert (sel.index[0, len(want):] == -1).all()
+        flat = {c: j for j, c in enumerate(want)}
+        for j, c in enumerate(want):
+            p = tree.parent[0, c]
+            assert sel.parent[0, j] == (-1 if p < 0 else flat[p])  # connected whatever m cuts off
+            assert sel.token[0, j] == tree.token[0, c]
+            assert sel.depth[0, j] == _level(c, k) - 1
+        if not by_confidence and m >= k * D:
+            # the reranked tree of the same size is at least as good under the paper's objective
+            full = ref.rerank(tree.token, tree.parent, tree.value, k, D, k * D)
+            assert np.exp(tree.value[0, full.index[0, :k * D]]).sum() >= \
+                np.exp(tree.value[0, want]).sum() - 1e-15
+
+
+def test_without_reranking_a_bad_frontier_is_reported():
+    k, D, m = 2, 3, 6
+    N = ref.n_nodes(k, D)
+    token = np.zeros((1, N), np.int32)
+    parent = np.array([[-1, -1, 0, 0, 1, 1, 2, 2, 3, 3]], np.int32)
+    value = np.zeros((1, N))
+    sel = ref.rerank_skipped(token, parent, value, np.array([[6, 99]], np.int32), k, D, m)
+    assert sel.status & ref.ST_BAD_TREE
+    assert sel.index[0, :int(sel.n_sel[0])].tolist() == [0, 1, 2, 3, 6]
