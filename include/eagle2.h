@@ -100,13 +100,14 @@ int eagle2_expand(const float* draft_logits, long long batch_stride, int B, int 
 
 /*
  * Expansion with a choice of ranking score (paper Section 5.2, the ablation "without value").
- * flags = 0 is eagle2_expand.  With EAGLE2_EXPAND_BY_CONFIDENCE a new node's stored score is its own
- * confidence alone, the log-probability the draft model gives the token after its path, instead of
- * the sum along the path; the children, their order and the tie rules are unchanged, and the next
- * frontier is the k best of the step by that score.  Scores are then no longer monotone along a
- * path: eagle2_rerank's ancestor rule is what keeps the selected set a connected tree.  Every other
- * argument, the workspace and the errors are those of eagle2_expand; an unknown flag bit is
- * EAGLE2_ERR_SHAPE.  All steps of one tree must use the same flags.
+ * The ablation compares expanding on the value with expanding on the confidence score, so only the
+ * choice of the nodes to expand changes.  flags = 0 is eagle2_expand.  With
+ * EAGLE2_EXPAND_BY_CONFIDENCE the next frontier is the k best new candidates by their own confidence
+ * (the log-probability the draft model gives the token after its path; ties: lower index) instead
+ * of by value.  Children, their order, tree_value (still the sum of log-probabilities along the
+ * path) and everything else are unchanged, so eagle2_rerank afterwards ranks by value as always.
+ * Every other argument, the workspace and the errors are those of eagle2_expand; an unknown flag
+ * bit is EAGLE2_ERR_SHAPE.
  */
 #define EAGLE2_EXPAND_BY_CONFIDENCE 1u
 int eagle2_expand_variant(const float* draft_logits, long long batch_stride, int B, int V, int k, int D,
@@ -152,6 +153,23 @@ int eagle2_rerank(const int32_t* tree_token, const int32_t* tree_parent, const d
                   int B, int k, int D, int m, int32_t* sel_index, int32_t* sel_parent,
                   int32_t* sel_token, int32_t* sel_depth, int32_t* n_sel, int32_t* d_status,
                   eagle2_stream_t stream);
+
+/*
+ * Step 2a without the reranking (paper Section 5.2, the ablation "without reranking").  The paper does
+ * not list the nodes verified in that case; the reading taken here is the selection the expansion
+ * phase made by itself: the frontier of every step, k nodes per step and at most kD in all, which is
+ * a connected tree.  They are the nodes that some node names as its parent, plus the last step's
+ * frontier, which the caller passes (the array eagle2_expand left after step D-1).  If there are
+ * more than m, the m lowest indices (shallowest levels) are kept.  Outputs, padding, limits and
+ * status bits are those of eagle2_rerank; n_sel[b] = min(m, number of such nodes); a frontier entry
+ * outside [0, N) raises EAGLE2_STATUS_BAD_TREE and is skipped.  tree_value is read only for the NaN
+ * check.
+ *   frontier  int32 [B][k]
+ */
+int eagle2_rerank_skipped(const int32_t* tree_token, const int32_t* tree_parent, const double* tree_value,
+                          const int32_t* frontier, int B, int k, int D, int m, int32_t* sel_index,
+                          int32_t* sel_parent, int32_t* sel_token, int32_t* sel_depth, int32_t* n_sel,
+                          int32_t* d_status, eagle2_stream_t stream);
 
 /*
  * Step 2b -- tree attention mask and position ids (paper Section 4.2: a draft token sees only its

@@ -118,6 +118,7 @@ static int expand_impl(const float* draft_logits, long long batch_stride, int B,
         double* val = tree_value + (long long)b * N;
         int32_t* fr = frontier + (long long)b * k;
         keyed_t* order = (keyed_t*)malloc(sizeof(keyed_t) * (size_t)V);
+        double* conf = (double*)malloc(sizeof(double) * (size_t)n_rows * (size_t)k);
         int st = 0;
 
         for (int r = 0; r < n_rows; ++r) {
@@ -138,7 +139,8 @@ static int expand_impl(const float* draft_logits, long long batch_stride, int B,
                 const long long node = base + (long long)r * k + c;
                 tok[node] = order[c].idx;
                 par[node] = parent;
-                val[node] = (by_confidence ? 0.0 : parent_value) + (order[c].key - lse);
+                val[node] = parent_value + (order[c].key - lse);
+                conf[r * k + c] = order[c].key - lse; /* the node's own confidence, log c_i */
             }
         }
         free(order);
@@ -147,12 +149,13 @@ static int expand_impl(const float* draft_logits, long long batch_stride, int B,
         const int n_new = n_rows * k;
         keyed_t* cand = (keyed_t*)malloc(sizeof(keyed_t) * (size_t)n_new);
         for (int i = 0; i < n_new; ++i) {
-            cand[i].key = val[base + i];
+            cand[i].key = by_confidence ? conf[i] : val[base + i];
             cand[i].idx = (int)(base + i);
         }
         qsort(cand, (size_t)n_new, sizeof(keyed_t), cmp_desc_key_asc_idx);
         for (int j = 0; j < k; ++j) fr[j] = cand[j].idx;
         free(cand);
+        free(conf);
         if (st) {
 #pragma omp atomic
             *status |= st;
@@ -169,11 +172,12 @@ int eagle2_expand_ref(const float* draft_logits, long long batch_stride, int B, 
 }
 
 /*
- * The ablation of Section 5.2 "w/o value": nodes are ranked by their own confidence c_i (the draft
- * model's probability of the token given its path) instead of the value V_i, the product of the
- * confidences along the path.  With by_confidence != 0 a node's stored value is log c_i alone; the
- * frontier and, later, the reranking then order by it (the reranking's ancestor clamp keeps the
- * selection closed).  by_confidence == 0 is eagle2_expand_ref.
+ * The ablation of Section 5.2 "w/o value", which the text describes as expanding on the confidence
+ * score instead of the value: with by_confidence != 0 the k nodes to expand next are the step's best
+ * by their own confidence c_i (the draft model's probability of the token given its path) instead
+ * of by V_i, the product of the confidences along the path.  Only that choice changes: the stored
+ * value of every node is still V_i, so a later reranking ranks by value as the paper's reranking
+ * does.  by_confidence == 0 is eagle2_expand_ref.
  */
 int eagle2_expand_variant_ref(const float* draft_logits, long long batch_stride, int B, int V, int k,
                               int D, int s, int by_confidence, int32_t* tree_token,

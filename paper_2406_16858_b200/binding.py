@@ -21,7 +21,8 @@ STATUS_TIMEOUT, STATUS_BOUNDS, STATUS_BAD_TREE = 8, 16, 32
 
 EXPORTS = ("eagle2_version", "eagle2_strerror", "eagle2_workspace_bytes", "eagle2_workspace_init",
            "eagle2_expand", "eagle2_rerank", "eagle2_tree_mask", "eagle2_tree_attention",
-           "eagle2_accept", "eagle2_kv_compact", "eagle2_expand_static", "eagle2_expand_variant")
+           "eagle2_accept", "eagle2_kv_compact", "eagle2_expand_static", "eagle2_expand_variant",
+           "eagle2_rerank_skipped")
 EXPAND_BY_CONFIDENCE = 1
 
 
@@ -60,6 +61,8 @@ def lib() -> C.CDLL:
                                             vp, vp]
         h.eagle2_expand_variant.restype = i32
         h.eagle2_rerank.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp]
+        h.eagle2_rerank_skipped.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp]
+        h.eagle2_rerank_skipped.restype = i32
         h.eagle2_tree_mask.argtypes = [vp, vp, vp, vp, i32, i32, vp, vp, vp, vp, vp]
         h.eagle2_tree_attention.argtypes = [vp, vp, vp, i64, vp, vp, vp, i32, i32, i32, i32, i32, i32,
                                             f32, vp, vp, vp, sz, vp, vp]
@@ -127,8 +130,8 @@ def expand(draft_logits, batch_stride: int, B: int, V: int, k: int, D: int, s: i
 
 def expand_variant(draft_logits, batch_stride: int, B: int, V: int, k: int, D: int, s: int, flags: int,
                    tree_token, tree_parent, tree_value, frontier, ws, d_status, stream=None) -> None:
-    """``expand`` with a choice of ranking score (``EXPAND_BY_CONFIDENCE``: a node's own
-    log-probability instead of the sum along its path)."""
+    """``expand`` with a choice of what ranks the next frontier (``EXPAND_BY_CONFIDENCE``: a node's
+    own log-probability instead of its value; stored values stay the path sums)."""
     p, n = _ws(ws)
     _check("eagle2_expand_variant", lib().eagle2_expand_variant(
         _ptr(draft_logits), batch_stride, B, V, k, D, s, flags, _ptr(tree_token), _ptr(tree_parent),
@@ -150,6 +153,15 @@ def rerank(tree_token, tree_parent, tree_value, B: int, k: int, D: int, m: int, 
         _ptr(tree_token), _ptr(tree_parent), _ptr(tree_value), B, k, D, m, _ptr(sel_index),
         _ptr(sel_parent), _ptr(sel_token), _ptr(sel_depth), _ptr(n_sel), _ptr(d_status),
         _stream(stream)))
+
+
+def rerank_skipped(tree_token, tree_parent, tree_value, frontier, B: int, k: int, D: int, m: int, sel_index,
+                   sel_parent, sel_token, sel_depth, n_sel, d_status, stream=None) -> None:
+    """The selection without reranking: the frontier nodes of every expansion step, flattened."""
+    _check("eagle2_rerank_skipped", lib().eagle2_rerank_skipped(
+        _ptr(tree_token), _ptr(tree_parent), _ptr(tree_value), _ptr(frontier), B, k, D, m,
+        _ptr(sel_index), _ptr(sel_parent), _ptr(sel_token), _ptr(sel_depth), _ptr(n_sel),
+        _ptr(d_status), _stream(stream)))
 
 
 def tree_mask(sel_parent, sel_depth, n_sel, kv_len, B: int, m: int, mask_bits, mask_dense, pos_ids,

@@ -239,7 +239,7 @@ expand_kernel(const float* __restrict__ draft_logits, long long batch_stride, in
         const long long prev_base = s >= 2 ? (long long)k + (long long)(s - 2) * k * k : 0;
         const long long prev_count = s >= 2 ? (long long)k * k : k;
         if (my_parent < prev_base || my_parent >= prev_base + prev_count) my_parent = -2;  // reported by the merger
-        else if (!by_confidence) my_parent_value = tree_value[(long long)b * N + my_parent];  // else log 1
+        else my_parent_value = tree_value[(long long)b * N + my_parent];
     }
 
     unsigned long long* list = s_list[warp];
@@ -699,11 +699,13 @@ expand_kernel(const float* __restrict__ draft_logits, long long batch_stride, in
             for (int q = 0; q < NR; ++q) {
                 if (valid[q] && lane < k) {
                     const long long node = base + (long long)r[q] * k + lane;
-                    const double v = parent_value[q] + ((double)key_value(mine[q]) - lse[q]);
+                    const double confidence = (double)key_value(mine[q]) - lse[q];  // log c_i
+                    const double v = parent_value[q] + confidence;
                     tok[node] = (int32_t)key_index(mine[q]);
                     par[node] = parent[q];
                     val[node] = v;
-                    s_rank[r[q] * k + lane] = order_code_f64(v);
+                    // the next frontier is ranked by value, or by confidence alone in the ablation
+                    s_rank[r[q] * k + lane] = order_code_f64(by_confidence ? confidence : v);
                 }
             }
         }

@@ -18,11 +18,13 @@ __device__ __forceinline__ unsigned long long value_code(double x) {
 
 // Values are compared as integer codes throughout (fp64 compares are slow on this part).  The
 // ranking is a bitonic sort of (code, index) pairs, padded to a power of two with code 0, which
-// sorts behind every real value.
+// sorts behind every real value.  With `frontier` given there is no ranking at all (the ablation
+// without reranking, Section 5.2): the selection is every node the expansion phase selected, i.e.
+// every node that is some node's parent plus the last step's frontier, lowest indices first.
 __global__ void __launch_bounds__(kRerankThreads)
 rerank_kernel(const int32_t* __restrict__ tree_token, const int32_t* __restrict__ tree_parent,
-              const double* __restrict__ tree_value, int k, int N, int P, int m, int keep,
-              int32_t* __restrict__ sel_index, int32_t* __restrict__ sel_parent,
+              const double* __restrict__ tree_value, const int32_t* __restrict__ frontier, int k, int N,
+              int P, int m, int most, int32_t* __restrict__ sel_index, int32_t* __restrict__ sel_parent,
               int32_t* __restrict__ sel_token, int32_t* __restrict__ sel_depth,
               int32_t* __restrict__ n_sel, int32_t* d_status) {
     extern __shared__ __align__(16) unsigned char s_dyn[];
@@ -57,6 +59,15 @@ rerank_kernel(const int32_t* __restrict__ tree_token, const int32_t* __restrict_
         s_flat[i] = -1;
     }
     __syncthreads();
+    if (frontier) {
+        for (int i = tid; i < N; i += kRerankThreads)
+            if (s_par[i] >= 0) s_flat[s_par[i]] = 0;  // several children store the same 0
+        if (tid < k) {
+            const int f = frontier[(long long)b * k + tid];
+            if (f < 0 || f >= N) status |= EAGLE2_STATUS_BAD_TREE;
+            else s_flat[f] = 0;
+        }
+    } else {
     // effective value = minimum of the values on the path from the root (parents have lower
     // indices, so the walk ends)
     for (int i = tid; i < P; i += kRerankThreads) {
@@ -100,7 +111,7 @@ rerank_kernel(const int32_t* __restrict__ tree_token, const int32_t* __restrict_
                 if (mine_first != keep_first) key = ok, idx = oi;
             }
         }
-        if (tid < keep) s_flat[idx] = 0;
+        if (tid < most) s_flat[idx] = 0;
     } else {
         for (int size = 2; size <= P; size <<= 1) {
             for (int stride = size >> 1; stride > 0; stride >>= 1) {
@@ -120,7 +131,8 @@ rerank_kernel(const int32_t* __restrict__ tree_token, const int32_t* __restrict_
                 __syncthreads();
             }
         }
-        for (int r = tid; r < keep; r += kRerankThreads) s_flat[s_idx[r]] = 0;
+        for (int r = tid; r < most; r += kRerankThreads) s_flat[s_idx[r]] = 0;
+    }
     }
     __syncthreads();
     // exclusive scan of the per-thread counts -> flat positions in ascending index
@@ -148,8 +160,12 @@ rerank_kernel(const int32_t* __restrict__ tree_token, const int32_t* __restrict_
     }
     __syncthreads();
     int pos = incl - mine + (warp ? s_scan[warp - 1] : 0);
+    const int keep = min(most, s_scan[kRerankThreads / 32 - 1]);  // fewer than `most` only without ranking
     for (int i = lo; i < hi; ++i)
-        if (s_flat[i] == 0) s_flat[i] = pos++;
+        if (s_flat[i] == 0) {
+            s_flat[i] = pos < most ? pos : -1;
+            ++pos;
+        }
     __syncthreads();
 
     int32_t* o_idx = sel_index + (long long)b * m;
@@ -226,10 +242,11 @@ tree_mask_kernel(const int32_t* __restrict__ sel_parent, const int32_t* __restri
 
 using namespace eagle2;
 
-extern "C" int eagle2_rerank(const int32_t* tree_token, const int32_t* tree_parent,
-                             const double* tree_value, int B, int k, int D, int m, int32_t* sel_index,
-                             int32_t* sel_parent, int32_t* sel_token, int32_t* sel_depth,
-                             int32_t* n_sel, int32_t* d_status, eagle2_stream_t stream) {
+// frontier == nullptr: the paper's reranking; else the selection the expansion phase made.
+static int rerank_launch(const int32_t* tree_token, const int32_t* tree_parent, const double* tree_value,
+                         const int32_t* frontier, int B, int k, int D, int m, int32_t* sel_index,
+                         int32_t* sel_parent, int32_t* sel_token, int32_t* sel_depth, int32_t* n_sel,
+                         int32_t* d_status, eagle2_stream_t stream) {
     if (!tree_token || !tree_parent || !tree_value || !sel_index || !sel_parent || !sel_token ||
         !sel_depth || !n_sel || !d_status)
         return EAGLE2_ERR_NULL;
@@ -239,7 +256,7 @@ extern "C" int eagle2_rerank(const int32_t* tree_token, const int32_t* tree_pare
     if (!aligned(tree_value, 8)) return EAGLE2_ERR_ALIGN;
     if (B == 0) return EAGLE2_OK;
     const int N = (int)nodes_of(k, D);
-    const int keep = m < N ? m : N;
+    const int most = m < N ? m : N;
     int P = 1;
     while (P < N) P <<= 1;
     const size_t dyn = (size_t)N * (sizeof(unsigned long long) + 2 * sizeof(int32_t)) +
@@ -249,8 +266,26 @@ extern "C" int eagle2_rerank(const int32_t* tree_token, const int32_t* tree_pare
             cudaSuccess)
         return EAGLE2_ERR_CUDA;
     return launch_chained(rerank_kernel, dim3(B), dim3(kRerankThreads), dyn, reinterpret_cast<cudaStream_t>(stream), 1,
-                          tree_token, tree_parent, tree_value, k, N, P, m, keep, sel_index, sel_parent, sel_token,
-                          sel_depth, n_sel, d_status);
+                          tree_token, tree_parent, tree_value, frontier, k, N, P, m, most, sel_index, sel_parent,
+                          sel_token, sel_depth, n_sel, d_status);
+}
+
+extern "C" int eagle2_rerank(const int32_t* tree_token, const int32_t* tree_parent,
+                             const double* tree_value, int B, int k, int D, int m, int32_t* sel_index,
+                             int32_t* sel_parent, int32_t* sel_token, int32_t* sel_depth,
+                             int32_t* n_sel, int32_t* d_status, eagle2_stream_t stream) {
+    return rerank_launch(tree_token, tree_parent, tree_value, nullptr, B, k, D, m, sel_index, sel_parent,
+                         sel_token, sel_depth, n_sel, d_status, stream);
+}
+
+extern "C" int eagle2_rerank_skipped(const int32_t* tree_token, const int32_t* tree_parent,
+                                     const double* tree_value, const int32_t* frontier, int B, int k,
+                                     int D, int m, int32_t* sel_index, int32_t* sel_parent,
+                                     int32_t* sel_token, int32_t* sel_depth, int32_t* n_sel,
+                                     int32_t* d_status, eagle2_stream_t stream) {
+    if (!frontier) return EAGLE2_ERR_NULL;
+    return rerank_launch(tree_token, tree_parent, tree_value, frontier, B, k, D, m, sel_index, sel_parent,
+                         sel_token, sel_depth, n_sel, d_status, stream);
 }
 
 extern "C" int eagle2_tree_mask(const int32_t* sel_parent, const int32_t* sel_depth,

@@ -22,7 +22,7 @@ def _frontier_gap(values_of_new, k):
     return np.inf if len(v) <= k else v[k - 1] - v[k]
 
 
-def _check_tree(cfg, draft, gpu: GpuTree, want: ref.Tree):
+def _check_tree(cfg, draft, gpu: GpuTree, want: ref.Tree, by_confidence=False):
     B, k, D = cfg.B, cfg.k, cfg.D
     tok, par, val, fr = host(gpu.token), host(gpu.parent), host(gpu.value), host(gpu.frontier)
     assert int(gpu.status.item()) == want.status
@@ -33,7 +33,10 @@ def _check_tree(cfg, draft, gpu: GpuTree, want: ref.Tree):
         for s in range(D):
             base = 0 if s == 0 else k + (s - 1) * k * k
             n_new = k if s == 0 else k * k
-            if _frontier_gap(want.value[b, base:base + n_new], k) < 1e-6:
+            score = want.value[b, base:base + n_new]
+            if by_confidence and s:  # the frontier was ranked by the node's own log-probability
+                score = score - want.value[b, want.parent[b, base:base + n_new]]
+            if _frontier_gap(score, k) < 1e-6:
                 exempt = True
         if exempt:
             continue

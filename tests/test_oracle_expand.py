@@ -39,8 +39,8 @@ def test_topk_ties_prefer_lower_token_id():
 
 
 def _brute(rows, V, k, D, by_confidence=False):
-    """Linear-space reconstruction: softmax probabilities multiplied along every root path (or, for the
-    ablation that ranks by confidence, each node's own probability alone)."""
+    """Linear-space reconstruction: softmax probabilities multiplied along every root path; the frontier
+    is ranked by that product, or by each node's own probability in the ablation."""
     prob = np.exp(rows.astype(np.float64) - rows.astype(np.float64).max(axis=1, keepdims=True))
     prob /= prob.sum(axis=1, keepdims=True)
     N = k + (D - 1) * k * k
@@ -64,8 +64,9 @@ def _brute(rows, V, k, D, by_confidence=False):
             while a >= 0:
                 prod *= edge[a]
                 a = parent[a]
-            lin[node] = edge[node] if by_confidence else prod
-        frontier = sorted(new, key=lambda n: (-lin[n], n))[:k]
+            lin[node] = prod
+        score = edge if by_confidence else lin
+        frontier = sorted(new, key=lambda n: (-score[n], n))[:k]
         frontiers.append(frontier)
     return token, parent, lin, frontiers
 
@@ -93,10 +94,10 @@ def test_values_and_frontier_match_linear_space_brute_force(seed):
 
 
 @pytest.mark.parametrize("seed", range(6))
-def test_ranking_by_confidence_alone_matches_brute_force(seed):
-    """Section 5.2, the ablation without the value: a node's score is its own softmax probability, and
-    the frontier is the k best of the step by that score.  The trees must also differ from the
-    value-ranked ones somewhere, or the switch would be untested."""
+def test_expanding_on_confidence_matches_brute_force(seed):
+    """Section 5.2, the ablation without the value: the nodes to expand are the k best of the step by
+    their own softmax probability; the stored value is still the path product.  The trees must also
+    differ from the value-ranked ones somewhere, or the switch would be untested."""
     V, k, D = 40, 3, 4
     rows = _small_rows(300 + seed, 1, ref.n_draft_rows(k, D), V)
     tree = ref.new_tree(1, k, D)
@@ -110,35 +111,20 @@ def test_ranking_by_confidence_alone_matches_brute_force(seed):
     np.testing.assert_allclose(np.exp(tree.value[0]), lin, rtol=1e-12)
     whole = ref.build_tree(rows, V, k, D, by_confidence=True)
     assert (whole.value[0] == tree.value[0]).all() and (whole.parent[0] == tree.parent[0]).all()
-    by_value = ref.build_tree(rows, V, k, D)
-    assert (by_value.value[0, :k] == tree.value[0, :k]).all()      # depth 1: value == confidence
-    # deeper rows differ as soon as the two frontiers do; where a node has the same parent and token
-    # in both trees, the path product is the smaller of the two scores
-    same = (by_value.parent[0] == tree.parent[0]) & (by_value.token[0] == tree.token[0])
-    same[:k] = False
-    assert same.any() and (by_value.value[0, same] < tree.value[0, same]).all()
+    for i in range(len(parent)):  # values are path products here too: never above the parent's
+        assert parent[i] < 0 or tree.value[0, i] <= tree.value[0, parent[i]]
 
 
-def test_confidence_ranked_tree_reranks_to_a_closed_selection():
-    """Confidences are not monotone along a path, so the m best by score alone need not contain their
-    ancestors; the reranking's ancestor rule must still return a connected tree."""
-    V, k, D, m = 64, 4, 5, 20
-    unclosed = 0
-    for seed in range(10):
-        rows = _small_rows(400 + seed, 1, ref.n_draft_rows(k, D), V)
-        t = ref.build_tree(rows, V, k, D, by_confidence=True)
-        N = ref.n_nodes(k, D)
-        plain = sorted(range(N), key=lambda i: (-t.value[0, i], i))[:m]
-        unclosed += any(t.parent[0, c] >= 0 and t.parent[0, c] not in plain for c in plain)
-        sel = ref.rerank(t.token, t.parent, t.value, k, D, m)
-        chosen = sel.index[0, :int(sel.n_sel[0])].tolist()
-        assert sel.status == 0 and len(chosen) == m
-        flat = {c: j for j, c in enumerate(chosen)}
-        for j, c in enumerate(chosen):
-            p = t.parent[0, c]
-            assert p < 0 or p in flat
-            assert sel.parent[0, j] == (-1 if p < 0 else flat[p]) and sel.parent[0, j] < j
-    assert unclosed > 0  # the case the ancestor rule exists for did occur
+def test_expanding_on_confidence_changes_some_frontier():
+    V, k, D = 40, 3, 4
+    changed = 0
+    for seed in range(6):
+        rows = _small_rows(300 + seed, 1, ref.n_draft_rows(k, D), V)
+        a = ref.build_tree(rows, V, k, D)
+        b = ref.build_tree(rows, V, k, D, by_confidence=True)
+        assert (a.value[0, :k + k * k] == b.value[0, :k + k * k]).all()  # two levels share their parents
+        changed += not (a.parent[0] == b.parent[0]).all()
+    assert changed > 0
 
 
 def test_tiny_config_generator_tree_is_consistent():

@@ -8,6 +8,10 @@ Recipe
                    +8 when the row is "easy" (probability p_easy), +2 otherwise
   target row     = the draft row that expanded the node (a fresh draft-style row for a node that
                    was never expanded) + N(0, std 0.5)
+  calibrated target row (acceptance-length studies only) = that same base row with one token
+                   raised above all others, the token drawn from the base row's softmax by the
+                   Gumbel-max trick: a greedy verifier then accepts a child with exactly the
+                   probability the draft gave it
   Q, K, V        ~ N(0,1) rounded to bf16
   uniforms       ~ U[0,1) fp32
   ragged lengths = round(exp(U(ln lo, ln hi)))
@@ -28,6 +32,7 @@ def rng_for(seed: int, stream: int) -> np.random.Generator:
 
 
 STREAM_DRAFT, STREAM_TARGET, STREAM_FRESH, STREAM_QKV, STREAM_U, STREAM_LEN, STREAM_EASY = range(7)
+STREAM_GUMBEL = 7
 
 
 def f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:
@@ -96,6 +101,30 @@ def target_rows(cfg: Config, seed: int, draft: np.ndarray, tree_parent: np.ndarr
                 row = int(nd[b, idx]) if idx >= 0 else -1
                 base = draft[b, row] if row >= 0 else _boosted_rows(fresh, 1, V, pe[b])[0]
             out[b, r] = base + np.float32(0.5) * noise.standard_normal(V, dtype=np.float32)
+    return out
+
+
+def target_rows_calibrated(cfg: Config, seed: int, draft: np.ndarray, tree_parent: np.ndarray,
+                           sel_index: np.ndarray) -> np.ndarray:
+    """fp32 [B, m+1, V] like ``target_rows``, but the row's largest logit sits on a token drawn from
+    the base row's own softmax (argmax of row + Gumbel noise), 4 above the previous maximum."""
+    B, m, V = cfg.B, cfg.m, cfg.V
+    nd = node_draft_rows(tree_parent, cfg.k, cfg.D)
+    pe = p_easy_per_sequence(cfg, seed)
+    out = np.empty((B, m + 1, V), np.float32)
+    for b in range(B):
+        fresh = rng_for(seed, STREAM_FRESH * 1000003 + b)
+        gum = rng_for(seed, STREAM_GUMBEL * 1000003 + b)
+        for r in range(m + 1):
+            if r == 0:
+                base = draft[b, 0]
+            else:
+                idx = int(sel_index[b, r - 1])
+                row = int(nd[b, idx]) if idx >= 0 else -1
+                base = draft[b, row] if row >= 0 else _boosted_rows(fresh, 1, V, pe[b])[0]
+            drawn = int(np.argmax(base.astype(np.float64) + gum.gumbel(size=V)))
+            out[b, r] = base
+            out[b, r, drawn] = base.max() + np.float32(4.0)
     return out
 
 
