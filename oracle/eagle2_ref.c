@@ -30,7 +30,8 @@
  * ancestor definition of Section 4.2 and the causal special case; attention
  * against closed forms and a library causal attention; greedy acceptance
  * against brute force; temperature-1 acceptance against exact enumeration of
- * the output law, the chain rule of Section 2.1 and a chi-square test.
+ * the output law, the chain rule of Section 2.1 and a chi-square test; the
+ * LM head against a library matrix product.
  * The worked example of the paper's method figure is an image that is not
  * available, so no printed value pins the oracle: "parity unpinned" by
  * printed values for that example only.
@@ -720,4 +721,29 @@ int eagle2_ref_num_threads(void) {
 #else
     return 1;
 #endif
+}
+
+/* ---------- before step 1: the LM head (Section 4.1) --------------------- */
+/*
+ * The draft model's feature of each frontier token goes through the LM head of the original LLM
+ * to give the draft distribution that step 1 ranks: logits[r][v] = sum_h hidden[r][h] * weight[v][h]
+ * (no bias).  bf16 operands as the GPU sees them, every product and the sum in double precision.
+ *   hidden [rows][H], weight [V][H]: bf16 bit patterns; logits [rows][V] double.
+ * Pins: numpy's matrix product on the same values; a one-hot feature selects a weight column.
+ */
+int eagle2_lm_head_ref(const uint16_t* hidden, const uint16_t* weight, int rows, int H, int V,
+                       double* logits) {
+    if (!hidden || !weight || !logits) return ERR_NULL;
+    if (rows < 0 || H < 1 || V < 1) return ERR_SHAPE;
+#pragma omp parallel for schedule(static)
+    for (int v = 0; v < V; ++v) {
+        const uint16_t* w = weight + (long long)v * H;
+        for (int r = 0; r < rows; ++r) {
+            const uint16_t* x = hidden + (long long)r * H;
+            double acc = 0.0;
+            for (int h = 0; h < H; ++h) acc += bf16_to_double(x[h]) * bf16_to_double(w[h]);
+            logits[(long long)r * V + v] = acc;
+        }
+    }
+    return 0;
 }

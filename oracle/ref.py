@@ -278,3 +278,15 @@ def kv_compact(k_layers, v_layers, kv_off, kv_len, acc_path, acc_len, m: int, D:
         _p(np.ascontiguousarray(acc_len, np.int32), C.c_int32), B, m, D, Hkv, d,
         _p(st, C.c_int32)), "eagle2_kv_compact_ref")
     return int(st[0])
+
+
+def lm_head(hidden: np.ndarray, weight: np.ndarray) -> np.ndarray:
+    """hidden uint16 (bf16 bits) [rows, H], weight uint16 [V, H] -> logits float64 [rows, V]."""
+    assert hidden.dtype == np.uint16 and weight.dtype == np.uint16 and hidden.shape[1] == weight.shape[1]
+    rows, H = hidden.shape
+    V = weight.shape[0]
+    out = np.zeros((rows, V), np.float64)
+    _check(lib().eagle2_lm_head_ref(_p(np.ascontiguousarray(hidden), C.c_uint16),
+                                    _p(np.ascontiguousarray(weight), C.c_uint16), rows, H, V,
+                                    _p(out, C.c_double)), "eagle2_lm_head_ref")
+    return out
