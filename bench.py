@@ -386,6 +386,53 @@ def draft_attention_extra(e2, dev, stream, hbm_peak, reps=200):
 # ------------------------------------------------------------------------------------------------
 # the CUDA path
 
+def lm_head_extra(e2, dev, stream, hbm_peak, reps=30):
+    """The LM head in front of each expansion step (Section 4.1) at the llama3_8b shape: k feature rows
+    of hidden size 4096 against a random bf16 [V][4096] weight matrix (1.05 GB, larger than L2), alone
+    and followed by the expansion that ranks its logits.  Algorithmic bytes per launch: the weight
+    matrix once, plus features and logits."""
+    import torch
+    cfg = get_config("llama3_8b")
+    H, V, k, D = 4096, cfg.V, cfg.k, cfg.D
+    g = torch.Generator(device=dev).manual_seed(5)
+    weight = (torch.randn((V, H), generator=g, device=dev) * (2.0 / math.sqrt(H))).to(torch.bfloat16)
+    hidden = torch.randn((k, H), generator=g, device=dev).to(torch.bfloat16)
+    logits = torch.zeros((k, V), dtype=torch.float32, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    N = k + (D - 1) * k * k
+    token = torch.zeros((1, N), dtype=torch.int32, device=dev)
+    parent = torch.zeros((1, N), dtype=torch.int32, device=dev)
+    value = torch.zeros((1, N), dtype=torch.float64, device=dev)
+    frontier = torch.zeros((1, k), dtype=torch.int32, device=dev)
+    ws = torch.empty(max(e2.workspace_bytes(e2.OP_EXPAND, B=1, V=V, k=k, D=D), 256), dtype=torch.uint8, device=dev)
+    e2.workspace_init(ws)
+    out = {}
+    for name in ("lm_head", "lm_head_then_expand"):
+        def calls():
+            e2.lm_head(hidden, weight, k, H, V, logits, status)
+            if name == "lm_head_then_expand":  # level 1 again from the first row, then level 2 from all k rows
+                e2.expand(logits, k * V, 1, V, k, D, 0, token, parent, value, frontier, ws, status)
+                e2.expand(logits, k * V, 1, V, k, D, 1, token, parent, value, frontier, ws, status)
+        with torch.cuda.stream(stream):
+            for _ in range(3):
+                calls()
+            stream.synchronize()
+            ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            ev0.record(stream)
+            for _ in range(reps):
+                calls()
+            ev1.record(stream)
+        torch.cuda.synchronize()
+        out[name + "_us"] = ev0.elapsed_time(ev1) * 1e3 / reps
+    assert int(status.item()) == 0
+    nbytes = 2.0 * V * H + 2.0 * k * H + 4.0 * k * V
+    out.update({"workload": f"llama3_8b-shaped LM head, {k} rows x {H} -> {V} logits, "
+                            f"bf16 weights {2.0 * V * H / 1e9:.2f} GB",
+                "bytes_per_launch": nbytes, "achieved_gbs": nbytes / (out["lm_head_us"] * 1e-6) / 1e9,
+                "frac_of_measured_hbm": nbytes / (out["lm_head_us"] * 1e-6) / 1e9 / hbm_peak})
+    return out
+
+
 def run_ours(args):
     import torch
 
@@ -409,7 +456,8 @@ def run_ours(args):
         print(json.dumps({"attention_batched": batched_attention_extra(e2, dev, stream, hbm_peak),
                           "expand_batched": batched_expand_extra(e2, dev, stream, hbm_peak),
                           "accept_batched": batched_accept_extra(e2, dev, stream, hbm_peak),
-                          "draft_attention": draft_attention_extra(e2, dev, stream, hbm_peak)}))
+                          "draft_attention": draft_attention_extra(e2, dev, stream, hbm_peak),
+                          "lm_head": lm_head_extra(e2, dev, stream, hbm_peak)}))
         return
     cfg = get_config(args.workload)
     if args.batch:
@@ -632,6 +680,7 @@ def run_ours(args):
         line["expand_batched"] = batched_expand_extra(e2, dev, stream, hbm_peak)
         line["accept_batched"] = batched_accept_extra(e2, dev, stream, hbm_peak)
         line["draft_attention"] = draft_attention_extra(e2, dev, stream, hbm_peak)
+        line["lm_head"] = lm_head_extra(e2, dev, stream, hbm_peak)
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

@@ -80,6 +80,21 @@ size_t eagle2_workspace_bytes(int op, int B, int V, int k, int D, int m, int Hq,
 int eagle2_workspace_init(void* ws, size_t ws_bytes, eagle2_stream_t stream);
 
 /*
+ * Before step 1 -- the LM head (paper Section 4.1: the draft model's feature of a token goes through
+ * the LM head of the original LLM to give the draft distribution):
+ *   logits[r][v] = sum_h hidden[r][h] * weight[v][h]      (no bias)
+ * bf16 operands, fp32 accumulation on the tensor path, fp32 result: the [rows][V] array that
+ * eagle2_expand takes as draft_logits (for B sequences pass rows = B*n_s and batch_stride = n_s*V).
+ *   hidden  bf16 [rows][H], 16-byte aligned
+ *   weight  bf16 [V][H], 16-byte aligned (the matrix is read once per call)
+ *   logits  fp32 [rows][V], written
+ * Limits: 0 <= rows <= 256, H a multiple of 64, V >= 1.  Needs no workspace.  A bounded wait that
+ * runs out raises EAGLE2_STATUS_TIMEOUT.
+ */
+int eagle2_lm_head(const void* hidden, const void* weight, int rows, int H, int V, float* logits,
+                   int32_t* d_status, eagle2_stream_t stream);
+
+/*
  * Step 1 -- expansion (paper Section 4.1, the value equation V_i = prod c_j over Path(root, t_i)).
  * Called for s = 0..D-1.  For each of the n_s input rows (n_s = 1 at s = 0, else k; row j belongs
  * to frontier[b][j]) it takes the log-softmax over the vocabulary, makes the k most probable tokens

@@ -22,7 +22,7 @@ STATUS_TIMEOUT, STATUS_BOUNDS, STATUS_BAD_TREE = 8, 16, 32
 EXPORTS = ("eagle2_version", "eagle2_strerror", "eagle2_workspace_bytes", "eagle2_workspace_init",
            "eagle2_expand", "eagle2_rerank", "eagle2_tree_mask", "eagle2_tree_attention",
            "eagle2_accept", "eagle2_kv_compact", "eagle2_expand_static", "eagle2_expand_variant",
-           "eagle2_rerank_skipped")
+           "eagle2_rerank_skipped", "eagle2_lm_head")
 EXPAND_BY_CONFIDENCE = 1
 
 
@@ -61,6 +61,8 @@ def lib() -> C.CDLL:
                                             vp, vp]
         h.eagle2_expand_variant.restype = i32
         h.eagle2_rerank.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp]
+        h.eagle2_lm_head.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp]
+        h.eagle2_lm_head.restype = i32
         h.eagle2_rerank_skipped.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp]
         h.eagle2_rerank_skipped.restype = i32
         h.eagle2_tree_mask.argtypes = [vp, vp, vp, vp, i32, i32, vp, vp, vp, vp, vp]
@@ -126,6 +128,12 @@ def expand(draft_logits, batch_stride: int, B: int, V: int, k: int, D: int, s: i
     _check("eagle2_expand", lib().eagle2_expand(
         _ptr(draft_logits), batch_stride, B, V, k, D, s, _ptr(tree_token), _ptr(tree_parent),
         _ptr(tree_value), _ptr(frontier), p, n, _ptr(d_status), _stream(stream)))
+
+
+def lm_head(hidden, weight, rows: int, H: int, V: int, logits, d_status, stream=None) -> None:
+    """logits fp32 [rows, V] = hidden bf16 [rows, H] . weight bf16 [V, H]^T (the draft logits of ``expand``)."""
+    _check("eagle2_lm_head", lib().eagle2_lm_head(_ptr(hidden), _ptr(weight), rows, H, V, _ptr(logits),
+                                                  _ptr(d_status), _stream(stream)))
 
 
 def expand_variant(draft_logits, batch_stride: int, B: int, V: int, k: int, D: int, s: int, flags: int,

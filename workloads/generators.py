@@ -12,6 +12,9 @@ Recipe
                    raised above all others, the token drawn from the base row's softmax by the
                    Gumbel-max trick: a greedy verifier then accepts a child with exactly the
                    probability the draft gave it
+  LM head        feature rows ~ N(0,1), weight [V][H] ~ N(0, (2/sqrt(H))^2), both rounded to bf16:
+                   logits of standard deviation 2 like the draft rows above (random weights of
+                   the right shape; no trained head is available)
   Q, K, V        ~ N(0,1) rounded to bf16
   uniforms       ~ U[0,1) fp32
   ragged lengths = round(exp(U(ln lo, ln hi)))
@@ -33,6 +36,7 @@ def rng_for(seed: int, stream: int) -> np.random.Generator:
 
 STREAM_DRAFT, STREAM_TARGET, STREAM_FRESH, STREAM_QKV, STREAM_U, STREAM_LEN, STREAM_EASY = range(7)
 STREAM_GUMBEL = 7
+STREAM_LM_HEAD = 8
 
 
 def f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:
@@ -160,3 +164,11 @@ def qkv_bf16(cfg: Config, seed: int, kv_len: np.ndarray, kv_off: np.ndarray, lay
     kc = f32_to_bf16_bits(rng.standard_normal((rows, cfg.Hkv, cfg.d), dtype=np.float32))
     vc = f32_to_bf16_bits(rng.standard_normal((rows, cfg.Hkv, cfg.d), dtype=np.float32))
     return q, kc, vc
+
+
+def lm_head_inputs(rows: int, H: int, V: int, seed: int):
+    """(hidden [rows,H], weight [V,H]) as uint16 bf16 bit patterns."""
+    rng = rng_for(seed, STREAM_LM_HEAD)
+    hidden = f32_to_bf16_bits(rng.standard_normal((rows, H), dtype=np.float32))
+    weight = f32_to_bf16_bits(rng.standard_normal((V, H), dtype=np.float32) * np.float32(2.0 / np.sqrt(H)))
+    return hidden, weight
