@@ -5,8 +5,11 @@
 // a few flops per byte.  It still is a dense contraction, so the arithmetic runs on the tensor path,
 // laid out so that the streamed operand fills the instruction: a tile of 128 vocabulary rows is the
 // M side of tcgen05.mma, the (padded) feature rows are its N side, and the accumulator in tensor
-// memory holds logits[vocabulary row][feature row].  One persistent block per SM walks the vocabulary
-// tiles, warp specialised:
+// memory holds logits[vocabulary row][feature row].  Persistent blocks walk the vocabulary tiles,
+// up to four resident per SM: one block's chain of copy, wait and issue sustains about 36 bytes per
+// nanosecond, a quarter short of an SM's share of HBM, and several short rings fill the gap better
+// than one long ring (measured: 199 us with one block of 8 stages per SM, 160 us with four of 3
+// stages, at 10 rows x 4096 x 128256).  A block is warp specialised:
 //   TMA warp       streams 128 x 64 weight boxes (and the matching 64 columns of the features, which
 //                  stay in L2) through a ring of stages;
 //   MMA warp       one thread issues four K = 16 instructions per stage into one of two accumulators;
@@ -43,10 +46,11 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
 }
 
 // n_pad: feature rows rounded up to a multiple of 16 (the instruction's N); acc_cols: accumulator
-// stride in tensor-memory columns (>= 32 so that a 32-column read stays inside the allocation).
-__global__ void __launch_bounds__(kLmThreads, 1)
+// stride in tensor-memory columns (>= 32 so that a 32-column read stays inside the allocation);
+// tmem_cols: the allocation, a power of two that holds the last 32-column read of either accumulator.
+__global__ void __launch_bounds__(kLmThreads, 4)
 lm_head_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant__ CUtensorMap h_map, int rows,
-               int n_pad, int H, int V, int stages, float* __restrict__ logits, int32_t* d_status) {
+               int n_pad, int H, int V, int stages, int tmem_cols, float* __restrict__ logits, int32_t* d_status) {
     extern __shared__ unsigned char smem_raw[];
     __shared__ LmBarriers bars;
     __shared__ uint32_t s_tmem_base;
@@ -74,7 +78,7 @@ lm_head_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant_
         fence_barrier_init();
     }
     if (warp == 1) {
-        tmem_alloc(smem_u32(&s_tmem_base), 512);
+        tmem_alloc(smem_u32(&s_tmem_base), (uint32_t)tmem_cols);
         tmem_relinquish();
     }
     if (warp == 0 && lane == 0) {
@@ -187,7 +191,7 @@ lm_head_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant_
     __syncthreads();
     if (warp == 1) {
         tc_fence_after();
-        tmem_dealloc(tmem, 512);
+        tmem_dealloc(tmem, (uint32_t)tmem_cols);
     }
     if (tid == 0 && s_abort) raise_status(d_status, EAGLE2_STATUS_TIMEOUT);
 }
@@ -220,18 +224,33 @@ extern "C" int eagle2_lm_head(const void* hidden, const void* weight, int rows, 
     if (!make_matrix_map(&w_map, weight, V, H, kLmTileV) || !make_matrix_map(&h_map, hidden, rows, H, n_pad))
         return EAGLE2_ERR_CUDA;
     const uint32_t stage_bytes = kLmWBytes + (uint32_t)n_pad * kLmTileK * 2;
-    int stages = (int)((200u * 1024u) / stage_bytes);
-    if (stages > kLmMaxStages) stages = kLmMaxStages;
+    const int acc_cols = n_pad < 32 ? 32 : n_pad;
+    int tmem_cols = 32;
+    while (tmem_cols < acc_cols + (rows + 31) / 32 * 32) tmem_cols <<= 1;
+    // resident blocks per SM: as many (at most 4) as leave each a ring of 3 stages and its share of
+    // the 512 tensor-memory columns; otherwise one block with the longest ring that fits
+    constexpr uint32_t kSmemPerSm = 227u * 1024u, kPerBlockOverhead = 2u * 1024u + 512u;
+    int resident = 1, stages = 0;
+    for (int c = 4; c >= 1; --c) {
+        const int s = (int)((kSmemPerSm / c - kPerBlockOverhead) / stage_bytes);
+        if ((s >= 3 && c * tmem_cols <= 512) || c == 1) {
+            resident = c;
+            stages = c == 1 ? (s > kLmMaxStages ? kLmMaxStages : s) : 3;
+            break;
+        }
+    }
     const size_t dyn = (size_t)stages * stage_bytes + 1024;
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) != cudaSuccess ||
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
-        cudaFuncSetAttribute(lm_head_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) != cudaSuccess) {
+        cudaFuncSetAttribute(lm_head_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) != cudaSuccess ||
+        cudaFuncSetAttribute(lm_head_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+                             cudaSharedmemCarveoutMaxShared) != cudaSuccess) {
         cudaGetLastError();
         return EAGLE2_ERR_CUDA;
     }
     const int n_tiles = (V + kLmTileV - 1) / kLmTileV;
-    const int grid = n_tiles < sms ? n_tiles : sms;
+    const int grid = n_tiles < resident * sms ? n_tiles : resident * sms;
     return launch_chained(lm_head_kernel, dim3(grid), dim3(kLmThreads), dyn, reinterpret_cast<cudaStream_t>(stream), 1,
-                          w_map, h_map, rows, n_pad, H, V, stages, logits, d_status);
+                          w_map, h_map, rows, n_pad, H, V, stages, tmem_cols, logits, d_status);
 }
