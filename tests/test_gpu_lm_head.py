@@ -122,3 +122,40 @@ def test_lm_head_feeds_the_expansion(name, H):
         assert np.abs(host(gpu.value) - want.value).max() < 1e-3
         assert (host(gpu.frontier) == want.frontier).all()
     assert checked > 0
+
+
+def test_lm_head_and_expansion_replay_from_a_captured_graph():
+    """Both calls only enqueue work, so the pair can be captured once and replayed: the replay on new
+    features must give the logits and the tree of the plain calls."""
+    cfg = get_config("tiny")
+    H = 128
+    hb, wb = gen.lm_head_inputs(cfg.R, H, cfg.V, seed=60)
+    hb2, _ = gen.lm_head_inputs(cfg.R, H, cfg.V, seed=61)
+    th, tw = dev(hb), dev(wb)
+    logits = torch.zeros((1, cfg.R, cfg.V), dtype=torch.float32, device=DEV)
+    st = new_status()
+    tree = GpuTree(1, cfg.V, cfg.k, cfg.D)
+    stream = torch.cuda.Stream()
+
+    def enqueue():
+        e2.lm_head(th, tw, cfg.R, H, cfg.V, logits, st, stream=stream)
+        for s in range(cfg.D):
+            lo = 0 if s == 0 else 1 + (s - 1) * cfg.k
+            e2.expand(logits.data_ptr() + lo * cfg.V * 4, cfg.R * cfg.V, 1, cfg.V, cfg.k, cfg.D, s, tree.token,
+                      tree.parent, tree.value, tree.frontier, tree.ws, tree.status, stream=stream)
+
+    with torch.cuda.stream(stream):
+        enqueue()
+        stream.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            enqueue()
+        th.copy_(dev(hb2))
+        graph.replay()
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0 and int(tree.status.item()) == 0
+    want_logits = ref.lm_head(hb2, wb)
+    assert (np.abs(host(logits)[0] - want_logits) <= _bound(hb2, wb, H)).all()
+    want = ref.build_tree(host(logits), cfg.V, cfg.k, cfg.D)  # the tree of exactly these fp32 logits
+    assert (host(tree.token) == want.token).all() and (host(tree.parent) == want.parent).all()
+    assert (host(tree.frontier) == want.frontier).all()

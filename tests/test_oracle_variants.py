@@ -72,3 +72,52 @@ def test_calibrated_targets_accept_a_child_with_its_confidence():
     keep = p * trials >= 5
     chi2 = ((counts[keep] - p[keep] * trials) ** 2 / (p[keep] * trials)).sum()
     assert chi2 < 45  # 99.99th percentile of chi-square with at most 11 degrees of freedom is below 40
+
+
+def test_dynamic_tree_accepts_more_than_the_fixed_shape_tree_of_the_same_size():
+    """The paper's central comparison (Section 3 against Section 4) on the calibrated workload: with the
+    same number of verified tokens and the same depth limit, the context-dependent tree has the larger
+    expected accepted length, and both measured means sit on their expectations."""
+    from scipy.special import logsumexp
+    from workloads import static_tree
+
+    k, D = 10, static_tree.N_LEVELS
+    index, parent, depth, rank, row_of = static_tree.shape(k)
+    n = len(index)
+    cfg = get_config("tiny", B=8, V=1000, k=k, D=D, m=n)
+    got = {"static": [], "dynamic": []}
+    want = {"static": [], "dynamic": []}
+    for seed in range(40):
+        draft = gen.draft_rows(cfg, seed)
+        ua, ub = gen.uniforms(cfg, seed)
+        # dynamic: the method itself
+        tree = ref.build_tree(draft, cfg.V, k, D)
+        sel = ref.rerank(tree.token, tree.parent, tree.value, k, D, n)
+        target = gen.target_rows_calibrated(cfg, seed, draft, tree.parent, sel.index)
+        got["dynamic"].append(ref.accept(target, None, sel, cfg.V, k, D, n, 0.0, ua, ub).acc_len)
+        want["dynamic"].append(np.exp(np.take_along_axis(tree.value, sel.index.astype(np.int64), axis=1)).sum(axis=1))
+        # static: the declared shape filled with per-position top tokens
+        tok = static_tree.tokens(draft, k)
+        ssel = ref.Selection(np.tile(index, (cfg.B, 1)), np.tile(parent, (cfg.B, 1)), tok,
+                             np.tile(depth, (cfg.B, 1)), np.full(cfg.B, n, np.int32))
+        parent_cand = np.full((cfg.B, cfg.N), -1, np.int32)  # which candidate expanded which slot
+        for x in range(n):
+            if parent[x] >= 0:
+                parent_cand[:, index[x]] = index[parent[x]]
+        starget = gen.target_rows_calibrated(cfg, seed, draft, parent_cand, ssel.index)
+        got["static"].append(ref.accept(starget, None, ssel, cfg.V, k, D, n, 0.0, ua, ub).acc_len)
+        expect = np.zeros(cfg.B)
+        for b in range(cfg.B):
+            logv = np.zeros(n)
+            for x in range(n):  # ascending index: parents first
+                row = 0 if parent[x] < 0 else int(row_of[parent[x]])
+                z = draft[b, row].astype(np.float64)
+                logv[x] = (0.0 if parent[x] < 0 else logv[parent[x]]) + z[tok[b, x]] - logsumexp(z)
+            expect[b] = np.exp(logv).sum()
+        want["static"].append(expect)
+    for name in got:
+        g, w = np.concatenate(got[name]).astype(np.float64), np.concatenate(want[name])
+        assert abs(g.mean() - w.mean()) < 4 * 1.2 / np.sqrt(len(g)), name
+        got[name], want[name] = g, w
+    assert want["dynamic"].mean() > want["static"].mean()
+    assert got["dynamic"].mean() > got["static"].mean()
