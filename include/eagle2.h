@@ -88,7 +88,8 @@ int eagle2_workspace_init(void* ws, size_t ws_bytes, eagle2_stream_t stream);
  *   hidden  bf16 [rows][H], 16-byte aligned
  *   weight  bf16 [V][H], 16-byte aligned (the matrix is read once per call)
  *   logits  fp32 [rows][V], written
- * Limits: 0 <= rows <= 256, H a multiple of 64, V >= 1.  Needs no workspace.  A bounded wait that
+ * Limits: rows >= 0, H a multiple of 64, V >= 1.  Up to 256 rows are one pass over the weights; more
+ * rows take one pass per 256.  Needs no workspace.  A bounded wait that
  * runs out raises EAGLE2_STATUS_TIMEOUT.
  */
 int eagle2_lm_head(const void* hidden, const void* weight, int rows, int H, int V, float* logits,

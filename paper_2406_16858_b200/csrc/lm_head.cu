@@ -212,12 +212,9 @@ static bool make_matrix_map(CUtensorMap* map, const void* base, long long n_rows
 
 using namespace eagle2;
 
-extern "C" int eagle2_lm_head(const void* hidden, const void* weight, int rows, int H, int V, float* logits,
-                              int32_t* d_status, eagle2_stream_t stream) {
-    if (!hidden || !weight || !logits || !d_status) return EAGLE2_ERR_NULL;
-    if (rows < 0 || rows > kLmMaxRows || H < kLmTileK || H % kLmTileK != 0 || V < 1) return EAGLE2_ERR_SHAPE;
-    if (!aligned(hidden, 16) || !aligned(weight, 16) || !aligned(logits, 4)) return EAGLE2_ERR_ALIGN;
-    if (rows == 0) return EAGLE2_OK;
+// One launch: up to kLmMaxRows feature rows against the whole weight matrix.
+static int lm_head_rows(const void* hidden, const void* weight, int rows, int H, int V, float* logits,
+                        int32_t* d_status, eagle2_stream_t stream) {
     const int n_pad = (rows + 15) / 16 * 16;
     CUtensorMap w_map, h_map;
     // feature rows past `rows` and vocabulary rows past V read as zero
@@ -253,4 +250,20 @@ extern "C" int eagle2_lm_head(const void* hidden, const void* weight, int rows, 
     const int grid = n_tiles < resident * sms ? n_tiles : resident * sms;
     return launch_chained(lm_head_kernel, dim3(grid), dim3(kLmThreads), dyn, reinterpret_cast<cudaStream_t>(stream), 1,
                           w_map, h_map, rows, n_pad, H, V, stages, tmem_cols, logits, d_status);
+}
+
+extern "C" int eagle2_lm_head(const void* hidden, const void* weight, int rows, int H, int V, float* logits,
+                              int32_t* d_status, eagle2_stream_t stream) {
+    if (!hidden || !weight || !logits || !d_status) return EAGLE2_ERR_NULL;
+    if (rows < 0 || H < kLmTileK || H % kLmTileK != 0 || V < 1) return EAGLE2_ERR_SHAPE;
+    if (!aligned(hidden, 16) || !aligned(weight, 16) || !aligned(logits, 4)) return EAGLE2_ERR_ALIGN;
+    // more rows than one instruction's N: one pass over the weights per 256 rows (at that width a
+    // pass is bound by the tensor pipe, not by the weight stream, so little is lost by re-reading)
+    for (int r0 = 0; r0 < rows; r0 += kLmMaxRows) {
+        const int n = rows - r0 < kLmMaxRows ? rows - r0 : kLmMaxRows;
+        const int rc = lm_head_rows(static_cast<const __nv_bfloat16*>(hidden) + (size_t)r0 * H, weight, n, H, V,
+                                    logits + (size_t)r0 * V, d_status, stream);
+        if (rc != EAGLE2_OK) return rc;
+    }
+    return EAGLE2_OK;
 }

@@ -37,6 +37,7 @@ def _bound(hb, wb, H):
 @pytest.mark.parametrize("rows,H,V", [
     (1, 64, 1), (1, 64, 128), (4, 128, 129), (10, 320, 1000), (13, 64, 5000), (16, 128, 127),
     (17, 192, 300), (40, 64, 1000), (51, 256, 2049), (200, 128, 777), (256, 64, 1000),
+    (257, 64, 300), (600, 128, 1000),  # more rows than one pass holds
 ])
 def test_small_shapes_tails_and_row_counts(rows, H, V):
     hb, wb = gen.lm_head_inputs(rows, H, V, seed=rows + V)
@@ -81,7 +82,7 @@ def test_refusals():
         e2.lm_head(th, tw, 4, 48, 100, out, st)      # H not a multiple of 64
     assert err.value.code == -2
     with pytest.raises(e2.Eagle2Error) as err:
-        e2.lm_head(th, tw, 257, 64, 100, out, st)    # too many rows
+        e2.lm_head(th, tw, -1, 64, 100, out, st)
     assert err.value.code == -2
     with pytest.raises(e2.Eagle2Error) as err:
         e2.lm_head(th.data_ptr() + 2, tw, 4, 64, 100, out, st)
