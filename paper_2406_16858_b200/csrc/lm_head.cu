@@ -224,15 +224,16 @@ static int lm_head_rows(const void* hidden, const void* weight, int rows, int H,
     const int acc_cols = n_pad < 32 ? 32 : n_pad;
     int tmem_cols = 32;
     while (tmem_cols < acc_cols + (rows + 31) / 32 * 32) tmem_cols <<= 1;
-    // resident blocks per SM: as many (at most 4) as leave each a ring of 3 stages and its share of
-    // the 512 tensor-memory columns; otherwise one block with the longest ring that fits
+    // resident blocks per SM: four with rings of 2-3 stages where shared memory and the 512
+    // tensor-memory columns allow (measured best up to 64 rows), else as many as keep 3 stages each,
+    // else one block with the longest ring that fits
     constexpr uint32_t kSmemPerSm = 227u * 1024u, kPerBlockOverhead = 2u * 1024u + 512u;
     int resident = 1, stages = 0;
     for (int c = 4; c >= 1; --c) {
         const int s = (int)((kSmemPerSm / c - kPerBlockOverhead) / stage_bytes);
-        if ((s >= 3 && c * tmem_cols <= 512) || c == 1) {
+        if ((s >= (c == 4 ? 2 : 3) && c * tmem_cols <= 512) || c == 1) {
             resident = c;
-            stages = c == 1 ? (s > kLmMaxStages ? kLmMaxStages : s) : 3;
+            stages = c == 1 ? (s > kLmMaxStages ? kLmMaxStages : s) : (s < 3 ? s : 3);
             break;
         }
     }

@@ -84,6 +84,17 @@ def test_null_and_shape_errors_are_found_on_the_host():
                  FAKE, FAKE, FAKE, None, FAKE) == -2
     # compaction: row bytes must be a multiple of 16
     assert _code(e2.kv_compact, FAKE, FAKE, 1, FAKE, FAKE, FAKE, FAKE, 1, 16, 3, 1, 4, FAKE) == -3
+    # the variants: unknown expansion flag, selection without a frontier
+    assert _code(e2.expand_variant, FAKE, 0, 1, 100, 4, 3, 0, 2, FAKE, FAKE, FAKE, FAKE, None, FAKE) == -2
+    assert _code(e2.expand_variant, FAKE, 0, 1, 100, 4, 3, 0, 1, FAKE, FAKE, FAKE, FAKE, None, FAKE) == -4
+    assert _code(e2.rerank_skipped, FAKE, FAKE, FAKE, None, 1, 4, 3, 16, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE) == -1
+    assert _code(e2.rerank_skipped, FAKE, FAKE, FAKE, FAKE, 1, 4, 3, 129, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE) == -2
+    # LM head: hidden size in whole 64-column blocks, 16-byte aligned operands
+    assert _code(e2.lm_head, FAKE, FAKE, 4, 96, 100, FAKE, FAKE) == -2
+    assert _code(e2.lm_head, FAKE, FAKE, -1, 64, 100, FAKE, FAKE) == -2
+    assert _code(e2.lm_head, FAKE + 2, FAKE, 4, 64, 100, FAKE, FAKE) == -3
+    assert _code(e2.lm_head, FAKE, None, 4, 64, 100, FAKE, FAKE) == -1
+    e2.lm_head(FAKE, FAKE, 0, 64, 100, FAKE, FAKE)  # no rows: nothing is launched
 
 
 def test_zero_batch_is_a_no_op():

@@ -56,7 +56,7 @@ def test_more_tiles_than_blocks_and_every_stage_reused():
     assert (np.abs(got - want) <= _bound(hb, wb, H)).all()
 
 
-@pytest.mark.parametrize("name,H", [("vicuna7b", 4096), ("llama3_8b", 4096)])
+@pytest.mark.parametrize("name,H", [("vicuna7b", 4096), ("llama3_8b", 4096), ("llama2_70b", 8192)])
 def test_model_shapes_sampled_vocabulary_rows(name, H):
     """Full vocabulary and hidden size on the device; the oracle computes a sample of 3000 vocabulary
     rows (the same weight rows handed to it as a smaller matrix) plus the first and last tile."""
