@@ -35,6 +35,7 @@ constexpr uint32_t kLmWBytes = kLmTileV * kLmTileK * 2;
 
 struct LmBarriers {
     unsigned long long full[kLmMaxStages], empty[kLmMaxStages], acc_full[2], acc_empty[2];
+    unsigned long long drain;  // used only after a wait ran out: the block's last instructions have retired
 };
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
@@ -75,6 +76,7 @@ lm_head_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant_
             mbar_init(smem_u32(&bars.acc_full[a]), 1);
             mbar_init(smem_u32(&bars.acc_empty[a]), 4);  // one arrival per store warp
         }
+        mbar_init(smem_u32(&bars.drain), 1);
         fence_barrier_init();
     }
     if (warp == 1) {
@@ -191,6 +193,17 @@ lm_head_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant_
     __syncthreads();
     if (warp == 1) {
         tc_fence_after();
+        if (s_abort) {
+            // instructions issued before the wait ran out may still be reading shared memory and
+            // writing tensor memory: let them retire (bounded) before either is given back
+            if (lane == 0) {
+                tc_commit(smem_u32(&bars.drain));
+                const long long t0 = clock64();
+                while (!mbar_try_wait(smem_u32(&bars.drain), 0) && clock64() - t0 < kWaitCycles) {}
+            }
+            __syncwarp();
+            tc_fence_after();
+        }
         tmem_dealloc(tmem, (uint32_t)tmem_cols);
     }
     if (tid == 0 && s_abort) raise_status(d_status, EAGLE2_STATUS_TIMEOUT);
