@@ -31,7 +31,7 @@ def _compare(cfg, draft, sel, target, ua, ub, temperature, point_mass=False, t_s
              d_stride=None):
     d_arg = None if (temperature == 0 or point_mass) else draft
     want = ref.accept(target, d_arg, sel, cfg.V, cfg.k, cfg.D, cfg.m, temperature, ua, ub,
-                      t_stride=t_stride, d_stride=d_stride)
+                      t_stride=t_stride, d_stride=d_stride, debug=temperature > 0)
     alen, apath, bonus, st = gpu_accept(target, d_arg, sel.index, sel.parent, sel.token, sel.n_sel,
                                         cfg.V, cfg.k, cfg.D, cfg.m, temperature, ua, ub,
                                         t_stride=t_stride, d_stride=d_stride)
@@ -44,7 +44,16 @@ def _compare(cfg, draft, sel, target, ua, ub, temperature, point_mass=False, t_s
         assert alen[b] == want.acc_len[b], (b, alen[b], want.acc_len[b])
         assert (apath[b] == want.acc_path[b]).all()
         if temperature > 0 and want.margins[b, 1] < 1e-5:
+            # the draw falls within 1e-5 of a step of the distribution function (always so when the
+            # drawn token itself holds less than 2e-5): the device may name a neighbour, but only one
+            # whose own step lies within that distance of the draw
             n_exempt += 1
+            p = want.p_final[b]
+            cdf = np.cumsum(p)
+            thr = float(ub[b]) * cdf[-1]
+            t = int(bonus[b])
+            assert 0 <= t < cfg.V and p[t] > 0
+            assert cdf[t] - p[t] - 1e-5 * cdf[-1] <= thr <= cdf[t] + 1e-5 * cdf[-1], (b, t, want.bonus_token[b])
             continue
         assert bonus[b] == want.bonus_token[b], (b, bonus[b], want.bonus_token[b], want.margins[b])
     return n_exempt, want

@@ -69,7 +69,7 @@ def test_acceptance(temperature, V, seed):
     B = 16
     draft, sel, target, ua, ub, n = _forest(B, V, seed)
     d_arg = draft if temperature > 0 else None
-    want = ref.accept(target, d_arg, sel, V, K, D, n, temperature, ua, ub)
+    want = ref.accept(target, d_arg, sel, V, K, D, n, temperature, ua, ub, debug=temperature > 0)
     alen, apath, bonus, st = gpu_accept(target, d_arg, sel.index, sel.parent, sel.token, sel.n_sel, V, K, D, n,
                                         temperature, ua, ub)
     assert st == want.status == 0
@@ -79,5 +79,11 @@ def test_acceptance(temperature, V, seed):
             continue
         assert alen[b] == want.acc_len[b] and (apath[b] == want.acc_path[b]).all()
         if temperature > 0 and want.margins[b, 1] < 1e-5:
+            # a draw within 1e-5 of a step of the distribution function: a neighbour is acceptable
+            # if its own step lies within that distance of the draw
+            p = want.p_final[b]
+            cdf = np.cumsum(p)
+            thr, t = float(ub[b]) * cdf[-1], int(bonus[b])
+            assert p[t] > 0 and cdf[t] - p[t] - 1e-5 * cdf[-1] <= thr <= cdf[t] + 1e-5 * cdf[-1]
             continue
         assert bonus[b] == want.bonus_token[b]
