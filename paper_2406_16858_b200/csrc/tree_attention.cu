@@ -98,7 +98,7 @@ static void attention_plan(int B, int m, int Hq, int Hkv, int d, int max_kv_len,
 }
 
 struct AttnWs {
-    float* o_part;  // [B][Hkv][splits][n_rb][mt*128][d]
+    __nv_bfloat16* o_part;  // [B][Hkv][splits][n_rb][mt*128][d], unnormalised, rounded once to bf16
     float2* ml;     // [B][Hkv][splits][n_rb][mt*128]  (reference maximum in log2 units, sum)
     uint32_t* order;  // ordered launches: [0] = items with tiles, [1 + i] = sequence * splits + split of item i
     int* tickets;     // merging launches: [B][Hkv][n_rb] arrival counters, left at zero
@@ -112,8 +112,8 @@ static size_t attention_ws_layout(int B, int Hkv, int d, const AttnPlan& p, void
     char* c = static_cast<char*>(base);
     if (p.splits > 1) {
         const size_t rows = (size_t)B * Hkv * p.splits * p.n_rb * p.mt * kRowsPerTile;
-        if (w) w->o_part = reinterpret_cast<float*>(c + off);
-        off += round_up(rows * d * sizeof(float), kWsAlign);
+        if (w) w->o_part = reinterpret_cast<__nv_bfloat16*>(c + off);
+        off += round_up(rows * d * sizeof(__nv_bfloat16), kWsAlign);
         if (w) w->ml = reinterpret_cast<float2*>(c + off);
         off += round_up(rows * sizeof(float2), kWsAlign);
     }
@@ -296,13 +296,14 @@ __device__ __forceinline__ void merge_row(const AttnPlan& plan, const AttnWs& ws
 #pragma unroll
             for (int u = 0; u < W; ++u) {
                 const int sl = min(s1 + u, n - 1);  // clamped: a repeated row gets weight 0 below
-                const float* src = ws.o_part + (first + (size_t)(s0 + sl) * stride) * DH + lane * PER;
+                const __nv_bfloat16* src = ws.o_part + (first + (size_t)(s0 + sl) * stride) * DH + lane * PER;
                 if (PER == 4) {
-                    const float4 t = *reinterpret_cast<const float4*>(src);
-                    v[u][0] = t.x, v[u][1] = t.y, v[u][PER - 2] = t.z, v[u][PER - 1] = t.w;
+                    const uint2 t = *reinterpret_cast<const uint2*>(src);
+                    v[u][0] = __uint_as_float(t.x << 16), v[u][1] = __uint_as_float(t.x & 0xffff0000u);
+                    v[u][PER - 2] = __uint_as_float(t.y << 16), v[u][PER - 1] = __uint_as_float(t.y & 0xffff0000u);
                 } else {
-                    const float2 t = *reinterpret_cast<const float2*>(src);
-                    v[u][0] = t.x, v[u][1] = t.y;
+                    const uint32_t t = *reinterpret_cast<const uint32_t*>(src);
+                    v[u][0] = __uint_as_float(t << 16), v[u][1] = __uint_as_float(t & 0xffff0000u);
                 }
             }
         };
@@ -850,12 +851,14 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
             const int col0 = half * NCOL;
             const uint32_t o_addr = tmem + lane_sel + kOCol + (uint32_t)wg * DH + (uint32_t)col0;
             const float l_tot = SPLIT ? l_run + s_xsum[half ^ 1][r_tile] : l_run;
-            const float inv = l_tot > 0.f ? 1.f / l_tot : 0.f;
+            // final rows are normalised here; a partial stays unnormalised (the merge divides by the
+            // combined sum) and is rounded to bf16 once, like a final row
+            const float inv = !direct ? 1.f : (l_tot > 0.f ? 1.f / l_tot : 0.f);
             unsigned char* stage = smem_gen + ((MT == 2 && wg == 0) ? 0u : (sK - smem_base));
-            // a staged row is DH fp32 (partial) or DH bf16 (final); 16-byte chunk c of row r sits at
-            // chunk c ^ (r mod chunks-per-row), which keeps both the row-wise writes and the
-            // chunk-wise reads free of bank conflicts
-            const int row_bytes = direct ? DH * 2 : DH * 4;
+            // a staged row is DH bf16; 16-byte chunk c of row r sits at chunk c ^ (r mod
+            // chunks-per-row), which keeps both the row-wise writes and the chunk-wise reads free of
+            // bank conflicts
+            constexpr int row_bytes = DH * 2;
             const int cmask = row_bytes / 16 - 1;
 #pragma unroll
             for (int c4 = 0; c4 < NCOL / 32; ++c4) {
@@ -863,7 +866,7 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
                 tmem_ld32(o_addr + c4 * 32, orow);
                 tc_wait_ld(orow);
                 unsigned char* srow = stage + (size_t)r_tile * row_bytes;
-                if (direct) {
+                {
 #pragma unroll
                     for (int c = 0; c < 32; c += 8) {
                         uint4 v;
@@ -873,13 +876,6 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
                         v.w = pack_bf16(__uint_as_float(orow[c + 6]) * inv, __uint_as_float(orow[c + 7]) * inv);
                         const int chunk = (col0 + c4 * 32 + c) >> 3;
                         *reinterpret_cast<uint4*>(srow + (((chunk ^ r_tile) & cmask) << 4)) = v;
-                    }
-                } else {
-#pragma unroll
-                    for (int c = 0; c < 32; c += 4) {
-                        const int chunk = (col0 + c4 * 32 + c) >> 2;
-                        *reinterpret_cast<uint4*>(srow + (((chunk ^ r_tile) & cmask) << 4)) =
-                            make_uint4(orow[c], orow[c + 1], orow[c + 2], orow[c + 3]);
                     }
                 }
             }
@@ -903,7 +899,7 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
                     __nv_bfloat16* dst = out + (((long long)b * m + p2 / g) * Hq + hk * g + p2 % g) * DH;
                     *reinterpret_cast<uint4*>(reinterpret_cast<unsigned char*>(dst) + cl * 16) = v;
                 } else {
-                    float* dst = ws.o_part + (part_row0 + wg * 128 + r) * DH;
+                    __nv_bfloat16* dst = ws.o_part + (part_row0 + wg * 128 + r) * DH;
                     *reinterpret_cast<uint4*>(reinterpret_cast<unsigned char*>(dst) + cl * 16) = v;
                 }
             }
