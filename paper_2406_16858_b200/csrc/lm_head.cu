@@ -254,7 +254,10 @@ static int lm_head_rows(const void* hidden, const void* weight, int rows, int H,
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) != cudaSuccess ||
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
-        cudaFuncSetAttribute(lm_head_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) != cudaSuccess ||
+        // always the device's opt-in maximum, whatever this call needs: concurrent callers with
+        // different row counts then set the same value
+        cudaFuncSetAttribute(lm_head_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemPerSm - 1024) !=
+            cudaSuccess ||
         cudaFuncSetAttribute(lm_head_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
                              cudaSharedmemCarveoutMaxShared) != cudaSuccess) {
         cudaGetLastError();
