@@ -121,7 +121,7 @@ static size_t attention_ws_layout(int B, int Hkv, int d, const AttnPlan& p, void
         if (w) w->order = reinterpret_cast<uint32_t*>(c + off);
         off += round_up(sizeof(uint32_t) * ((size_t)B * p.splits + 1), kWsAlign);
     }
-    if (p.fused_merge) {
+    if (p.fused_merge) {  // (cleared by the launch's own list kernel: other operations' scratch may overlap it)
         if (w) w->tickets = reinterpret_cast<int*>(c + off);
         off += round_up(sizeof(int) * (size_t)B * Hkv * p.n_rb, kWsAlign);
     }
@@ -935,10 +935,13 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
 // changes nothing but the schedule).
 __global__ void __launch_bounds__(1024)
 tree_attention_schedule_kernel(const int64_t* __restrict__ kv_off, const int32_t* __restrict__ kv_len, int B, int m,
-                               long long cache_rows, int max_kv_len, AttnPlan plan, uint32_t* __restrict__ order) {
+                               long long cache_rows, int max_kv_len, AttnPlan plan, uint32_t* __restrict__ order,
+                               int* __restrict__ tickets, int n_tickets) {
     __shared__ int s_bin[kMaxTilesPerSplitOrdered + 1];  // per tile count: items, then the next free place
     chain_wait();
     chain_release();
+    // the merging blocks' arrival counters start at zero whatever shared this workspace since
+    for (int i = threadIdx.x; i < n_tickets; i += blockDim.x) tickets[i] = 0;
     const int S = plan.splits;
     const long long n = (long long)B * S;
     for (int i = threadIdx.x; i <= kMaxTilesPerSplitOrdered; i += blockDim.x) s_bin[i] = 0;
@@ -1020,7 +1023,7 @@ static int launch_attention(const CUtensorMap& k_map, const CUtensorMap& v_map, 
     if (blocks > 0x7fffffffLL || (long long)B * plan.splits > 0x7fffffffLL) return EAGLE2_ERR_SHAPE;
     if (plan.ordered &&
         launch_chained(tree_attention_schedule_kernel, dim3(1), dim3(1024), 0, st, 1, kv_off, kv_len, B, m, cache_rows,
-                       max_kv_len, plan, ws.order) != EAGLE2_OK)
+                       max_kv_len, plan, ws.order, ws.tickets, plan.fused_merge ? B * Hkv * plan.n_rb : 0) != EAGLE2_OK)
         return EAGLE2_ERR_CUDA;
     if (launch_chained(kern, dim3((unsigned)blocks), dim3(kAttnThreads), plan.smem, st, PAIR ? 2u : 1u, k_map, v_map, q_map,
                        static_cast<const __nv_bfloat16*>(q), kv_off, kv_len, mask_bits, m, Hq, Hkv, cache_rows, max_kv_len,
