@@ -101,11 +101,18 @@ class ClockSampler:
 # ------------------------------------------------------------------------------------------------
 # CPU oracle timing (cpu_baseline leg and --impl reference)
 
-def oracle_cycle_seconds(cfg, seed: int = 0, attn_samples: int = 96):
+def oracle_cycle_seconds(cfg, seed: int = 0, attn_samples: int = 96, threads: int | None = None):
     """Times the oracle on a bounded sample of one cycle and extrapolates to the whole cycle.
     Logit steps and tree steps run whole; attention runs `attn_samples` query rows of one layer and is
-    scaled to n_layers * m * Hq rows; compaction runs on one layer and is scaled to n_layers."""
+    scaled to n_layers * m * Hq rows; compaction runs on one layer and is scaled to n_layers.
+    `threads`: run the oracle's loops over independent units on that many threads (default: all)."""
     from oracle import ref
+    if threads is not None:
+        before = ref.set_threads(threads)
+        try:
+            return oracle_cycle_seconds(cfg, seed, attn_samples)
+        finally:
+            ref.set_threads(before)
     small = cfg.with_(B=1)
     t = {}
     draft = gen.draft_rows(small, seed)
@@ -209,6 +216,7 @@ def batched_attention_extra(e2, dev, stream, hbm_peak, B=32, n_layers=3, reps=10
     ws = torch.empty(max(e2.workspace_bytes(e2.OP_TREE_ATTENTION, B=B, m=cfg.m, Hq=cfg.Hq, Hkv=cfg.Hkv, d=cfg.d,
                                             max_kv_len=max_len), 256), dtype=torch.uint8, device=dev)
     e2.workspace_init(ws)
+    torch.cuda.synchronize()  # inputs were made on the default stream; the timed work runs on `stream`
 
     def layers():
         for kc, vc in zip(ks, vs):
@@ -232,13 +240,16 @@ def batched_attention_extra(e2, dev, stream, hbm_peak, B=32, n_layers=3, reps=10
             "us_per_layer": us, "algorithmic_bytes_per_layer": nbytes, "achieved_gbs": gbs, "frac_of_measured_hbm": gbs / hbm_peak}
 
 
-def batched_expand_extra(e2, dev, stream, hbm_peak, B=128, n_sets=4, reps=20):
+def batched_expand_extra(e2, dev, stream, hbm_peak, B=128, n_sets=None, reps=20):
     """One expansion step (k rows per sequence) alone at a batch that gives a launch enough bytes
     (B*k*V*4 = 0.66 GB) for the HBM fraction to be about the kernel; a few distinct logit sets
     larger than L2."""
     import torch
     cfg = get_config("llama3_8b").with_(B=B)
     k, V, D = cfg.k, cfg.V, cfg.D
+    if n_sets is None:
+        n_sets = int(max(4, math.ceil(300e6 / (B * k * V * 4.0))))
+    reps = max(2, min(reps, 400 // n_sets))
     g = torch.Generator(device=dev).manual_seed(7)
     logits = [torch.randn((B, k, V), generator=g, device=dev) for _ in range(n_sets)]
     N = k + (D - 1) * k * k
@@ -250,6 +261,7 @@ def batched_expand_extra(e2, dev, stream, hbm_peak, B=128, n_sets=4, reps=20):
     status = torch.zeros(1, dtype=torch.int32, device=dev)
     ws = torch.empty(e2.workspace_bytes(e2.OP_EXPAND, B=B, V=V, k=k, D=D), dtype=torch.uint8, device=dev)
     e2.workspace_init(ws)
+    torch.cuda.synchronize()  # inputs were made on the default stream; the timed work runs on `stream`
 
     def steps():
         for z in logits:
@@ -265,7 +277,7 @@ def batched_expand_extra(e2, dev, stream, hbm_peak, B=128, n_sets=4, reps=20):
             steps()
         ev1.record(stream)
     torch.cuda.synchronize()
-    assert int(status.item()) == 0
+    assert int(status.item()) == 0, f"device status {int(status.item())} in the expansion sweep at B={B}"
     us = ev0.elapsed_time(ev1) * 1e3 / (reps * n_sets)  # includes the 5 KB frontier reset per call
     nbytes = float(B) * k * V * 4
     gbs = nbytes / (us * 1e-6) / 1e9
@@ -285,6 +297,7 @@ def batched_accept_extra(e2, dev, stream, hbm_peak, B=16, reps=10):
     g = torch.Generator(device=dev).manual_seed(11)
     draft = torch.from_numpy(gen.draft_rows(cfg, 5)).to(dev)
     kv_len = torch.zeros(B, dtype=torch.int32, device=dev)
+    torch.cuda.synchronize()
     with torch.cuda.stream(stream):
         buf.expand_all(draft)
         buf.rerank_and_mask(kv_len)
@@ -303,6 +316,7 @@ def batched_accept_extra(e2, dev, stream, hbm_peak, B=16, reps=10):
     del base
     ua_h, ub_h = gen.uniforms(cfg, 5)
     ua, ub = torch.from_numpy(ua_h).to(dev), torch.from_numpy(ub_h).to(dev)
+    torch.cuda.synchronize()
     with torch.cuda.stream(stream):
         for _ in range(3):
             buf.accept(target, draft, ua, ub)
@@ -355,6 +369,7 @@ def draft_attention_extra(e2, dev, stream, hbm_peak, reps=200):
         ws = torch.empty(max(e2.workspace_bytes(e2.OP_TREE_ATTENTION, B=1, m=m, Hq=cfg.Hq, Hkv=cfg.Hkv, d=cfg.d,
                                                 max_kv_len=L), 256), dtype=torch.uint8, device=dev)
         e2.workspace_init(ws)
+        torch.cuda.synchronize()  # inputs were made on the default stream; the timed work runs on `stream`
 
         def calls():
             for kc, vc in zip(ks, vs):
@@ -406,6 +421,7 @@ def lm_head_extra(e2, dev, stream, hbm_peak, reps=30):
     frontier = torch.zeros((1, k), dtype=torch.int32, device=dev)
     ws = torch.empty(max(e2.workspace_bytes(e2.OP_EXPAND, B=1, V=V, k=k, D=D), 256), dtype=torch.uint8, device=dev)
     e2.workspace_init(ws)
+    torch.cuda.synchronize()  # inputs were made on the default stream; the timed work runs on `stream`
     out = {}
     for name in ("lm_head", "lm_head_then_expand"):
         def calls():
@@ -462,6 +478,8 @@ def run_ours(args):
     cfg = get_config(args.workload)
     if args.batch:
         cfg = cfg.with_(B=args.batch)
+    if args.temperature is not None:
+        cfg = cfg.with_(temperature=args.temperature)
     seed = replica_seed(rank)
     kv_len_h = gen.kv_lengths(cfg, seed)
     kv_off_h = gen.kv_offsets(kv_len_h, cfg.m)
@@ -486,9 +504,14 @@ def run_ours(args):
     kv_len0 = torch.from_numpy(kv_len_h).to(dev)
     kv_len = kv_len0.clone()
 
-    buf = CycleBuffers(shape, dev)
+    # one set of tree/selection arrays per logit set (a set's acceptance reads its own tree's selection);
+    # the scratch workspace is shared
+    bufs = [CycleBuffers(shape, dev) for _ in range(N_SETS)]
+    for bb in bufs[1:]:
+        bb.ws = bufs[0].ws
     sets = []
     for i in range(N_SETS):
+        buf = bufs[i]
         draft_h = gen.draft_rows(cfg, seed + 17 * i)
         draft = torch.from_numpy(draft_h).to(dev)
         # the target rows depend on which nodes were selected: build the tree once to find them
@@ -505,13 +528,14 @@ def run_ours(args):
         base = torch.gather(draft, 1, torch.from_numpy(src_rows).to(dev)[:, :, None].expand(-1, -1, cfg.V))
         target = base + 0.5 * torch.randn(base.shape, generator=g, device=dev)
         ua_h, ub_h = gen.uniforms(cfg, seed + 17 * i)
-        sets.append(dict(draft=draft, target=target.contiguous(), ua=torch.from_numpy(ua_h).to(dev),
+        sets.append(dict(buf=buf, draft=draft, target=target.contiguous(), ua=torch.from_numpy(ua_h).to(dev),
                          ub=torch.from_numpy(ub_h).to(dev)))
-    assert int(buf.status.item()) == 0, "device status raised while preparing inputs"
+    assert all(int(bb.status.item()) == 0 for bb in bufs), "device status raised while preparing inputs"
+    buf = bufs[0]
 
     def one_cycle(s):
         kv_len.copy_(kv_len0)  # the cache length is caller state: start every cycle from the same prefix
-        enqueue_cycle(buf, s["draft"], s["target"], s["ua"], s["ub"], q_layers, k_layers, v_layers,
+        enqueue_cycle(s["buf"], s["draft"], s["target"], s["ua"], s["ub"], q_layers, k_layers, v_layers,
                       out_layers, k_ptrs, v_ptrs, kv_off, kv_len, scale)
 
     stream = torch.cuda.Stream(device=dev)
@@ -530,14 +554,16 @@ def run_ours(args):
             for qq, kc, vc, oo in zip(q_layers, k_layers, v_layers, out_layers):
                 buf.attention(qq, kc, vc, kv_off, kv_len0, oo, scale)
         # the other steps on their own, for the per-step breakdown
-        step_graphs = {}
-        for name, fn in (("expand_x%d" % cfg.D, lambda: buf.expand_all(sets[0]["draft"])),
-                         ("rerank_mask", lambda: buf.rerank_and_mask(kv_len0)),
-                         ("accept", lambda: buf.accept(sets[0]["target"], sets[0]["draft"], sets[0]["ua"], sets[0]["ub"]))):
-            gr = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(gr, stream=stream):
-                fn()
-            step_graphs[name] = gr
+        step_graphs = {}  # one graph per logit set and step, replayed in rotation: the logits come from HBM
+        for name, fn in (("expand_x%d" % cfg.D, lambda z: z["buf"].expand_all(z["draft"])),
+                         ("rerank_mask", lambda z: z["buf"].rerank_and_mask(kv_len0)),
+                         ("accept", lambda z: z["buf"].accept(z["target"], z["draft"], z["ua"], z["ub"]))):
+            step_graphs[name] = []
+            for z in sets:
+                gr = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(gr, stream=stream):
+                    fn(z)
+                step_graphs[name].append(gr)
     torch.cuda.synchronize()
 
     def barrier():
@@ -556,17 +582,59 @@ def run_ours(args):
         barrier()
         return max_over_ranks(ev0.elapsed_time(ev1), world, dev)
 
+    def timed_each(fn, steps):
+        """Per-step device times (ms): an event between consecutive steps."""
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+        barrier()
+        with torch.cuda.stream(stream):
+            evs[0].record(stream)
+            for i in range(steps):
+                fn(i)
+                evs[i + 1].record(stream)
+        barrier()
+        return [evs[i].elapsed_time(evs[i + 1]) for i in range(steps)]
+
+    def spread(ms_list, per=1.0):
+        a = np.asarray(ms_list) * 1e3 / per
+        return {"median": float(np.median(a)), "p10": float(np.percentile(a, 10)), "p90": float(np.percentile(a, 90)),
+                "n": int(a.size)}
+
+    kv_bytes = float(sum(2 * (int(L) + cfg.m) * cfg.Hkv * cfg.d * 2 for L in kv_len_h))
+    qo_bytes = float(2 * cfg.B * cfg.m * cfg.Hq * cfg.d * 2)
+    attn_bytes = kv_bytes + qo_bytes  # algorithmic bytes of one tree-attention call (one layer)
+
     K, W = args.steps, max(args.warmup, 3)
     with ClockSampler(local) as clocks:
         timed(lambda i: graphs[i % N_SETS].replay(), W)
         ms_total = timed(lambda i: graphs[i % N_SETS].replay(), K)
+        cycle_spread = spread(timed_each(lambda i: graphs[i % N_SETS].replay(), max(20, min(K, 200))))
         attn_reps = max(20, min(K, 400))
         timed(lambda i: attn_graph.replay(), 3)
         ms_attn = timed(lambda i: attn_graph.replay(), attn_reps)
+        attn_spread = spread(timed_each(lambda i: attn_graph.replay(), min(attn_reps, 100)), per=cfg.n_layers)
         breakdown = {"tree_attention_x%d" % cfg.n_layers: ms_attn * 1e3 / attn_reps}
-        for name, gr in step_graphs.items():
+        breakdown_spread = {}
+        for name, grs in step_graphs.items():
+            timed(lambda i: grs[i % N_SETS].replay(), 4)
+            breakdown[name] = timed(lambda i: grs[i % N_SETS].replay(), 48) * 1e3 / 48
+            breakdown_spread[name] = spread(timed_each(lambda i: grs[i % N_SETS].replay(), 48))
+        # launch-granularity floor: what a stream of plain device-to-device copies of the same sizes
+        # costs per launch when replayed as a graph (one layer's K/V + Q/O bytes; one expansion call's logits)
+        floor = {}
+        for name, nbytes in (("attention_layer", int(attn_bytes)), ("expand_call", cfg.B * cfg.k * cfg.V * 4)):
+            n_src = int(min(32, max(2, math.ceil(400e6 / nbytes))))  # together larger than L2
+            src = [torch.empty(nbytes, dtype=torch.uint8, device=dev).random_(0, 255) for _ in range(n_src)]
+            dst = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+            with torch.cuda.stream(stream):
+                gr = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(gr, stream=stream):
+                    for t in src:
+                        dst.copy_(t)
             timed(lambda i: gr.replay(), 3)
-            breakdown[name] = timed(lambda i: gr.replay(), 50) * 1e3 / 50
+            us = timed(lambda i: gr.replay(), 20) * 1e3 / (20 * n_src)
+            floor[name] = {"bytes_per_launch": nbytes, "us_per_launch": us, "read_gbs": nbytes / (us * 1e-6) / 1e9,
+                           "note": f"graph of {n_src} cudaMemcpyAsync device-to-device, distinct sources (larger than L2 together), one destination"}
+            del src, dst, gr
 
         # ---- end to end: inputs start in pinned host memory, results end in host memory -------------
         host_in = {
@@ -611,43 +679,87 @@ def run_ours(args):
                 ev_in[j].record(copy_stream)
             for layer in range(cfg.n_layers):
                 q_layers[layer].copy_(host_in["q"][layer], non_blocking=True)
-                for j, (_, r) in enumerate(tree_rows):
-                    k_layers[layer][r:r + cfg.m].copy_(host_in["tree_k"][layer][j], non_blocking=True)
-                    v_layers[layer][r:r + cfg.m].copy_(host_in["tree_v"][layer][j], non_blocking=True)
-            stream.wait_event(ev_in[j])
-            graphs[j].replay()
+                for seq, (_, r) in enumerate(tree_rows):
+                    k_layers[layer][r:r + cfg.m].copy_(host_in["tree_k"][layer][seq], non_blocking=True)
+                    v_layers[layer][r:r + cfg.m].copy_(host_in["tree_v"][layer][seq], non_blocking=True)
+            stream.wait_event(ev_in[j])  # this step's logits are in place (every upload is thereby ordered before
+            graphs[j].replay()           # the closing event, which is recorded on the compute stream)
             ev_free[j].record(stream)
-            host_out["acc_len"].copy_(buf.acc_len, non_blocking=True)
-            host_out["acc_path"].copy_(buf.acc_path, non_blocking=True)
-            host_out["bonus"].copy_(buf.bonus_token, non_blocking=True)
+            host_out["acc_len"].copy_(s["buf"].acc_len, non_blocking=True)
+            host_out["acc_path"].copy_(s["buf"].acc_path, non_blocking=True)
+            host_out["bonus"].copy_(s["buf"].bonus_token, non_blocking=True)
             for layer in range(cfg.n_layers):
                 host_out["o"][layer].copy_(out_layers[layer], non_blocking=True)
 
         e2e_steps = max(5, min(K, 50))
         timed(e2e_step, 3)
         ms_e2e = timed(e2e_step, e2e_steps)
-    assert int(buf.status.item()) == 0, "device status raised during the timed region"
+    assert all(int(bb.status.item()) == 0 for bb in bufs), "device status raised during the timed region"
 
     us_cycle = ms_total * 1e3 / (K * world)
     us_attn = ms_attn * 1e3 / (attn_reps * cfg.n_layers)
-    hbm_peak, _, peak_kind = _peaks()
-    kv_bytes = float(sum(2 * (int(L) + cfg.m) * cfg.Hkv * cfg.d * 2 for L in kv_len_h))
-    qo_bytes = float(2 * cfg.B * cfg.m * cfg.Hq * cfg.d * 2)
-    attn_bytes = kv_bytes + qo_bytes
+    hbm_peak, tensor_peak, peak_kind = _peaks()
     achieved = attn_bytes / (us_attn * 1e-6) / 1e9
     # accepted length of the synthetic workload (tokens per cycle = accepted draft tokens + 1)
     acc = []
     with torch.cuda.stream(stream):
-        for gr in graphs:
+        for gr, z in zip(graphs, sets):
             gr.replay()
             stream.synchronize()
-            acc.append(buf.acc_len.float().mean().item())
+            acc.append(z["buf"].acc_len.float().mean().item())
     tau = float(np.mean(acc)) + 1.0
 
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
+
+    # ---- every floor of the attention call (one layer), and which one binds ---------------------------
+    clk = clocks.summary()
+    sm_hz = 1e6 * float(clk["sm_mhz"] or clk["sm_max_mhz"] or 1965)
+    sms = torch.cuda.get_device_properties(dev).multi_processor_count
+    g_heads = cfg.Hq // cfg.Hkv
+    keys = [int(L) + cfg.m for L in kv_len_h]
+    tiles = [(n + 127) // 128 for n in keys]
+    rows_padded = ((cfg.m * g_heads + 127) // 128) * 128 if cfg.m * g_heads <= 256 else 256 * math.ceil(cfg.m * g_heads / 256)
+    flops_useful = float(sum(4 * cfg.m * cfg.Hq * n * cfg.d for n in keys))
+    flops_issued = float(sum(4 * rows_padded * cfg.Hkv * 128 * t * cfg.d for t in tiles))
+    exps = float(sum(cfg.m * cfg.Hq * n for n in keys))
+    t_hbm = attn_bytes / (hbm_peak * 1e9) * 1e6
+    t_tensor = flops_useful / (tensor_peak * 1e12) * 1e6
+    t_tensor_issued = flops_issued / (tensor_peak * 1e12) * 1e6
+    t_mufu = exps / (16.0 * sms * sm_hz) * 1e6
+    floors = {"hbm": t_hbm, "tensor": t_tensor, "mufu": t_mufu}
+    roofline_all = {
+        "per": "one tree-attention call (one layer)", "measured_us": us_attn,
+        "hbm_us": t_hbm, "tensor_us": t_tensor, "tensor_us_with_padding": t_tensor_issued, "mufu_us": t_mufu,
+        "binding": max(floors, key=floors.get), "frac_of_binding_floor": max(floors.values()) / us_attn,
+        "inputs": {"bytes": attn_bytes, "flops": flops_useful, "flops_issued": flops_issued, "exponentials": exps,
+                   "hbm_gbs": hbm_peak, "bf16_tflops_sustained": tensor_peak,
+                   "mufu": f"16 ex2 per clock per SM x {sms} SMs x {sm_hz / 1e6:.0f} MHz (sampled)"}}
+
+    # ---- the vocabulary steps at this config, against the same HBM peak ----------------------------------
+    us_expand, us_accept = breakdown["expand_x%d" % cfg.D], breakdown["accept"]
+    expand_bytes = float(cfg.B) * cfg.R * cfg.V * 4
+    parents = 0  # nodes (the root included) with a selected child, over the logit sets (mean)
+    for z in sets:
+        sp, si = z["buf"].sel_parent.cpu().numpy(), z["buf"].sel_index.cpu().numpy()
+        parents += sum(len(set(int(q) for q, i in zip(sp[b], si[b]) if i >= 0)) for b in range(cfg.B))
+    parents /= len(sets)
+    if cfg.temperature > 0:
+        accept_bytes_def = float(cfg.B * (cfg.m + 1) + parents) * cfg.V * 4   # every target row + the parents' draft rows
+        accept_bytes_read = float(parents + cfg.B) * 2 * cfg.V * 4           # rows the kernels actually read
+    else:
+        accept_bytes_def = accept_bytes_read = float(cfg.B * (cfg.m + 1)) * cfg.V * 4
+    step_rooflines = {
+        "expand": {"us": us_expand, "calls": cfg.D, "algorithmic_bytes": expand_bytes,
+                   "achieved_gbs": expand_bytes / (us_expand * 1e-6) / 1e9,
+                   "frac_of_measured_hbm": expand_bytes / (us_expand * 1e-6) / 1e9 / hbm_peak},
+        "accept": {"us": us_accept, "temperature": cfg.temperature, "parents_with_selected_children": parents,
+                   "algorithmic_bytes": accept_bytes_def, "bytes_read": accept_bytes_read,
+                   "frac_of_measured_hbm": accept_bytes_def / (us_accept * 1e-6) / 1e9 / hbm_peak,
+                   "frac_of_measured_hbm_on_bytes_read": accept_bytes_read / (us_accept * 1e-6) / 1e9 / hbm_peak},
+    }
 
     line = {
         "metric": METRIC, "value": us_cycle, "unit": "us", "n_gpus": world, "steps": K, "warmup": W,
@@ -659,7 +771,8 @@ def run_ours(args):
                    "l2": f"inputs larger than L2: {cfg.n_layers} distinct KV layers "
                          f"({kv_bytes * cfg.n_layers / 1e6:.0f} MB) and {N_SETS} rotating logit sets",
                    "replicas": world, "synthetic_tau": tau},
-        "clocks": clocks.summary(),
+        "clocks": clk,
+        "per_replay_us": {"cycle": cycle_spread, "attention_layer": attn_spread, **breakdown_spread},
         "e2e": {"value": ms_e2e * 1e3 / (e2e_steps * world), "unit": "us", "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h,
                 "overlap": "a step's logit upload (copy stream, alternate input set) may run under the previous step's cycle"},
@@ -671,14 +784,23 @@ def run_ours(args):
     }
     if world == 1 and not args.no_cpu_baseline:
         total, parts, sample, cores = oracle_cycle_seconds(cfg)
+        total1, parts1, _, _ = oracle_cycle_seconds(cfg, attn_samples=24, threads=1)
         line["cpu_baseline"] = {"value": total * 1e6, "unit": "us", "cores": cores, "kind": "oracle",
-                                "sample": sample, "parts_us": {k: v * 1e6 for k, v in parts.items()}}
+                                "sample": sample, "parts_us": {k: v * 1e6 for k, v in parts.items()},
+                                "single_thread": {"value": total1 * 1e6, "unit": "us", "cores": 1,
+                                                  "parts_us": {k: v * 1e6 for k, v in parts1.items()}}}
     line["roofline"]["traffic"] = NCU_DRAM_BYTES_PER_LAUNCH.get(cfg.name)
-    line["breakdown_us"] = breakdown  # each step replayed alone (warm logits for the small steps)
+    line["breakdown_us"] = breakdown  # each step replayed alone, rotating over the logit sets
+    line["step_rooflines"] = step_rooflines
+    line["roofline_all"] = roofline_all
+    line["launch_floor"] = floor
     if world == 1 and not args.no_extras:
         line["attention_batched"] = batched_attention_extra(e2, dev, stream, hbm_peak)
         line["expand_batched"] = batched_expand_extra(e2, dev, stream, hbm_peak)
+        line["expand_sweep"] = [dict(B=b, **{k_: v for k_, v in batched_expand_extra(e2, dev, stream, hbm_peak, B=b).items()
+                                             if k_ != "workload"}) for b in (1, 8, 32)]
         line["accept_batched"] = batched_accept_extra(e2, dev, stream, hbm_peak)
+        line["accept_batched_b32"] = batched_accept_extra(e2, dev, stream, hbm_peak, B=32)
         line["draft_attention"] = draft_attention_extra(e2, dev, stream, hbm_peak)
         line["lm_head"] = lm_head_extra(e2, dev, stream, hbm_peak)
     print(json.dumps(line))
@@ -694,6 +816,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama3_8b")
     ap.add_argument("--batch", type=int, default=0, help="override the number of sequences")
+    ap.add_argument("--temperature", type=float, default=None, help="override the acceptance temperature")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="skip the batched attention, expansion and acceptance side measurements")
     ap.add_argument("--extras-only", action="store_true", help="run only those side measurements (no bench line)")

@@ -51,7 +51,7 @@ typedef struct CUstream_st* eagle2_stream_t; /* a cudaStream_t */
 #define EAGLE2_STATUS_NOT_CLOSED 2      /* a selected node's parent was not selected */
 #define EAGLE2_STATUS_KV_OVERFLOW 4     /* a sequence's rows exceed the stated cache capacity */
 #define EAGLE2_STATUS_TIMEOUT 8         /* a bounded device-side wait ran out */
-#define EAGLE2_STATUS_BOUNDS 16         /* an index check failed in a checked build */
+/* (bit 16 is not used) */
 #define EAGLE2_STATUS_BAD_TREE 32       /* parent/path arrays are not a valid topological tree */
 
 /* limits */
@@ -78,6 +78,19 @@ size_t eagle2_workspace_bytes(int op, int B, int V, int k, int D, int m, int Hq,
 
 /* Zero a freshly allocated workspace (asynchronous on `stream`). */
 int eagle2_workspace_init(void* ws, size_t ws_bytes, eagle2_stream_t stream);
+
+/*
+ * Bound of the device-side waits (no counterpart in the paper; it belongs to the library's failure
+ * detection).  The tensor-path kernels (tree attention, LM head) and the streaming expansion hand
+ * tiles and candidates between warps through barriers and queues; every such wait gives up after
+ * `cycles` SM clock cycles, the kernel then lets its copies and tensor instructions in flight
+ * finish, frees what it holds, raises EAGLE2_STATUS_TIMEOUT and ends normally, its outputs
+ * undefined.  The default is 2^31 cycles (about a second); cycles <= 0 restores it.  The value is
+ * process-wide, read on the host when a call is made and passed with the launch, so it applies to
+ * calls made after it was set.  A deployment may lower it to learn of a stuck kernel sooner; a
+ * test sets a few cycles to see the give-up path run.  Returns the bound in force before the call.
+ */
+long long eagle2_set_wait_limit(long long cycles);
 
 /*
  * Before step 1 -- the LM head (paper Section 4.1: the draft model's feature of a token goes through
@@ -139,11 +152,14 @@ int eagle2_expand_variant(const float* draft_logits, long long batch_stride, int
  * host loop in which a cudaMalloc is unacceptable because it synchronises the whole device.  The
  * scratch memory is a fixed array of EAGLE2_EXPAND_STATIC_BYTES that is part of the library image:
  * every GPU context that loads the library holds it until the process exits.
- *   - Sizes whose scratch need (what eagle2_workspace_bytes(EAGLE2_OP_EXPAND, ...) reports for the
- *     step) exceeds EAGLE2_EXPAND_STATIC_BYTES are refused with EAGLE2_ERR_STATIC_LIMIT; nothing is
- *     launched.  The call itself never allocates or frees device memory.
+ *   - Sizes whose scratch need (what eagle2_workspace_bytes(EAGLE2_OP_EXPAND, B, V, k, ...) reports:
+ *     the larger of the first step's and the later steps' need, so every step s of one tree gets the
+ *     same answer) exceeds EAGLE2_EXPAND_STATIC_BYTES are refused with EAGLE2_ERR_STATIC_LIMIT;
+ *     nothing is launched.  The call itself never allocates or frees device memory.
  *   - The first call on a device looks up the array's device address (one runtime query, made with
- *     that device current); make that first call outside any stream capture.
+ *     that device current); make that first call outside any stream capture.  The address is kept
+ *     per device ordinal for the life of the process: a process that destroys the device's context
+ *     (cudaDeviceReset) must not call this entry point on that device afterwards.
  *   - All calls on a device share the one array.  Each call clears the few counters that must
  *     start at zero, on `stream`, before its kernel.  Two calls that can run on the GPU at the same
  *     time (different streams, no dependency) would overwrite each other's partial results: order

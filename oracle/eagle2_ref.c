@@ -723,6 +723,19 @@ int eagle2_ref_num_threads(void) {
 #endif
 }
 
+/* Threads the loops over independent sequences / queries may use from now on (timing only: the
+ * arithmetic of every unit is the same whatever the count).  Returns the count in force before. */
+int eagle2_ref_set_threads(int n) {
+#ifdef _OPENMP
+    const int before = omp_get_max_threads();
+    if (n >= 1) omp_set_num_threads(n);
+    return before;
+#else
+    (void)n;
+    return 1;
+#endif
+}
+
 /* ---------- before step 1: the LM head (Section 4.1) --------------------- */
 /*
  * The draft model's feature of each frontier token goes through the LM head of the original LLM

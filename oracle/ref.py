@@ -49,6 +49,11 @@ def num_threads() -> int:
     return int(lib().eagle2_ref_num_threads())
 
 
+def set_threads(n: int) -> int:
+    """Threads for the loops over independent units (timing only); returns the previous count."""
+    return int(lib().eagle2_ref_set_threads(int(n)))
+
+
 def n_nodes(k: int, D: int) -> int:
     return k + (D - 1) * k * k
 

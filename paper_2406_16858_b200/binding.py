@@ -17,12 +17,12 @@ _LIB_PATH = os.path.join(_PKG, "libeagle2.so")
 
 OP_EXPAND, OP_RERANK, OP_TREE_MASK, OP_TREE_ATTENTION, OP_ACCEPT, OP_KV_COMPACT = range(6)
 STATUS_NONFINITE_LOGIT, STATUS_NOT_CLOSED, STATUS_KV_OVERFLOW = 1, 2, 4
-STATUS_TIMEOUT, STATUS_BOUNDS, STATUS_BAD_TREE = 8, 16, 32
+STATUS_TIMEOUT, STATUS_BAD_TREE = 8, 32
 
 EXPORTS = ("eagle2_version", "eagle2_strerror", "eagle2_workspace_bytes", "eagle2_workspace_init",
            "eagle2_expand", "eagle2_rerank", "eagle2_tree_mask", "eagle2_tree_attention",
            "eagle2_accept", "eagle2_kv_compact", "eagle2_expand_static", "eagle2_expand_variant",
-           "eagle2_rerank_skipped", "eagle2_lm_head")
+           "eagle2_rerank_skipped", "eagle2_lm_head", "eagle2_set_wait_limit")
 EXPAND_BY_CONFIDENCE = 1
 
 
@@ -54,6 +54,8 @@ def lib() -> C.CDLL:
         h.eagle2_workspace_bytes.restype = sz
         h.eagle2_workspace_bytes.argtypes = [i32] * 10
         h.eagle2_workspace_init.argtypes = [vp, sz, vp]
+        h.eagle2_set_wait_limit.restype = i64
+        h.eagle2_set_wait_limit.argtypes = [i64]
         h.eagle2_expand.argtypes = [vp, i64, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, sz, vp, vp]
         h.eagle2_expand_static.argtypes = [vp, i64, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp]
         h.eagle2_expand_static.restype = i32
@@ -115,6 +117,12 @@ def _ws(ws):
 def workspace_bytes(op: int, B: int = 1, V: int = 1, k: int = 1, D: int = 1, m: int = 1, Hq: int = 1,
                     Hkv: int = 1, d: int = 128, max_kv_len: int = 0) -> int:
     return int(lib().eagle2_workspace_bytes(op, B, V, k, D, m, Hq, Hkv, d, max_kv_len))
+
+
+def set_wait_limit(cycles: int) -> int:
+    """Bound (SM clock cycles) of the device-side waits of later calls; <= 0 restores the default.
+    Returns the bound that was in force."""
+    return int(lib().eagle2_set_wait_limit(int(cycles)))
 
 
 def workspace_init(ws, stream=None) -> None:

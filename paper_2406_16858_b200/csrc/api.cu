@@ -1,7 +1,15 @@
 // Library-level entry points: version, error strings, workspace sizing and initialisation.
+#include <atomic>
+
 #include "common.cuh"
 
 namespace eagle2 {
+static std::atomic<long long> g_wait_limit{0};  // 0: the built-in default
+long long wait_limit_cycles() {
+    const long long v = g_wait_limit.load(std::memory_order_relaxed);
+    return v > 0 ? v : (1LL << 31);
+}
+
 size_t expand_workspace_bytes(int B, int V, int k);
 size_t accept_workspace_bytes(int B, int V, int k, int D, int m);
 size_t attention_workspace_bytes(int B, int m, int Hq, int Hkv, int d, int max_kv_len);
@@ -38,6 +46,12 @@ extern "C" size_t eagle2_workspace_bytes(int op, int B, int V, int k, int D, int
         default:
             return 0;  // rerank, tree mask and KV compaction work in place
     }
+}
+
+extern "C" long long eagle2_set_wait_limit(long long cycles) {
+    const long long before = eagle2::wait_limit_cycles();
+    eagle2::g_wait_limit.store(cycles > 0 ? cycles : 0, std::memory_order_relaxed);
+    return before;
 }
 
 extern "C" int eagle2_workspace_init(void* ws, size_t ws_bytes, eagle2_stream_t stream) {

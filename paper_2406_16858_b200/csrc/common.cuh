@@ -24,6 +24,31 @@ inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_
 
 inline int launch_result() { return cudaGetLastError() == cudaSuccess ? EAGLE2_OK : EAGLE2_ERR_CUDA; }
 
+// Bound, in clock cycles, that the next launches give their device-side waits (eagle2_set_wait_limit).
+long long wait_limit_cycles();
+
+// Streaming multiprocessors of the current device, queried once per device ordinal and kept for
+// the life of the process.  Launch plans and workspace sizes are both derived from it, so they
+// agree.  Without a usable device (a size query on a machine that has none) the B200's 148.
+inline int sm_count() {
+    constexpr int kMaxDevices = 64, kDefault = 148;
+    static int cached[kMaxDevices] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+        cudaGetLastError();
+        return kDefault;
+    }
+    if (cached[dev] == 0) {
+        int sms = 0;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) {
+            cudaGetLastError();
+            sms = kDefault;
+        }
+        cached[dev] = sms;
+    }
+    return cached[dev];
+}
+
 // Every kernel of the library is launched with programmatic stream serialisation and begins with
 // chain_wait(): it may be scheduled while its predecessor in the stream is still draining, and it
 // touches no global memory before that predecessor (and, by induction, everything before it) has

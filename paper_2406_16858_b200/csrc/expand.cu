@@ -31,7 +31,8 @@ constexpr int kMergeKeysMax = 1024;  // segment winners per row that the merge h
 // up) x (cost of a block).  Never more segments per row than the merge can take, whole tiles per
 // segment.
 static bool expand_plan(long long rows, int V, int k, ExpandPlan* p) {
-    constexpr int kSMs = 148, kBlockFixed = 6;
+    constexpr int kBlockFixed = 6;
+    const long long kSMs = sm_count();
     const int tiles = (V + kTileTokens - 1) / kTileTokens;
     long long g_max = kMergeKeysMax / k;
     if (g_max > tiles) g_max = tiles;
@@ -128,7 +129,6 @@ __device__ __forceinline__ void warp_sort_desc_u64_n(unsigned long long (&v)[N])
 }
 
 constexpr int kQueue = 256;                              // candidate keys in flight to the selector warp
-constexpr long long kExpandWaitCycles = 1LL << 31;       // ~1 s bound of every wait below
 
 // Sorts a bitonic sequence of one key per lane (first rising then falling, or the reverse) into
 // descending order.
@@ -166,7 +166,7 @@ __global__ void __launch_bounds__(STREAM ? kScanThreads + 32 : kScanThreads, 3)
 expand_kernel(const float* __restrict__ draft_logits, long long batch_stride, int V, int k, int D,
               int s, int n_s, int chunks, int tpb, int by_confidence, int32_t* __restrict__ tree_token,
               int32_t* __restrict__ tree_parent, double* __restrict__ tree_value,
-              int32_t* __restrict__ frontier, ExpandWs ws, int32_t* d_status) {
+              int32_t* __restrict__ frontier, ExpandWs ws, long long wait_limit, int32_t* d_status) {
     constexpr int VPT = 4, NE = 16;
     constexpr float kLog2e = 1.4426950408889634f;
     extern __shared__ __align__(16) float s_ring[];  // [kScanWarps][kDepth][512] (vector path)
@@ -250,7 +250,7 @@ expand_kernel(const float* __restrict__ draft_logits, long long batch_stride, in
         if (pos - *reinterpret_cast<volatile int*>(&s_head) >= kQueue) {  // the slot still holds entry pos - kQueue
             const long long w0 = clock64();
             while (pos - *reinterpret_cast<volatile int*>(&s_head) >= kQueue) {
-                if (clock64() - w0 > kExpandWaitCycles) {
+                if (clock64() - w0 > wait_limit) {
                     timed_out = 1;
                     return;
                 }
@@ -424,7 +424,7 @@ expand_kernel(const float* __restrict__ draft_logits, long long batch_stride, in
         const int take = min(tail - head, 32);
         if (take <= 0) {
             if (done == kScanWarps) break;  // every reservation was made before its warp counted itself
-            if (clock64() - w0 > 4 * kExpandWaitCycles) {
+            if (clock64() - w0 > 4 * wait_limit) {
                 timed_out = 1;
                 break;
             }
@@ -436,7 +436,7 @@ expand_kernel(const float* __restrict__ draft_logits, long long batch_stride, in
             volatile unsigned long long* slot = &s_queue[(head + lane) & (kQueue - 1)];
             const long long w1 = clock64();
             while ((key = *slot) == 0ull) {  // reserved, not yet written
-                if (clock64() - w1 > kExpandWaitCycles) {
+                if (clock64() - w1 > wait_limit) {
                     timed_out = 1;
                     break;
                 }
@@ -749,7 +749,7 @@ static int launch_expand_as(const float* draft_logits, long long batch_stride, i
     return launch_chained(expand_kernel<VEC, STREAM>, dim3((unsigned)blocks),
                           dim3(STREAM ? kScanThreads + 32 : kScanThreads), dyn, stream, 1, draft_logits, batch_stride, V,
                           k, D, s, n_s, plan.chunks, plan.tpb, by_confidence, tree_token, tree_parent, tree_value,
-                          frontier, ws, d_status);
+                          frontier, ws, wait_limit_cycles(), d_status);
 }
 
 // Blocks that stream several tiles get the selector warp; one-tile blocks rank within the block.
@@ -857,8 +857,9 @@ extern "C" int eagle2_expand_static(const float* draft_logits, long long batch_s
     ExpandPlan plan;
     if (!expand_plan((long long)B * n_s, V, k, &plan)) return EAGLE2_ERR_SHAPE;
     if ((long long)B * n_s * plan.chunks > 0x7fffffffLL) return EAGLE2_ERR_SHAPE;
-    if (expand_ws_layout(B, n_s, plan.chunks, k, nullptr, nullptr) > (size_t)EAGLE2_EXPAND_STATIC_BYTES)
-        return EAGLE2_ERR_STATIC_LIMIT;
+    // the figure eagle2_workspace_bytes reports (the larger of the first step's and the later steps'
+    // need) decides, so that every step of one tree is accepted or refused alike
+    if (expand_workspace_bytes(B, V, k) > (size_t)EAGLE2_EXPAND_STATIC_BYTES) return EAGLE2_ERR_STATIC_LIMIT;
     void* scratch = nullptr;
     const int rc = expand_scratch_address(&scratch);
     if (rc != EAGLE2_OK) return rc;

@@ -51,11 +51,12 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
 // tmem_cols: the allocation, a power of two that holds the last 32-column read of either accumulator.
 __global__ void __launch_bounds__(kLmThreads, 4)
 lm_head_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant__ CUtensorMap h_map, int rows,
-               int n_pad, int H, int V, int stages, int tmem_cols, float* __restrict__ logits, int32_t* d_status) {
+               int n_pad, int H, int V, int stages, int tmem_cols, long long wait_limit, float* __restrict__ logits,
+               int32_t* d_status) {
     extern __shared__ unsigned char smem_raw[];
     __shared__ LmBarriers bars;
     __shared__ uint32_t s_tmem_base;
-    __shared__ int s_abort;
+    __shared__ WaitCtl s_ctl;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -64,10 +65,12 @@ lm_head_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant_
     const int acc_cols = n_pad < 32 ? 32 : n_pad;
     const int n_tiles = (V + kLmTileV - 1) / kLmTileV;
     const int n_kb = H / kLmTileK;
-    volatile int* abort_flag = &s_abort;
+    volatile WaitCtl* ctl = &s_ctl;
+    long long issued = 0;  // producer lane: weight stages requested so far
 
     if (tid == 0) {
-        s_abort = 0;
+        s_ctl.abort = 0;
+        s_ctl.limit = wait_limit;
         for (int s = 0; s < kLmMaxStages; ++s) {
             mbar_init(smem_u32(&bars.full[s]), 1);
             mbar_init(smem_u32(&bars.empty[s]), 1);
@@ -97,13 +100,12 @@ lm_head_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant_
     if (warp == 0) {
         // ===== producer =============================================================================
         if (lane == 0) {
-            long long issued = 0;
             bool ok = true;
             for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
                 for (int kb = 0; kb < n_kb; ++kb, ++issued) {
                     const int st = (int)(issued % stages);
                     const uint32_t ph = (uint32_t)((issued / stages) & 1);
-                    if (issued >= stages) ok = mbar_wait_spin(smem_u32(&bars.empty[st]), ph ^ 1u, abort_flag);
+                    if (issued >= stages) ok = mbar_wait_spin(smem_u32(&bars.empty[st]), ph ^ 1u, ctl);
                     if (!ok) break;
                     const uint32_t dst = smem_base + (uint32_t)st * stage_bytes;
                     const uint32_t bar = smem_u32(&bars.full[st]);
@@ -112,21 +114,13 @@ lm_head_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant_
                     tma_load_2d(dst + kLmWBytes, &h_map, kb * kLmTileK, 0, bar);
                 }
             }
-            if (!ok) {
-                // every copy issued for the newest use of each stage must land before the block leaves
-                for (long long j = issued > stages ? issued - stages : 0; j < issued; ++j) {
-                    const long long t0 = clock64();
-                    while (!mbar_try_wait(smem_u32(&bars.full[j % stages]), (uint32_t)((j / stages) & 1)) &&
-                           clock64() - t0 < kWaitCycles) {}
-                }
-            }
         }
     } else if (warp == 1) {
         // ===== MMA issuer (the warp walks the loop, lane 0 waits and issues) =========================
         const uint32_t idesc = instr_desc(n_pad, false, kLmTileV);
         auto wait_all = [&](uint32_t bar, uint32_t parity) {
             int r = 1;
-            if (lane == 0) r = mbar_wait_spin(bar, parity, abort_flag) ? 1 : 0;
+            if (lane == 0) r = mbar_wait_spin(bar, parity, ctl) ? 1 : 0;
             r = __shfl_sync(0xffffffffu, r, 0);
             return r != 0;
         };
@@ -166,7 +160,7 @@ lm_head_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant_
         for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++i) {
             const int acc = i & 1;
             int r = 1;
-            if (lane == 0) r = mbar_wait(smem_u32(&bars.acc_full[acc]), (uint32_t)((i >> 1) & 1), abort_flag) ? 1 : 0;
+            if (lane == 0) r = mbar_wait(smem_u32(&bars.acc_full[acc]), (uint32_t)((i >> 1) & 1), ctl) ? 1 : 0;
             ok = __shfl_sync(0xffffffffu, r, 0) != 0;
             if (!ok) break;
             tc_fence_after();
@@ -193,20 +187,25 @@ lm_head_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant_
     __syncthreads();
     if (warp == 1) {
         tc_fence_after();
-        if (s_abort) {
+        if (s_ctl.abort) {
             // instructions issued before the wait ran out may still be reading shared memory and
             // writing tensor memory: let them retire (bounded) before either is given back
             if (lane == 0) {
                 tc_commit(smem_u32(&bars.drain));
-                const long long t0 = clock64();
-                while (!mbar_try_wait(smem_u32(&bars.drain), 0) && clock64() - t0 < kWaitCycles) {}
+                mbar_drain(smem_u32(&bars.drain), 0);
             }
             __syncwarp();
             tc_fence_after();
         }
         tmem_dealloc(tmem, (uint32_t)tmem_cols);
     }
-    if (tid == 0 && s_abort) raise_status(d_status, EAGLE2_STATUS_TIMEOUT);
+    if (warp == 0 && lane == 0 && s_ctl.abort) {
+        // whoever gave up, and whenever: every copy requested for the newest use of each stage
+        // must have landed before the block's shared memory is given back
+        for (long long j = issued > stages ? issued - stages : 0; j < issued; ++j)
+            mbar_drain(smem_u32(&bars.full[j % stages]), (uint32_t)((j / stages) & 1));
+    }
+    if (tid == 0 && s_ctl.abort) raise_status(d_status, EAGLE2_STATUS_TIMEOUT);
 }
 
 static bool make_matrix_map(CUtensorMap* map, const void* base, long long n_rows, int H, int box_rows) {
@@ -266,7 +265,7 @@ static int lm_head_rows(const void* hidden, const void* weight, int rows, int H,
     const int n_tiles = (V + kLmTileV - 1) / kLmTileV;
     const int grid = n_tiles < resident * sms ? n_tiles : resident * sms;
     return launch_chained(lm_head_kernel, dim3(grid), dim3(kLmThreads), dyn, reinterpret_cast<cudaStream_t>(stream), 1,
-                          w_map, h_map, rows, n_pad, H, V, stages, tmem_cols, logits, d_status);
+                          w_map, h_map, rows, n_pad, H, V, stages, tmem_cols, wait_limit_cycles(), logits, d_status);
 }
 
 extern "C" int eagle2_lm_head(const void* hidden, const void* weight, int rows, int H, int V, float* logits,

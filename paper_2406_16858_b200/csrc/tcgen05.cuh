@@ -12,7 +12,8 @@
 
 namespace eagle2 {
 
-constexpr long long kWaitCycles = 1LL << 31;  // ~1 s bound of a barrier wait
+constexpr long long kWaitCycles = 1LL << 31;  // ~1 s: default bound of a barrier wait, and the fixed bound
+                                              // of the drains that follow a wait that ran out
 constexpr uint32_t kSuspendNs = 400;          // a waiting thread sleeps in hardware at most this long per try
 
 using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -70,31 +71,47 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-// The same bounded wait, polling without ever sleeping: for the single lanes whose reaction time
-// is on the critical path (MMA issue, producer).
-__device__ __forceinline__ bool mbar_wait_spin(uint32_t bar, uint32_t parity, volatile int* abort) {
+// What the waits of one block share: the flag a role raises when its wait ran out (every other
+// role then gives up at its next unsatisfied wait) and the bound itself, in clock cycles, which the
+// host passes with the launch (eagle2_set_wait_limit; kWaitCycles unless changed).
+struct WaitCtl {
+    int abort;
+    int pad_;
+    long long limit;
+};
+// Bounded wait, polling without ever sleeping: for the single lanes whose reaction time is on the
+// critical path (MMA issue, producer).
+__device__ __forceinline__ bool mbar_wait_spin(uint32_t bar, uint32_t parity, volatile WaitCtl* ctl) {
     if (mbar_test_wait(bar, parity)) return true;
-    const long long t0 = clock64();
+    const long long t0 = clock64(), limit = ctl->limit;
+    const int check = limit < 65536 ? 0 : 1023;  // short bounds are looked at on every poll
     for (int spin = 1;; ++spin) {
         if (mbar_test_wait(bar, parity)) return true;
-        if ((spin & 1023) == 0 && (*abort || clock64() - t0 > kWaitCycles)) {
-            *abort = 1;
+        if ((spin & check) == 0 && (ctl->abort || clock64() - t0 > limit)) {
+            ctl->abort = 1;
             return false;
         }
     }
 }
 // Bounded wait for the phase of the given parity.  Returns false when the bound ran out or another
-// role of the block has already given up (*abort != 0).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort) {
+// role of the block has already given up (ctl->abort != 0).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile WaitCtl* ctl) {
     if (mbar_try_wait(bar, parity)) return true;
-    const long long t0 = clock64();
+    const long long t0 = clock64(), limit = ctl->limit;
+    const int check = limit < 65536 ? 0 : 15;
     for (int spin = 1;; ++spin) {
         if (mbar_try_wait(bar, parity)) return true;
-        if ((spin & 15) == 0 && (*abort || clock64() - t0 > kWaitCycles)) {
-            *abort = 1;
+        if ((spin & check) == 0 && (ctl->abort || clock64() - t0 > limit)) {
+            ctl->abort = 1;
             return false;
         }
     }
+}
+// After a wait ran out: waits (fixed ~1 s bound, whatever the launch's limit) for a phase that
+// copies or tensor instructions already in flight will complete.
+__device__ __forceinline__ void mbar_drain(uint32_t bar, uint32_t parity) {
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity) && clock64() - t0 < kWaitCycles) {}
 }
 __device__ __forceinline__ void fence_proxy_async() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");

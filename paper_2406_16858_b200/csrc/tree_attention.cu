@@ -58,23 +58,27 @@ struct AttnPlan {
     int fused_merge;  // 1 (ordered launches with several splits): the last block of a (sequence, KV head, row
                       // block) to finish combines the splits' partials itself, while other blocks still run
     size_t smem;
+    long long wait_limit;  // bound of every device-side wait of the launch, in clock cycles
 };
 
 static void attention_plan(int B, int m, int Hq, int Hkv, int d, int max_kv_len, AttnPlan* p) {
     p->g = Hq / Hkv;
     p->M = m * p->g;
-    p->n_rb = (p->M + 2 * kRowsPerTile - 1) / (2 * kRowsPerTile);
+    // A block holds at most 256 packed rows, i.e. at most 256/g whole tokens (g need not divide 256).
+    const int per_tok_max = (2 * kRowsPerTile) / p->g;
+    p->n_rb = (m + per_tok_max - 1) / per_tok_max;
     p->per_tok = (m + p->n_rb - 1) / p->n_rb;
-    p->per = p->per_tok * p->g;  // never above 256: n_rb >= m*g/256
+    p->per = p->per_tok * p->g;  // <= per_tok_max * g <= 256
     p->mt = p->per > kRowsPerTile ? 2 : 1;
     p->q_tma = (kRowsPerTile % p->g) == 0;
     const long long items = (long long)B * Hkv * p->n_rb;
+    const int sms = sm_count(), tpcs = sms / 2;  // a pair needs both SMs of a TPC
     // Pairs pay off while the launch is short of blocks and every sequence is cut into several
     // splits (they halve the query and partial traffic); a launch that fills the device without
     // splitting is better served by independent blocks.
-    p->pair = (p->mt == 2 && p->q_tma && d == 128 && items * 2 <= 74) ? 1 : 0;
+    p->pair = (p->mt == 2 && p->q_tma && d == 128 && items * 2 <= tpcs) ? 1 : 0;
     const int tiles = (max_kv_len + m + kTK - 1) / kTK;
-    long long s = (p->pair ? 74 : 148) / (items > 0 ? items : 1);
+    long long s = (p->pair ? tpcs : sms) / (items > 0 ? items : 1);
     if (s < 1) s = 1;
     if (s > tiles) s = tiles;
     int per_split = (int)((tiles + s - 1) / s);
@@ -90,6 +94,7 @@ static void attention_plan(int B, int m, int Hq, int Hkv, int d, int max_kv_len,
     int stages = (int)((220 * 1024 - p->mt * unit) / (2 * unit));
     p->stages = stages > 4 ? 4 : (stages < 2 ? 2 : stages);
     p->smem = (p->mt + 2 * (size_t)p->stages) * unit + 1024;
+    p->wait_limit = wait_limit_cycles();
     p->setup_first = B == 1;  // ragged batches leave many splits without tiles: those leave at once
     if (p->pair) {  // per block: one 128-row query tile, half-size K and V stages
         p->stages = 4;
@@ -238,6 +243,7 @@ struct AttnBarriers {
     // pair mode, used in the pair's first block: the other block's query tile / K half / V half
     // has landed (and its V tail is cleared)
     unsigned long long q_peer, k_peer[4], v_peer[4];
+    unsigned long long drain;  // after a wait ran out: the tensor instructions issued so far have retired
 };
 
 // Visibility of the 128 keys of a tile that reaches past the committed cache, as four 32-bit words:
@@ -373,7 +379,7 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
     extern __shared__ unsigned char smem_raw[];
     __shared__ AttnBarriers bars;
     __shared__ uint32_t s_tmem_base;
-    __shared__ int s_abort;
+    __shared__ WaitCtl s_ctl;
 
     const int g = plan.g, M = plan.M, S = plan.splits, NST = plan.stages;
     const uint32_t rank = PAIR ? cluster_ctarank() : 0u;  // 0: the block that issues the pair's MMAs
@@ -387,7 +393,8 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
     // ---- set-up: barriers, tensor memory (reads nothing an earlier kernel could have written) ----
     auto set_up = [&]() {
         if (tid == 0) {
-            s_abort = 0;
+            s_ctl.abort = 0;
+            s_ctl.limit = plan.wait_limit;
             mbar_init(smem_u32(&bars.q_full), plan.q_tma ? 1 : kSoftmaxThreads);
             for (int s = 0; s < 4; ++s) {
                 mbar_init(smem_u32(&bars.k_full[s]), 1);
@@ -405,6 +412,7 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
                 mbar_init(smem_u32(&bars.v_peer[s]), 1);
             }
             for (int s = 0; s < 4; ++s) mbar_init(smem_u32(&bars.o_done[s >> 1][s & 1]), 1);
+            mbar_init(smem_u32(&bars.drain), 1);
             fence_barrier_init();
         }
         if (warp == kMmaWarp) {
@@ -478,14 +486,14 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
         set_up();
     }
     const uint32_t tmem = s_tmem_base;
-    volatile int* abort_flag = &s_abort;
+    volatile WaitCtl* abort_flag = &s_ctl;
+    int k_issued = 0, v_issued = 0;  // TMA lane: K and V tiles requested so far
     const int n_items = nt * MT;  // item i = (tile i / MT, row tile i % MT), score slot i % 2
 
     if (active) {
     if (warp == kTmaWarp) {
         // ===== TMA producer =======================================================================
         if (lane == 0) {
-            int issued = 0;
             bool ok = true;
             if (plan.q_tma) {
                 mbar_expect_tx(smem_u32(&bars.q_full), MT * kTile);
@@ -508,11 +516,9 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
                 for (int h = 0; h < HALVES; ++h)  // a pair block takes its 64 of the tile's 128 keys
                     tma_load_3d(sK + st * kKTile + h * kKPanel, &k_map, h * 64, hk, row + (int)rank * (kTK / 2),
                                 smem_u32(&bars.k_full[st]));
+                k_issued = j + 1;
                 if (j >= NST) ok = mbar_wait(smem_u32(&bars.v_empty[st]), ph ^ 1u, abort_flag);
-                if (!ok) {  // K of this tile is in flight, V is not
-                    mbar_wait(smem_u32(&bars.k_full[st]), ph, abort_flag);
-                    break;
-                }
+                if (!ok) break;
                 mbar_expect_tx(smem_u32(&bars.v_full[st]), kVTile);
                 if (PAIR) {  // all keys, this block's 64 of the 128 columns
                     tma_load_3d(sV + st * kVTile, &v_map, (int)rank * 64, hk, row, smem_u32(&bars.v_full[st]));
@@ -521,22 +527,7 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
                     for (int h = 0; h < HALVES; ++h)
                         tma_load_3d(sV + st * kTile + h * kPanel, &v_map, h * 64, hk, row, smem_u32(&bars.v_full[st]));
                 }
-                issued = j + 1;
-            }
-            if (*abort_flag) {
-                if (plan.q_tma) {
-                    const long long t0 = clock64();
-                    while (!mbar_try_wait(smem_u32(&bars.q_full), 0) && clock64() - t0 < kWaitCycles) {}
-                }
-                // drain: every copy issued for the newest tile of each stage must have landed before
-                // the block may leave (bounded by the clock only, the flag is already up)
-                for (int j = max(0, issued - NST); j < issued; ++j) {
-                    const int st = j % NST;
-                    const uint32_t ph = (uint32_t)((j / NST) & 1);
-                    const long long t0 = clock64();
-                    while (!mbar_try_wait(smem_u32(&bars.k_full[st]), ph) && clock64() - t0 < kWaitCycles) {}
-                    while (!mbar_try_wait(smem_u32(&bars.v_full[st]), ph) && clock64() - t0 < kWaitCycles) {}
-                }
+                v_issued = j + 1;
             }
         }
     } else if (warp == kMmaWarp) {
@@ -918,15 +909,44 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
     }
 
     // ---- teardown ----------------------------------------------------------------------------------
+    // A block whose wait ran out tells its pair block (every thread that sees the flag on its way
+    // here repeats the store; whoever raised it comes by after raising it), so that both take the
+    // same path below.
+    if (PAIR && s_ctl.abort) {
+        uint32_t remote;
+        asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(smem_u32(&s_ctl.abort)), "r"(rank ^ 1u));
+        asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(remote), "r"(1u) : "memory");
+    }
     tc_fence_before();
     if (PAIR) cluster_sync_all();  // tensor memory is released by both blocks together
     else __syncthreads();
     tc_fence_after();
+    if (s_ctl.abort) {
+        // Whoever gave up, and whenever: the tensor instructions issued so far may still read shared
+        // memory and write tensor memory, and copies may still be on their way into the rings.  Both
+        // must have finished before either memory is given back (fixed bound, about a second).
+        if (warp == kMmaWarp && lane == 0 && rank == 0) {
+            if (PAIR) tc_commit2(smem_u32(&bars.drain));
+            else tc_commit(smem_u32(&bars.drain));
+            mbar_drain(smem_u32(&bars.drain), 0);
+        }
+        if (warp == kTmaWarp && lane == 0) {
+            if (plan.q_tma) mbar_drain(smem_u32(&bars.q_full), 0);
+            for (int j = max(0, k_issued - NST); j < k_issued; ++j)
+                mbar_drain(smem_u32(&bars.k_full[j % NST]), (uint32_t)((j / NST) & 1));
+            for (int j = max(0, v_issued - NST); j < v_issued; ++j)
+                mbar_drain(smem_u32(&bars.v_full[j % NST]), (uint32_t)((j / NST) & 1));
+        }
+        tc_fence_before();
+        if (PAIR) cluster_sync_all();
+        else __syncthreads();
+        tc_fence_after();
+    }
     if (warp == kMmaWarp) {
         if (PAIR) tmem_dealloc2(tmem, kTmemCols);
         else tmem_dealloc(tmem, kTmemCols);
     }
-    if (tid == 0 && s_abort) raise_status(d_status, EAGLE2_STATUS_TIMEOUT);
+    if (tid == 0 && s_ctl.abort) raise_status(d_status, EAGLE2_STATUS_TIMEOUT);
     if (PAIR) cluster_sync_all();  // neither block leaves while the other may still signal it
 }
 
@@ -1032,7 +1052,7 @@ static int launch_attention(const CUtensorMap& k_map, const CUtensorMap& v_map, 
     if (plan.splits > 1 && !plan.fused_merge) {
         const long long warps = (long long)B * Hkv * plan.M;
         long long mblocks = (warps + 7) / 8;
-        if (mblocks > 8 * 148) mblocks = 8 * 148;
+        if (mblocks > 8LL * sm_count()) mblocks = 8LL * sm_count();
         if (launch_chained(tree_attention_merge_kernel<DH>, dim3((unsigned)mblocks), dim3(256), 0, st, 1, kv_off, kv_len, B, m,
                            Hq, Hkv, cache_rows, max_kv_len, plan, ws, static_cast<__nv_bfloat16*>(out), lse) != EAGLE2_OK)
             return EAGLE2_ERR_CUDA;
@@ -1061,6 +1081,7 @@ extern "C" int eagle2_tree_attention(const void* q, const void* k_cache, const v
     if (B == 0) return EAGLE2_OK;
     AttnPlan plan;
     attention_plan(B, m, Hq, Hkv, d, max_kv_len, &plan);
+    if (plan.per > plan.mt * kRowsPerTile || plan.per_tok * plan.n_rb < m) return EAGLE2_ERR_SHAPE;  // (cannot happen)
     AttnWs w = {nullptr, nullptr, nullptr, nullptr};
     if (plan.splits > 1 || plan.ordered) {
         if (!ws || !aligned(ws, kWsAlign)) return EAGLE2_ERR_WORKSPACE;

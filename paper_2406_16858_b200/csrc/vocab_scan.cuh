@@ -135,7 +135,7 @@ __device__ __forceinline__ unsigned long long warp_sort_desc_u64(unsigned long l
 // Choose elements per chunk (as float4 per thread: 1, 2 or 4) so that a launch fills the GPU when
 // it can and no row is cut into more pieces than the merge step can hold.
 inline int scan_pick_vpt(long long rows, int V) {
-    const long long want_blocks = 2 * 148;
+    const long long want_blocks = 2LL * sm_count();
     for (int vpt = 4; vpt >= 2; vpt >>= 1) {
         const long long chunks = (V + kScanThreads * 4 * vpt - 1) / (kScanThreads * 4 * vpt);
         if (rows * chunks >= want_blocks) return vpt;

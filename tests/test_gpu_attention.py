@@ -80,6 +80,26 @@ def test_shapes_tails_and_gqa(m, Hq, Hkv, d, lens):
 
 
 @pytest.mark.parametrize("m,Hq,Hkv,d,lens", [
+    # query heads per KV head that do not divide 256: a row block holds whole tokens only, so the
+    # blocks are sized from 256 // g tokens (g = 7: 36 tokens = 252 rows; g = 6: 42 tokens = 252 rows)
+    (73, 7, 1, 128, [900]),           # three row blocks, several splits (one sequence, one KV head)
+    (73, 7, 1, 128, [40] * 40),       # the same rows written directly: one split per sequence
+    (128, 6, 1, 128, [1500]),         # four row blocks of 32 tokens
+    (128, 6, 1, 64, [77] * 30),
+    (109, 7, 1, 64, [300, 5]),
+    (85, 6, 2, 128, [2000, 130]),
+])
+def test_row_blocks_when_the_group_size_does_not_divide_256(m, Hq, Hkv, d, lens):
+    q, kc, vc, off, kl, bits = _inputs(17, len(lens), m, Hq, Hkv, d, lens)
+    rng = np.random.default_rng(m)
+    n = 500
+    samples = np.stack([rng.integers(0, len(lens), n), rng.integers(0, Hq, n),
+                        rng.integers(0, m, n)], axis=1).astype(np.int32)
+    samples[:Hq] = [(0, h, m - 1) for h in range(Hq)]  # the last token's rows: the tail of the last row block
+    _compare(q, kc, vc, off, kl, bits, 1.0 / np.sqrt(d), samples=samples)
+
+
+@pytest.mark.parametrize("m,Hq,Hkv,d,lens", [
     # many (sequence, KV head) pairs leave one split per sequence: several tiles per block, so the
     # K/V ring and the score slots are reused; ragged lengths leave some blocks a single tile
     (60, 16, 16, 128, [700, 100, 1500, 40, 2100, 300, 900, 5]),      # one 128-row tile per block
@@ -251,7 +271,71 @@ def test_full_size_one_layer_sampled(name):
                                     1.0 / np.sqrt(cfg.d), samples=samples)
     got = out.float().cpu().numpy().astype(np.float64)
     for t, (b, h, i) in enumerate(samples):
-        assert np.abs(got[b, i, h] - want[t]).max() <= TOL
+        err = np.abs(got[b, i, h] - want[t]).max()
+        assert err <= TOL
+        # Design budget.  With thousands of N(0,1) keys the outputs have rms ~0.02-0.03: the bar above
+        # alone could not see a wrong tree mask here (removing every ancestor moves these outputs by
+        # ~3e-3).  Probabilities rounded to bf16 (2^-9 relative, random sign) and one bf16 rounding of
+        # the row give ~3e-3 * |o| ~ 1e-4; 1e-3 leaves a margin of ten and is a third of a mask's worth.
+        assert err <= 1e-3
     # property that holds at any size: rows are finite and bounded by the largest |v|
     assert torch.isfinite(out.float()).all()
     assert out.float().abs().max() <= tv.float().abs().max()
+
+
+@pytest.mark.parametrize("mode,B,Hq,Hkv,lens", [
+    ("block pairs, several splits", 1, 32, 8, [4096]),
+    ("block pairs, two row blocks", 1, 64, 8, [8192]),
+    ("one row tile per block", 1, 32, 32, [1024]),
+    ("two row tiles per block", 8, 32, 8, [2000] * 8),
+    ("ordered launch, splits merged in the kernel", 24, 32, 8,
+     [9000, 300, 4500, 20, 70, 5200, 1300, 0, 4037, 4036, 8100, 64, 2500, 1, 700, 3100, 128, 4097, 0, 950, 6000,
+      33, 2047, 410]),
+])
+def test_full_size_tree_keys_dominate(mode, B, Hq, Hkv, lens):
+    """Full-size launches of every mode in which the tree tokens' keys and all queries share one
+    direction (a score offset of sqrt(d) = 11.3 for every tree key), so that the tree keys a row may
+    see carry most of its softmax weight: an ancestor mask applied wrongly (a bit dropped, a sibling
+    let in, a row's word shifted) then moves the output by O(1), far above the bar.  The tree is a
+    random forest; the oracle computes sampled rows one by one."""
+    m, d = 60, 128
+    rng = np.random.default_rng(len(mode))
+    kv_len = np.array(lens, np.int32)
+    kv_off = gen.kv_offsets(kv_len, m)
+    rows = int(kv_off[-1] + kv_len[-1] + m)
+    g = torch.Generator(device=DEV).manual_seed(77)
+    w = torch.randn(d, generator=g, device=DEV)
+    w = w / w.norm() * float(np.sqrt(d))
+    tq = (torch.randn((B, m, Hq, d), generator=g, device=DEV) + w).to(torch.bfloat16)
+    tk = torch.randn((rows, Hkv, d), generator=g, device=DEV)
+    for b in range(B):
+        lo = int(kv_off[b] + kv_len[b])
+        tk[lo:lo + m] += w  # tree keys: q.k / sqrt(d) gains |w|^2 / sqrt(d) = sqrt(d)
+    tk = tk.to(torch.bfloat16)
+    tv = torch.randn((rows, Hkv, d), generator=g, device=DEV).to(torch.bfloat16)
+    bits = _random_forest_mask(rng, B, m, kv_len)
+    out = torch.zeros_like(tq)
+    st = new_status()
+    max_len = int(kv_len.max())
+    ws = make_ws(e2.workspace_bytes(e2.OP_TREE_ATTENTION, B=B, m=m, Hq=Hq, Hkv=Hkv, d=d, max_kv_len=max_len))
+    e2.tree_attention(tq, tk, tv, rows, dev(kv_off), dev(kv_len), dev(bits), B, m, Hq, Hkv, d, max_len,
+                      1.0 / np.sqrt(d), out, None, ws, st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    n = 160
+    samples = np.stack([rng.integers(0, B, n), rng.integers(0, Hq, n), rng.integers(0, m, n)], axis=1).astype(np.int32)
+    samples[:8, 2] = m - 1  # deep rows: the most ancestors
+    samples[8:16, 0] = int(np.argmax(kv_len))
+    hq, hk, hv = (host(t.view(torch.int16), np.uint16) for t in (tq, tk, tv))
+    _, want, _ = ref.tree_attention(hq, hk, hv, kv_off, kv_len, bits, 1.0 / np.sqrt(d), samples=samples)
+    # the same rows with every ancestor hidden (each row sees itself and the cache): how far a wrong mask moves them
+    self_only = np.zeros_like(bits)
+    for i in range(m):
+        self_only[:, i, i // 64] = np.uint64(1) << np.uint64(i % 64)
+    _, blind, _ = ref.tree_attention(hq, hk, hv, kv_off, kv_len, self_only, 1.0 / np.sqrt(d), samples=samples)
+    has_anc = np.array([bin(int(bits[b, i, 0])).count("1") > 1 for b, _, i in samples])
+    assert np.median(np.abs(want - blind).max(axis=1)[has_anc]) > 0.3  # the case does what it is for
+    got = out.float().cpu().numpy().astype(np.float64)
+    for t, (b, h, i) in enumerate(samples):
+        # outputs reach |o| ~ 3 here, where bf16 steps are 2^-6: the bar scales with rows above 1
+        assert np.abs(got[b, i, h] - want[t]).max() <= TOL * max(1.0, np.abs(want[t]).max())

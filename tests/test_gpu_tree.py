@@ -17,12 +17,17 @@ from harness import DEV, GpuSelection, GpuTree, dev, host
 pytestmark = pytest.mark.gpu
 
 
+# Exemptions are counted over the whole module and held to a ceiling by the module's last test: a
+# predicate that exempted everything would otherwise turn every check below into a no-op.
+COUNTS = {"trees": 0, "exempt": 0}
+
+
 def _frontier_gap(values_of_new, k):
     v = np.sort(values_of_new)[::-1]
     return np.inf if len(v) <= k else v[k - 1] - v[k]
 
 
-def _check_tree(cfg, draft, gpu: GpuTree, want: ref.Tree, by_confidence=False):
+def _check_tree(cfg, draft, gpu: GpuTree, want: ref.Tree, by_confidence=False, ties_by_design=False):
     B, k, D = cfg.B, cfg.k, cfg.D
     tok, par, val, fr = host(gpu.token), host(gpu.parent), host(gpu.value), host(gpu.frontier)
     assert int(gpu.status.item()) == want.status
@@ -38,7 +43,9 @@ def _check_tree(cfg, draft, gpu: GpuTree, want: ref.Tree, by_confidence=False):
                 score = score - want.value[b, want.parent[b, base:base + n_new]]
             if _frontier_gap(score, k) < 1e-6:
                 exempt = True
+        COUNTS["trees"] += not ties_by_design
         if exempt:
+            COUNTS["exempt"] += not ties_by_design
             continue
         assert (tok[b] == want.token[b]).all()
         assert (par[b] == want.parent[b]).all()
@@ -134,7 +141,8 @@ def test_many_tiles_per_block_and_ordered_rows(kind, V):
     assert (host(gpu.parent) == want.parent).all()
     assert np.abs(host(gpu.value) - want.value).max() < 3e-6
     cfg = get_config("tiny", B=B, V=V, k=k, D=D)
-    _check_tree(cfg, draft, gpu, want)
+    # (rows made of a handful of levels tie by construction: their exemptions are not counted)
+    _check_tree(cfg, draft, gpu, want, ties_by_design=(kind == "plateaus"))
 
 
 @pytest.mark.parametrize("V,k,D,B", [(40000, 32, 2, 8),    # widest frontier: 256 rows, all 32 lanes of the selector in use
@@ -239,3 +247,9 @@ def test_rerank_arbitrary_values_and_bad_parents():
     got = GpuSelection(dev(token), dev(parent), dev(value), B, k, D, m)
     assert want.status & ref.ST_BAD_TREE and int(got.status.item()) & e2.STATUS_BAD_TREE
     assert (host(got.index) == want.index).all() and (host(got.parent) == want.parent).all()
+
+
+def test_zz_exempt_trees_stay_rare():
+    """Runs after the tests above (file order).  On the seeded inputs of this module the oracle
+    exempts no tree at all; the ceiling allows for one."""
+    assert COUNTS["exempt"] <= 1 + COUNTS["trees"] // 200, COUNTS

@@ -49,6 +49,39 @@ def test_static_scratch_expansion_matches_workspace_expansion(name, B):
         assert np.abs(got - want).max() <= 1e-5 * max(1.0, np.abs(want).max())
 
 
+def test_static_scratch_expansion_takes_no_device_memory():
+    """What the entry point is for: its calls leave the device's free memory exactly as they found
+    it.  After a first tree (whose first call looks the built-in buffer up), the free bytes the
+    driver reports and the bytes torch's allocator holds are read before and after two more trees
+    whose output arrays already exist; neither may move."""
+    cfg = get_config("vicuna7b").with_(B=2)
+    B, V, k, D = cfg.B, cfg.V, cfg.k, cfg.D
+    draft = dev(gen.draft_rows(cfg, 9))
+    N, R = cfg.N, cfg.R
+    token = torch.full((B, N), -1, dtype=torch.int32, device=DEV)
+    parent = torch.full((B, N), -2, dtype=torch.int32, device=DEV)
+    value = torch.full((B, N), float("-inf"), dtype=torch.float64, device=DEV)
+    frontier = torch.zeros((B, k), dtype=torch.int32, device=DEV)
+    status = new_status()
+
+    def one_tree():
+        for s in range(D):
+            lo = 0 if s == 0 else 1 + (s - 1) * k
+            e2.expand_static(draft.data_ptr() + lo * V * 4, R * V, B, V, k, D, s, token, parent, value, frontier,
+                             status)
+        torch.cuda.synchronize()
+
+    one_tree()
+    free_before, _ = torch.cuda.mem_get_info()
+    held_before = torch.cuda.memory_reserved()
+    one_tree()
+    one_tree()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before
+    assert torch.cuda.memory_reserved() == held_before
+    assert int(status.item()) == 0
+
+
 def test_sizes_beyond_the_built_in_buffer_are_refused():
     cfg = get_config("llama3_8b")
     B = 2048  # 2048 sequences x 10 rows x (10 keys + statistics) exceed the 1 MiB buffer
