@@ -35,7 +35,8 @@ constexpr int kMaxTilesPerSplit = 16; // a block never streams more than 2048 ke
 constexpr int kMaxTilesPerSplitOrdered = 32;  // ... 4096 when the launch runs its longest blocks first
 constexpr int kTmemCols = 512;
 constexpr int kSlots = 2;             // score slots in tensor memory
-constexpr int kAttnThreads = 320;     // 8 softmax warps, the TMA warp, the MMA warp
+constexpr int kSoftmaxThreads = 512;  // 16 softmax warps: four per SM sub-partition
+constexpr int kAttnThreads = kSoftmaxThreads + 64;  // ... the TMA warp, the MMA warp
 
 struct AttnPlan {
     int g, M;
@@ -243,6 +244,7 @@ struct AttnBarriers {
     // pair mode, used in the pair's first block: the other block's query tile / K half / V half
     // has landed (and its V tail is cleared)
     unsigned long long q_peer, k_peer[4], v_peer[4];
+    unsigned long long v_landed, v_clean;  // the block's last V tile has landed / its rows past the sequence's last key are cleared
     unsigned long long drain;  // after a wait ran out: the tensor instructions issued so far have retired
 };
 
@@ -363,11 +365,7 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
     constexpr int HALVES = DH / 64;                    // 64-column (128-byte) panels per operand tile
     constexpr uint32_t kPanel = kTK * 128;             // bytes of one panel: 128 rows x 128 bytes
     constexpr uint32_t kTile = HALVES * kPanel;
-    // Two row tiles: a warp group (4 warps, thread = row) per tile.  One row tile: both warp groups
-    // serve it, each thread taking half of the columns of its row (SPLIT).
-    constexpr bool SPLIT = MT == 1;
-    constexpr int kSoftmaxThreads = 256;
-    constexpr int kTmaWarp = 8, kMmaWarp = 9;
+    constexpr int kTmaWarp = kSoftmaxThreads / 32, kMmaWarp = kTmaWarp + 1;
     constexpr uint32_t kIdescQK = instr_desc(kTK, false, PAIR ? 256 : 128);
     constexpr uint32_t kIdescPV = instr_desc(DH, true, PAIR ? 256 : 128);
     constexpr uint32_t kOCol = kSlots * kTK;           // first accumulator column of O
@@ -404,7 +402,7 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
             }
             for (int s = 0; s < kSlots; ++s) {
                 mbar_init(smem_u32(&bars.s_full[s]), 1);
-                mbar_init(smem_u32(&bars.p_full[s]), PAIR ? 16 : (SPLIT ? 8 : 4));  // one arrival per softmax warp
+                mbar_init(smem_u32(&bars.p_full[s]), (PAIR ? 2 : 1) * (kSoftmaxThreads / 32));  // one arrival per softmax warp
             }
             mbar_init(smem_u32(&bars.q_peer), 1);
             for (int s = 0; s < 4; ++s) {
@@ -413,6 +411,8 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
             }
             for (int s = 0; s < 4; ++s) mbar_init(smem_u32(&bars.o_done[s >> 1][s & 1]), 1);
             mbar_init(smem_u32(&bars.drain), 1);
+            mbar_init(smem_u32(&bars.v_clean), 1);
+            mbar_init(smem_u32(&bars.v_landed), 1);
             fence_barrier_init();
         }
         if (warp == kMmaWarp) {
@@ -531,126 +531,151 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
             }
         }
     } else if (warp == kMmaWarp) {
-        // ===== MMA issuer (whole warp walks the loop, lane 0 waits and issues) =====================
-        auto wait_all = [&](uint32_t bar, uint32_t parity) {  // lane 0 polls, the warp gets the outcome
-            int r = 1;
-            if (lane == 0) r = mbar_wait_spin(bar, parity, abort_flag) ? 1 : 0;
-            r = __shfl_sync(0xffffffffu, r, 0);
-            __syncwarp();
-            return r != 0;
-        };
-        // rows past the sequence's last key hold whatever follows it in the cache: clear them in
-        // this block's V tile so that a zero probability times a non-finite value cannot reach O
-        auto clear_v_tail = [&](int j, int st) {
-            const int valid = n_keys - (t_begin + j) * kTK;
-            if (valid < kTK) {
-                constexpr int PANELS = PAIR ? 1 : HALVES;
-                const int chunks = (kTK - valid) * 8;
-                for (int idx = lane; idx < chunks * PANELS; idx += 32) {
-                    const int h = idx / chunks, rem = idx % chunks;
-                    const int r = valid + rem / 8, c = rem % 8;
-                    *reinterpret_cast<uint4*>(smem_gen + (sV - smem_base) + st * kVTile + h * kPanel + r * 128 +
-                                              c * 16) = make_uint4(0, 0, 0, 0);
+        // ===== MMA issuer: lane 0 alone walks the tiles, waits and issues; nothing in its loop
+        // involves the other lanes (a hand-off through the whole warp cost more than the eight
+        // instructions it guards).  The other lanes have one job: the only tile of this block that can
+        // reach past the sequence's last key is its last one, and rows past that key hold whatever
+        // follows the sequence in the cache.  Lane 0 tells them when that V tile has landed (it follows
+        // the ring's barriers phase by phase; a late joiner could not tell one use of a stage from the
+        // next), they clear those rows in this block's V tile, so that a zero probability times a
+        // non-finite value cannot reach O, and tell lane 0.
+        const int jt = nt - 1;                                  // the block's last tile
+        const int valid_t = n_keys - (t_begin + jt) * kTK;      // keys that exist in it
+        const bool has_tail = valid_t < kTK;
+        if (lane != 0) {
+            if (has_tail) {
+                const int st = jt % NST;
+                if (mbar_wait(smem_u32(&bars.v_landed), 0, abort_flag)) {
+                    constexpr int PANELS = PAIR ? 1 : HALVES;
+                    const int chunks = (kTK - valid_t) * 8;
+                    for (int idx = lane - 1; idx < chunks * PANELS; idx += 31) {
+                        const int h = idx / chunks, rem = idx % chunks;
+                        const int r = valid_t + rem / 8, c = rem % 8;
+                        *reinterpret_cast<uint4*>(smem_gen + (sV - smem_base) + st * kVTile + h * kPanel + r * 128 +
+                                                  c * 16) = make_uint4(0, 0, 0, 0);
+                    }
+                    fence_proxy_async();
+                    __syncwarp(0xfffffffeu);
+                    if (lane == 1) mbar_arrive(smem_u32(&bars.v_clean));
                 }
-                fence_proxy_async();
-                __syncwarp();
-            }
-        };
-        bool ok = wait_all(smem_u32(&bars.q_full), 0);
-        if (PAIR && rank != 0) {
-            // The second block of a pair issues no MMA: this warp tells the first block when this
-            // block's query tile, K half and V half are in place.
-            if (ok && lane == 0) mbar_arrive_in(smem_u32(&bars.q_peer), 0);
-            for (int j = 0; j < nt && ok; ++j) {
-                const int st = j % NST;
-                const uint32_t ph = (uint32_t)((j / NST) & 1);
-                ok = wait_all(smem_u32(&bars.k_full[st]), ph);
-                if (!ok) break;
-                if (lane == 0) mbar_arrive_in(smem_u32(&bars.k_peer[st]), 0);
-                ok = wait_all(smem_u32(&bars.v_full[st]), ph);
-                if (!ok) break;
-                clear_v_tail(j, st);
-                if (lane == 0) mbar_arrive_in(smem_u32(&bars.v_peer[st]), 0);
-                __syncwarp();
             }
         } else {
-            if (PAIR) ok = ok && wait_all(smem_u32(&bars.q_peer), 0);
-            auto commit = [&](uint32_t bar) {
-                if (PAIR) tc_commit2(bar);
-                else tc_commit(bar);
-            };
-            auto issue_qk = [&](int i) {  // S[slot] = Q[row tile] . K[tile]^T
-                const int j = i / MT, t = i % MT, st = j % NST;
-                if (t == 0) {
-                    ok = ok && wait_all(smem_u32(&bars.k_full[st]), (uint32_t)((j / NST) & 1));
-                    if (PAIR) ok = ok && wait_all(smem_u32(&bars.k_peer[st]), (uint32_t)((j / NST) & 1));
+            auto wait1 = [&](uint32_t bar, uint32_t parity) { return mbar_wait_spin(bar, parity, abort_flag); };
+            bool ok = wait1(smem_u32(&bars.q_full), 0);
+            if (PAIR && rank != 0) {
+                // The second block of a pair issues no MMA: this lane tells the first block when this
+                // block's query tile, K half and V half are in place.
+                if (ok) mbar_arrive_in(smem_u32(&bars.q_peer), 0);
+                int st = 0;
+                uint32_t ph = 0;
+                for (int j = 0; j < nt && ok; ++j) {
+                    ok = wait1(smem_u32(&bars.k_full[st]), ph);
+                    if (!ok) break;
+                    mbar_arrive_in(smem_u32(&bars.k_peer[st]), 0);
+                    ok = wait1(smem_u32(&bars.v_full[st]), ph);
+                    if (ok && has_tail && j == jt) {
+                        mbar_arrive(smem_u32(&bars.v_landed));
+                        ok = wait1(smem_u32(&bars.v_clean), 0);
+                    }
+                    if (!ok) break;
+                    mbar_arrive_in(smem_u32(&bars.v_peer[st]), 0);
+                    if (++st == NST) st = 0, ph ^= 1u;
                 }
-                if (!ok) return;
-                tc_fence_after();
-                if (lane == 0) {
-                    const uint32_t d_tmem = tmem + (uint32_t)(i % kSlots) * kTK;
-                    const uint64_t qd0 = smem_desc(sQ + t * kTile, 16), kd0 = smem_desc(sK + st * kKTile, 16);
+            } else {
+                if (PAIR) ok = ok && wait1(smem_u32(&bars.q_peer), 0);
+                auto commit = [&](uint32_t bar) {
+                    if (PAIR) tc_commit2(bar);
+                    else tc_commit(bar);
+                };
+                // Descriptor words of the three operand layouts (low word: address and leading offset
+                // in 16-byte units; high word: the layout's constants).
+                constexpr int CG = PAIR ? 2 : 1;
+                const uint64_t qd_first = smem_desc(sQ, 16), kd_first = smem_desc(sK, 16), vd_first = smem_desc(sV, kPanel);
+                const uint32_t q_lo0 = (uint32_t)qd_first, k_lo0 = (uint32_t)kd_first, v_lo0 = (uint32_t)vd_first;
+                const uint32_t qk_hi = (uint32_t)(qd_first >> 32), v_hi = (uint32_t)(vd_first >> 32);
+                int k_st = 0, v_st = 0;        // ring stage of the K tile the next Q.K^T reads, of the V tile the next P.V reads
+                uint32_t k_ph = 0, v_ph = 0;   // and the phases of their barriers
+                auto issue_qk = [&](int i) {  // S[slot] = Q[row tile] . K[tile]^T
+                    const int t = i & (MT - 1);
+                    if (t == 0) {
+                        ok = ok && wait1(smem_u32(&bars.k_full[k_st]), k_ph);
+                        if (PAIR) ok = ok && wait1(smem_u32(&bars.k_peer[k_st]), k_ph);
+                    }
+                    if (!ok) return;
+                    tc_fence_after();
+                    const uint32_t d_tmem = tmem + (uint32_t)(i & 1) * kTK;
+                    const uint32_t q_lo = q_lo0 + (uint32_t)t * (kTile >> 4), k_lo = k_lo0 + (uint32_t)k_st * (kKTile >> 4);
 #pragma unroll
                     for (int ks = 0; ks < DH / 16; ++ks) {
-                        const uint64_t qd = desc_advance(qd0, (uint32_t)(ks / 4) * kPanel + (uint32_t)(ks % 4) * 32u);
-                        const uint64_t kd = desc_advance(kd0, (uint32_t)(ks / 4) * kKPanel + (uint32_t)(ks % 4) * 32u);
-                        if (PAIR) mma2_ss(d_tmem, qd, kd, kIdescQK, ks > 0);
-                        else mma_ss(d_tmem, qd, kd, kIdescQK, ks > 0);
+                        const uint32_t qo = ((uint32_t)(ks / 4) * kPanel + (uint32_t)(ks % 4) * 32u) >> 4;
+                        const uint32_t ko = ((uint32_t)(ks / 4) * kKPanel + (uint32_t)(ks % 4) * 32u) >> 4;
+                        if (ks == 0) umma_ss<CG, 0>(d_tmem, q_lo + qo, qk_hi, k_lo + ko, qk_hi, kIdescQK);
+                        else umma_ss<CG, 1>(d_tmem, q_lo + qo, qk_hi, k_lo + ko, qk_hi, kIdescQK);
                     }
-                    commit(smem_u32(&bars.s_full[i % kSlots]));
-                    if (t == MT - 1) commit(smem_u32(&bars.k_empty[st]));
-                }
-                __syncwarp();
-            };
-            auto issue_pv = [&](int i) {  // O[row tile] += P[slot] . V[tile]
-                const int j = i / MT, t = i % MT, st = j % NST;
-                if (t == 0) {
-                    ok = ok && wait_all(smem_u32(&bars.v_full[st]), (uint32_t)((j / NST) & 1));
+                    commit(smem_u32(&bars.s_full[i & 1]));
+                    if (t == MT - 1) {
+                        commit(smem_u32(&bars.k_empty[k_st]));
+                        if (++k_st == NST) k_st = 0, k_ph ^= 1u;
+                    }
+                };
+                auto issue_pv = [&](int i) {  // O[row tile] += P[slot] . V[tile]
+                    const int t = i & (MT - 1), j = MT == 1 ? i : (i >> 1);
+                    if (t == 0) {
+                        ok = ok && wait1(smem_u32(&bars.v_full[v_st]), v_ph);
+                        if (ok && has_tail && j == jt) {
+                            mbar_arrive(smem_u32(&bars.v_landed));
+                            ok = wait1(smem_u32(&bars.v_clean), 0);
+                        }
+                        if (PAIR) ok = ok && wait1(smem_u32(&bars.v_peer[v_st]), v_ph);
+                    }
+                    ok = ok && wait1(smem_u32(&bars.p_full[i & 1]), (uint32_t)((i >> 1) & 1));
                     if (!ok) return;
-                    clear_v_tail(j, st);
-                    if (PAIR) ok = ok && wait_all(smem_u32(&bars.v_peer[st]), (uint32_t)((j / NST) & 1));
-                }
-                ok = ok && wait_all(smem_u32(&bars.p_full[i % kSlots]), (uint32_t)((i / kSlots) & 1));
-                if (!ok) return;
-                tc_fence_after();
-                if (lane == 0) {
+                    tc_fence_after();
                     const uint32_t d_tmem = tmem + kOCol + (uint32_t)t * DH;
-                    const uint32_t a_tmem = tmem + (uint32_t)(i % kSlots) * kTK;
-                    const uint64_t vd0 = smem_desc(sV + st * kVTile, kPanel);
+                    const uint32_t a_tmem = tmem + (uint32_t)(i & 1) * kTK;
+                    const uint32_t v_lo = v_lo0 + (uint32_t)v_st * (kVTile >> 4);
 #pragma unroll
                     for (int ks = 0; ks < kTK / 16; ++ks) {
-                        const uint64_t vd = desc_advance(vd0, ks * 2048u);
-                        const uint32_t acc = (j > 0 || ks > 0) ? 1u : 0u;
-                        if (PAIR) mma2_ts(d_tmem, a_tmem + ks * 8, vd, kIdescPV, acc);
-                        else mma_ts(d_tmem, a_tmem + ks * 8, vd, kIdescPV, acc);
+                        const uint32_t vo = (uint32_t)ks * (2048u >> 4);
+                        if (ks == 0) umma_ts<CG, 2>(d_tmem, a_tmem, v_lo, v_hi, kIdescPV, j > 0 ? 1u : 0u);
+                        else umma_ts<CG, 1>(d_tmem, a_tmem + ks * 8, v_lo + vo, v_hi, kIdescPV);
                     }
                     commit(smem_u32(&bars.o_done[t][j & 1]));
-                    if (t == MT - 1) commit(smem_u32(&bars.v_empty[st]));
+                    if (t == MT - 1) {
+                        commit(smem_u32(&bars.v_empty[v_st]));
+                        if (++v_st == NST) v_st = 0, v_ph ^= 1u;
+                    }
+                };
+                static_assert(kSlots == 2, "slot = item & 1");
+                for (int i = 0; i < kSlots && i < n_items && ok; ++i) issue_qk(i);
+                for (int i = 0; i < n_items && ok; ++i) {
+                    issue_pv(i);
+                    if (ok && i + kSlots < n_items) issue_qk(i + kSlots);
                 }
-                __syncwarp();
-            };
-            for (int i = 0; i < kSlots && i < n_items && ok; ++i) issue_qk(i);
-            for (int i = 0; i < n_items && ok; ++i) {
-                issue_pv(i);
-                if (ok && i + kSlots < n_items) issue_qk(i + kSlots);
             }
         }
+        __syncwarp();
     } else {
-        // ===== softmax warps: thread = packed query row ============================================
-        __shared__ float s_xmax[2][2][128];               // SPLIT: row maxima of the two column halves
-        __shared__ float s_xsum[2][128];                  // SPLIT: row sums of the two column halves
-        const int wg = SPLIT ? 0 : warp >> 2;             // row tile of this warp group
-        const int half = SPLIT ? warp >> 2 : 0;           // SPLIT: which half of the columns
-        const int r_tile = ((warp & 3) << 5) | lane;      // row inside the tile = tensor-memory lane
-        const int r_blk = wg * 128 + r_tile;              // row inside the block
-        const bool row_ok = r_blk < rows_here;
-        const int pr = row_ok ? row0 + r_blk : rb * plan.per;  // packed row = token * g + head in group
-        const int tok = pr / g, hq = hk * g + pr % g;
-        const uint32_t lane_sel = (uint32_t)((warp & 3) << 5) << 16;
-
+        // ===== softmax warps: thread = (packed query row, quarter of a tile's keys) ================
+        // Warp w reads the tensor-memory lanes of its sub-partition, 32 * (w % 4) .. + 31: the four
+        // warps w % 4 == s ("a quad") share 32 query rows and take 32 of the tile's 128 keys each.
+        // They exchange their row maxima through shared memory behind one barrier of the quad, which
+        // also separates every read of the scores from the writes of the probabilities over them.
+        // With two row tiles the sixteen warps serve the items (K/V tile, row tile) one after another.
+        __shared__ float s_xmax[2][4][128];               // [item parity][quarter][row]: row maxima of the quarters
+        __shared__ float s_xsum[MT][4][128];              // epilogue: row sums of the quarters
+        const int quad = warp & 3, quarter = warp >> 2;
+        const int r_tile = (quad << 5) | lane;            // row inside the tile = tensor-memory lane
+        const uint32_t lane_sel = (uint32_t)(quad << 5) << 16;
         const int W = (m + 63) >> 6;
-        const unsigned long long mlo = mask_bits[((long long)b * m + tok) * W];
-        const unsigned long long mhi = W > 1 ? mask_bits[((long long)b * m + tok) * W + 1] : 0ull;
+        unsigned long long mlo[MT], mhi[MT];
+#pragma unroll
+        for (int t = 0; t < MT; ++t) {
+            const int r_blk = t * 128 + r_tile;
+            const int pr = r_blk < rows_here ? row0 + r_blk : rb * plan.per;  // packed row = token * g + head in group
+            mlo[t] = mask_bits[((long long)b * m + pr / g) * W];
+            mhi[t] = W > 1 ? mask_bits[((long long)b * m + pr / g) * W + 1] : 0ull;
+        }
         if (!plan.q_tma) {
             // query rows into shared memory by hand, 128-byte swizzled (chunk c of row r at
             // c ^ (r & 7)); all copies of a thread are in flight together, absent rows zero-filled
@@ -670,155 +695,92 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
             mbar_arrive(smem_u32(&bars.q_full));
         }
 
-        float m_ref = -INFINITY, l_run = 0.f;
+        float m_ref[MT], l_run[MT];
+#pragma unroll
+        for (int t = 0; t < MT; ++t) m_ref[t] = -INFINITY, l_run[t] = 0.f;
         bool ok = true;
-        for (int j = 0; j < nt; ++j) {
-            const int i = j * MT + wg, slot = i % kSlots;
-            ok = mbar_wait(smem_u32(&bars.s_full[slot]), (uint32_t)((i / kSlots) & 1), abort_flag);
+        const int quad_bar = 2 + quad;  // named barrier of this quad's 128 threads
+        for (int i = 0; i < n_items; ++i) {
+            const int j = i / MT, slot = i % kSlots;
+            const int t = MT == 1 ? 0 : (i & 1);
+            ok = ok && mbar_wait(smem_u32(&bars.s_full[slot]), (uint32_t)((i / kSlots) & 1), abort_flag);
             ok = __all_sync(0xffffffffu, ok);  // the tensor-memory accesses below need the whole warp
-            if (!SPLIT && !ok) break;          // SPLIT: all eight warps leave together, a few lines down
-            tc_fence_after();
             const uint32_t s_addr = tmem + lane_sel + (uint32_t)slot * kTK;
             const int key0 = (t_begin + j) * kTK;
             const bool tail = key0 + kTK > L;  // the tile holds tree keys or runs past the last key
-            uint32_t vis[4] = {~0u, ~0u, ~0u, ~0u};
-            if (tail) tile_visibility(mlo, mhi, key0, L, n_keys, vis);
-
-            if constexpr (SPLIT) {
-                // This thread owns columns [64*half, 64*half+64) of its row; the thread of the other
-                // warp group owns the rest.  They exchange their maxima through shared memory; the
-                // barrier of that exchange also separates every read of S from the writes of P.
-                ok = named_barrier_and(2, kSoftmaxThreads, ok);
-                if (!ok) break;
-                uint32_t bufa[32], bufb[32];
-                tmem_ld32(s_addr + half * 64, bufa);
-                tmem_ld32(s_addr + half * 64 + 32, bufb);
-                tc_wait_ld(bufa);
-                tc_wait_ld(bufb);
-                float mx = -INFINITY;
-                mx = tail ? chunk_rowmax<true>(bufa, vis[half * 2], mx) : chunk_rowmax<false>(bufa, 0, mx);
-                mx = tail ? chunk_rowmax<true>(bufb, vis[half * 2 + 1], mx) : chunk_rowmax<false>(bufb, 0, mx);
-                s_xmax[j & 1][half][r_tile] = mx;
-                asm volatile("bar.sync 2, %0;" ::"n"(kSoftmaxThreads) : "memory");
-                mx = fmaxf(mx, s_xmax[j & 1][half ^ 1][r_tile]) * scale_log2;
-
-                const float m_new = fmaxf(m_ref, mx);
-                const bool grow = m_new > m_ref + 8.f;
-                if (__any_sync(0xffffffffu, grow)) {
-                    const float factor = !grow ? 1.f : (m_ref == -INFINITY ? 0.f : ex2(m_ref - m_new));
-                    if (grow) m_ref = m_new, l_run *= factor;
-                    bool waited = true;
-                    if (j > 0)
-                        waited = mbar_wait(smem_u32(&bars.o_done[0][(j - 1) & 1]), (uint32_t)(((j - 1) >> 1) & 1), abort_flag);
-                    waited = __all_sync(0xffffffffu, waited);
-                    if (!waited) ok = false;  // every warp learns it at the top of the next tile
-                    if (j > 0 && waited) {
-                        tc_fence_after();
-                        const uint32_t o_half = tmem + lane_sel + kOCol + (uint32_t)half * (DH / 2);
-                        uint32_t orow[32];
-#pragma unroll
-                        for (int c4 = 0; c4 < DH / 64; ++c4) {
-                            tmem_ld32(o_half + c4 * 32, orow);
-                            tc_wait_ld(orow);
-#pragma unroll
-                            for (int c = 0; c < 32; ++c) orow[c] = __float_as_uint(__uint_as_float(orow[c]) * factor);
-                            tmem_st32(o_half + c4 * 32, orow);
-                        }
-                    }
-                }
-                const float neg_ref = m_ref == -INFINITY ? 0.f : -m_ref;
-                const float2 scale2 = make_float2(scale_log2, scale_log2), neg_ref2 = make_float2(neg_ref, neg_ref);
-                float2 sum_a = make_float2(0.f, 0.f), sum_b = make_float2(0.f, 0.f);
-                uint32_t pk[32];
-                if (tail) {
-                    chunk_probs<true>(bufa, vis[half * 2], scale2, neg_ref2, sum_a, sum_b, pk);
-                    chunk_probs<true>(bufb, vis[half * 2 + 1], scale2, neg_ref2, sum_a, sum_b, pk + 16);
-                } else {
-                    chunk_probs<false>(bufa, 0, scale2, neg_ref2, sum_a, sum_b, pk);
-                    chunk_probs<false>(bufb, 0, scale2, neg_ref2, sum_a, sum_b, pk + 16);
-                }
-                tmem_st32(s_addr + half * 32, pk);  // keys [64*half, +64) as 32 packed columns
-                l_run += (sum_a.x + sum_a.y) + (sum_b.x + sum_b.y);
-                tc_wait_st();
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) {
-                    if (PAIR) mbar_arrive_in(smem_u32(&bars.p_full[slot]), 0);
-                    else mbar_arrive(smem_u32(&bars.p_full[slot]));
-                }
-                continue;
+            uint32_t visw = ~0u;
+            if (tail) {
+                uint32_t vis[4];
+                tile_visibility(t == 0 ? mlo[0] : mlo[MT - 1], t == 0 ? mhi[0] : mhi[MT - 1], key0, L, n_keys, vis);
+                visw = vis[quarter];
             }
-
-            // Both passes walk the row in four 32-column chunks through two register buffers: the
-            // load of the next chunk is in flight while the current one is processed.  A tile that
-            // lies wholly inside the committed cache takes the branch without mask arithmetic.
-            uint32_t bufa[32], bufb[32];
-            // pass 1: row maximum of the raw scores (the scale is positive)
+            uint32_t buf[32];
             float mx = -INFINITY;
-            tmem_ld32(s_addr, bufa);
-            tc_wait_ld(bufa);
-            tmem_ld32(s_addr + 32, bufb);
-            mx = tail ? chunk_rowmax<true>(bufa, vis[0], mx) : chunk_rowmax<false>(bufa, 0, mx);
-            tc_wait_ld(bufb);
-            tmem_ld32(s_addr + 64, bufa);
-            mx = tail ? chunk_rowmax<true>(bufb, vis[1], mx) : chunk_rowmax<false>(bufb, 0, mx);
-            tc_wait_ld(bufa);
-            tmem_ld32(s_addr + 96, bufb);
-            mx = tail ? chunk_rowmax<true>(bufa, vis[2], mx) : chunk_rowmax<false>(bufa, 0, mx);
-            tc_wait_ld(bufb);
-            tmem_ld32(s_addr, bufa);  // first chunk of pass 2
-            mx = tail ? chunk_rowmax<true>(bufb, vis[3], mx) : chunk_rowmax<false>(bufb, 0, mx);
+            if (ok) {
+                tc_fence_after();
+                tmem_ld32(s_addr + quarter * 32, buf);
+                tc_wait_ld(buf);
+                mx = tail ? chunk_rowmax<true>(buf, visw, mx) : chunk_rowmax<false>(buf, 0, mx);
+                s_xmax[i & 1][quarter][r_tile] = mx;
+            }
+            // every warp of the quad has its scores in registers (or all of them leave together)
+            ok = named_barrier_and(quad_bar, 128, ok);
+            if (!ok) break;
+#pragma unroll
+            for (int o = 1; o < 4; ++o) mx = fmaxf(mx, s_xmax[i & 1][(quarter + o) & 3][r_tile]);
             mx *= scale_log2;
 
-            // lazily rescaled reference maximum: probabilities stay below 2^8 in between
-            const float m_new = fmaxf(m_ref, mx);
-            const bool grow = m_new > m_ref + 8.f;
+            // lazily rescaled reference maximum: probabilities stay below 2^8 in between.  The four
+            // threads of a row hold the same reference: they derive it from the same four maxima.
+            float mr = t == 0 ? m_ref[0] : m_ref[MT - 1];
+            const float m_new = fmaxf(mr, mx);
+            const bool grow = m_new > mr + 8.f;
             if (__any_sync(0xffffffffu, grow)) {
-                const float factor = !grow ? 1.f : (m_ref == -INFINITY ? 0.f : ex2(m_ref - m_new));
-                if (grow) m_ref = m_new, l_run *= factor;
-                // O may be rescaled once the previous P.V of this row tile has finished
+                const float factor = !grow ? 1.f : (mr == -INFINITY ? 0.f : ex2(mr - m_new));
+                if (grow) {
+                    mr = m_new;
+                    if (MT == 1 || t == 0) m_ref[0] = mr, l_run[0] *= factor;
+                    else m_ref[MT - 1] = mr, l_run[MT - 1] *= factor;
+                }
+                // O may be rescaled once the previous P.V of this row tile has finished; this thread
+                // owns a quarter of the row's columns
+                bool waited = true;
                 if (j > 0)
-                    ok = mbar_wait(smem_u32(&bars.o_done[wg][(j - 1) & 1]), (uint32_t)(((j - 1) >> 1) & 1), abort_flag);
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) break;
-                if (j > 0) {
+                    waited = mbar_wait(smem_u32(&bars.o_done[t][(j - 1) & 1]), (uint32_t)(((j - 1) >> 1) & 1), abort_flag);
+                waited = __all_sync(0xffffffffu, waited);
+                if (!waited) ok = false;  // the quad learns it at its next barrier
+                if (j > 0 && waited) {
                     tc_fence_after();
-                    const uint32_t o_addr = tmem + lane_sel + kOCol + (uint32_t)wg * DH;
+                    const uint32_t o_q = tmem + lane_sel + kOCol + (uint32_t)t * DH + (uint32_t)quarter * (DH / 4);
+                    if constexpr (DH == 128) {
+                        uint32_t orow[32];
+                        tmem_ld32(o_q, orow);
+                        tc_wait_ld(orow);
 #pragma unroll
-                    for (int c4 = 0; c4 < DH / 32; ++c4) {
-                        tmem_ld32(o_addr + c4 * 32, bufb);
-                        tc_wait_ld(bufb);
+                        for (int c = 0; c < 32; ++c) orow[c] = __float_as_uint(__uint_as_float(orow[c]) * factor);
+                        tmem_st32(o_q, orow);
+                    } else {
+                        uint32_t orow[16];
+                        tmem_ld16(o_q, orow);
+                        tc_wait_ld16(orow);
 #pragma unroll
-                        for (int c = 0; c < 32; ++c) bufb[c] = __float_as_uint(__uint_as_float(bufb[c]) * factor);
-                        tmem_st32(o_addr + c4 * 32, bufb);
+                        for (int c = 0; c < 16; ++c) orow[c] = __float_as_uint(__uint_as_float(orow[c]) * factor);
+                        tmem_st16(o_q, orow);
                     }
                 }
             }
-            // pass 2: P = 2^(s * scale - reference) as bf16 over the first 64 columns of the slot;
-            // packed columns [0,32) are written once score columns [0,64) are in registers, [32,64)
-            // after the rest
-            const float neg_ref = m_ref == -INFINITY ? 0.f : -m_ref;
+            // P = 2^(s * scale - reference) as bf16: this thread's 32 keys become 16 packed columns
+            // over the first half of the slot
+            const float neg_ref = mr == -INFINITY ? 0.f : -mr;
             const float2 scale2 = make_float2(scale_log2, scale_log2), neg_ref2 = make_float2(neg_ref, neg_ref);
             float2 sum_a = make_float2(0.f, 0.f), sum_b = make_float2(0.f, 0.f);
-            uint32_t pk[32];
-            tc_wait_ld(bufa);
-            tmem_ld32(s_addr + 32, bufb);
-            if (tail) chunk_probs<true>(bufa, vis[0], scale2, neg_ref2, sum_a, sum_b, pk);
-            else chunk_probs<false>(bufa, 0, scale2, neg_ref2, sum_a, sum_b, pk);
-            tc_wait_ld(bufb);
-            tmem_ld32(s_addr + 64, bufa);
-            if (tail) chunk_probs<true>(bufb, vis[1], scale2, neg_ref2, sum_a, sum_b, pk + 16);
-            else chunk_probs<false>(bufb, 0, scale2, neg_ref2, sum_a, sum_b, pk + 16);
-            tc_wait_ld(bufa);
-            tmem_ld32(s_addr + 96, bufb);
-            tmem_st32(s_addr, pk);
-            if (tail) chunk_probs<true>(bufa, vis[2], scale2, neg_ref2, sum_a, sum_b, pk);
-            else chunk_probs<false>(bufa, 0, scale2, neg_ref2, sum_a, sum_b, pk);
-            tc_wait_ld(bufb);
-            if (tail) chunk_probs<true>(bufb, vis[3], scale2, neg_ref2, sum_a, sum_b, pk + 16);
-            else chunk_probs<false>(bufb, 0, scale2, neg_ref2, sum_a, sum_b, pk + 16);
-            tmem_st32(s_addr + 32, pk);
-            l_run += (sum_a.x + sum_a.y) + (sum_b.x + sum_b.y);
+            uint32_t pk[16];
+            if (tail) chunk_probs<true>(buf, visw, scale2, neg_ref2, sum_a, sum_b, pk);
+            else chunk_probs<false>(buf, 0, scale2, neg_ref2, sum_a, sum_b, pk);
+            tmem_st16(s_addr + quarter * 16, pk);
+            const float add = (sum_a.x + sum_a.y) + (sum_b.x + sum_b.y);
+            if (MT == 1 || t == 0) l_run[0] += add;
+            else l_run[MT - 1] += add;
             tc_wait_st();
             tc_fence_before();
             __syncwarp();  // every lane's P is in tensor memory: one arrival speaks for the warp
@@ -829,68 +791,75 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
         }
 
         // ---- epilogue: O rows leave tensor memory through shared memory, so that the global
-        // stores are whole contiguous rows.  Row tile 0 of two stages in the query region (both row
-        // tiles' Q.K^T are complete once any last P.V is), the other one - and a single tile - in the
-        // K ring.  The threads that share a staging area first agree that none of them gave up.
-        ok = ok && mbar_wait(smem_u32(&bars.o_done[wg][(nt - 1) & 1]), (uint32_t)(((nt - 1) >> 1) & 1), abort_flag);
-        const int epi_id = SPLIT ? 2 : 1 + wg, epi_threads = SPLIT ? kSoftmaxThreads : 128;
-        if (SPLIT) s_xsum[half][r_tile] = l_run;
-        ok = named_barrier_and(epi_id, epi_threads, ok);
+        // stores are whole contiguous rows.  Row tile t is staged where its queries were: every
+        // Q.K^T has completed once the last P.V of a row tile has.  All softmax threads first agree
+        // that none of them gave up.
+#pragma unroll
+        for (int t = 0; t < MT; ++t) {
+            ok = ok && mbar_wait(smem_u32(&bars.o_done[t][(nt - 1) & 1]), (uint32_t)(((nt - 1) >> 1) & 1), abort_flag);
+            s_xsum[t][quarter][r_tile] = l_run[t];
+        }
+        ok = named_barrier_and(1, kSoftmaxThreads, ok);
         if (ok) {
             tc_fence_after();
-            constexpr int NCOL = SPLIT ? DH / 2 : DH;          // columns of O this thread owns
-            const int col0 = half * NCOL;
-            const uint32_t o_addr = tmem + lane_sel + kOCol + (uint32_t)wg * DH + (uint32_t)col0;
-            const float l_tot = SPLIT ? l_run + s_xsum[half ^ 1][r_tile] : l_run;
-            // final rows are normalised here; a partial stays unnormalised (the merge divides by the
-            // combined sum) and is rounded to bf16 once, like a final row
-            const float inv = !direct ? 1.f : (l_tot > 0.f ? 1.f / l_tot : 0.f);
-            unsigned char* stage = smem_gen + ((MT == 2 && wg == 0) ? 0u : (sK - smem_base));
+            constexpr int NCOL = DH / 4;  // columns of O this thread owns
+            constexpr int row_bytes = DH * 2;
+            const int cmask = row_bytes / 16 - 1;
             // a staged row is DH bf16; 16-byte chunk c of row r sits at chunk c ^ (r mod
             // chunks-per-row), which keeps both the row-wise writes and the chunk-wise reads free of
             // bank conflicts
-            constexpr int row_bytes = DH * 2;
-            const int cmask = row_bytes / 16 - 1;
 #pragma unroll
-            for (int c4 = 0; c4 < NCOL / 32; ++c4) {
-                uint32_t orow[32];
-                tmem_ld32(o_addr + c4 * 32, orow);
-                tc_wait_ld(orow);
-                unsigned char* srow = stage + (size_t)r_tile * row_bytes;
-                {
+            for (int t = 0; t < MT; ++t) {
+                const int r_blk = t * 128 + r_tile;
+                const float l_tot = (s_xsum[t][0][r_tile] + s_xsum[t][1][r_tile]) + (s_xsum[t][2][r_tile] + s_xsum[t][3][r_tile]);
+                // final rows are normalised here; a partial stays unnormalised (the merge divides by the
+                // combined sum) and is rounded to bf16 once, like a final row
+                const float inv = !direct ? 1.f : (l_tot > 0.f ? 1.f / l_tot : 0.f);
+                unsigned char* srow = smem_gen + t * kTile + (size_t)r_tile * row_bytes;
+                const uint32_t o_q = tmem + lane_sel + kOCol + (uint32_t)t * DH + (uint32_t)quarter * NCOL;
+                uint32_t orow[NCOL];
+                if constexpr (DH == 128) {
+                    tmem_ld32(o_q, orow);
+                    tc_wait_ld(orow);
+                } else {
+                    tmem_ld16(o_q, orow);
+                    tc_wait_ld16(orow);
+                }
 #pragma unroll
-                    for (int c = 0; c < 32; c += 8) {
-                        uint4 v;
-                        v.x = pack_bf16(__uint_as_float(orow[c + 0]) * inv, __uint_as_float(orow[c + 1]) * inv);
-                        v.y = pack_bf16(__uint_as_float(orow[c + 2]) * inv, __uint_as_float(orow[c + 3]) * inv);
-                        v.z = pack_bf16(__uint_as_float(orow[c + 4]) * inv, __uint_as_float(orow[c + 5]) * inv);
-                        v.w = pack_bf16(__uint_as_float(orow[c + 6]) * inv, __uint_as_float(orow[c + 7]) * inv);
-                        const int chunk = (col0 + c4 * 32 + c) >> 3;
-                        *reinterpret_cast<uint4*>(srow + (((chunk ^ r_tile) & cmask) << 4)) = v;
+                for (int c = 0; c < NCOL; c += 8) {
+                    uint4 v;
+                    v.x = pack_bf16(__uint_as_float(orow[c + 0]) * inv, __uint_as_float(orow[c + 1]) * inv);
+                    v.y = pack_bf16(__uint_as_float(orow[c + 2]) * inv, __uint_as_float(orow[c + 3]) * inv);
+                    v.z = pack_bf16(__uint_as_float(orow[c + 4]) * inv, __uint_as_float(orow[c + 5]) * inv);
+                    v.w = pack_bf16(__uint_as_float(orow[c + 6]) * inv, __uint_as_float(orow[c + 7]) * inv);
+                    const int chunk = (quarter * NCOL + c) >> 3;
+                    *reinterpret_cast<uint4*>(srow + (((chunk ^ r_tile) & cmask) << 4)) = v;
+                }
+                if (r_blk < rows_here && quarter == 0) {
+                    const int pr = row0 + r_blk;
+                    if (direct) {
+                        if (lse)
+                            lse[((long long)b * Hq + hk * g + pr % g) * m + pr / g] =
+                                ((MT == 1 ? m_ref[0] : m_ref[t]) + log2f(l_tot)) * 0.69314718055994531f;
+                    } else {
+                        ws.ml[part_row0 + r_blk] = make_float2(MT == 1 ? m_ref[0] : m_ref[t], l_tot);
                     }
                 }
             }
-            if (row_ok && half == 0) {
-                if (direct) {
-                    if (lse) lse[((long long)b * Hq + hq) * m + tok] = (m_ref + log2f(l_tot)) * 0.69314718055994531f;
-                } else {
-                    ws.ml[part_row0 + r_blk] = make_float2(m_ref, l_tot);
-                }
-            }
-            asm volatile("bar.sync %0, %1;" ::"r"(epi_id), "r"(epi_threads) : "memory");  // rows are staged
-            const int rows_tile = min(128, rows_here - wg * 128);
-            const int lanes_per_row = row_bytes / 16;       // 16 or 32 (8 for a 64-wide bf16 row)
+            asm volatile("bar.sync 1, %0;" ::"n"(kSoftmaxThreads) : "memory");  // rows are staged
+            const int lanes_per_row = row_bytes / 16;       // 16 lanes (8 for a 64-wide bf16 row)
             const int rows_per_pass = 32 / lanes_per_row;
             const int sub = lane / lanes_per_row, cl = lane % lanes_per_row;
-            const int cw = SPLIT ? warp : (warp & 3), ncw = SPLIT ? 8 : 4;  // copying warps of this tile
-            for (int r = cw * rows_per_pass + sub; r < rows_tile; r += ncw * rows_per_pass) {
-                const uint4 v = *reinterpret_cast<const uint4*>(stage + (size_t)r * row_bytes + (((cl ^ r) & cmask) << 4));
+            for (int r = warp * rows_per_pass + sub; r < rows_here; r += (kSoftmaxThreads / 32) * rows_per_pass) {
+                const int t = r >> 7, rr = r & 127;
+                const uint4 v = *reinterpret_cast<const uint4*>(smem_gen + t * kTile + (size_t)rr * row_bytes +
+                                                                (((cl ^ rr) & cmask) << 4));
                 if (direct) {
-                    const int p2 = row0 + wg * 128 + r;
+                    const int p2 = row0 + r;
                     __nv_bfloat16* dst = out + (((long long)b * m + p2 / g) * Hq + hk * g + p2 % g) * DH;
                     *reinterpret_cast<uint4*>(reinterpret_cast<unsigned char*>(dst) + cl * 16) = v;
                 } else {
-                    __nv_bfloat16* dst = ws.o_part + (part_row0 + wg * 128 + r) * DH;
+                    __nv_bfloat16* dst = ws.o_part + (part_row0 + r) * DH;
                     *reinterpret_cast<uint4*>(reinterpret_cast<unsigned char*>(dst) + cl * 16) = v;
                 }
             }
