@@ -205,13 +205,13 @@ __device__ __forceinline__ float chunk_rowmax(const uint32_t (&r)[32], uint32_t 
     }
     return fmaxf(m0, m1);
 }
-// p = 2^(s * scale - reference) for a 32-column chunk, packed to 16 bf16 pairs; the sums of the
+// p = 2^(s * scale - reference) for a chunk of NC columns, packed to NC/2 bf16 pairs; the sums of the
 // unrounded probabilities accumulate in two packed registers.
-template <bool TAIL>
-__device__ __forceinline__ void chunk_probs(const uint32_t (&r)[32], uint32_t visw, float2 scale2, float2 neg_ref2,
-                                            float2& sum_a, float2& sum_b, uint32_t* pk) {
+template <bool TAIL, int NC>
+__device__ __forceinline__ void chunk_probs(const uint32_t (&r)[NC], uint32_t visw, float2 scale2, float2 neg_ref2,
+                                            float2& sum_a, float2& sum_b, uint32_t (&pk)[NC / 2]) {
 #pragma unroll
-    for (int c = 0; c < 32; c += 4) {
+    for (int c = 0; c < NC; c += 4) {
         float2 a = __ffma2_rn(make_float2(__uint_as_float(r[c]), __uint_as_float(r[c + 1])), scale2, neg_ref2);
         float2 bq = __ffma2_rn(make_float2(__uint_as_float(r[c + 2]), __uint_as_float(r[c + 3])), scale2, neg_ref2);
         if (TAIL) {
@@ -223,8 +223,8 @@ __device__ __forceinline__ void chunk_probs(const uint32_t (&r)[32], uint32_t vi
         const float2 pa = make_float2(ex2(a.x), ex2(a.y)), pb = make_float2(ex2(bq.x), ex2(bq.y));
         sum_a = __fadd2_rn(sum_a, pa);
         sum_b = __fadd2_rn(sum_b, pb);
-        pk[c >> 1] = pack_bf16(pa.x, pa.y);
-        pk[(c >> 1) + 1] = pack_bf16(pb.x, pb.y);
+        pk[c >> 1] = pack_bf16_alu(pa.x, pa.y);
+        pk[(c >> 1) + 1] = pack_bf16_alu(pb.x, pb.y);
     }
 }
 
@@ -638,7 +638,7 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
                     for (int ks = 0; ks < kTK / 16; ++ks) {
                         const uint32_t vo = (uint32_t)ks * (2048u >> 4);
                         if (ks == 0) umma_ts<CG, 2>(d_tmem, a_tmem, v_lo, v_hi, kIdescPV, j > 0 ? 1u : 0u);
-                        else umma_ts<CG, 1>(d_tmem, a_tmem + ks * 8, v_lo + vo, v_hi, kIdescPV);
+                        else umma_ts<CG, 1>(d_tmem, a_tmem + (ks >> 1) * 32 + (ks & 1) * 8, v_lo + vo, v_hi, kIdescPV);
                     }
                     commit(smem_u32(&bars.o_done[t][j & 1]));
                     if (t == MT - 1) {
@@ -659,8 +659,8 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
         // ===== softmax warps: thread = (packed query row, quarter of a tile's keys) ================
         // Warp w reads the tensor-memory lanes of its sub-partition, 32 * (w % 4) .. + 31: the four
         // warps w % 4 == s ("a quad") share 32 query rows and take 32 of the tile's 128 keys each.
-        // They exchange their row maxima through shared memory behind one barrier of the quad, which
-        // also separates every read of the scores from the writes of the probabilities over them.
+        // They exchange their row maxima through shared memory behind one barrier of the quad; each
+        // writes its probabilities over its own scores.
         // With two row tiles the sixteen warps serve the items (K/V tile, row tile) one after another.
         __shared__ float s_xmax[2][4][128];               // [item parity][quarter][row]: row maxima of the quarters
         __shared__ float s_xsum[MT][4][128];              // epilogue: row sums of the quarters
@@ -714,16 +714,17 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
                 tile_visibility(t == 0 ? mlo[0] : mlo[MT - 1], t == 0 ? mhi[0] : mhi[MT - 1], key0, L, n_keys, vis);
                 visw = vis[quarter];
             }
-            uint32_t buf[32];
             float mx = -INFINITY;
             if (ok) {
+                // pass 1: the largest raw score of this thread's 32 keys (the scale is positive)
+                uint32_t buf[32];
                 tc_fence_after();
                 tmem_ld32(s_addr + quarter * 32, buf);
                 tc_wait_ld(buf);
                 mx = tail ? chunk_rowmax<true>(buf, visw, mx) : chunk_rowmax<false>(buf, 0, mx);
                 s_xmax[i & 1][quarter][r_tile] = mx;
             }
-            // every warp of the quad has its scores in registers (or all of them leave together)
+            // the quarters' maxima meet here (or all four warps leave together)
             ok = named_barrier_and(quad_bar, 128, ok);
             if (!ok) break;
 #pragma unroll
@@ -769,15 +770,26 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
                     }
                 }
             }
-            // P = 2^(s * scale - reference) as bf16: this thread's 32 keys become 16 packed columns
-            // over the first half of the slot
+            // pass 2: P = 2^(s * scale - reference) as bf16.  The scores are read again, 16 keys at a
+            // time, and each 16 keys become 8 packed columns written over the thread's own scores
+            // (columns 32 * quarter + 8 * half ..): no thread ever writes a column another one reads.
             const float neg_ref = mr == -INFINITY ? 0.f : -mr;
             const float2 scale2 = make_float2(scale_log2, scale_log2), neg_ref2 = make_float2(neg_ref, neg_ref);
             float2 sum_a = make_float2(0.f, 0.f), sum_b = make_float2(0.f, 0.f);
-            uint32_t pk[16];
-            if (tail) chunk_probs<true>(buf, visw, scale2, neg_ref2, sum_a, sum_b, pk);
-            else chunk_probs<false>(buf, 0, scale2, neg_ref2, sum_a, sum_b, pk);
-            tmem_st16(s_addr + quarter * 16, pk);
+            uint32_t b0[16], b1[16];
+            tmem_ld16(s_addr + quarter * 32, b0);
+            tmem_ld16(s_addr + quarter * 32 + 16, b1);
+            tc_wait_ld16(b0);
+            tc_wait_ld16(b1);
+            {
+                uint32_t pk[8];
+                if (tail) chunk_probs<true, 16>(b0, visw, scale2, neg_ref2, sum_a, sum_b, pk);
+                else chunk_probs<false, 16>(b0, 0, scale2, neg_ref2, sum_a, sum_b, pk);
+                tmem_st8(s_addr + quarter * 32, pk);
+                if (tail) chunk_probs<true, 16>(b1, visw >> 16, scale2, neg_ref2, sum_a, sum_b, pk);
+                else chunk_probs<false, 16>(b1, 0, scale2, neg_ref2, sum_a, sum_b, pk);
+                tmem_st8(s_addr + quarter * 32 + 8, pk);
+            }
             const float add = (sum_a.x + sum_a.y) + (sum_b.x + sum_b.y);
             if (MT == 1 || t == 0) l_run[0] += add;
             else l_run[MT - 1] += add;
