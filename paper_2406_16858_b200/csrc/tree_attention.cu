@@ -237,8 +237,8 @@ struct AttnBarriers {
     unsigned long long q_full;
     unsigned long long k_full[4], k_empty[4], v_full[4], v_empty[4];
     unsigned long long s_full[kSlots], p_full[kSlots];
-    // Per row tile, two barriers used by alternate K/V tiles: P.V of tile j completes a phase of
-    // o_done[t][j & 1].  A waiter may skip phases (it only looks when it must rescale O, and at the
+    // Per accumulator (= score slot = item parity), two barriers used by its alternate uses: the
+    // u-th P.V into accumulator e completes a phase of o_done[e][u & 1].  A waiter may skip phases (it only looks when it must rescale O, and at the
     // end); with two barriers the one it consults is never more than one phase ahead of it.
     unsigned long long o_done[2][2];
     // pair mode, used in the pair's first block: the other block's query tile / K half / V half
@@ -402,7 +402,7 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
             }
             for (int s = 0; s < kSlots; ++s) {
                 mbar_init(smem_u32(&bars.s_full[s]), 1);
-                mbar_init(smem_u32(&bars.p_full[s]), (PAIR ? 2 : 1) * (kSoftmaxThreads / 32));  // one arrival per softmax warp
+                mbar_init(smem_u32(&bars.p_full[s]), (PAIR ? 2 : 1) * (kSoftmaxThreads / 64));  // one arrival per warp of the slot's group
             }
             mbar_init(smem_u32(&bars.q_peer), 1);
             for (int s = 0; s < 4; ++s) {
@@ -631,16 +631,16 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
                     ok = ok && wait1(smem_u32(&bars.p_full[i & 1]), (uint32_t)((i >> 1) & 1));
                     if (!ok) return;
                     tc_fence_after();
-                    const uint32_t d_tmem = tmem + kOCol + (uint32_t)t * DH;
+                    const uint32_t d_tmem = tmem + kOCol + (uint32_t)(i & 1) * DH;  // accumulator = slot = item parity
                     const uint32_t a_tmem = tmem + (uint32_t)(i & 1) * kTK;
                     const uint32_t v_lo = v_lo0 + (uint32_t)v_st * (kVTile >> 4);
 #pragma unroll
                     for (int ks = 0; ks < kTK / 16; ++ks) {
                         const uint32_t vo = (uint32_t)ks * (2048u >> 4);
-                        if (ks == 0) umma_ts<CG, 2>(d_tmem, a_tmem, v_lo, v_hi, kIdescPV, j > 0 ? 1u : 0u);
-                        else umma_ts<CG, 1>(d_tmem, a_tmem + (ks >> 1) * 32 + (ks & 1) * 8, v_lo + vo, v_hi, kIdescPV);
+                        if (ks == 0) umma_ts<CG, 2>(d_tmem, a_tmem, v_lo, v_hi, kIdescPV, i >= 2 ? 1u : 0u);
+                        else umma_ts<CG, 1>(d_tmem, a_tmem + ks * 16, v_lo + vo, v_hi, kIdescPV);
                     }
-                    commit(smem_u32(&bars.o_done[t][j & 1]));
+                    commit(smem_u32(&bars.o_done[i & 1][(i >> 1) & 1]));
                     if (t == MT - 1) {
                         commit(smem_u32(&bars.v_empty[v_st]));
                         if (++v_st == NST) v_st = 0, v_ph ^= 1u;
@@ -656,25 +656,31 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
         }
         __syncwarp();
     } else {
-        // ===== softmax warps: thread = (packed query row, quarter of a tile's keys) ================
-        // Warp w reads the tensor-memory lanes of its sub-partition, 32 * (w % 4) .. + 31: the four
-        // warps w % 4 == s ("a quad") share 32 query rows and take 32 of the tile's 128 keys each.
-        // They exchange their row maxima through shared memory behind one barrier of the quad; each
-        // writes its probabilities over its own scores.
-        // With two row tiles the sixteen warps serve the items (K/V tile, row tile) one after another.
-        __shared__ float s_xmax[2][4][128];               // [item parity][quarter][row]: row maxima of the quarters
-        __shared__ float s_xsum[MT][4][128];              // epilogue: row sums of the quarters
-        const int quad = warp & 3, quarter = warp >> 2;
+        // ===== softmax warps: two groups of eight, each serving every other item ====================
+        // A pass over one item (128 rows x 128 keys) is a chain of dependent steps - scores out of
+        // tensor memory, row maximum, exchange, exponentials, probabilities back - and a group of
+        // warps running it is mostly waiting; two groups on different items keep each other's
+        // gaps filled.  Group e serves the items i with i % 2 == e: score slot e and accumulator e.
+        // With two row tiles that is row tile e; with one row tile both groups serve it, each with
+        // its own reference maximum, row sums and accumulator, and the epilogue combines the two.
+        // Inside a group, warp w reads the tensor-memory lanes of its sub-partition, 32 * (w % 4) ..
+        // + 31, and the two warps with the same w % 4 share 32 query rows, taking 64 of the tile's 128
+        // keys each; they exchange their row maxima through shared memory behind a barrier of those 64
+        // threads.  Every thread writes its probabilities over its own scores.
+        __shared__ float s_xmax[2][2][2][128];            // [use parity][group][half][row]: row maxima of the halves
+        __shared__ float s_xsum[2][2][128];               // epilogue: [group][half][row] row sums
+        __shared__ float s_xref[2][128];                  // epilogue, one row tile: [group][row] reference maxima
+        const int grp = warp >> 3, quad = warp & 3, half = (warp >> 2) & 1;
         const int r_tile = (quad << 5) | lane;            // row inside the tile = tensor-memory lane
         const uint32_t lane_sel = (uint32_t)(quad << 5) << 16;
+        const int t_own = MT == 2 ? grp : 0;              // row tile this group's items belong to
         const int W = (m + 63) >> 6;
-        unsigned long long mlo[MT], mhi[MT];
-#pragma unroll
-        for (int t = 0; t < MT; ++t) {
-            const int r_blk = t * 128 + r_tile;
+        unsigned long long mlo, mhi;
+        {
+            const int r_blk = t_own * 128 + r_tile;
             const int pr = r_blk < rows_here ? row0 + r_blk : rb * plan.per;  // packed row = token * g + head in group
-            mlo[t] = mask_bits[((long long)b * m + pr / g) * W];
-            mhi[t] = W > 1 ? mask_bits[((long long)b * m + pr / g) * W + 1] : 0ull;
+            mlo = mask_bits[((long long)b * m + pr / g) * W];
+            mhi = W > 1 ? mask_bits[((long long)b * m + pr / g) * W + 1] : 0ull;
         }
         if (!plan.q_tma) {
             // query rows into shared memory by hand, 128-byte swizzled (chunk c of row r at
@@ -695,167 +701,170 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
             mbar_arrive(smem_u32(&bars.q_full));
         }
 
-        float m_ref[MT], l_run[MT];
-#pragma unroll
-        for (int t = 0; t < MT; ++t) m_ref[t] = -INFINITY, l_run[t] = 0.f;
+        float m_ref = -INFINITY, l_run = 0.f;
         bool ok = true;
-        const int quad_bar = 2 + quad;  // named barrier of this quad's 128 threads
-        for (int i = 0; i < n_items; ++i) {
-            const int j = i / MT, slot = i % kSlots;
-            const int t = MT == 1 ? 0 : (i & 1);
-            ok = ok && mbar_wait(smem_u32(&bars.s_full[slot]), (uint32_t)((i / kSlots) & 1), abort_flag);
+        const int pair_bar = 2 + grp * 4 + quad;  // named barrier of the two warps that share this thread's rows
+        const uint32_t s_addr = tmem + lane_sel + (uint32_t)grp * kTK + (uint32_t)half * 64;  // this thread's 64 score columns
+        const uint32_t o_acc = tmem + lane_sel + kOCol + (uint32_t)grp * DH;                    // this group's accumulator
+        for (int i = grp; i < n_items; i += 2) {
+            const int u = i >> 1;                          // the u-th use of this group's slot and accumulator
+            const int j = MT == 2 ? u : i;                 // K/V tile of the item
+            ok = ok && mbar_wait(smem_u32(&bars.s_full[grp]), (uint32_t)(u & 1), abort_flag);
             ok = __all_sync(0xffffffffu, ok);  // the tensor-memory accesses below need the whole warp
-            const uint32_t s_addr = tmem + lane_sel + (uint32_t)slot * kTK;
             const int key0 = (t_begin + j) * kTK;
             const bool tail = key0 + kTK > L;  // the tile holds tree keys or runs past the last key
-            uint32_t visw = ~0u;
+            uint32_t vis0 = ~0u, vis1 = ~0u;   // visibility of this thread's keys 0..31 and 32..63
             if (tail) {
                 uint32_t vis[4];
-                tile_visibility(t == 0 ? mlo[0] : mlo[MT - 1], t == 0 ? mhi[0] : mhi[MT - 1], key0, L, n_keys, vis);
-                visw = vis[quarter];
+                tile_visibility(mlo, mhi, key0, L, n_keys, vis);
+                vis0 = half ? vis[2] : vis[0];
+                vis1 = half ? vis[3] : vis[1];
             }
             float mx = -INFINITY;
             if (ok) {
-                // pass 1: the largest raw score of this thread's 32 keys (the scale is positive)
-                uint32_t buf[32];
+                // pass 1: the largest raw score of this thread's 64 keys (the scale is positive)
+                uint32_t ba[32];
                 tc_fence_after();
-                tmem_ld32(s_addr + quarter * 32, buf);
-                tc_wait_ld(buf);
-                mx = tail ? chunk_rowmax<true>(buf, visw, mx) : chunk_rowmax<false>(buf, 0, mx);
-                s_xmax[i & 1][quarter][r_tile] = mx;
+                tmem_ld32(s_addr, ba);
+                tc_wait_ld(ba);
+                mx = tail ? chunk_rowmax<true>(ba, vis0, mx) : chunk_rowmax<false>(ba, 0, mx);
+                tmem_ld32(s_addr + 32, ba);
+                tc_wait_ld(ba);
+                mx = tail ? chunk_rowmax<true>(ba, vis1, mx) : chunk_rowmax<false>(ba, 0, mx);
+                s_xmax[u & 1][grp][half][r_tile] = mx;
             }
-            // the quarters' maxima meet here (or all four warps leave together)
-            ok = named_barrier_and(quad_bar, 128, ok);
+            // the halves' maxima meet here (or both warps leave together)
+            ok = named_barrier_and(pair_bar, 64, ok);
             if (!ok) break;
-#pragma unroll
-            for (int o = 1; o < 4; ++o) mx = fmaxf(mx, s_xmax[i & 1][(quarter + o) & 3][r_tile]);
-            mx *= scale_log2;
+            mx = fmaxf(mx, s_xmax[u & 1][grp][half ^ 1][r_tile]) * scale_log2;
 
-            // lazily rescaled reference maximum: probabilities stay below 2^8 in between.  The four
-            // threads of a row hold the same reference: they derive it from the same four maxima.
-            float mr = t == 0 ? m_ref[0] : m_ref[MT - 1];
-            const float m_new = fmaxf(mr, mx);
-            const bool grow = m_new > mr + 8.f;
+            // lazily rescaled reference maximum: probabilities stay below 2^8 in between.  The two
+            // threads of a row hold the same reference: they derive it from the same two maxima.
+            const float m_new = fmaxf(m_ref, mx);
+            const bool grow = m_new > m_ref + 8.f;
             if (__any_sync(0xffffffffu, grow)) {
-                const float factor = !grow ? 1.f : (mr == -INFINITY ? 0.f : ex2(mr - m_new));
-                if (grow) {
-                    mr = m_new;
-                    if (MT == 1 || t == 0) m_ref[0] = mr, l_run[0] *= factor;
-                    else m_ref[MT - 1] = mr, l_run[MT - 1] *= factor;
-                }
-                // O may be rescaled once the previous P.V of this row tile has finished; this thread
-                // owns a quarter of the row's columns
+                const float factor = !grow ? 1.f : (m_ref == -INFINITY ? 0.f : ex2(m_ref - m_new));
+                if (grow) m_ref = m_new, l_run *= factor;
+                // the accumulator may be rescaled once the group's previous P.V has finished; this
+                // thread owns half of the row's columns
                 bool waited = true;
-                if (j > 0)
-                    waited = mbar_wait(smem_u32(&bars.o_done[t][(j - 1) & 1]), (uint32_t)(((j - 1) >> 1) & 1), abort_flag);
+                if (u > 0)
+                    waited = mbar_wait(smem_u32(&bars.o_done[grp][(u - 1) & 1]), (uint32_t)(((u - 1) >> 1) & 1), abort_flag);
                 waited = __all_sync(0xffffffffu, waited);
-                if (!waited) ok = false;  // the quad learns it at its next barrier
-                if (j > 0 && waited) {
+                if (!waited) ok = false;  // the other warp learns it at the next barrier
+                if (u > 0 && waited) {
                     tc_fence_after();
-                    const uint32_t o_q = tmem + lane_sel + kOCol + (uint32_t)t * DH + (uint32_t)quarter * (DH / 4);
-                    if constexpr (DH == 128) {
+#pragma unroll
+                    for (int c0 = 0; c0 < DH / 2; c0 += 32) {
                         uint32_t orow[32];
-                        tmem_ld32(o_q, orow);
+                        tmem_ld32(o_acc + (uint32_t)half * (DH / 2) + c0, orow);
                         tc_wait_ld(orow);
 #pragma unroll
                         for (int c = 0; c < 32; ++c) orow[c] = __float_as_uint(__uint_as_float(orow[c]) * factor);
-                        tmem_st32(o_q, orow);
-                    } else {
-                        uint32_t orow[16];
-                        tmem_ld16(o_q, orow);
-                        tc_wait_ld16(orow);
-#pragma unroll
-                        for (int c = 0; c < 16; ++c) orow[c] = __float_as_uint(__uint_as_float(orow[c]) * factor);
-                        tmem_st16(o_q, orow);
+                        tmem_st32(o_acc + (uint32_t)half * (DH / 2) + c0, orow);
                     }
                 }
             }
             // pass 2: P = 2^(s * scale - reference) as bf16.  The scores are read again, 16 keys at a
-            // time, and each 16 keys become 8 packed columns written over the thread's own scores
-            // (columns 32 * quarter + 8 * half ..): no thread ever writes a column another one reads.
-            const float neg_ref = mr == -INFINITY ? 0.f : -mr;
+            // time, and each 16 keys become 8 packed columns written over the first half of those 16
+            // score columns: no thread ever writes a column another one reads.
+            const float neg_ref = m_ref == -INFINITY ? 0.f : -m_ref;
             const float2 scale2 = make_float2(scale_log2, scale_log2), neg_ref2 = make_float2(neg_ref, neg_ref);
             float2 sum_a = make_float2(0.f, 0.f), sum_b = make_float2(0.f, 0.f);
-            uint32_t b0[16], b1[16];
-            tmem_ld16(s_addr + quarter * 32, b0);
-            tmem_ld16(s_addr + quarter * 32 + 16, b1);
-            tc_wait_ld16(b0);
-            tc_wait_ld16(b1);
-            {
-                uint32_t pk[8];
-                if (tail) chunk_probs<true, 16>(b0, visw, scale2, neg_ref2, sum_a, sum_b, pk);
+#pragma unroll
+            for (int c2 = 0; c2 < 2; ++c2) {
+                uint32_t b0[16], b1[16], pk[8];
+                tmem_ld16(s_addr + c2 * 32, b0);
+                tmem_ld16(s_addr + c2 * 32 + 16, b1);
+                tc_wait_ld16(b0);
+                tc_wait_ld16(b1);
+                const uint32_t vw = c2 ? vis1 : vis0;
+                if (tail) chunk_probs<true, 16>(b0, vw, scale2, neg_ref2, sum_a, sum_b, pk);
                 else chunk_probs<false, 16>(b0, 0, scale2, neg_ref2, sum_a, sum_b, pk);
-                tmem_st8(s_addr + quarter * 32, pk);
-                if (tail) chunk_probs<true, 16>(b1, visw >> 16, scale2, neg_ref2, sum_a, sum_b, pk);
+                tmem_st8(s_addr + c2 * 32, pk);
+                if (tail) chunk_probs<true, 16>(b1, vw >> 16, scale2, neg_ref2, sum_a, sum_b, pk);
                 else chunk_probs<false, 16>(b1, 0, scale2, neg_ref2, sum_a, sum_b, pk);
-                tmem_st8(s_addr + quarter * 32 + 8, pk);
+                tmem_st8(s_addr + c2 * 32 + 16, pk);
             }
-            const float add = (sum_a.x + sum_a.y) + (sum_b.x + sum_b.y);
-            if (MT == 1 || t == 0) l_run[0] += add;
-            else l_run[MT - 1] += add;
+            l_run += (sum_a.x + sum_a.y) + (sum_b.x + sum_b.y);
             tc_wait_st();
             tc_fence_before();
             __syncwarp();  // every lane's P is in tensor memory: one arrival speaks for the warp
             if (lane == 0) {
-                if (PAIR) mbar_arrive_in(smem_u32(&bars.p_full[slot]), 0);  // the pair's first block issues P.V
-                else mbar_arrive(smem_u32(&bars.p_full[slot]));
+                if (PAIR) mbar_arrive_in(smem_u32(&bars.p_full[grp]), 0);  // the pair's first block issues P.V
+                else mbar_arrive(smem_u32(&bars.p_full[grp]));
             }
         }
 
         // ---- epilogue: O rows leave tensor memory through shared memory, so that the global
         // stores are whole contiguous rows.  Row tile t is staged where its queries were: every
-        // Q.K^T has completed once the last P.V of a row tile has.  All softmax threads first agree
-        // that none of them gave up.
-#pragma unroll
-        for (int t = 0; t < MT; ++t) {
-            ok = ok && mbar_wait(smem_u32(&bars.o_done[t][(nt - 1) & 1]), (uint32_t)(((nt - 1) >> 1) & 1), abort_flag);
-            s_xsum[t][quarter][r_tile] = l_run[t];
-        }
+        // Q.K^T has completed once the last P.V has.  All softmax threads first agree that none of
+        // them gave up.  A group that served no item (a block with a single item) contributes nothing.
+        const int n_uses = (n_items - grp + 1) / 2;  // items this group served
+        if (n_uses > 0)
+            ok = ok && mbar_wait(smem_u32(&bars.o_done[grp][(n_uses - 1) & 1]), (uint32_t)(((n_uses - 1) >> 1) & 1), abort_flag);
+        s_xsum[grp][half][r_tile] = l_run;
+        if (half == 0) s_xref[grp][r_tile] = m_ref;
         ok = named_barrier_and(1, kSoftmaxThreads, ok);
         if (ok) {
             tc_fence_after();
-            constexpr int NCOL = DH / 4;  // columns of O this thread owns
+            constexpr int NCOL = MT == 2 ? DH / 2 : DH / 4;  // columns of an output row this thread produces
             constexpr int row_bytes = DH * 2;
             const int cmask = row_bytes / 16 - 1;
             // a staged row is DH bf16; 16-byte chunk c of row r sits at chunk c ^ (r mod
             // chunks-per-row), which keeps both the row-wise writes and the chunk-wise reads free of
             // bank conflicts
+            const int r_blk = t_own * 128 + r_tile;
+            // One row tile: the two groups hold partial results of the same rows under their own
+            // references; each thread combines a quarter of the row's columns.  Two row tiles: the
+            // group's accumulator is the row tile's result and each thread takes half of the columns.
+            const int col0 = MT == 2 ? half * NCOL : (2 * half + grp) * NCOL;
+            float w_own = 1.f, w_oth = 0.f, l_tot, m_tot = m_ref;
+            if (MT == 2) {
+                l_tot = s_xsum[grp][0][r_tile] + s_xsum[grp][1][r_tile];
+            } else {
+                const float m0 = s_xref[0][r_tile], m1 = s_xref[1][r_tile];
+                m_tot = fmaxf(m0, m1);
+                const float w0 = m0 == -INFINITY ? 0.f : ex2(m0 - m_tot), w1 = m1 == -INFINITY ? 0.f : ex2(m1 - m_tot);
+                l_tot = (s_xsum[0][0][r_tile] + s_xsum[0][1][r_tile]) * w0 + (s_xsum[1][0][r_tile] + s_xsum[1][1][r_tile]) * w1;
+                w_own = grp ? w1 : w0, w_oth = grp ? w0 : w1;
+                if (n_items < 2) w_own = grp ? 0.f : w0, w_oth = grp ? w0 : 0.f;  // accumulator 1 was never written
+            }
+            // final rows are normalised here; a partial stays unnormalised (the merge divides by the
+            // combined sum) and is rounded to bf16 once, like a final row
+            const float inv = !direct ? 1.f : (l_tot > 0.f ? 1.f / l_tot : 0.f);
+            unsigned char* srow = smem_gen + t_own * kTile + (size_t)r_tile * row_bytes;
 #pragma unroll
-            for (int t = 0; t < MT; ++t) {
-                const int r_blk = t * 128 + r_tile;
-                const float l_tot = (s_xsum[t][0][r_tile] + s_xsum[t][1][r_tile]) + (s_xsum[t][2][r_tile] + s_xsum[t][3][r_tile]);
-                // final rows are normalised here; a partial stays unnormalised (the merge divides by the
-                // combined sum) and is rounded to bf16 once, like a final row
-                const float inv = !direct ? 1.f : (l_tot > 0.f ? 1.f / l_tot : 0.f);
-                unsigned char* srow = smem_gen + t * kTile + (size_t)r_tile * row_bytes;
-                const uint32_t o_q = tmem + lane_sel + kOCol + (uint32_t)t * DH + (uint32_t)quarter * NCOL;
-                uint32_t orow[NCOL];
-                if constexpr (DH == 128) {
-                    tmem_ld32(o_q, orow);
-                    tc_wait_ld(orow);
+            for (int c0 = 0; c0 < NCOL; c0 += 16) {
+                uint32_t oa[16], ob[16];
+                tmem_ld16(o_acc + (uint32_t)(col0 + c0), oa);
+                if (MT == 1) tmem_ld16(tmem + lane_sel + kOCol + (uint32_t)(grp ^ 1) * DH + (uint32_t)(col0 + c0), ob);
+                tc_wait_ld16(oa);
+                if (MT == 1) tc_wait_ld16(ob);
+                float v[16];
+#pragma unroll
+                for (int c = 0; c < 16; ++c) {
+                    float x = w_own != 0.f ? __uint_as_float(oa[c]) * w_own : 0.f;
+                    if (MT == 1 && w_oth != 0.f) x += __uint_as_float(ob[c]) * w_oth;
+                    v[c] = MT == 2 ? __uint_as_float(oa[c]) * inv : x * inv;
+                }
+#pragma unroll
+                for (int c = 0; c < 16; c += 8) {
+                    uint4 pkt;
+                    pkt.x = pack_bf16(v[c + 0], v[c + 1]);
+                    pkt.y = pack_bf16(v[c + 2], v[c + 3]);
+                    pkt.z = pack_bf16(v[c + 4], v[c + 5]);
+                    pkt.w = pack_bf16(v[c + 6], v[c + 7]);
+                    const int chunk = (col0 + c0 + c) >> 3;
+                    *reinterpret_cast<uint4*>(srow + (((chunk ^ r_tile) & cmask) << 4)) = pkt;
+                }
+            }
+            if (r_blk < rows_here && half == 0 && (MT == 2 || grp == 0)) {
+                const int pr = row0 + r_blk;
+                if (direct) {
+                    if (lse) lse[((long long)b * Hq + hk * g + pr % g) * m + pr / g] = (m_tot + log2f(l_tot)) * 0.69314718055994531f;
                 } else {
-                    tmem_ld16(o_q, orow);
-                    tc_wait_ld16(orow);
-                }
-#pragma unroll
-                for (int c = 0; c < NCOL; c += 8) {
-                    uint4 v;
-                    v.x = pack_bf16(__uint_as_float(orow[c + 0]) * inv, __uint_as_float(orow[c + 1]) * inv);
-                    v.y = pack_bf16(__uint_as_float(orow[c + 2]) * inv, __uint_as_float(orow[c + 3]) * inv);
-                    v.z = pack_bf16(__uint_as_float(orow[c + 4]) * inv, __uint_as_float(orow[c + 5]) * inv);
-                    v.w = pack_bf16(__uint_as_float(orow[c + 6]) * inv, __uint_as_float(orow[c + 7]) * inv);
-                    const int chunk = (quarter * NCOL + c) >> 3;
-                    *reinterpret_cast<uint4*>(srow + (((chunk ^ r_tile) & cmask) << 4)) = v;
-                }
-                if (r_blk < rows_here && quarter == 0) {
-                    const int pr = row0 + r_blk;
-                    if (direct) {
-                        if (lse)
-                            lse[((long long)b * Hq + hk * g + pr % g) * m + pr / g] =
-                                ((MT == 1 ? m_ref[0] : m_ref[t]) + log2f(l_tot)) * 0.69314718055994531f;
-                    } else {
-                        ws.ml[part_row0 + r_blk] = make_float2(MT == 1 ? m_ref[0] : m_ref[t], l_tot);
-                    }
+                    ws.ml[part_row0 + r_blk] = make_float2(m_tot, l_tot);
                 }
             }
             asm volatile("bar.sync 1, %0;" ::"n"(kSoftmaxThreads) : "memory");  // rows are staged
@@ -877,7 +886,6 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
             }
         }
     }
-
     }  // active
 
     // ---- merging launches: whoever finishes a (sequence, KV head, row block) last combines its splits
