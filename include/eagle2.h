@@ -215,6 +215,12 @@ int eagle2_tree_mask(const int32_t* sel_parent, const int32_t* sel_depth, const 
                      const int32_t* kv_len, int B, int m, uint64_t* mask_bits, uint8_t* mask_dense,
                      int32_t* pos_ids, int32_t* d_status, eagle2_stream_t stream);
 
+/* Kernels one eagle2_tree_attention call launches at these sizes (bookkeeping for benchmarks and
+ * graph builders; 0 for sizes the call would refuse): the attention kernel, a list kernel in front
+ * of it when a ragged batch is served longest first, and a merge kernel behind it when the splits of
+ * a sequence are not combined inside the attention kernel. */
+int eagle2_tree_attention_launches(int B, int m, int Hq, int Hkv, int d, int max_kv_len);
+
 /*
  * Step 3 -- tree-masked attention of the verification pass (paper Section 4.2), one layer per call:
  *   out[b,i,h,:] = sum_j softmax_j(scale * q[b,i,h,:].k[j,h/g,:]) v[j,h/g,:]

@@ -22,7 +22,8 @@ STATUS_TIMEOUT, STATUS_BAD_TREE = 8, 32
 EXPORTS = ("eagle2_version", "eagle2_strerror", "eagle2_workspace_bytes", "eagle2_workspace_init",
            "eagle2_expand", "eagle2_rerank", "eagle2_tree_mask", "eagle2_tree_attention",
            "eagle2_accept", "eagle2_kv_compact", "eagle2_expand_static", "eagle2_expand_variant",
-           "eagle2_rerank_skipped", "eagle2_lm_head", "eagle2_set_wait_limit")
+           "eagle2_rerank_skipped", "eagle2_lm_head", "eagle2_set_wait_limit",
+           "eagle2_tree_attention_launches")
 EXPAND_BY_CONFIDENCE = 1
 
 
@@ -54,6 +55,8 @@ def lib() -> C.CDLL:
         h.eagle2_workspace_bytes.restype = sz
         h.eagle2_workspace_bytes.argtypes = [i32] * 10
         h.eagle2_workspace_init.argtypes = [vp, sz, vp]
+        h.eagle2_tree_attention_launches.restype = i32
+        h.eagle2_tree_attention_launches.argtypes = [i32] * 6
         h.eagle2_set_wait_limit.restype = i64
         h.eagle2_set_wait_limit.argtypes = [i64]
         h.eagle2_expand.argtypes = [vp, i64, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, sz, vp, vp]
@@ -123,6 +126,11 @@ def set_wait_limit(cycles: int) -> int:
     """Bound (SM clock cycles) of the device-side waits of later calls; <= 0 restores the default.
     Returns the bound that was in force."""
     return int(lib().eagle2_set_wait_limit(int(cycles)))
+
+
+def tree_attention_launches(B: int, m: int, Hq: int, Hkv: int, d: int, max_kv_len: int) -> int:
+    """Kernels one ``tree_attention`` call launches at these sizes."""
+    return int(lib().eagle2_tree_attention_launches(B, m, Hq, Hkv, d, max_kv_len))
 
 
 def workspace_init(ws, stream=None) -> None:

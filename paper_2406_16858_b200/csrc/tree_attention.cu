@@ -293,6 +293,7 @@ __device__ __forceinline__ void merge_row(const AttnPlan& plan, const AttnWs& ws
 #pragma unroll
     for (int e = 0; e < PER; ++e) acc[e] = 0.f;
     float l = 0.f, mmax = -INFINITY;
+    // (Every load of a partial goes to L2: other SMs wrote the rows, possibly during this kernel.)
     // W partial rows are fetched before any is used: 16 when the sequence has many splits (one round
     // trip for the batch-1 layer's nine), fewer when it has few, so that short lists do not fetch the
     // same row over and over.  The first batch of rows is requested together with the splits'
@@ -306,26 +307,26 @@ __device__ __forceinline__ void merge_row(const AttnPlan& plan, const AttnWs& ws
                 const int sl = min(s1 + u, n - 1);  // clamped: a repeated row gets weight 0 below
                 const __nv_bfloat16* src = ws.o_part + (first + (size_t)(s0 + sl) * stride) * DH + lane * PER;
                 if (PER == 4) {
-                    const uint2 t = *reinterpret_cast<const uint2*>(src);
+                    const uint2 t = __ldcg(reinterpret_cast<const uint2*>(src));
                     v[u][0] = __uint_as_float(t.x << 16), v[u][1] = __uint_as_float(t.x & 0xffff0000u);
                     v[u][PER - 2] = __uint_as_float(t.y << 16), v[u][PER - 1] = __uint_as_float(t.y & 0xffff0000u);
                 } else {
-                    const uint32_t t = *reinterpret_cast<const uint32_t*>(src);
+                    const uint32_t t = __ldcg(reinterpret_cast<const uint32_t*>(src));
                     v[u][0] = __uint_as_float(t << 16), v[u][1] = __uint_as_float(t & 0xffff0000u);
                 }
             }
         };
         const int n0 = min(32, S_b);
-        const float2 ml0 = lane < n0 ? ws.ml[first + (size_t)lane * stride] : make_float2(-INFINITY, 0.f);
+        const float2 ml0 = lane < n0 ? __ldcg(ws.ml + first + (size_t)lane * stride) : make_float2(-INFINITY, 0.f);
         fetch(0, 0, n0);
         mmax = ml0.x;
         for (int s0 = 32; s0 < S_b; s0 += 32)
-            if (s0 + lane < S_b) mmax = fmaxf(mmax, ws.ml[first + (size_t)(s0 + lane) * stride].x);
+            if (s0 + lane < S_b) mmax = fmaxf(mmax, __ldcg(ws.ml + first + (size_t)(s0 + lane) * stride).x);
         mmax = warp_max_f32(mmax);
         for (int s0 = 0; s0 < S_b; s0 += 32) {
             const int n = min(32, S_b - s0);
             float2 ml = ml0;
-            if (s0) ml = lane < n ? ws.ml[first + (size_t)(s0 + lane) * stride] : make_float2(-INFINITY, 0.f);
+            if (s0) ml = lane < n ? __ldcg(ws.ml + first + (size_t)(s0 + lane) * stride) : make_float2(-INFINITY, 0.f);
             float w = 0.f;  // weight of split s0 + lane
             if (lane < n && ml.x != -INFINITY) w = exp2f(ml.x - mmax), l += ml.y * w;
             for (int s1 = 0; s1 < n; s1 += W) {
@@ -1052,6 +1053,15 @@ static int launch_attention(const CUtensorMap& k_map, const CUtensorMap& v_map, 
 }  // namespace eagle2
 
 using namespace eagle2;
+
+extern "C" int eagle2_tree_attention_launches(int B, int m, int Hq, int Hkv, int d, int max_kv_len) {
+    if (B < 1 || m < 1 || m > EAGLE2_MAX_M || Hq < 1 || Hkv < 1 || Hq % Hkv || Hq / Hkv > 8 || (d != 64 && d != 128) ||
+        max_kv_len < 0)
+        return 0;
+    AttnPlan plan;
+    attention_plan(B, m, Hq, Hkv, d, max_kv_len, &plan);
+    return 1 + (plan.ordered ? 1 : 0) + ((plan.splits > 1 && !plan.fused_merge) ? 1 : 0);
+}
 
 extern "C" int eagle2_tree_attention(const void* q, const void* k_cache, const void* v_cache,
                                      long long cache_rows, const int64_t* kv_off, const int32_t* kv_len,

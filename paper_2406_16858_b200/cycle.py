@@ -105,9 +105,7 @@ class CycleBuffers:
     def launches_per_cycle(self) -> int:
         """Kernel launches of this library in one cycle (for bookkeeping in benchmarks)."""
         s = self.shape
-        attn = e2.workspace_bytes(e2.OP_TREE_ATTENTION, B=s.B, m=s.m, Hq=s.Hq, Hkv=s.Hkv, d=s.d,
-                                  max_kv_len=s.max_kv_len)
-        per_layer = 2 if attn > 0 else 1  # split-KV adds the merge kernel
+        per_layer = e2.tree_attention_launches(s.B, s.m, s.Hq, s.Hkv, s.d, s.max_kv_len)
         return s.D + 2 + s.n_layers * per_layer + (2 if s.temperature > 0 else 1) + 2
 
 
