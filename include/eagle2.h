@@ -67,6 +67,7 @@ typedef struct CUstream_st* eagle2_stream_t; /* a cudaStream_t */
 #define EAGLE2_OP_TREE_ATTENTION 3
 #define EAGLE2_OP_ACCEPT 4
 #define EAGLE2_OP_KV_COMPACT 5
+#define EAGLE2_OP_LM_HEAD_EXPAND 6
 
 int eagle2_version(void);
 const char* eagle2_strerror(int code);
@@ -107,6 +108,29 @@ long long eagle2_set_wait_limit(long long cycles);
  */
 int eagle2_lm_head(const void* hidden, const void* weight, int rows, int H, int V, float* logits,
                    int32_t* d_status, eagle2_stream_t stream);
+
+/*
+ * The LM head and the expansion of one step in one pass over the weights (paper Section 4.1: the
+ * draft features go through the original LLM's LM head, and the expansion keeps every row's k most
+ * probable tokens).  Same result as eagle2_lm_head followed by eagle2_expand on its logits, but the
+ * logits are never written: the kernel that forms them folds them into per-row maxima, sums of
+ * exponentials and k best (value, token) keys, and a merge launch builds the tree level and the
+ * next frontier from those.  Meant for many feature rows (B * k of the order of 100 and more),
+ * where the logits would cost as much traffic as the weights; with few rows the two separate calls
+ * are as fast.
+ *   hidden  bf16 [B][n_s][H] (n_s = 1 at s == 0, else k: the features of frontier slot j of sequence b
+ *           at row b * n_s + j), 16-byte aligned;  weight  bf16 [V][H], 16-byte aligned
+ *   tree_token, tree_parent, tree_value, frontier: as for eagle2_expand (level s + 1 is written,
+ *           frontier is read at s > 0 and overwritten)
+ *   ws      eagle2_workspace_bytes(EAGLE2_OP_LM_HEAD_EXPAND, B, V, k, ...) bytes
+ * Limits: those of eagle2_expand, and k <= 16, H a multiple of 64.  Logits are fp32 sums of bf16
+ * products, as eagle2_lm_head forms them; a row's k-th and (k+1)-th logits closer than that sum's
+ * rounding may come out in either order.  Status bits as for eagle2_expand; a bounded wait that
+ * runs out raises EAGLE2_STATUS_TIMEOUT.
+ */
+int eagle2_lm_head_expand(const void* hidden, const void* weight, int H, int B, int V, int k, int D, int s,
+                          int32_t* tree_token, int32_t* tree_parent, double* tree_value, int32_t* frontier,
+                          void* ws, size_t ws_bytes, int32_t* d_status, eagle2_stream_t stream);
 
 /*
  * Step 1 -- expansion (paper Section 4.1, the value equation V_i = prod c_j over Path(root, t_i)).

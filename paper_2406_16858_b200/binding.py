@@ -15,7 +15,7 @@ import torch
 _PKG = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_PKG, "libeagle2.so")
 
-OP_EXPAND, OP_RERANK, OP_TREE_MASK, OP_TREE_ATTENTION, OP_ACCEPT, OP_KV_COMPACT = range(6)
+OP_EXPAND, OP_RERANK, OP_TREE_MASK, OP_TREE_ATTENTION, OP_ACCEPT, OP_KV_COMPACT, OP_LM_HEAD_EXPAND = range(7)
 STATUS_NONFINITE_LOGIT, STATUS_NOT_CLOSED, STATUS_KV_OVERFLOW = 1, 2, 4
 STATUS_TIMEOUT, STATUS_BAD_TREE = 8, 32
 
@@ -23,7 +23,7 @@ EXPORTS = ("eagle2_version", "eagle2_strerror", "eagle2_workspace_bytes", "eagle
            "eagle2_expand", "eagle2_rerank", "eagle2_tree_mask", "eagle2_tree_attention",
            "eagle2_accept", "eagle2_kv_compact", "eagle2_expand_static", "eagle2_expand_variant",
            "eagle2_rerank_skipped", "eagle2_lm_head", "eagle2_set_wait_limit",
-           "eagle2_tree_attention_launches")
+           "eagle2_tree_attention_launches", "eagle2_lm_head_expand")
 EXPAND_BY_CONFIDENCE = 1
 
 
@@ -55,6 +55,8 @@ def lib() -> C.CDLL:
         h.eagle2_workspace_bytes.restype = sz
         h.eagle2_workspace_bytes.argtypes = [i32] * 10
         h.eagle2_workspace_init.argtypes = [vp, sz, vp]
+        h.eagle2_lm_head_expand.restype = i32
+        h.eagle2_lm_head_expand.argtypes = [vp, vp, i32, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, sz, vp, vp]
         h.eagle2_tree_attention_launches.restype = i32
         h.eagle2_tree_attention_launches.argtypes = [i32] * 6
         h.eagle2_set_wait_limit.restype = i64
@@ -150,6 +152,15 @@ def lm_head(hidden, weight, rows: int, H: int, V: int, logits, d_status, stream=
     """logits fp32 [rows, V] = hidden bf16 [rows, H] . weight bf16 [V, H]^T (the draft logits of ``expand``)."""
     _check("eagle2_lm_head", lib().eagle2_lm_head(_ptr(hidden), _ptr(weight), rows, H, V, _ptr(logits),
                                                   _ptr(d_status), _stream(stream)))
+
+
+def lm_head_expand(hidden, weight, H: int, B: int, V: int, k: int, D: int, s: int, tree_token, tree_parent,
+                   tree_value, frontier, ws, d_status, stream=None) -> None:
+    """``lm_head`` and ``expand`` of one step in one pass over the weights (the logits are never written)."""
+    p, n = _ws(ws)
+    _check("eagle2_lm_head_expand", lib().eagle2_lm_head_expand(
+        _ptr(hidden), _ptr(weight), H, B, V, k, D, s, _ptr(tree_token), _ptr(tree_parent), _ptr(tree_value),
+        _ptr(frontier), p, n, _ptr(d_status), _stream(stream)))
 
 
 def expand_variant(draft_logits, batch_stride: int, B: int, V: int, k: int, D: int, s: int, flags: int,

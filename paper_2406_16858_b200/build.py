@@ -18,7 +18,7 @@ _CSRC = os.path.join(_PKG, "csrc")
 _OBJ = os.path.join(_PKG, "_build")
 LIB_PATH = os.path.join(_PKG, "libeagle2.so")
 
-SOURCES = ["api.cu", "expand.cu", "rerank_mask.cu", "tree_attention.cu", "accept.cu", "kv_compact.cu", "lm_head.cu"]
+SOURCES = ["api.cu", "expand.cu", "rerank_mask.cu", "tree_attention.cu", "accept.cu", "kv_compact.cu", "lm_head.cu", "lm_head_topk.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xptxas", "-v", "-I", os.path.join(_ROOT, "include"), "-I", _CSRC]
 

@@ -13,6 +13,7 @@ long long wait_limit_cycles() {
 size_t expand_workspace_bytes(int B, int V, int k);
 size_t accept_workspace_bytes(int B, int V, int k, int D, int m);
 size_t attention_workspace_bytes(int B, int m, int Hq, int Hkv, int d, int max_kv_len);
+size_t lm_head_expand_workspace_bytes(int B, int V, int k);
 }  // namespace eagle2
 
 extern "C" int eagle2_version(void) { return 100; }
@@ -43,6 +44,9 @@ extern "C" size_t eagle2_workspace_bytes(int op, int B, int V, int k, int D, int
         case EAGLE2_OP_TREE_ATTENTION:
             if (m < 1 || Hq < 1 || Hkv < 1 || Hq % Hkv || (d != 64 && d != 128) || max_kv_len < 0) return 0;
             return eagle2::attention_workspace_bytes(B, m, Hq, Hkv, d, max_kv_len);
+        case EAGLE2_OP_LM_HEAD_EXPAND:
+            if (V < 1 || k < 1 || k > 16) return 0;
+            return eagle2::lm_head_expand_workspace_bytes(B, V, k);
         default:
             return 0;  // rerank, tree mask and KV compaction work in place
     }

@@ -143,6 +143,206 @@ __device__ __forceinline__ unsigned long long warp_bitonic_merge_desc(unsigned l
     return v;
 }
 
+// What the block that arrives last for a sequence does, a warp per row: the rows' log-sum-exp from
+// the segments' statistics (fp64), the k best of the segments' winners, the new tree level (token,
+// parent, value = parent value + log-probability) and the next frontier, ranked by value.  Also the
+// whole of a merge-only launch, whose partials another kernel wrote in the same layout.
+// my_parent / my_parent_value: thread r < n_s holds frontier slot r's node and its value.
+__device__ __forceinline__ void expand_finish(int b, int V, int k, int D, int s, int n_s, int chunks, int by_confidence,
+                                              int my_parent, double my_parent_value, int32_t* __restrict__ tree_token,
+                                              int32_t* __restrict__ tree_parent, double* __restrict__ tree_value,
+                                              int32_t* __restrict__ frontier, const ExpandWs& ws,
+                                              unsigned long long (*s_list)[kWarpList], unsigned long long* s_rank,
+                                              int32_t* d_status) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const long long N = nodes_of(k, D);
+    (void)V;
+    __shared__ int s_parent[EAGLE2_MAX_K];
+    __shared__ double s_pvalue[EAGLE2_MAX_K];
+    const long long base = s ? (long long)k + (long long)(s - 1) * k * k : 0;
+    const int n_new = n_s * k;
+    const int keys_per_row = chunks * k;
+    int32_t* tok = tree_token + (long long)b * N;
+    int32_t* par = tree_parent + (long long)b * N;
+    double* val = tree_value + (long long)b * N;
+    int32_t* fr = frontier + (long long)b * k;
+    if (threadIdx.x < n_s) s_parent[threadIdx.x] = my_parent, s_pvalue[threadIdx.x] = my_parent_value;
+    __syncthreads();
+    int status = 0;
+
+    // A warp merges NR rows at a time, r and r + 8: the work of a row is a chain of dependent
+    // shuffles, so when there are more rows than warps (the ten rows of a step on eight warps) the
+    // second row rides along in the first one's latency instead of taking a second pass.
+    auto merge_rows = [&](auto nr_tag, auto batch_tag) {
+        constexpr int NR = decltype(nr_tag)::value;
+        constexpr int BATCH = decltype(batch_tag)::value;  // chunk winners per lane and pass
+        for (int r_base = warp; r_base < n_s; r_base += kScanWarps * NR) {
+            int r[NR];
+            bool valid[NR];
+            size_t p0[NR];
+            unsigned long long cand[NR][BATCH + 1];
+            double2 st0[NR];
+            int parent[NR];
+            double parent_value[NR], lse[NR];
+            // everything the rows need is requested before any of it is used
+#pragma unroll
+            for (int q = 0; q < NR; ++q) {
+                r[q] = r_base + q * kScanWarps;
+                valid[q] = r[q] < n_s;
+                p0[q] = ((size_t)b * n_s + (valid[q] ? r[q] : 0)) * chunks;
+#pragma unroll
+                for (int t = 0; t < BATCH; ++t)
+                    cand[q][t] = (valid[q] && lane + 32 * t < keys_per_row) ? ws.keys[p0[q] * k + lane + 32 * t] : 0ull;
+                st0[q] = make_double2(-INFINITY, 0.0);
+                if (valid[q] && lane < chunks) st0[q] = ws.stats[p0[q] + lane];
+                parent[q] = (s && valid[q]) ? s_parent[r[q]] : -1;
+                parent_value[q] = (s && valid[q]) ? s_pvalue[r[q]] : 0.0;
+                if (parent[q] < -1) {
+                    status |= EAGLE2_STATUS_BAD_TREE;
+                    parent[q] = (int)(s >= 2 ? (long long)k + (long long)(s - 2) * k * k : 0);
+                }
+            }
+            // log-sum-exp of the rows from the chunk partials, in double
+#pragma unroll
+            for (int q = 0; q < NR; ++q) {
+                double m = st0[q].x;
+                if (valid[q])
+                    for (int c = lane + 32; c < chunks; c += 32) m = fmax(m, ws.stats[p0[q] + c].x);
+                m = warp_max_f64(m);
+                double sum = st0[q].x > -INFINITY ? st0[q].y * exp(st0[q].x - m) : 0.0;
+                if (valid[q])
+                    for (int c = lane + 32; c < chunks; c += 32) {
+                        const double2 st = ws.stats[p0[q] + c];
+                        if (st.x > -INFINITY) sum += st.y * exp(st.x - m);
+                    }
+                sum = warp_sum_f64(sum);
+                if (valid[q] && !(m > -INFINITY)) status |= EAGLE2_STATUS_NONFINITE_LOGIT;
+                lse[q] = m + log(sum);
+            }
+            // top-k of the chunk winners, 32*BATCH at a time together with the best so far; lane c ends
+            // up holding the c-th.  The k-th largest lane maximum is a threshold no winner can be below;
+            // when at most 32 keys reach it (the usual case) they are sorted across the lanes, otherwise
+            // k rounds of maximum extraction do the same job.
+            unsigned long long mine[NR];
+#pragma unroll
+            for (int q = 0; q < NR; ++q) mine[q] = 0ull;
+            for (int e0 = 0; e0 < keys_per_row; e0 += 32 * BATCH) {
+                unsigned long long thr[NR];
+                int cnt[NR], incl[NR], total[NR];
+#pragma unroll
+                for (int q = 0; q < NR; ++q) {
+                    if (e0) {
+#pragma unroll
+                        for (int t = 0; t < BATCH; ++t)
+                            cand[q][t] = (valid[q] && e0 + lane + 32 * t < keys_per_row)
+                                             ? ws.keys[p0[q] * k + e0 + lane + 32 * t]
+                                             : 0ull;
+                    }
+                    cand[q][BATCH] = mine[q];
+                }
+                unsigned long long lane_best[NR];
+#pragma unroll
+                for (int q = 0; q < NR; ++q) {
+                    lane_best[q] = 0;
+#pragma unroll
+                    for (int t = 0; t <= BATCH; ++t) lane_best[q] = cand[q][t] > lane_best[q] ? cand[q][t] : lane_best[q];
+                }
+                warp_sort_desc_u64_n<NR>(lane_best);
+#pragma unroll
+                for (int q = 0; q < NR; ++q) {
+                    thr[q] = __shfl_sync(0xffffffffu, lane_best[q], k - 1);
+                    cnt[q] = 0;
+#pragma unroll
+                    for (int t = 0; t <= BATCH; ++t) cnt[q] += cand[q][t] >= thr[q] && cand[q][t] != 0ull;
+                    incl[q] = cnt[q];
+                }
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+#pragma unroll
+                    for (int q = 0; q < NR; ++q) {
+                        const int up = __shfl_up_sync(0xffffffffu, incl[q], o);
+                        if (lane >= o) incl[q] += up;
+                    }
+                }
+                bool packed = true;
+                unsigned long long next[NR];
+#pragma unroll
+                for (int q = 0; q < NR; ++q) {
+                    total[q] = __shfl_sync(0xffffffffu, incl[q], 31);
+                    packed = packed && total[q] <= 32;
+                    next[q] = 0ull;
+                }
+                if (packed) {  // every row of the warp: pack, then sort the rows side by side
+#pragma unroll
+                    for (int q = 0; q < NR; ++q) {
+                        unsigned long long* s_pack = s_list[warp] + q * 32;  // free: the segment scan is over
+                        int pos = incl[q] - cnt[q];
+#pragma unroll
+                        for (int t = 0; t <= BATCH; ++t)
+                            if (cand[q][t] >= thr[q] && cand[q][t] != 0ull) s_pack[pos++] = cand[q][t];
+                    }
+                    __syncwarp();
+#pragma unroll
+                    for (int q = 0; q < NR; ++q) next[q] = lane < total[q] ? s_list[warp][q * 32 + lane] : 0ull;
+                    warp_sort_desc_u64_n<NR>(next);
+                    __syncwarp();
+#pragma unroll
+                    for (int q = 0; q < NR; ++q)
+                        if (lane >= k) next[q] = 0ull;
+                } else {
+#pragma unroll
+                    for (int q = 0; q < NR; ++q) {
+                        for (int c = 0; c < k; ++c) {
+                            unsigned long long best = 0;
+#pragma unroll
+                            for (int t = 0; t <= BATCH; ++t) best = cand[q][t] > best ? cand[q][t] : best;
+                            const unsigned long long top = warp_max_u64(best);
+#pragma unroll
+                            for (int t = 0; t <= BATCH; ++t) cand[q][t] = (cand[q][t] == top) ? 0ull : cand[q][t];
+                            if (lane == c) next[q] = top;
+                        }
+                    }
+                }
+#pragma unroll
+                for (int q = 0; q < NR; ++q) mine[q] = next[q];
+            }
+#pragma unroll
+            for (int q = 0; q < NR; ++q) {
+                if (valid[q] && lane < k) {
+                    const long long node = base + (long long)r[q] * k + lane;
+                    const double confidence = (double)key_value(mine[q]) - lse[q];  // log c_i
+                    const double v = parent_value[q] + confidence;
+                    tok[node] = (int32_t)key_index(mine[q]);
+                    par[node] = parent[q];
+                    val[node] = v;
+                    // the next frontier is ranked by value, or by confidence alone in the ablation
+                    s_rank[r[q] * k + lane] = order_code_f64(by_confidence ? confidence : v);
+                }
+            }
+        }
+    };
+    if (warp < kScanWarps) {
+        using std::integral_constant;
+        if (n_s > kScanWarps && n_s <= 2 * kScanWarps && keys_per_row <= 32 * 10)
+            merge_rows(integral_constant<int, 2>{}, integral_constant<int, 10>{});
+        else
+            merge_rows(integral_constant<int, 1>{}, integral_constant<int, 16>{});
+    }
+    __syncthreads();  // all rows merged (the old frontier was read when the kernel started)
+
+    // next frontier: rank the new candidates by (value desc, index asc); ranks < k are kept
+    for (int i = threadIdx.x; i < n_new && threadIdx.x < kScanThreads; i += kScanThreads) {
+        const unsigned long long ci = s_rank[i];
+        int rank = 0;
+        for (int j = 0; j < n_new; ++j) {
+            const unsigned long long cj = s_rank[j];
+            rank += (cj > ci) || (cj == ci && j < i);
+        }
+        if (rank < k) fr[rank] = (int32_t)(base + i);
+    }
+    if (status && lane == 0) raise_status(d_status, status);
+}
+
 // Phase 1 has no block-wide barrier inside the streaming loop.  Every streaming warp keeps, per
 // lane, a running (max, sum of exponentials) of the elements it has seen, and filters its elements
 // against a bar: a value that the k-th best element of the segment so far is known to reach, so that
@@ -546,190 +746,53 @@ expand_kernel(const float* __restrict__ draft_logits, long long batch_stride, in
     // ---- the last block of this sequence merges: a warp per row -------------------------------
     if (!last_block_arrives(ws.counters + b, chunks * n_s, &s_flag)) return;
 
-    __shared__ int s_parent[EAGLE2_MAX_K];
-    __shared__ double s_pvalue[EAGLE2_MAX_K];
-    const long long base = s ? (long long)k + (long long)(s - 1) * k * k : 0;
-    const int n_new = n_s * k;
-    const int keys_per_row = chunks * k;
-    int32_t* tok = tree_token + (long long)b * N;
-    int32_t* par = tree_parent + (long long)b * N;
-    double* val = tree_value + (long long)b * N;
-    int32_t* fr = frontier + (long long)b * k;
-    if (threadIdx.x < n_s) s_parent[threadIdx.x] = my_parent, s_pvalue[threadIdx.x] = my_parent_value;
-    __syncthreads();
-    int status = 0;
+    expand_finish(b, V, k, D, s, n_s, chunks, by_confidence, my_parent, my_parent_value, tree_token, tree_parent, tree_value,
+                  frontier, ws, s_list, s_rank, d_status);
+}
 
-    // A warp merges NR rows at a time, r and r + 8: the work of a row is a chain of dependent
-    // shuffles, so when there are more rows than warps (the ten rows of a step on eight warps) the
-    // second row rides along in the first one's latency instead of taking a second pass.
-    auto merge_rows = [&](auto nr_tag, auto batch_tag) {
-        constexpr int NR = decltype(nr_tag)::value;
-        constexpr int BATCH = decltype(batch_tag)::value;  // chunk winners per lane and pass
-        for (int r_base = warp; r_base < n_s; r_base += kScanWarps * NR) {
-            int r[NR];
-            bool valid[NR];
-            size_t p0[NR];
-            unsigned long long cand[NR][BATCH + 1];
-            double2 st0[NR];
-            int parent[NR];
-            double parent_value[NR], lse[NR];
-            // everything the rows need is requested before any of it is used
-#pragma unroll
-            for (int q = 0; q < NR; ++q) {
-                r[q] = r_base + q * kScanWarps;
-                valid[q] = r[q] < n_s;
-                p0[q] = ((size_t)b * n_s + (valid[q] ? r[q] : 0)) * chunks;
-#pragma unroll
-                for (int t = 0; t < BATCH; ++t)
-                    cand[q][t] = (valid[q] && lane + 32 * t < keys_per_row) ? ws.keys[p0[q] * k + lane + 32 * t] : 0ull;
-                st0[q] = make_double2(-INFINITY, 0.0);
-                if (valid[q] && lane < chunks) st0[q] = ws.stats[p0[q] + lane];
-                parent[q] = (s && valid[q]) ? s_parent[r[q]] : -1;
-                parent_value[q] = (s && valid[q]) ? s_pvalue[r[q]] : 0.0;
-                if (parent[q] < -1) {
-                    status |= EAGLE2_STATUS_BAD_TREE;
-                    parent[q] = (int)(s >= 2 ? (long long)k + (long long)(s - 2) * k * k : 0);
-                }
-            }
-            // log-sum-exp of the rows from the chunk partials, in double
-#pragma unroll
-            for (int q = 0; q < NR; ++q) {
-                double m = st0[q].x;
-                if (valid[q])
-                    for (int c = lane + 32; c < chunks; c += 32) m = fmax(m, ws.stats[p0[q] + c].x);
-                m = warp_max_f64(m);
-                double sum = st0[q].x > -INFINITY ? st0[q].y * exp(st0[q].x - m) : 0.0;
-                if (valid[q])
-                    for (int c = lane + 32; c < chunks; c += 32) {
-                        const double2 st = ws.stats[p0[q] + c];
-                        if (st.x > -INFINITY) sum += st.y * exp(st.x - m);
-                    }
-                sum = warp_sum_f64(sum);
-                if (valid[q] && !(m > -INFINITY)) status |= EAGLE2_STATUS_NONFINITE_LOGIT;
-                lse[q] = m + log(sum);
-            }
-            // top-k of the chunk winners, 32*BATCH at a time together with the best so far; lane c ends
-            // up holding the c-th.  The k-th largest lane maximum is a threshold no winner can be below;
-            // when at most 32 keys reach it (the usual case) they are sorted across the lanes, otherwise
-            // k rounds of maximum extraction do the same job.
-            unsigned long long mine[NR];
-#pragma unroll
-            for (int q = 0; q < NR; ++q) mine[q] = 0ull;
-            for (int e0 = 0; e0 < keys_per_row; e0 += 32 * BATCH) {
-                unsigned long long thr[NR];
-                int cnt[NR], incl[NR], total[NR];
-#pragma unroll
-                for (int q = 0; q < NR; ++q) {
-                    if (e0) {
-#pragma unroll
-                        for (int t = 0; t < BATCH; ++t)
-                            cand[q][t] = (valid[q] && e0 + lane + 32 * t < keys_per_row)
-                                             ? ws.keys[p0[q] * k + e0 + lane + 32 * t]
-                                             : 0ull;
-                    }
-                    cand[q][BATCH] = mine[q];
-                }
-                unsigned long long lane_best[NR];
-#pragma unroll
-                for (int q = 0; q < NR; ++q) {
-                    lane_best[q] = 0;
-#pragma unroll
-                    for (int t = 0; t <= BATCH; ++t) lane_best[q] = cand[q][t] > lane_best[q] ? cand[q][t] : lane_best[q];
-                }
-                warp_sort_desc_u64_n<NR>(lane_best);
-#pragma unroll
-                for (int q = 0; q < NR; ++q) {
-                    thr[q] = __shfl_sync(0xffffffffu, lane_best[q], k - 1);
-                    cnt[q] = 0;
-#pragma unroll
-                    for (int t = 0; t <= BATCH; ++t) cnt[q] += cand[q][t] >= thr[q] && cand[q][t] != 0ull;
-                    incl[q] = cnt[q];
-                }
-#pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-#pragma unroll
-                    for (int q = 0; q < NR; ++q) {
-                        const int up = __shfl_up_sync(0xffffffffu, incl[q], o);
-                        if (lane >= o) incl[q] += up;
-                    }
-                }
-                bool packed = true;
-                unsigned long long next[NR];
-#pragma unroll
-                for (int q = 0; q < NR; ++q) {
-                    total[q] = __shfl_sync(0xffffffffu, incl[q], 31);
-                    packed = packed && total[q] <= 32;
-                    next[q] = 0ull;
-                }
-                if (packed) {  // every row of the warp: pack, then sort the rows side by side
-#pragma unroll
-                    for (int q = 0; q < NR; ++q) {
-                        unsigned long long* s_pack = s_list[warp] + q * 32;  // free: the segment scan is over
-                        int pos = incl[q] - cnt[q];
-#pragma unroll
-                        for (int t = 0; t <= BATCH; ++t)
-                            if (cand[q][t] >= thr[q] && cand[q][t] != 0ull) s_pack[pos++] = cand[q][t];
-                    }
-                    __syncwarp();
-#pragma unroll
-                    for (int q = 0; q < NR; ++q) next[q] = lane < total[q] ? s_list[warp][q * 32 + lane] : 0ull;
-                    warp_sort_desc_u64_n<NR>(next);
-                    __syncwarp();
-#pragma unroll
-                    for (int q = 0; q < NR; ++q)
-                        if (lane >= k) next[q] = 0ull;
-                } else {
-#pragma unroll
-                    for (int q = 0; q < NR; ++q) {
-                        for (int c = 0; c < k; ++c) {
-                            unsigned long long best = 0;
-#pragma unroll
-                            for (int t = 0; t <= BATCH; ++t) best = cand[q][t] > best ? cand[q][t] : best;
-                            const unsigned long long top = warp_max_u64(best);
-#pragma unroll
-                            for (int t = 0; t <= BATCH; ++t) cand[q][t] = (cand[q][t] == top) ? 0ull : cand[q][t];
-                            if (lane == c) next[q] = top;
-                        }
-                    }
-                }
-#pragma unroll
-                for (int q = 0; q < NR; ++q) mine[q] = next[q];
-            }
-#pragma unroll
-            for (int q = 0; q < NR; ++q) {
-                if (valid[q] && lane < k) {
-                    const long long node = base + (long long)r[q] * k + lane;
-                    const double confidence = (double)key_value(mine[q]) - lse[q];  // log c_i
-                    const double v = parent_value[q] + confidence;
-                    tok[node] = (int32_t)key_index(mine[q]);
-                    par[node] = parent[q];
-                    val[node] = v;
-                    // the next frontier is ranked by value, or by confidence alone in the ablation
-                    s_rank[r[q] * k + lane] = order_code_f64(by_confidence ? confidence : v);
-                }
-            }
-        }
-    };
-    if (warp < kScanWarps) {
-        using std::integral_constant;
-        if (n_s > kScanWarps && n_s <= 2 * kScanWarps && keys_per_row <= 32 * 10)
-            merge_rows(integral_constant<int, 2>{}, integral_constant<int, 10>{});
-        else
-            merge_rows(integral_constant<int, 1>{}, integral_constant<int, 16>{});
+// Merge-only launch: one block per sequence finishes a step whose per-row partials (statistics and k
+// best keys per producer, in this file's workspace layout with `chunks` producers per row) were
+// written by another kernel - the LM head that ranks its own logits.
+__global__ void __launch_bounds__(kScanThreads)
+expand_merge_kernel(int V, int k, int D, int s, int n_s, int chunks, int by_confidence, int32_t* __restrict__ tree_token,
+                    int32_t* __restrict__ tree_parent, double* __restrict__ tree_value,
+                    int32_t* __restrict__ frontier, ExpandWs ws, int32_t* d_status) {
+    __shared__ unsigned long long s_list[kScanWarps][kWarpList];
+    __shared__ unsigned long long s_rank[EAGLE2_MAX_K * EAGLE2_MAX_K];
+    chain_wait();
+    chain_release();
+    const int b = blockIdx.x;
+    const long long N = nodes_of(k, D);
+    int my_parent = -1;
+    double my_parent_value = 0.0;
+    if (s && threadIdx.x < n_s) {
+        my_parent = frontier[(long long)b * k + threadIdx.x];
+        const long long prev_base = s >= 2 ? (long long)k + (long long)(s - 2) * k * k : 0;
+        const long long prev_count = s >= 2 ? (long long)k * k : k;
+        if (my_parent < prev_base || my_parent >= prev_base + prev_count) my_parent = -2;  // reported by the merger
+        else my_parent_value = tree_value[(long long)b * N + my_parent];
     }
-    __syncthreads();  // all rows merged (the old frontier was read when the kernel started)
+    expand_finish(b, V, k, D, s, n_s, chunks, by_confidence, my_parent, my_parent_value, tree_token, tree_parent, tree_value,
+                  frontier, ws, s_list, s_rank, d_status);
+}
 
-    // next frontier: rank the new candidates by (value desc, index asc); ranks < k are kept
-    for (int i = threadIdx.x; i < n_new && threadIdx.x < kScanThreads; i += kScanThreads) {
-        const unsigned long long ci = s_rank[i];
-        int rank = 0;
-        for (int j = 0; j < n_new; ++j) {
-            const unsigned long long cj = s_rank[j];
-            rank += (cj > ci) || (cj == ci && j < i);
-        }
-        if (rank < k) fr[rank] = (int32_t)(base + i);
-    }
-    if (status && lane == 0) raise_status(d_status, status);
+// For the kernels of other files that write such partials: where they go in a workspace, how much of
+// it they need, and the launch that finishes the step from them.
+size_t expand_partials_bytes(int B, int n_s, int chunks, int k) { return expand_ws_layout(B, n_s, chunks, k, nullptr, nullptr); }
+bool expand_partials_layout(int B, int n_s, int chunks, int k, void* ws, size_t ws_bytes, double2** stats,
+                            unsigned long long** keys) {
+    ExpandWs w;
+    if (expand_ws_layout(B, n_s, chunks, k, ws, &w) > ws_bytes) return false;
+    *stats = w.stats, *keys = w.keys;
+    return true;
+}
+int launch_expand_merge(int B, int V, int k, int D, int s, int chunks, int32_t* tree_token, int32_t* tree_parent,
+                        double* tree_value, int32_t* frontier, void* ws, int32_t* d_status, cudaStream_t stream) {
+    const int n_s = s ? k : 1;
+    ExpandWs w;
+    expand_ws_layout(B, n_s, chunks, k, ws, &w);
+    return launch_chained(expand_merge_kernel, dim3((unsigned)B), dim3(kScanThreads), 0, stream, 1, V, k, D, s, n_s, chunks,
+                          0, tree_token, tree_parent, tree_value, frontier, w, d_status);
 }
 
 template <bool VEC, bool STREAM>

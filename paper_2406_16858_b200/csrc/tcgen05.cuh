@@ -234,8 +234,13 @@ __device__ __forceinline__ void mma2_ts(uint32_t d_tmem, uint32_t a_tmem, uint64
 // CG: 1 or 2 blocks per instruction; ACC: 0 overwrite D, 1 accumulate.
 template <int CG, int ACC>
 __device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
-                                        uint32_t idesc) {
-    if constexpr (CG == 1) {
+                                        uint32_t idesc, uint32_t acc = 1) {
+    if constexpr (ACC == 2) {  // accumulate iff `acc` != 0 (a run-time flag); one block per instruction only
+        static_assert(CG == 1 || ACC != 2, "run-time accumulate flag: single-block form only");
+        asm volatile("{\n\t.reg .b64 da, db;\n\t.reg .pred p;\n\tsetp.ne.b32 p, %6, 0;\n\tmov.b64 da, {%1, %2};\n\tmov.b64 db, {%3, %4};\n\t"
+                     "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n\t}"
+                     ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(acc) : "memory");
+    } else if constexpr (CG == 1) {
         if constexpr (ACC == 0)
             asm volatile("{\n\t.reg .b64 da, db;\n\tmov.b64 da, {%1, %2};\n\tmov.b64 db, {%3, %4};\n\t"
                          "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, 0;\n\t}"
