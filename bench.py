@@ -449,6 +449,64 @@ def lm_head_extra(e2, dev, stream, hbm_peak, reps=30):
     return out
 
 
+def lm_head_fused_extra(e2, dev, stream, hbm_peak, reps=10):
+    """The LM head in front of a batched expansion step at the llama3_8b shape, 16 and 32 sequences
+    (160 and 320 feature rows): the two chained calls (logits written, then ranked) against the fused
+    call that never writes them.  Algorithmic bytes of the fused step: the weight matrix once per
+    256 rows."""
+    import torch
+    cfg = get_config("llama3_8b")
+    H, V, k, D = 4096, cfg.V, cfg.k, cfg.D
+    g = torch.Generator(device=dev).manual_seed(6)
+    weight = (torch.randn((V, H), generator=g, device=dev) * (2.0 / math.sqrt(H))).to(torch.bfloat16)
+    out = []
+    for B in (16, 32):
+        rows = B * k
+        hidden = torch.randn((rows, H), generator=g, device=dev).to(torch.bfloat16)
+        logits = torch.zeros((rows, V), dtype=torch.float32, device=dev)
+        N = k + (D - 1) * k * k
+        token = torch.zeros((B, N), dtype=torch.int32, device=dev)
+        parent = torch.zeros((B, N), dtype=torch.int32, device=dev)
+        value = torch.zeros((B, N), dtype=torch.float64, device=dev)
+        frontier0 = torch.arange(k, dtype=torch.int32, device=dev).repeat(B, 1).contiguous()
+        frontier = frontier0.clone()
+        status = torch.zeros(1, dtype=torch.int32, device=dev)
+        ws = torch.empty(max(e2.workspace_bytes(e2.OP_EXPAND, B=B, V=V, k=k, D=D),
+                             e2.workspace_bytes(e2.OP_LM_HEAD_EXPAND, B=B, V=V, k=k, D=D), 256), dtype=torch.uint8, device=dev)
+        e2.workspace_init(ws)
+        torch.cuda.synchronize()
+        res = {"B": B, "rows": rows}
+        for name in ("chained", "fused"):
+            def calls():
+                frontier.copy_(frontier0)  # every call expands the same level
+                if name == "chained":
+                    e2.lm_head(hidden, weight, rows, H, V, logits, status)
+                    e2.expand(logits, k * V, B, V, k, D, 1, token, parent, value, frontier, ws, status)
+                else:
+                    e2.lm_head_expand(hidden, weight, H, B, V, k, D, 1, token, parent, value, frontier, ws, status)
+            with torch.cuda.stream(stream):
+                for _ in range(2):
+                    calls()
+                stream.synchronize()
+                ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                ev0.record(stream)
+                for _ in range(reps):
+                    calls()
+                ev1.record(stream)
+            torch.cuda.synchronize()
+            res[name + "_us"] = ev0.elapsed_time(ev1) * 1e3 / reps
+        assert int(status.item()) == 0
+        passes = (rows + 255) // 256
+        nbytes = 2.0 * V * H * passes + 2.0 * rows * H
+        res.update({"fused_algorithmic_bytes": nbytes, "fused_achieved_gbs": nbytes / (res["fused_us"] * 1e-6) / 1e9,
+                    "fused_frac_of_measured_hbm": nbytes / (res["fused_us"] * 1e-6) / 1e9 / hbm_peak,
+                    "chained_logit_bytes_written_and_read": 8.0 * rows * V,
+                    "fused_tflops": 2.0 * rows * V * H / (res["fused_us"] * 1e-6) / 1e12})
+        out.append(res)
+        del hidden, logits, ws
+    return {"workload": f"llama3_8b-shaped LM head ({H} -> {V}) + expansion step 1, bf16 weights {2.0 * V * H / 1e9:.2f} GB", "cases": out}
+
+
 def run_ours(args):
     import torch
 
@@ -473,7 +531,8 @@ def run_ours(args):
                           "expand_batched": batched_expand_extra(e2, dev, stream, hbm_peak),
                           "accept_batched": batched_accept_extra(e2, dev, stream, hbm_peak),
                           "draft_attention": draft_attention_extra(e2, dev, stream, hbm_peak),
-                          "lm_head": lm_head_extra(e2, dev, stream, hbm_peak)}))
+                          "lm_head": lm_head_extra(e2, dev, stream, hbm_peak),
+                          "lm_head_fused": lm_head_fused_extra(e2, dev, stream, hbm_peak)}))
         return
     cfg = get_config(args.workload)
     if args.batch:
@@ -803,6 +862,7 @@ def run_ours(args):
         line["accept_batched_b32"] = batched_accept_extra(e2, dev, stream, hbm_peak, B=32)
         line["draft_attention"] = draft_attention_extra(e2, dev, stream, hbm_peak)
         line["lm_head"] = lm_head_extra(e2, dev, stream, hbm_peak)
+        line["lm_head_fused"] = lm_head_fused_extra(e2, dev, stream, hbm_peak)
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

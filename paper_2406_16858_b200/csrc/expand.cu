@@ -776,6 +776,83 @@ expand_merge_kernel(int V, int k, int D, int s, int n_s, int chunks, int by_conf
                   frontier, ws, s_list, s_rank, d_status);
 }
 
+// Row-merge launch: one block per row folds the row's `chunks` partials into a single one (the same
+// statistics and k best keys a lone producer would have written).  With a partial per SM a row has
+// a few thousand keys, and a step's rows are independent: merging them side by side, a block each,
+// leaves the per-sequence launch above only k keys per row.  Keys of a row are distinct (a token is
+// ranked by exactly one producer) except for the empty slots, which hold 0.
+constexpr int kRowMergeMaxKeysPerThread = 16;
+__global__ void __launch_bounds__(kScanThreads)
+expand_row_merge_kernel(int chunks, int k, const double2* __restrict__ stats_in,
+                        const unsigned long long* __restrict__ keys_in, double2* __restrict__ stats_out,
+                        unsigned long long* __restrict__ keys_out) {
+    __shared__ unsigned long long s_top[kScanWarps * EAGLE2_MAX_K];  // every warp's k largest thread maxima
+    __shared__ unsigned long long s_cand[kScanThreads];
+    __shared__ unsigned long long s_thr;
+    __shared__ int s_n;
+    chain_wait();
+    chain_release();
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const size_t row = blockIdx.x;
+    const int n = chunks * k;
+    const unsigned long long* kin = keys_in + row * (size_t)n;
+    unsigned long long mine[kRowMergeMaxKeysPerThread];
+    unsigned long long mx[1] = {0ull};
+#pragma unroll
+    for (int t = 0; t < kRowMergeMaxKeysPerThread; ++t) {
+        const int i = tid + t * kScanThreads;
+        mine[t] = i < n ? kin[i] : 0ull;
+        mx[0] = mine[t] > mx[0] ? mine[t] : mx[0];
+    }
+    if (tid == 0) s_n = 0, s_thr = 0ull;
+    // The k-th largest of the threads' maxima is reached by at least k keys, and only the k threads
+    // whose maximum reaches it can hold such keys: at most k * keys-per-thread candidates.
+    warp_sort_desc_u64_n<1>(mx);
+    if (lane < k) s_top[warp * k + lane] = mx[0];
+    __syncthreads();
+    if (tid < kScanWarps * k) {
+        const unsigned long long v = s_top[tid];
+        int above = 0;
+        for (int j = 0; j < kScanWarps * k; ++j) {
+            const unsigned long long w = s_top[j];
+            above += (w > v) || (w == v && j < tid);
+        }
+        if (above == k - 1) s_thr = v;  // 0 when the row has fewer than k keys: every key is kept
+    }
+    // the row's log-sum-exp statistics from its partials, in double (one warp)
+    if (warp == kScanWarps - 1) {
+        const double2* sin = stats_in + row * (size_t)chunks;
+        double m = -INFINITY;
+        for (int c = lane; c < chunks; c += 32) m = fmax(m, sin[c].x);
+        m = warp_max_f64(m);
+        double sum = 0.0;
+        for (int c = lane; c < chunks; c += 32) {
+            const double2 st = sin[c];
+            if (st.x > -INFINITY) sum += st.y * exp(st.x - m);
+        }
+        sum = warp_sum_f64(sum);
+        if (lane == 0) stats_out[row] = make_double2(m, sum);
+    }
+    __syncthreads();
+    const unsigned long long thr = s_thr;
+#pragma unroll
+    for (int t = 0; t < kRowMergeMaxKeysPerThread; ++t) {
+        if (mine[t] != 0ull && mine[t] >= thr) {
+            const int pos = atomicAdd(&s_n, 1);
+            if (pos < kScanThreads) s_cand[pos] = mine[t];
+        }
+    }
+    __syncthreads();
+    const int nc = min(s_n, kScanThreads);
+    if (tid < nc) {
+        const unsigned long long v = s_cand[tid];
+        int above = 0;
+        for (int j = 0; j < nc; ++j) above += s_cand[j] > v;
+        if (above < k) keys_out[row * k + above] = v;
+    }
+    if (tid >= nc && tid < k) keys_out[row * k + tid] = 0ull;
+}
+
 // For the kernels of other files that write such partials: where they go in a workspace, how much of
 // it they need, and the launch that finishes the step from them.
 size_t expand_partials_bytes(int B, int n_s, int chunks, int k) { return expand_ws_layout(B, n_s, chunks, k, nullptr, nullptr); }
@@ -793,6 +870,19 @@ int launch_expand_merge(int B, int V, int k, int D, int s, int chunks, int32_t* 
     expand_ws_layout(B, n_s, chunks, k, ws, &w);
     return launch_chained(expand_merge_kernel, dim3((unsigned)B), dim3(kScanThreads), 0, stream, 1, V, k, D, s, n_s, chunks,
                           0, tree_token, tree_parent, tree_value, frontier, w, d_status);
+}
+
+// Folds every row's partials (in `ws`, `chunks` per row) into one per row, written in the same layout
+// with one producer per row into `ws_rows`.  Refuses more keys per row than the row-merge block holds.
+int launch_expand_row_merge(int B, int n_s, int chunks, int k, void* ws, void* ws_rows, cudaStream_t stream) {
+    if ((long long)chunks * k > (long long)kRowMergeMaxKeysPerThread * kScanThreads ||
+        (long long)k * ((chunks * k + kScanThreads - 1) / kScanThreads) > kScanThreads)
+        return EAGLE2_ERR_SHAPE;
+    ExpandWs in, out;
+    expand_ws_layout(B, n_s, chunks, k, ws, &in);
+    expand_ws_layout(B, n_s, 1, k, ws_rows, &out);
+    return launch_chained(expand_row_merge_kernel, dim3((unsigned)(B * n_s)), dim3(kScanThreads), 0, stream, 1, chunks, k,
+                          in.stats, in.keys, out.stats, out.keys);
 }
 
 template <bool VEC, bool STREAM>

@@ -82,6 +82,27 @@ def test_fused_tree_against_the_oracle_pipeline(B, k, D, H, V):
     assert exempt <= max(2, checked)
 
 
+def test_full_vocabulary_of_the_llama3_shape():
+    """The whole 128256-entry vocabulary (501 tiles over 148 blocks, 1480 keys per row for the merge)
+    with 160 rows; the hidden size is kept small so that the oracle's LM head stays within seconds."""
+    B, k, D, H, V = 16, 10, 2, 128, 128256
+    R = 1 + (D - 1) * k
+    hb, wb = gen.lm_head_inputs(B * R, H, V, seed=77)
+    want_logits = ref.lm_head(hb, wb).reshape(B, R, V)
+    tree = ref.build_tree(want_logits.astype(np.float32), V, k, D)
+    tok, par, val, fr, st = _device_tree(hb.reshape(B, R, H), wb, B, V, k, D, H)
+    assert st == 0
+    checked = 0
+    for b in range(B):
+        if _decided_by_rounding(want_logits, tree, b, k, D):
+            continue
+        checked += 1
+        assert (tok[b] == tree.token[b]).all() and (par[b] == tree.parent[b]).all()
+        assert np.abs(val[b] - tree.value[b]).max() < 1e-3
+        assert (fr[b] == tree.frontier[b]).all()
+    assert checked >= B // 2
+
+
 def test_fused_equals_the_two_separate_calls():
     """The same features through ``lm_head`` + ``expand``: identical tokens, parents and frontier
     wherever the separate path's own fp32 logits leave no near-tie."""

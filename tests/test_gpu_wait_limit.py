@@ -100,6 +100,41 @@ def test_lm_head_gives_up_and_recovers(short_wait):
     assert (np.abs(host(out) - want) <= (H / 16 + 16) * 2.0 ** -23 * S + 1e-30).all()
 
 
+def test_fused_lm_head_gives_up_and_recovers(short_wait):
+    B, k, D, H, V = 16, 10, 2, 128, 40000  # 160 rows; more vocabulary tiles than blocks
+    hb, wb = gen.lm_head_inputs(B * k, H, V, seed=9)
+    th, tw = dev(hb), dev(wb)
+    N = k + (D - 1) * k * k
+    token = torch.full((B, N), -1, dtype=torch.int32, device=DEV)
+    parent = torch.full((B, N), -2, dtype=torch.int32, device=DEV)
+    value = torch.full((B, N), float("-inf"), dtype=torch.float64, device=DEV)
+    frontier = torch.arange(k, dtype=torch.int32, device=DEV).repeat(B, 1).contiguous()
+    value[:, :k] = 0.0  # level 1 as if already built: every parent has value log 1
+    ws = make_ws(e2.workspace_bytes(e2.OP_LM_HEAD_EXPAND, B=B, V=V, k=k, D=D))
+
+    def call():
+        st = new_status()
+        fr = frontier.clone()
+        e2.lm_head_expand(th, tw, H, B, V, k, D, 1, token, parent, value, fr, ws, st)
+        torch.cuda.synchronize()
+        return int(st.item()), fr
+
+    assert call()[0] & e2.STATUS_TIMEOUT
+    assert call()[0] & e2.STATUS_TIMEOUT
+    e2.set_wait_limit(0)
+    status, fr = call()
+    assert status == 0
+    # level 2 of every sequence: the k best tokens of each of its k rows (the oracle's LM head)
+    want_logits = ref.lm_head(hb, wb).reshape(B, k, V)
+    got = host(token)[:, k:k + k * k].reshape(B, k, k)
+    for b in range(B):
+        for r in range(k):
+            top = -np.sort(-want_logits[b, r])[:k + 1]
+            if (np.diff(-top) < 1e-4).any():
+                continue
+            assert (got[b, r] == np.argsort(-want_logits[b, r], kind="stable")[:k]).all()
+
+
 def test_streaming_expansion_gives_up_and_recovers(short_wait):
     V, k, D, B = 70004, 5, 2, 32  # 160 rows at the second step: several tiles per block, selector warp
     rng = np.random.default_rng(8)
