@@ -783,9 +783,9 @@ expand_merge_kernel(int V, int k, int D, int s, int n_s, int chunks, int by_conf
 // ranked by exactly one producer) except for the empty slots, which hold 0.
 constexpr int kRowMergeMaxKeysPerThread = 16;
 __global__ void __launch_bounds__(kScanThreads)
-expand_row_merge_kernel(int chunks, int k, const double2* __restrict__ stats_in,
-                        const unsigned long long* __restrict__ keys_in, double2* __restrict__ stats_out,
-                        unsigned long long* __restrict__ keys_out) {
+expand_row_merge_kernel(int slots, int split_row, int chunks_lo, int chunks_hi, int k,
+                        const double2* __restrict__ stats_in, const unsigned long long* __restrict__ keys_in,
+                        double2* __restrict__ stats_out, unsigned long long* __restrict__ keys_out) {
     __shared__ unsigned long long s_top[kScanWarps * EAGLE2_MAX_K];  // every warp's k largest thread maxima
     __shared__ unsigned long long s_cand[kScanThreads];
     __shared__ unsigned long long s_thr;
@@ -794,8 +794,9 @@ expand_row_merge_kernel(int chunks, int k, const double2* __restrict__ stats_in,
     chain_release();
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const size_t row = blockIdx.x;
+    const int chunks = (int)row < split_row ? chunks_lo : chunks_hi;  // producers that wrote this row
     const int n = chunks * k;
-    const unsigned long long* kin = keys_in + row * (size_t)n;
+    const unsigned long long* kin = keys_in + row * (size_t)slots * k;
     unsigned long long mine[kRowMergeMaxKeysPerThread];
     unsigned long long mx[1] = {0ull};
 #pragma unroll
@@ -821,7 +822,7 @@ expand_row_merge_kernel(int chunks, int k, const double2* __restrict__ stats_in,
     }
     // the row's log-sum-exp statistics from its partials, in double (one warp)
     if (warp == kScanWarps - 1) {
-        const double2* sin = stats_in + row * (size_t)chunks;
+        const double2* sin = stats_in + row * (size_t)slots;
         double m = -INFINITY;
         for (int c = lane; c < chunks; c += 32) m = fmax(m, sin[c].x);
         m = warp_max_f64(m);
@@ -872,17 +873,23 @@ int launch_expand_merge(int B, int V, int k, int D, int s, int chunks, int32_t* 
                           0, tree_token, tree_parent, tree_value, frontier, w, d_status);
 }
 
-// Folds every row's partials (in `ws`, `chunks` per row) into one per row, written in the same layout
-// with one producer per row into `ws_rows`.  Refuses more keys per row than the row-merge block holds.
-int launch_expand_row_merge(int B, int n_s, int chunks, int k, void* ws, void* ws_rows, cudaStream_t stream) {
-    if ((long long)chunks * k > (long long)kRowMergeMaxKeysPerThread * kScanThreads ||
-        (long long)k * ((chunks * k + kScanThreads - 1) / kScanThreads) > kScanThreads)
+// Folds every row's partials into one per row, written in the same layout with one producer per row
+// into `ws_rows`.  `ws` holds `slots` partial places per row, of which the first chunks_lo are filled
+// for the rows below split_row and the first chunks_hi for the others (passes over the rows may use
+// different numbers of producers).  Refuses more keys per row than the row-merge block holds.
+int launch_expand_row_merge(int B, int n_s, int slots, long long split_row, int chunks_lo, int chunks_hi, int k, void* ws,
+                            void* ws_rows, cudaStream_t stream) {
+    const int most = chunks_lo > chunks_hi ? chunks_lo : chunks_hi;
+    if (most > slots || (long long)most * k > (long long)kRowMergeMaxKeysPerThread * kScanThreads ||
+        (long long)k * ((most * k + kScanThreads - 1) / kScanThreads) > kScanThreads)
         return EAGLE2_ERR_SHAPE;
     ExpandWs in, out;
-    expand_ws_layout(B, n_s, chunks, k, ws, &in);
+    expand_ws_layout(B, n_s, slots, k, ws, &in);
     expand_ws_layout(B, n_s, 1, k, ws_rows, &out);
-    return launch_chained(expand_row_merge_kernel, dim3((unsigned)(B * n_s)), dim3(kScanThreads), 0, stream, 1, chunks, k,
-                          in.stats, in.keys, out.stats, out.keys);
+    const long long rows = (long long)B * n_s;
+    return launch_chained(expand_row_merge_kernel, dim3((unsigned)rows), dim3(kScanThreads), 0, stream, 1, slots,
+                          (int)(split_row < rows ? split_row : rows), chunks_lo, chunks_hi, k, in.stats, in.keys, out.stats,
+                          out.keys);
 }
 
 template <bool VEC, bool STREAM>

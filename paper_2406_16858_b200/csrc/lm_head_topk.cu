@@ -36,7 +36,8 @@ bool expand_partials_layout(int B, int n_s, int chunks, int k, void* ws, size_t 
                             unsigned long long** keys);
 int launch_expand_merge(int B, int V, int k, int D, int s, int chunks, int32_t* tree_token, int32_t* tree_parent,
                         double* tree_value, int32_t* frontier, void* ws, int32_t* d_status, cudaStream_t stream);
-int launch_expand_row_merge(int B, int n_s, int chunks, int k, void* ws, void* ws_rows, cudaStream_t stream);
+int launch_expand_row_merge(int B, int n_s, int slots, long long split_row, int chunks_lo, int chunks_hi, int k, void* ws,
+                            void* ws_rows, cudaStream_t stream);
 
 constexpr int kFzThreads = 64 + 256;  // TMA warp, MMA warp, eight epilogue warps
 constexpr int kFzTileV = 256;         // vocabulary entries per tile = N of the instruction
@@ -80,12 +81,12 @@ __device__ __forceinline__ unsigned long long fz_insert(unsigned long long (&lis
 }
 
 // rows: feature rows of this pass (<= 128, pair: <= 256); row0: first of them among all rows of the
-// call; chunks: partials per row (= blocks or pairs of the launch); stats/keys: the expansion's
-// partial arrays.
+// call; chunks: producers per row (= blocks or pairs of the launch); slots: partial places per row in
+// stats/keys, the expansion's partial arrays (>= chunks).
 template <bool PAIR>
 __global__ void __launch_bounds__(kFzThreads, 1)
 lm_head_topk_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant__ CUtensorMap h_map, int rows,
-                    int row0, int H, int V, int k, int stages, int chunks, long long wait_limit,
+                    int row0, int H, int V, int k, int stages, int chunks, int slots, long long wait_limit,
                     double2* __restrict__ stats, unsigned long long* __restrict__ keys, int32_t* d_status) {
     extern __shared__ unsigned char smem_raw[];
     __shared__ FzBarriers bars;
@@ -345,7 +346,7 @@ lm_head_topk_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_cons
                             const unsigned long long key = c_keys[j * 128 + r_local];
                             if (key) fz_insert(list, key, k);
                         }
-                    const size_t part = (size_t)(row0 + (int)rank * 128 + r_local) * chunks + unit;
+                    const size_t part = (size_t)(row0 + (int)rank * 128 + r_local) * slots + unit;
                     stats[part] = make_double2((double)m, (double)sum);
 #pragma unroll
                     for (int j = 0; j < kFzMaxK; ++j)
@@ -416,20 +417,29 @@ static int fz_chunks(int V, bool pair) {
     return n_tiles < units ? n_tiles : units;
 }
 
-// Rows per pass over the weights: all of them up to 128 (single blocks); otherwise as few passes of
-// block pairs as 256 rows each allow, of equal size.
-static void fz_passes(long long rows, bool* pair, int* n_pass, int* per_pass) {
-    *pair = rows > 128;
-    *n_pass = rows > 128 ? (int)((rows + 255) / 256) : 1;
-    *per_pass = (int)((rows + *n_pass - 1) / *n_pass);
+// Passes over the weights: all rows in one pass of single blocks up to 128 rows; otherwise passes of
+// block pairs with 256 rows each, and the rest in a pass of its own (single blocks up to 128 rows).
+struct FzPasses {
+    int full;        // pair passes of 256 rows
+    int rest;        // rows of the last pass (0: none)
+    bool rest_pair;  // the last pass uses block pairs
+    int chunks_pair, chunks_single, slots;
+};
+static FzPasses fz_passes(long long rows, int V) {
+    FzPasses p;
+    p.full = rows > 128 ? (int)(rows / 256) : 0;
+    p.rest = (int)(rows - (long long)p.full * 256);
+    p.rest_pair = p.rest > 128;
+    p.chunks_pair = fz_chunks(V, true), p.chunks_single = fz_chunks(V, false);
+    p.slots = (p.rest && !p.rest_pair) ? p.chunks_single : p.chunks_pair;
+    if (p.full && p.chunks_pair > p.slots) p.slots = p.chunks_pair;
+    return p;
 }
 
-// Two areas: the producers' partials (`chunks` per row), then the rows' merged partials (one per row).
+// Two areas: the producers' partials (`slots` per row), then the rows' merged partials (one per row).
 static size_t fz_ws_bytes(int B, int n_s, int V, int k, size_t* second) {
-    bool pair;
-    int n_pass, per;
-    fz_passes((long long)B * n_s, &pair, &n_pass, &per);
-    const size_t first = round_up(expand_partials_bytes(B, n_s, fz_chunks(V, pair), k), kWsAlign);
+    const FzPasses p = fz_passes((long long)B * n_s, V);
+    const size_t first = round_up(expand_partials_bytes(B, n_s, p.slots, k), kWsAlign);
     if (second) *second = first;
     return first + expand_partials_bytes(B, n_s, 1, k);
 }
@@ -440,7 +450,7 @@ size_t lm_head_expand_workspace_bytes(int B, int V, int k) {
 }
 
 template <bool PAIR>
-static int fz_launch(const CUtensorMap& w_map, const CUtensorMap& h_map, int rows, int row0, int H, int V, int k, int chunks,
+static int fz_launch(const CUtensorMap& w_map, const CUtensorMap& h_map, int rows, int row0, int H, int V, int k, int chunks, int slots,
                      double2* stats, unsigned long long* keys, int32_t* d_status, cudaStream_t st) {
     constexpr uint32_t kStageBytes = kFzABytes + (PAIR ? kFzTileV / 2 : kFzTileV) * kFzTileK * 2;
     const int stages = PAIR ? 6 : 4;
@@ -450,7 +460,7 @@ static int fz_launch(const CUtensorMap& w_map, const CUtensorMap& h_map, int row
         return EAGLE2_ERR_CUDA;
     }
     return launch_chained(lm_head_topk_kernel<PAIR>, dim3((unsigned)(chunks * (PAIR ? 2 : 1))), dim3(kFzThreads), dyn, st,
-                          PAIR ? 2u : 1u, w_map, h_map, rows, row0, H, V, k, stages, chunks, wait_limit_cycles(), stats, keys,
+                          PAIR ? 2u : 1u, w_map, h_map, rows, row0, H, V, k, stages, chunks, slots, wait_limit_cycles(), stats, keys,
                           d_status);
 }
 
@@ -471,30 +481,28 @@ extern "C" int eagle2_lm_head_expand(const void* hidden, const void* weight, int
     const long long rows = (long long)B * n_s;
     if (rows > 0x7fffffffLL) return EAGLE2_ERR_SHAPE;
     if (!ws || !aligned(ws, kWsAlign)) return EAGLE2_ERR_WORKSPACE;
-    bool pair;
-    int n_pass, per_pass;
-    fz_passes(rows, &pair, &n_pass, &per_pass);
-    const int chunks = fz_chunks(V, pair);
+    const FzPasses p = fz_passes(rows, V);
     size_t second = 0;
     if (fz_ws_bytes(B, n_s, V, k, &second) > ws_bytes) return EAGLE2_ERR_WORKSPACE;
     void* ws_rows = static_cast<char*>(ws) + second;
     double2* stats = nullptr;
     unsigned long long* keys = nullptr;
-    if (!expand_partials_layout(B, n_s, chunks, k, ws, second, &stats, &keys)) return EAGLE2_ERR_WORKSPACE;
-    CUtensorMap w_map, h_map;
+    if (!expand_partials_layout(B, n_s, p.slots, k, ws, second, &stats, &keys)) return EAGLE2_ERR_WORKSPACE;
+    CUtensorMap w_pair, w_single, h_map;
     // vocabulary rows past V and feature rows past the last one read as zero
-    if (!fz_matrix_map(&w_map, weight, V, H, pair ? kFzTileV / 2 : kFzTileV) || !fz_matrix_map(&h_map, hidden, rows, H, 128))
+    if (!fz_matrix_map(&w_pair, weight, V, H, kFzTileV / 2) || !fz_matrix_map(&w_single, weight, V, H, kFzTileV) ||
+        !fz_matrix_map(&h_map, hidden, rows, H, 128))
         return EAGLE2_ERR_CUDA;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-    for (int p = 0; p < n_pass; ++p) {
-        const long long r0 = (long long)p * per_pass;
-        const int n = (int)(rows - r0 < per_pass ? rows - r0 : per_pass);
-        if (n <= 0) break;
-        const int rc = pair ? fz_launch<true>(w_map, h_map, n, (int)r0, H, V, k, chunks, stats, keys, d_status, st)
-                            : fz_launch<false>(w_map, h_map, n, (int)r0, H, V, k, chunks, stats, keys, d_status, st);
-        if (rc != EAGLE2_OK) return rc;
-    }
-    int rc = launch_expand_row_merge(B, n_s, chunks, k, ws, ws_rows, st);
+    int rc = EAGLE2_OK;
+    for (int i = 0; i < p.full && rc == EAGLE2_OK; ++i)
+        rc = fz_launch<true>(w_pair, h_map, 256, i * 256, H, V, k, p.chunks_pair, p.slots, stats, keys, d_status, st);
+    if (rc == EAGLE2_OK && p.rest)
+        rc = p.rest_pair ? fz_launch<true>(w_pair, h_map, p.rest, p.full * 256, H, V, k, p.chunks_pair, p.slots, stats, keys, d_status, st)
+                         : fz_launch<false>(w_single, h_map, p.rest, p.full * 256, H, V, k, p.chunks_single, p.slots, stats, keys, d_status, st);
+    if (rc != EAGLE2_OK) return rc;
+    rc = launch_expand_row_merge(B, n_s, p.slots, (long long)p.full * 256, p.chunks_pair,
+                                 p.rest_pair ? p.chunks_pair : p.chunks_single, k, ws, ws_rows, st);
     if (rc != EAGLE2_OK) return rc;
     return launch_expand_merge(B, V, k, D, s, 1, tree_token, tree_parent, tree_value, frontier, ws_rows, d_status, st);
 }
