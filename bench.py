@@ -507,6 +507,26 @@ def lm_head_fused_extra(e2, dev, stream, hbm_peak, reps=10):
     return {"workload": f"llama3_8b-shaped LM head ({H} -> {V}) + expansion step 1, bf16 weights {2.0 * V * H / 1e9:.2f} GB", "cases": out}
 
 
+def side_measurements(e2, dev, stream, hbm_peak, only=""):
+    """The measurements beside the bench line, by key; `only`: comma-separated keys (default: all)."""
+    table = {
+        "attention_batched": lambda: batched_attention_extra(e2, dev, stream, hbm_peak),
+        "expand_batched": lambda: batched_expand_extra(e2, dev, stream, hbm_peak),
+        "expand_sweep": lambda: [dict(B=b, **{k_: v for k_, v in batched_expand_extra(e2, dev, stream, hbm_peak, B=b).items()
+                                              if k_ != "workload"}) for b in (1, 8, 32)],
+        "accept_batched": lambda: batched_accept_extra(e2, dev, stream, hbm_peak),
+        "accept_batched_b32": lambda: batched_accept_extra(e2, dev, stream, hbm_peak, B=32),
+        "draft_attention": lambda: draft_attention_extra(e2, dev, stream, hbm_peak),
+        "lm_head": lambda: lm_head_extra(e2, dev, stream, hbm_peak),
+        "lm_head_fused": lambda: lm_head_fused_extra(e2, dev, stream, hbm_peak),
+    }
+    want = [w for w in only.split(",") if w] or list(table)
+    unknown = [w for w in want if w not in table]
+    if unknown:
+        raise SystemExit(f"unknown side measurement(s) {unknown}; known: {sorted(table)}")
+    return {w: table[w]() for w in want}
+
+
 def run_ours(args):
     import torch
 
@@ -524,15 +544,9 @@ def run_ours(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
 
-    if args.extras_only:  # the two batched side measurements alone (one GPU; also what the ncu summaries capture)
+    if args.extras_only:  # side measurements alone (one GPU; also what the ncu summaries capture)
         stream = torch.cuda.Stream(device=dev)
-        hbm_peak = _peaks()[0]
-        print(json.dumps({"attention_batched": batched_attention_extra(e2, dev, stream, hbm_peak),
-                          "expand_batched": batched_expand_extra(e2, dev, stream, hbm_peak),
-                          "accept_batched": batched_accept_extra(e2, dev, stream, hbm_peak),
-                          "draft_attention": draft_attention_extra(e2, dev, stream, hbm_peak),
-                          "lm_head": lm_head_extra(e2, dev, stream, hbm_peak),
-                          "lm_head_fused": lm_head_fused_extra(e2, dev, stream, hbm_peak)}))
+        print(json.dumps(side_measurements(e2, dev, stream, _peaks()[0], args.extras)))
         return
     cfg = get_config(args.workload)
     if args.batch:
@@ -854,15 +868,7 @@ def run_ours(args):
     line["roofline_all"] = roofline_all
     line["launch_floor"] = floor
     if world == 1 and not args.no_extras:
-        line["attention_batched"] = batched_attention_extra(e2, dev, stream, hbm_peak)
-        line["expand_batched"] = batched_expand_extra(e2, dev, stream, hbm_peak)
-        line["expand_sweep"] = [dict(B=b, **{k_: v for k_, v in batched_expand_extra(e2, dev, stream, hbm_peak, B=b).items()
-                                             if k_ != "workload"}) for b in (1, 8, 32)]
-        line["accept_batched"] = batched_accept_extra(e2, dev, stream, hbm_peak)
-        line["accept_batched_b32"] = batched_accept_extra(e2, dev, stream, hbm_peak, B=32)
-        line["draft_attention"] = draft_attention_extra(e2, dev, stream, hbm_peak)
-        line["lm_head"] = lm_head_extra(e2, dev, stream, hbm_peak)
-        line["lm_head_fused"] = lm_head_fused_extra(e2, dev, stream, hbm_peak)
+        line.update(side_measurements(e2, dev, stream, hbm_peak, args.extras))
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
@@ -880,6 +886,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="skip the batched attention, expansion and acceptance side measurements")
     ap.add_argument("--extras-only", action="store_true", help="run only those side measurements (no bench line)")
+    ap.add_argument("--extras", default="", help="comma-separated side measurements to run (default: all)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
