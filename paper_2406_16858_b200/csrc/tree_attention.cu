@@ -85,13 +85,20 @@ static void attention_plan(int B, int m, int Hq, int Hkv, int d, int max_kv_len,
     int per_split = (int)((tiles + s - 1) / s);
     // a batch whose longest sequence needs several blocks anyway: order them, and let each stream more
     p->ordered = (B > 1 && !p->pair && per_split > kMaxTilesPerSplit) ? 1 : 0;
+    // An ordered launch with few (sequence, KV head) items - up to one and a half per TPC - runs on
+    // pairs as well: with so few items the longest sequences decide the time, and a pair puts two SMs
+    // on each of their splits (measured per layer, ragged batches of the LLaMA3-8B shape: B = 8 86 ->
+    // 67 us, B = 12 112 -> 104 us; with more items pairs lose: B = 16 112 -> 119 us, B = 32 181 -> 216 us).
+    const bool ordered_pair = p->ordered && p->mt == 2 && p->q_tma && d == 128 && 2 * items <= 3 * tpcs;
+    if (ordered_pair) p->pair = 1;
+    const int units = p->pair ? tpcs : sms;  // blocks (pairs) resident at once
     if (p->ordered) {
         // Only the longest length is known here and a ragged batch holds far fewer tiles than
         // sequences x longest: aim at two blocks per SM by that count, within 8..32 tiles per block
         // (long blocks leave a batch of a few sequences to a handful of SMs; short ones cost partials
         // and a block's start-up each).  Measured per layer at B = 8 / 16: 110 / 111 us with 32 tiles,
         // 105 / 121 us when aiming at four blocks per SM.
-        const long long want = (tiles * items + 2LL * sms - 1) / (2LL * sms);
+        const long long want = (tiles * items + 2LL * units - 1) / (2LL * units);
         per_split = (int)(want < 8 ? 8 : (want > kMaxTilesPerSplitOrdered ? kMaxTilesPerSplitOrdered : want));
     } else if (per_split > kMaxTilesPerSplitOrdered) {
         per_split = kMaxTilesPerSplitOrdered;  // more blocks than the device holds at once: several waves
@@ -107,8 +114,8 @@ static void attention_plan(int B, int m, int Hq, int Hkv, int d, int max_kv_len,
     p->wait_limit = wait_limit_cycles();
     p->setup_first = B == 1;  // ragged batches leave many splits without tiles: those leave at once
     if (p->pair) {  // per block: one 128-row query tile, half-size K and V stages
-        p->stages = 4;
-        p->smem = unit + 4 * unit + 1024;
+        p->stages = p->ordered ? 5 : 4;
+        p->smem = unit + (size_t)p->stages * unit + 1024;
     }
 }
 
@@ -138,7 +145,7 @@ static size_t attention_ws_layout(int B, int Hkv, int d, const AttnPlan& p, void
     }
     if (p.fused_merge) {  // (cleared by the launch's own list kernel: other operations' scratch may overlap it)
         if (w) w->tickets = reinterpret_cast<int*>(c + off);
-        off += round_up(sizeof(int) * (size_t)B * Hkv * p.n_rb, kWsAlign);
+        off += round_up(sizeof(int) * (size_t)B * Hkv * p.n_rb * (p.pair ? 2 : 1), kWsAlign);
     }
     return off;
 }
@@ -242,9 +249,10 @@ __device__ __forceinline__ bool sequence_ok(int L, long long row_base, int m, in
     return L >= 0 && L <= max_kv_len && row_base >= 0 && row_base + L + m <= cache_rows;
 }
 
+constexpr int kMaxStages = 6;  // K/V ring depth the barrier arrays allow
 struct AttnBarriers {
     unsigned long long q_full;
-    unsigned long long k_full[4], k_empty[4], v_full[4], v_empty[4];
+    unsigned long long k_full[kMaxStages], k_empty[kMaxStages], v_full[kMaxStages], v_empty[kMaxStages];
     unsigned long long s_full[kSlots], p_full[kSlots];
     // Per accumulator (= score slot = item parity), two barriers used by its alternate uses: the
     // u-th P.V into accumulator e completes a phase of o_done[e][u & 1].  A waiter may skip phases (it only looks when it must rescale O, and at the
@@ -252,7 +260,7 @@ struct AttnBarriers {
     unsigned long long o_done[2][2];
     // pair mode, used in the pair's first block: the other block's query tile / K half / V half
     // has landed (and its V tail is cleared)
-    unsigned long long q_peer, k_peer[4], v_peer[4];
+    unsigned long long q_peer, k_peer[kMaxStages], v_peer[kMaxStages];
     unsigned long long v_landed, v_clean;  // the block's last V tile has landed / its rows past the sequence's last key are cleared
     unsigned long long drain;  // after a wait ran out: the tensor instructions issued so far have retired
 };
@@ -404,7 +412,7 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
             s_ctl.abort = 0;
             s_ctl.limit = plan.wait_limit;
             mbar_init(smem_u32(&bars.q_full), plan.q_tma ? 1 : kSoftmaxThreads);
-            for (int s = 0; s < 4; ++s) {
+            for (int s = 0; s < kMaxStages; ++s) {
                 mbar_init(smem_u32(&bars.k_full[s]), 1);
                 mbar_init(smem_u32(&bars.k_empty[s]), 1);
                 mbar_init(smem_u32(&bars.v_full[s]), 1);
@@ -415,7 +423,7 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
                 mbar_init(smem_u32(&bars.p_full[s]), (PAIR ? 2 : 1) * (kSoftmaxThreads / 64));  // one arrival per warp of the slot's group
             }
             mbar_init(smem_u32(&bars.q_peer), 1);
-            for (int s = 0; s < 4; ++s) {
+            for (int s = 0; s < kMaxStages; ++s) {
                 mbar_init(smem_u32(&bars.k_peer[s]), 1);
                 mbar_init(smem_u32(&bars.v_peer[s]), 1);
             }
@@ -450,7 +458,7 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
 
     int bid = PAIR ? blockIdx.x >> 1 : blockIdx.x;
     int split, rb, hk, b;
-    if (!PAIR && plan.ordered) {  // item-major: the list says which (sequence, split) this block serves
+    if (plan.ordered) {  // item-major: the list says which (sequence, split) this block serves
         rb = bid % plan.n_rb;
         bid /= plan.n_rb;
         hk = bid % Hkv;
@@ -899,11 +907,13 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
     }  // active
 
     // ---- merging launches: whoever finishes a (sequence, KV head, row block) last combines its splits
-    if (!PAIR && plan.fused_merge && !direct) {  // uniform over the block; blocks without tiles left long ago
+    // (a pair's blocks count and merge on their own, each for its 128 rows)
+    if (plan.fused_merge && !direct) {  // uniform over the block; blocks without tiles left long ago
         __shared__ int s_last;
-        if (last_block_arrives(ws.tickets + ((size_t)b * Hkv + hk) * plan.n_rb + rb, S_b, &s_last)) {
-            for (int r = warp; r < rows_blk; r += kAttnThreads / 32)
-                merge_row<DH>(plan, ws, b, hk, rb * plan.per + r, S_b, m, Hq, Hkv, out, lse);
+        int* ticket = ws.tickets + (((size_t)b * Hkv + hk) * plan.n_rb + rb) * (PAIR ? 2 : 1) + rank;
+        if (last_block_arrives(ticket, S_b, &s_last)) {
+            for (int r = warp; r < rows_here; r += kAttnThreads / 32)
+                merge_row<DH>(plan, ws, b, hk, row0 + r, S_b, m, Hq, Hkv, out, lse);
         }
     }
 
@@ -1042,7 +1052,7 @@ static int launch_attention(const CUtensorMap& k_map, const CUtensorMap& v_map, 
     if (blocks > 0x7fffffffLL || (long long)B * plan.splits > 0x7fffffffLL) return EAGLE2_ERR_SHAPE;
     if (plan.ordered &&
         launch_chained(tree_attention_schedule_kernel, dim3(1), dim3(1024), 0, st, 1, kv_off, kv_len, B, m, cache_rows,
-                       max_kv_len, plan, ws.order, ws.tickets, plan.fused_merge ? B * Hkv * plan.n_rb : 0) != EAGLE2_OK)
+                       max_kv_len, plan, ws.order, ws.tickets, plan.fused_merge ? B * Hkv * plan.n_rb * (plan.pair ? 2 : 1) : 0) != EAGLE2_OK)
         return EAGLE2_ERR_CUDA;
     if (launch_chained(kern, dim3((unsigned)blocks), dim3(kAttnThreads), plan.smem, st, PAIR ? 2u : 1u, k_map, v_map, q_map,
                        static_cast<const __nv_bfloat16*>(q), kv_off, kv_len, mask_bits, m, Hq, Hkv, cache_rows, max_kv_len,
