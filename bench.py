@@ -567,10 +567,17 @@ def run_ours(args):
     def randn_bf16(*shape_):
         return torch.randn(shape_, generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
 
-    k_layers = [randn_bf16(rows, cfg.Hkv, cfg.d) for _ in range(cfg.n_layers)]
-    v_layers = [randn_bf16(rows, cfg.Hkv, cfg.d) for _ in range(cfg.n_layers)]
-    q_layers = [randn_bf16(cfg.B, cfg.m, cfg.Hq, cfg.d) for _ in range(cfg.n_layers)]
-    out_layers = [torch.zeros_like(qq) for qq in q_layers]
+    # One allocation each for all layers' K, V, Q and O, handed to the library layer by layer: the end
+    # to end region below then moves a cycle's per-layer inputs and results in a handful of copies.
+    k_all = torch.empty((cfg.n_layers, rows, cfg.Hkv, cfg.d), dtype=torch.bfloat16, device=dev)
+    v_all = torch.empty_like(k_all)
+    for layer in range(cfg.n_layers):
+        k_all[layer].copy_(randn_bf16(rows, cfg.Hkv, cfg.d))
+        v_all[layer].copy_(randn_bf16(rows, cfg.Hkv, cfg.d))
+    q_all = randn_bf16(cfg.n_layers, cfg.B, cfg.m, cfg.Hq, cfg.d)
+    out_all = torch.zeros_like(q_all)
+    k_layers, v_layers = list(k_all.unbind(0)), list(v_all.unbind(0))
+    q_layers, out_layers = list(q_all.unbind(0)), list(out_all.unbind(0))
     k_ptrs = torch.tensor([t.data_ptr() for t in k_layers], dtype=torch.int64, device=dev)
     v_ptrs = torch.tensor([t.data_ptr() for t in v_layers], dtype=torch.int64, device=dev)
     kv_off = torch.from_numpy(kv_off_h).to(dev)
@@ -713,23 +720,23 @@ def run_ours(args):
         host_in = {
             "draft": sets[0]["draft"].cpu().pin_memory(), "target": sets[0]["target"].cpu().pin_memory(),
             "ua": sets[0]["ua"].cpu().pin_memory(), "ub": sets[0]["ub"].cpu().pin_memory(),
-            "q": [t.cpu().pin_memory() for t in q_layers],
+            "q": q_all.cpu().pin_memory(),
         }
         # the K/V of the m tree tokens are this cycle's new cache rows, one block per layer
         tree_rows = [(b, int(kv_off_h[b] + kv_len_h[b])) for b in range(cfg.B)]
-        host_in["tree_k"] = [torch.stack([kc[r:r + cfg.m] for _, r in tree_rows]).cpu().pin_memory()
-                             for kc in k_layers]
-        host_in["tree_v"] = [torch.stack([vc[r:r + cfg.m] for _, r in tree_rows]).cpu().pin_memory()
-                             for vc in v_layers]
+        # [layer][K or V][sequence][m][Hkv][d]: one upload into a staging tensor, then one strided
+        # device copy per sequence and operand puts the rows behind the sequence's prefix in every layer
+        host_in["tree_kv"] = torch.stack([torch.stack([c[:, r:r + cfg.m] for _, r in tree_rows], dim=1)
+                                          for c in (k_all, v_all)], dim=1).cpu().pin_memory()
+        tree_kv_dev = torch.empty_like(host_in["tree_kv"], device=dev)
         host_out = {"acc_len": torch.zeros(cfg.B, dtype=torch.int32).pin_memory(),
                     "acc_path": torch.zeros((cfg.B, cfg.D), dtype=torch.int32).pin_memory(),
                     "bonus": torch.zeros(cfg.B, dtype=torch.int32).pin_memory(),
-                    "o": [torch.zeros_like(t, device="cpu").pin_memory() for t in out_layers]}
+                    "o": torch.zeros_like(out_all, device="cpu").pin_memory()}
         h2d = sum(t.numel() * t.element_size() for t in
-                  [host_in["draft"], host_in["target"], host_in["ua"], host_in["ub"], *host_in["q"],
-                   *host_in["tree_k"], *host_in["tree_v"]])
+                  [host_in["draft"], host_in["target"], host_in["ua"], host_in["ub"], host_in["q"], host_in["tree_kv"]])
         d2h = sum(t.numel() * t.element_size() for t in
-                  [host_out["acc_len"], host_out["acc_path"], host_out["bonus"], *host_out["o"]])
+                  [host_out["acc_len"], host_out["acc_path"], host_out["bonus"], host_out["o"]])
 
         # Two input sets alternate: the logits of a step travel on a copy stream and may overlap the
         # compute of the step before (which works on the other set); the per-layer inputs, the cycle
@@ -750,19 +757,18 @@ def run_ours(args):
                 s["ua"].copy_(host_in["ua"], non_blocking=True)
                 s["ub"].copy_(host_in["ub"], non_blocking=True)
                 ev_in[j].record(copy_stream)
-            for layer in range(cfg.n_layers):
-                q_layers[layer].copy_(host_in["q"][layer], non_blocking=True)
-                for seq, (_, r) in enumerate(tree_rows):
-                    k_layers[layer][r:r + cfg.m].copy_(host_in["tree_k"][layer][seq], non_blocking=True)
-                    v_layers[layer][r:r + cfg.m].copy_(host_in["tree_v"][layer][seq], non_blocking=True)
+            q_all.copy_(host_in["q"], non_blocking=True)
+            tree_kv_dev.copy_(host_in["tree_kv"], non_blocking=True)
+            for seq, (_, r) in enumerate(tree_rows):
+                k_all[:, r:r + cfg.m].copy_(tree_kv_dev[:, 0, seq])
+                v_all[:, r:r + cfg.m].copy_(tree_kv_dev[:, 1, seq])
             stream.wait_event(ev_in[j])  # this step's logits are in place (every upload is thereby ordered before
             graphs[j].replay()           # the closing event, which is recorded on the compute stream)
             ev_free[j].record(stream)
             host_out["acc_len"].copy_(s["buf"].acc_len, non_blocking=True)
             host_out["acc_path"].copy_(s["buf"].acc_path, non_blocking=True)
             host_out["bonus"].copy_(s["buf"].bonus_token, non_blocking=True)
-            for layer in range(cfg.n_layers):
-                host_out["o"][layer].copy_(out_layers[layer], non_blocking=True)
+            host_out["o"].copy_(out_all, non_blocking=True)
 
         e2e_steps = max(5, min(K, 50))
         timed(e2e_step, 3)
