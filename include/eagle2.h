@@ -123,6 +123,9 @@ int eagle2_lm_head(const void* hidden, const void* weight, int rows, int H, int 
  *   tree_token, tree_parent, tree_value, frontier: as for eagle2_expand (level s + 1 is written,
  *           frontier is read at s > 0 and overwritten)
  *   ws      eagle2_workspace_bytes(EAGLE2_OP_LM_HEAD_EXPAND, B, V, k, ...) bytes
+ * Up to 128 rows (B * n_s) ride on one pass over the weights, one block per SM; up to 256 on one
+ * pass of block pairs; more rows take a pass per 256 and one for the rest.  Three kinds of launch per
+ * call: the passes, a merge of every row's partial results, and the expansion's own merge.
  * Limits: those of eagle2_expand, and k <= 16, H a multiple of 64.  Logits are fp32 sums of bf16
  * products, as eagle2_lm_head forms them; a row's k-th and (k+1)-th logits closer than that sum's
  * rounding may come out in either order.  Status bits as for eagle2_expand; a bounded wait that
