@@ -2,25 +2,28 @@
 // features go through the LM head of the original LLM, and the expansion keeps the k most probable
 // tokens of every row).  For many feature rows (rows = sequences x frontier size) the logits are as
 // large as the weights, and writing them only to read them back once is most of the step's traffic.
-// Here they never leave the SM: a block walks vocabulary tiles, the tensor pipe leaves
-// logits[feature row][256 vocabulary entries] in tensor memory, and the epilogue threads fold each
-// tile into their row's running maximum, sum of exponentials and k best (value, token) keys while
-// the tensor pipe already works on the next tile (two accumulators).  When a block has walked its
-// tiles it writes one partial per row, in the expansion's own workspace layout; a row-merge launch
-// folds a row's partials into one, and the expansion's merge launch finishes the step from those.
+// Here they never leave the SM: a block walks tiles of 128 vocabulary entries, the tensor pipe leaves
+// logits[vocabulary entry][feature row] in tensor memory, writer warps turn 32 rows at a time through
+// shared memory, and scanner threads - one per feature row - fold them into the row's running
+// maximum, sum of exponentials and k best (value, token) keys while the tensor pipe already works on
+// the next tile (two accumulators).  When a block has walked its tiles it writes one partial per row,
+// in the expansion's own workspace layout; a row-merge launch folds a row's partials into one, and the
+// expansion's merge launch finishes the step from those.
 //
-// Operand roles are swapped against the plain LM head: the feature rows are the M side of
-// tcgen05.mma, a vocabulary tile is its N = 256, so that a thread's tensor-memory lane is a feature
-// row and its columns are that row's logits.  A block holds 128 feature rows.  Up to 128 rows: one
-// block per SM (cta_group::1).  More: two blocks on one TPC form a pair (cta_group::2, M = 256),
-// each holding 128 rows and copying half of every weight box, so that the weights cross from L2
-// into shared memory once per pair; tensor memory then still has room for two accumulators.
-//   TMA warp        streams [256 (pair: 128) vocabulary rows x 64 hidden columns] weight boxes and
-//                   the matching 64 columns of the block's features (from L2) through a ring;
-//   MMA warp        one lane (of the pair's first block) issues four K = 16 instructions per stage;
-//                   the second block's lane tells it when that block's halves have landed;
-//   8 epilogue warps two per tensor-memory lane quadrant, one for columns 0..127 and one for columns
-//                   128..255 of every tile; the two halves of a row are combined at the end.
+// The vocabulary is the M side of tcgen05.mma (128 entries per block) and the feature rows are its
+// N side, N = the rows of the pass rounded up to 16: the tensor work is proportional to the rows
+// (with the rows on the M side it was padded to 128 or 256, which at 160 rows made it as long as the
+// weight stream).  Up to 128 rows: one block per SM (cta_group::1).  More: two blocks on one TPC form
+// a pair (cta_group::2, M = 256 vocabulary entries), each copying half of the feature rows, so that
+// the features cross from L2 into shared memory once per pair.
+//   TMA warp         streams [128 vocabulary rows x 64 hidden columns] weight boxes and the matching
+//                    64 columns of the block's feature rows (from L2) through a ring;
+//   MMA warp         one lane (of the pair's first block) issues four K = 16 instructions per stage;
+//                    the second block's lane tells it when that block's boxes have landed;
+//   4 writer warps   one per tensor-memory lane quadrant: 32 feature rows (columns) of the finished
+//                    accumulator at a time into one of two shared-memory buffers, transposed
+//                    ([row][vocabulary entry], rows 129 words apart: no bank conflicts either way);
+//   8 scanner warps  warp c owns feature rows 32c .. 32c+31 of the pass, a thread one row.
 // Every wait on an mbarrier is bounded (EAGLE2_STATUS_TIMEOUT, copies drained, tensor memory freed).
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -39,18 +42,23 @@ int launch_expand_merge(int B, int V, int k, int D, int s, int chunks, int32_t* 
 int launch_expand_row_merge(int B, int n_s, int slots, long long split_row, int chunks_lo, int chunks_hi, int k, void* ws,
                             void* ws_rows, cudaStream_t stream);
 
-constexpr int kFzThreads = 64 + 256;  // TMA warp, MMA warp, eight epilogue warps
-constexpr int kFzTileV = 256;         // vocabulary entries per tile = N of the instruction
-constexpr int kFzTileK = 64;          // hidden columns per stage (128 bytes, the swizzle span)
-constexpr int kFzMaxK = 16;           // keys a row's list holds (children per node the fused path supports)
-constexpr int kFzMaxStages = 6;
-constexpr uint32_t kFzABytes = 128 * kFzTileK * 2;  // the block's feature rows' share of a stage
+constexpr int kFzWriterWarps = 4, kFzScanWarps = 8;
+constexpr int kFzThreads = (2 + kFzWriterWarps + kFzScanWarps) * 32;
+constexpr int kFzTileV = 128;   // vocabulary entries per block and tile = the block's M
+constexpr int kFzTileK = 64;    // hidden columns per stage (128 bytes, the swizzle span)
+constexpr int kFzMaxK = 16;     // keys a row's list holds (children per node the fused path supports)
+constexpr int kFzMaxRows = 256; // feature rows per pass = N of the instruction at most
+constexpr int kFzMaxStages = 8;
+constexpr uint32_t kFzABytes = kFzTileV * kFzTileK * 2;     // the weight box of a stage
+constexpr int kFzTStride = 33;                              // words between rows of a transposition unit
+constexpr uint32_t kFzTBytes = 32 * kFzTStride * 4;         // one unit: 32 feature rows x 32 vocabulary entries
 
 struct FzBarriers {
     unsigned long long full[kFzMaxStages], empty[kFzMaxStages];
-    unsigned long long peer[kFzMaxStages];  // first block of a pair: the second block's halves have landed
+    unsigned long long peer[kFzMaxStages];  // first block of a pair: the second block's boxes have landed
     unsigned long long acc_full[2], acc_empty[2];  // an accumulator is complete / has been read
-    unsigned long long comb;                       // the upper column half's results are in shared memory
+    // unit (c, q) = feature rows 32c.., vocabulary entries 32q.. of the tile: written / scanned
+    unsigned long long t_full[kFzScanWarps][4], t_empty[kFzScanWarps][4];
     unsigned long long drain;
 };
 
@@ -80,32 +88,36 @@ __device__ __forceinline__ unsigned long long fz_insert(unsigned long long (&lis
     return kth;
 }
 
-// rows: feature rows of this pass (<= 128, pair: <= 256); row0: first of them among all rows of the
-// call; chunks: producers per row (= blocks or pairs of the launch); slots: partial places per row in
-// stats/keys, the expansion's partial arrays (>= chunks).
+// rows: feature rows of this pass (<= 128, pair: <= 256); n_pad: rows rounded up to 16 (= N); row0:
+// first of them among all rows of the call; units: blocks (pairs) of the launch, unit u walks tiles
+// u, u + units, ...; slots: partial places per row in stats/keys, the expansion's partial arrays
+// (a block writes place blockIdx.x); b_bytes: bytes of the block's feature box of a stage.
 template <bool PAIR>
 __global__ void __launch_bounds__(kFzThreads, 1)
 lm_head_topk_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant__ CUtensorMap h_map, int rows,
-                    int row0, int H, int V, int k, int stages, int chunks, int slots, long long wait_limit,
-                    double2* __restrict__ stats, unsigned long long* __restrict__ keys, int32_t* d_status) {
+                    int n_pad, int row0, int H, int V, int k, int stages, int t_slots, int units, int slots, uint32_t b_bytes,
+                    long long wait_limit, double2* __restrict__ stats, unsigned long long* __restrict__ keys,
+                    int32_t* d_status) {
     extern __shared__ unsigned char smem_raw[];
     __shared__ FzBarriers bars;
     __shared__ uint32_t s_tmem_base;
     __shared__ WaitCtl s_ctl;
     constexpr int CG = PAIR ? 2 : 1;
-    constexpr uint32_t kBBytes = (PAIR ? kFzTileV / 2 : kFzTileV) * kFzTileK * 2;  // this block's weight box
-    constexpr uint32_t kStageBytes = kFzABytes + kBBytes;
-    constexpr uint32_t kTmemCols = 2 * kFzTileV;  // two accumulators: all of tensor memory
+    constexpr uint32_t kTmemCols = 2 * kFzMaxRows;  // two accumulators: all of tensor memory
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t rank = PAIR ? cluster_ctarank() : 0u;
-    const int unit = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;  // walks tiles unit, unit + chunks, ...
+    const int unit = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     unsigned char* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
-    const int n_tiles = (V + kFzTileV - 1) / kFzTileV;
+    const uint32_t stage_bytes = kFzABytes + b_bytes;
+    float* t_buf = reinterpret_cast<float*>(smem_gen + (size_t)stages * stage_bytes);  // [chunk][t_slots][32][kFzTStride]
+    const int tile_v = CG * kFzTileV;  // vocabulary entries of a tile of the unit
+    const int n_tiles = (V + tile_v - 1) / tile_v;
     const int n_kb = H / kFzTileK;
-    const int my_tiles = unit < n_tiles ? (n_tiles - unit + chunks - 1) / chunks : 0;
-    const int rows_here = max(0, min(128, rows - (int)rank * 128));  // feature rows this block holds
+    const int my_tiles = unit < n_tiles ? (n_tiles - unit + units - 1) / units : 0;
+    const int n_chunks = (rows + 31) / 32;  // groups of 32 feature rows = scanner warps with work
+    const int b_rows = PAIR ? n_pad / 2 : n_pad;  // feature rows this block copies
     volatile WaitCtl* ctl = &s_ctl;
     long long issued = 0;  // producer lane: stages requested so far
 
@@ -119,9 +131,13 @@ lm_head_topk_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_cons
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(smem_u32(&bars.acc_full[a]), 1);
-            mbar_init(smem_u32(&bars.acc_empty[a]), 8 * CG);  // one arrival per epilogue warp of every block
+            mbar_init(smem_u32(&bars.acc_empty[a]), kFzWriterWarps * CG);  // one arrival per writer warp of every block
         }
-        mbar_init(smem_u32(&bars.comb), 4);
+        for (int c = 0; c < kFzScanWarps; ++c)
+            for (int q = 0; q < 4; ++q) {
+                mbar_init(smem_u32(&bars.t_full[c][q]), 1);
+                mbar_init(smem_u32(&bars.t_empty[c][q]), 1);
+            }
         mbar_init(smem_u32(&bars.drain), 1);
         fence_barrier_init();
     }
@@ -153,17 +169,17 @@ lm_head_topk_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_cons
             int st = 0;
             uint32_t ph = 0;
             for (int i = 0; i < my_tiles && ok; ++i) {
-                const int t = unit + i * chunks;
+                // this block's 128 vocabulary rows of the tile; rows past V read as zero, and so do
+                // feature rows past the call's last one
+                const int vrow = (unit + i * units) * tile_v + (int)rank * kFzTileV;
                 for (int kb = 0; kb < n_kb; ++kb, ++issued) {
                     if (issued >= stages) ok = mbar_wait_spin(smem_u32(&bars.empty[st]), ph ^ 1u, ctl);
                     if (!ok) break;
-                    const uint32_t dst = smem_base + (uint32_t)st * kStageBytes;
+                    const uint32_t dst = smem_base + (uint32_t)st * stage_bytes;
                     const uint32_t bar = smem_u32(&bars.full[st]);
-                    mbar_expect_tx(bar, kStageBytes);
-                    // feature rows past the last one and vocabulary rows past V read as zero; a pair
-                    // block takes its 128 of the tile's 256 vocabulary rows
-                    fz_tma_2d(dst, &h_map, kb * kFzTileK, row0 + (int)rank * 128, bar);
-                    fz_tma_2d(dst + kFzABytes, &w_map, kb * kFzTileK, t * kFzTileV + (int)rank * (kFzTileV / 2), bar);
+                    mbar_expect_tx(bar, stage_bytes);
+                    fz_tma_2d(dst, &w_map, kb * kFzTileK, vrow, bar);
+                    fz_tma_2d(dst + kFzABytes, &h_map, kb * kFzTileK, row0 + (int)rank * b_rows, bar);
                     if (++st == stages) st = 0, ph ^= 1u;
                 }
             }
@@ -175,7 +191,7 @@ lm_head_topk_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_cons
             uint32_t ph = 0;
             bool ok = true;
             if (PAIR && rank != 0) {
-                // the second block of a pair issues nothing: it tells the first when its halves are in place
+                // the second block of a pair issues nothing: it tells the first when its boxes are in place
                 for (long long j = 0; j < (long long)my_tiles * n_kb && ok; ++j) {
                     ok = mbar_wait_spin(smem_u32(&bars.full[st]), ph, ctl);
                     if (!ok) break;
@@ -183,7 +199,7 @@ lm_head_topk_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_cons
                     if (++st == stages) st = 0, ph ^= 1u;
                 }
             } else {
-                constexpr uint32_t idesc = instr_desc(kFzTileV, false, PAIR ? 256 : 128);
+                const uint32_t idesc = instr_desc(n_pad, false, PAIR ? 256 : 128);
                 const uint64_t d0 = smem_desc(smem_base, 16);
                 const uint32_t lo0 = (uint32_t)d0, hi = (uint32_t)(d0 >> 32);
                 auto commit = [&](uint32_t bar) {
@@ -195,13 +211,13 @@ lm_head_topk_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_cons
                     if (i >= 2) ok = mbar_wait_spin(smem_u32(&bars.acc_empty[a]), (uint32_t)(((i >> 1) - 1) & 1), ctl);
                     if (!ok) break;
                     tc_fence_after();
-                    const uint32_t d_tmem = tmem + (uint32_t)a * kFzTileV;
+                    const uint32_t d_tmem = tmem + (uint32_t)a * kFzMaxRows;
                     for (int kb = 0; kb < n_kb; ++kb) {
                         ok = mbar_wait_spin(smem_u32(&bars.full[st]), ph, ctl);
                         if (PAIR) ok = ok && mbar_wait_spin(smem_u32(&bars.peer[st]), ph, ctl);
                         if (!ok) break;
                         tc_fence_after();
-                        const uint32_t a_lo = lo0 + (uint32_t)st * (kStageBytes >> 4);
+                        const uint32_t a_lo = lo0 + (uint32_t)st * (stage_bytes >> 4);
                         const uint32_t b_lo = a_lo + (kFzABytes >> 4);
                         if (kb == 0) umma_ss<CG, 0>(d_tmem, a_lo, hi, b_lo, hi, idesc);
                         else umma_ss<CG, 1>(d_tmem, a_lo, hi, b_lo, hi, idesc);
@@ -215,23 +231,17 @@ lm_head_topk_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_cons
                 }
             }
         }
-    } else {
-        // ===== epilogue warps: thread = feature row, warp = (lane quadrant, column half) ================
-        // Warp w reads the tensor-memory lanes 32 * (w % 4) .. + 31; warps 2..5 take columns 0..127 of
-        // every tile, warps 6..9 columns 128..255.
-        constexpr float kLog2e = 1.4426950408889634f;
-        const int quad = warp & 3, half = (warp - 2) >> 2;
-        const int r_local = quad * 32 + lane;
-        const bool row_ok = r_local < rows_here;
-        const bool warp_live = quad * 32 < rows_here;  // a warp without rows only keeps the barriers going
-        const uint32_t t_lane = tmem + ((uint32_t)(quad << 5) << 16) + (uint32_t)half * (kFzTileV / 2);
-        float m_run = -INFINITY, s_run = 0.f;  // running maximum and sum of exp(x - maximum)
-        unsigned long long list[kFzMaxK];       // the row's best keys so far, descending
-#pragma unroll
-        for (int j = 0; j < kFzMaxK; ++j) list[j] = 0ull;
-        // Value of the k-th best once k keys are held.  Entries come in ascending token order, so one
-        // that only equals it loses the tie: nothing at or below the bar can enter.
-        float bar_f = -INFINITY;
+    } else if (warp < 2 + kFzWriterWarps) {
+        // ===== writer warps: thread = vocabulary entry (tensor-memory lane) ==============================
+        // Warp q reads the lanes 32q .. 32q+31 (q = warp % 4).  Columns 32c .. 32c+31 of the accumulator
+        // are the logits of feature rows 32c .. for this thread's entry: unit (c, q), which goes to
+        // slot q % t_slots of scanner warp c as [row][entry].  The slot's previous occupant is the unit
+        // t_slots quadrants back - of the same tile, or of the tile before - and this warp has waited for
+        // every earlier release of that unit, so the phase it looks at cannot be mistaken for another.
+        const int q = warp & 3;
+        const uint32_t t_lane = tmem + ((uint32_t)(q << 5) << 16);
+        const int q_prev = (q + 4 - t_slots) & 3;      // the quadrant whose unit held the slot before
+        const int tile_back = q < t_slots ? 1 : 0;     // ... in the tile before this one
         bool ok = true;
         for (int i = 0; i < my_tiles && ok; ++i) {
             const int a = i & 1;
@@ -240,26 +250,72 @@ lm_head_topk_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_cons
             ok = __shfl_sync(0xffffffffu, r, 0) != 0;
             if (!ok) break;
             tc_fence_after();
-            if (warp_live) {
-                const int v0 = (unit + i * chunks) * kFzTileV + half * (kFzTileV / 2);
 #pragma unroll 1
-                for (int c0 = 0; c0 < kFzTileV / 2; c0 += 32) {
-                    const int n_valid = V - (v0 + c0);  // vocabulary entries of this chunk that exist
-                    if (n_valid <= 0) break;            // (uniform over the block)
-                    uint32_t x[32];
-                    tmem_ld32(t_lane + (uint32_t)(a * kFzTileV + c0), x);
-                    tc_wait_ld(x);
+            for (int c = 0; c < n_chunks; ++c) {
+                uint32_t x[32];
+                tmem_ld32(t_lane + (uint32_t)(a * kFzMaxRows + c * 32), x);
+                if (i - tile_back >= 0) {
+                    r = 1;
+                    if (lane == 0)
+                        r = mbar_wait(smem_u32(&bars.t_empty[c][q_prev]), (uint32_t)((i - tile_back) & 1), ctl) ? 1 : 0;
+                    ok = __shfl_sync(0xffffffffu, r, 0) != 0;
+                }
+                tc_wait_ld(x);
+                if (!ok) break;
+                float* dst = t_buf + (size_t)(c * t_slots + (q % t_slots)) * (32 * kFzTStride) + lane;
+#pragma unroll
+                for (int j = 0; j < 32; ++j) dst[j * kFzTStride] = __uint_as_float(x[j]);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&bars.t_full[c][q]));
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0 && ok) {
+                if (PAIR) mbar_arrive_in(smem_u32(&bars.acc_empty[a]), 0);
+                else mbar_arrive(smem_u32(&bars.acc_empty[a]));
+            }
+        }
+    } else {
+        // ===== scanner warps: thread = feature row ======================================================
+        constexpr float kLog2e = 1.4426950408889634f;
+        const int c = warp - (2 + kFzWriterWarps);  // this warp's group of 32 rows
+        const int r_local = c * 32 + lane;
+        const bool row_ok = r_local < rows;
+        if (c < n_chunks) {
+            float m_run = -INFINITY, s_run = 0.f;  // running maximum and sum of exp(x - maximum)
+            unsigned long long list[kFzMaxK];       // the row's best keys so far, descending
+#pragma unroll
+            for (int j = 0; j < kFzMaxK; ++j) list[j] = 0ull;
+            // Value of the k-th best once k keys are held.  Entries come in ascending token order, so one
+            // that only equals it loses the tie: nothing at or below the bar can enter.
+            float bar_f = -INFINITY;
+            bool ok = true;
+            for (int i = 0; i < my_tiles && ok; ++i) {
+                const int v0 = (unit + i * units) * tile_v + (int)rank * kFzTileV;
+#pragma unroll 1
+                for (int q = 0; q < 4 && ok; ++q) {
+                    const int c0 = q * 32;
+                    int r = 1;
+                    if (lane == 0) r = mbar_wait(smem_u32(&bars.t_full[c][q]), (uint32_t)(i & 1), ctl) ? 1 : 0;
+                    ok = __shfl_sync(0xffffffffu, r, 0) != 0;
+                    __syncwarp();
+                    if (!ok) break;
+                    const float* src = t_buf + (size_t)(c * t_slots + (q % t_slots)) * (32 * kFzTStride) + lane * kFzTStride;
+                    float x[32];
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) x[e] = src[e];
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&bars.t_empty[c][q]));  // the unit is in registers
+                    const int n_valid = V - (v0 + c0);  // vocabulary entries of this unit that exist
+                    if (n_valid <= 0) continue;         // (uniform over the block; the units are still taken)
                     if (n_valid < 32) {
 #pragma unroll
-                        for (int c = 0; c < 32; ++c)
-                            if (c >= n_valid) x[c] = __float_as_uint(-INFINITY);
+                        for (int e = 0; e < 32; ++e)
+                            if (e >= n_valid) x[e] = -INFINITY;
                     }
                     float cm0 = -INFINITY, cm1 = -INFINITY;
 #pragma unroll
-                    for (int c = 0; c < 32; c += 2) {
-                        cm0 = fmaxf(cm0, __uint_as_float(x[c]));
-                        cm1 = fmaxf(cm1, __uint_as_float(x[c + 1]));
-                    }
+                    for (int e = 0; e < 32; e += 2) cm0 = fmaxf(cm0, x[e]), cm1 = fmaxf(cm1, x[e + 1]);
                     const float cm = fmaxf(cm0, cm1);
                     if (cm > m_run) {
                         s_run *= ex2((m_run - cm) * kLog2e);  // 0 when nothing was summed yet
@@ -269,9 +325,9 @@ lm_head_topk_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_cons
                         float acc0 = 0.f, acc1 = 0.f;
                         const float nm = m_run > -INFINITY ? -m_run * kLog2e : 0.f;
 #pragma unroll
-                        for (int c = 0; c < 32; c += 2) {
-                            acc0 += ex2(fmaf(__uint_as_float(x[c]), kLog2e, nm));
-                            acc1 += ex2(fmaf(__uint_as_float(x[c + 1]), kLog2e, nm));
+                        for (int e = 0; e < 32; e += 2) {
+                            acc0 += ex2(fmaf(x[e], kLog2e, nm));
+                            acc1 += ex2(fmaf(x[e + 1], kLog2e, nm));
                         }
                         s_run += acc0 + acc1;
                     }
@@ -281,78 +337,38 @@ lm_head_topk_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_cons
                     uint32_t cand = 0u;
                     if (row_ok && cm > bar_f) {
 #pragma unroll
-                        for (int c = 0; c < 32; ++c)
-                            if (__uint_as_float(x[c]) > bar_f) cand |= 1u << c;
+                        for (int e = 0; e < 32; ++e)
+                            if (x[e] > bar_f) cand |= 1u << e;
                     }
                     while (__any_sync(0xffffffffu, cand != 0u)) {
                         if (cand) {
-                            const int c = __ffs(cand) - 1;
+                            const int e = __ffs(cand) - 1;
                             cand &= cand - 1u;
-                            uint32_t y16[16], y8[8], y4[4], y2[2];
+                            float y16[16], y8[8], y4[4], y2[2];
 #pragma unroll
-                            for (int j = 0; j < 16; ++j) y16[j] = (c & 16) ? x[16 + j] : x[j];
+                            for (int j = 0; j < 16; ++j) y16[j] = (e & 16) ? x[16 + j] : x[j];
 #pragma unroll
-                            for (int j = 0; j < 8; ++j) y8[j] = (c & 8) ? y16[8 + j] : y16[j];
+                            for (int j = 0; j < 8; ++j) y8[j] = (e & 8) ? y16[8 + j] : y16[j];
 #pragma unroll
-                            for (int j = 0; j < 4; ++j) y4[j] = (c & 4) ? y8[4 + j] : y8[j];
+                            for (int j = 0; j < 4; ++j) y4[j] = (e & 4) ? y8[4 + j] : y8[j];
 #pragma unroll
-                            for (int j = 0; j < 2; ++j) y2[j] = (c & 2) ? y4[2 + j] : y4[j];
-                            const float f = __uint_as_float((c & 1) ? y2[1] : y2[0]);
+                            for (int j = 0; j < 2; ++j) y2[j] = (e & 2) ? y4[2 + j] : y4[j];
+                            const float f = (e & 1) ? y2[1] : y2[0];
                             if (f > bar_f) {  // the bar may have risen since the bits were set
-                                const unsigned long long kth = fz_insert(list, make_key(f, (uint32_t)(v0 + c0 + c)), k);
+                                const unsigned long long kth = fz_insert(list, make_key(f, (uint32_t)(v0 + c0 + e)), k);
                                 if (kth) bar_f = key_value(kth);
                             }
                         }
                     }
                 }
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) {
-                if (PAIR) mbar_arrive_in(smem_u32(&bars.acc_empty[a]), 0);
-                else mbar_arrive(smem_u32(&bars.acc_empty[a]));
-            }
-        }
-        // ---- the two column halves of a row become one partial ------------------------------------------
-        // The ring is free: the last accumulator's completion covered every instruction that read it,
-        // and every copy into it had landed before that.
-        if (ok) {
-            float2* c_ms = reinterpret_cast<float2*>(smem_gen);                              // [128]
-            unsigned long long* c_keys = reinterpret_cast<unsigned long long*>(smem_gen + 1024);  // [kFzMaxK][128]
-            if (half == 1) {
-                if (row_ok) {
-                    c_ms[r_local] = make_float2(m_run, s_run);
+            if (ok && row_ok) {
+                const size_t part = (size_t)(row0 + r_local) * slots + blockIdx.x;
+                stats[part] = make_double2((double)m_run, (double)s_run);
 #pragma unroll
-                    for (int j = 0; j < kFzMaxK; ++j)
-                        if (j < k) c_keys[j * 128 + r_local] = list[j];
-                }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&bars.comb));
-            } else {
-                int r = 1;
-                if (lane == 0) r = mbar_wait(smem_u32(&bars.comb), 0, ctl) ? 1 : 0;
-                ok = __shfl_sync(0xffffffffu, r, 0) != 0;
-                if (ok && row_ok) {
-                    const float2 o = c_ms[r_local];
-                    const float m = fmaxf(m_run, o.x);
-                    float sum = 0.f;
-                    if (m_run > -INFINITY) sum += s_run * ex2((m_run - m) * kLog2e);
-                    if (o.x > -INFINITY) sum += o.y * ex2((o.x - m) * kLog2e);
-                    if (!(m_run > -INFINITY) && s_run != s_run) sum = s_run;  // NaN among nothing but -inf
-                    if (!(o.x > -INFINITY) && o.y != o.y) sum = o.y;
-#pragma unroll
-                    for (int j = 0; j < kFzMaxK; ++j)
-                        if (j < k) {
-                            const unsigned long long key = c_keys[j * 128 + r_local];
-                            if (key) fz_insert(list, key, k);
-                        }
-                    const size_t part = (size_t)(row0 + (int)rank * 128 + r_local) * slots + unit;
-                    stats[part] = make_double2((double)m, (double)sum);
-#pragma unroll
-                    for (int j = 0; j < kFzMaxK; ++j)
-                        if (j < k) keys[part * k + j] = list[j];
-                    if (!(m < INFINITY) || sum != sum) raise_status(d_status, EAGLE2_STATUS_NONFINITE_LOGIT);
-                }
+                for (int j = 0; j < kFzMaxK; ++j)
+                    if (j < k) keys[part * k + j] = list[j];
+                if (!(m_run < INFINITY) || s_run != s_run) raise_status(d_status, EAGLE2_STATUS_NONFINITE_LOGIT);
             }
         }
     }
@@ -407,12 +423,13 @@ static bool fz_matrix_map(CUtensorMap* map, const void* base, long long n_rows, 
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// Partials per row: one per block (pair of blocks) of the launch, a block per SM or fewer when the
-// vocabulary has fewer tiles; never more than the row merge holds.
-static int fz_chunks(int V, bool pair) {
-    const int n_tiles = (V + kFzTileV - 1) / kFzTileV;
+// Units of a launch: blocks (pairs) that walk vocabulary tiles, one per SM (TPC) or fewer when the
+// vocabulary has fewer tiles.  Every block writes one partial per row.
+static int fz_units(int V, bool pair) {
+    const int tile_v = pair ? 2 * kFzTileV : kFzTileV;
+    const int n_tiles = (V + tile_v - 1) / tile_v;
     int units = pair ? sm_count() / 2 : sm_count();
-    if (units > 160) units = 160;
+    if (units > (pair ? 80 : 160)) units = pair ? 80 : 160;  // never more partials than the row merge holds
     if (units < 1) units = 1;
     return n_tiles < units ? n_tiles : units;
 }
@@ -423,16 +440,22 @@ struct FzPasses {
     int full;        // pair passes of 256 rows
     int rest;        // rows of the last pass (0: none)
     bool rest_pair;  // the last pass uses block pairs
-    int chunks_pair, chunks_single, slots;
+    int units_pair, units_single;
+    int producers_pair, producers_single;  // blocks = partials per row of such a pass
+    int slots;                             // partial places per row: the larger of those in use
 };
 static FzPasses fz_passes(long long rows, int V) {
     FzPasses p;
-    p.full = rows > 128 ? (int)(rows / 256) : 0;
-    p.rest = (int)(rows - (long long)p.full * 256);
+    p.full = rows > 128 ? (int)(rows / kFzMaxRows) : 0;
+    p.rest = (int)(rows - (long long)p.full * kFzMaxRows);
     p.rest_pair = p.rest > 128;
-    p.chunks_pair = fz_chunks(V, true), p.chunks_single = fz_chunks(V, false);
-    p.slots = (p.rest && !p.rest_pair) ? p.chunks_single : p.chunks_pair;
-    if (p.full && p.chunks_pair > p.slots) p.slots = p.chunks_pair;
+    p.units_pair = fz_units(V, true), p.units_single = fz_units(V, false);
+    p.producers_pair = 2 * p.units_pair, p.producers_single = p.units_single;
+    const bool any_pair = p.full > 0 || (p.rest && p.rest_pair), any_single = p.rest && !p.rest_pair;
+    p.slots = 0;
+    if (any_pair) p.slots = p.producers_pair;
+    if (any_single && p.producers_single > p.slots) p.slots = p.producers_single;
+    if (p.slots < 1) p.slots = 1;
     return p;
 }
 
@@ -449,19 +472,36 @@ size_t lm_head_expand_workspace_bytes(int B, int V, int k) {
     return a > b ? a : b;
 }
 
+// One pass: `rows` feature rows starting at row0 of the call's `rows_total`.
 template <bool PAIR>
-static int fz_launch(const CUtensorMap& w_map, const CUtensorMap& h_map, int rows, int row0, int H, int V, int k, int chunks, int slots,
-                     double2* stats, unsigned long long* keys, int32_t* d_status, cudaStream_t st) {
-    constexpr uint32_t kStageBytes = kFzABytes + (PAIR ? kFzTileV / 2 : kFzTileV) * kFzTileK * 2;
-    const int stages = PAIR ? 6 : 4;
-    const size_t dyn = (size_t)stages * kStageBytes + 1024;
+static int fz_launch(const CUtensorMap& w_map, const void* hidden, long long rows_total, int rows, int row0, int H, int V,
+                     int k, int units, int slots, double2* stats, unsigned long long* keys, int32_t* d_status,
+                     cudaStream_t st) {
+    const int n_pad = (rows + 15) / 16 * 16;       // N of the instruction
+    const int b_rows = PAIR ? n_pad / 2 : n_pad;   // feature rows a block copies: a multiple of 8
+    const uint32_t b_bytes = (uint32_t)b_rows * kFzTileK * 2;
+    const uint32_t stage_bytes = kFzABytes + b_bytes;
+    CUtensorMap h_map;
+    if (!fz_matrix_map(&h_map, hidden, rows_total, H, b_rows)) return EAGLE2_ERR_CUDA;
+    // As many stages as fit beside the transposition units: two per scanner warp with work if that
+    // leaves six stages, else one (static shared memory: the barriers).
+    constexpr size_t kDynMax = 229000;
+    const int n_chunks = (rows + 31) / 32;
+    int t_slots = 2;
+    int stages = (int)((kDynMax - 1024 - (size_t)n_chunks * t_slots * kFzTBytes) / stage_bytes);
+    if (stages < 6) {
+        t_slots = 1;
+        stages = (int)((kDynMax - 1024 - (size_t)n_chunks * t_slots * kFzTBytes) / stage_bytes);
+    }
+    if (stages > kFzMaxStages) stages = kFzMaxStages;
+    const size_t dyn = 1024 + (size_t)stages * stage_bytes + (size_t)n_chunks * t_slots * kFzTBytes;
     if (cudaFuncSetAttribute(lm_head_topk_kernel<PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) != cudaSuccess) {
         cudaGetLastError();
         return EAGLE2_ERR_CUDA;
     }
-    return launch_chained(lm_head_topk_kernel<PAIR>, dim3((unsigned)(chunks * (PAIR ? 2 : 1))), dim3(kFzThreads), dyn, st,
-                          PAIR ? 2u : 1u, w_map, h_map, rows, row0, H, V, k, stages, chunks, slots, wait_limit_cycles(), stats, keys,
-                          d_status);
+    return launch_chained(lm_head_topk_kernel<PAIR>, dim3((unsigned)(units * (PAIR ? 2 : 1))), dim3(kFzThreads), dyn, st,
+                          PAIR ? 2u : 1u, w_map, h_map, rows, n_pad, row0, H, V, k, stages, t_slots, units, slots, b_bytes,
+                          wait_limit_cycles(), stats, keys, d_status);
 }
 
 }  // namespace eagle2
@@ -488,21 +528,22 @@ extern "C" int eagle2_lm_head_expand(const void* hidden, const void* weight, int
     double2* stats = nullptr;
     unsigned long long* keys = nullptr;
     if (!expand_partials_layout(B, n_s, p.slots, k, ws, second, &stats, &keys)) return EAGLE2_ERR_WORKSPACE;
-    CUtensorMap w_pair, w_single, h_map;
-    // vocabulary rows past V and feature rows past the last one read as zero
-    if (!fz_matrix_map(&w_pair, weight, V, H, kFzTileV / 2) || !fz_matrix_map(&w_single, weight, V, H, kFzTileV) ||
-        !fz_matrix_map(&h_map, hidden, rows, H, 128))
-        return EAGLE2_ERR_CUDA;
+    CUtensorMap w_map;  // vocabulary rows past V read as zero
+    if (!fz_matrix_map(&w_map, weight, V, H, kFzTileV)) return EAGLE2_ERR_CUDA;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     int rc = EAGLE2_OK;
     for (int i = 0; i < p.full && rc == EAGLE2_OK; ++i)
-        rc = fz_launch<true>(w_pair, h_map, 256, i * 256, H, V, k, p.chunks_pair, p.slots, stats, keys, d_status, st);
+        rc = fz_launch<true>(w_map, hidden, rows, kFzMaxRows, i * kFzMaxRows, H, V, k, p.units_pair, p.slots, stats, keys,
+                             d_status, st);
     if (rc == EAGLE2_OK && p.rest)
-        rc = p.rest_pair ? fz_launch<true>(w_pair, h_map, p.rest, p.full * 256, H, V, k, p.chunks_pair, p.slots, stats, keys, d_status, st)
-                         : fz_launch<false>(w_single, h_map, p.rest, p.full * 256, H, V, k, p.chunks_single, p.slots, stats, keys, d_status, st);
+        rc = p.rest_pair ? fz_launch<true>(w_map, hidden, rows, p.rest, p.full * kFzMaxRows, H, V, k, p.units_pair, p.slots,
+                                           stats, keys, d_status, st)
+                         : fz_launch<false>(w_map, hidden, rows, p.rest, p.full * kFzMaxRows, H, V, k, p.units_single, p.slots,
+                                            stats, keys, d_status, st);
     if (rc != EAGLE2_OK) return rc;
-    rc = launch_expand_row_merge(B, n_s, p.slots, (long long)p.full * 256, p.chunks_pair,
-                                 p.rest_pair ? p.chunks_pair : p.chunks_single, k, ws, ws_rows, st);
+    const int rest_producers = p.rest_pair ? p.producers_pair : p.producers_single;
+    rc = launch_expand_row_merge(B, n_s, p.slots, (long long)p.full * kFzMaxRows, p.full ? p.producers_pair : rest_producers,
+                                 p.rest ? rest_producers : p.producers_pair, k, ws, ws_rows, st);
     if (rc != EAGLE2_OK) return rc;
     return launch_expand_merge(B, V, k, D, s, 1, tree_token, tree_parent, tree_value, frontier, ws_rows, d_status, st);
 }
