@@ -485,7 +485,12 @@ static int fz_launch(const CUtensorMap& w_map, const void* hidden, long long row
     if (!fz_matrix_map(&h_map, hidden, rows_total, H, b_rows)) return EAGLE2_ERR_CUDA;
     // As many stages as fit beside the transposition units: two per scanner warp with work if that
     // leaves six stages, else one (static shared memory: the barriers).
-    constexpr size_t kDynMax = 229000;
+    cudaFuncAttributes fa;
+    if (cudaFuncGetAttributes(&fa, lm_head_topk_kernel<PAIR>) != cudaSuccess) {
+        cudaGetLastError();
+        return EAGLE2_ERR_CUDA;
+    }
+    const size_t kDynMax = (size_t)227 * 1024 - fa.sharedSizeBytes;  // what a block may hold, less the static part
     const int n_chunks = (rows + 31) / 32;
     int t_slots = 2;
     int stages = (int)((kDynMax - 1024 - (size_t)n_chunks * t_slots * kFzTBytes) / stage_bytes);
