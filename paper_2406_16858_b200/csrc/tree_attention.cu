@@ -613,14 +613,18 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
                 const uint32_t qk_hi = (uint32_t)(qd_first >> 32), v_hi = (uint32_t)(vd_first >> 32);
                 int k_st = 0, v_st = 0;        // ring stage of the K tile the next Q.K^T reads, of the V tile the next P.V reads
                 uint32_t k_ph = 0, v_ph = 0;   // and the phases of their barriers
-                auto issue_qk = [&](int i) {  // S[slot] = Q[row tile] . K[tile]^T
-                    const int t = i & (MT - 1);
-                    if (t == 0) {
+                // Waits and issues are separate steps: the loop below first makes sure that everything
+                // the next sixteen instructions read is in place, then issues them back to back (the
+                // lane's own instructions between two groups of eight - waits, commits, address
+                // arithmetic - otherwise leave the tensor pipe idle for ~0.2 us each time).
+                auto wait_qk = [&](int i) {   // the K tile of item i has landed (both halves of a pair)
+                    if ((i & (MT - 1)) == 0) {
                         ok = ok && wait1(smem_u32(&bars.k_full[k_st]), k_ph);
                         if (PAIR) ok = ok && wait1(smem_u32(&bars.k_peer[k_st]), k_ph);
                     }
-                    if (!ok) return;
-                    tc_fence_after();
+                };
+                auto issue_qk = [&](int i) {  // S[slot] = Q[row tile] . K[tile]^T
+                    const int t = i & (MT - 1);
                     const uint32_t d_tmem = tmem + (uint32_t)(i & 1) * kTK;
                     const uint32_t q_lo = q_lo0 + (uint32_t)t * (kTile >> 4), k_lo = k_lo0 + (uint32_t)k_st * (kKTile >> 4);
 #pragma unroll
@@ -636,7 +640,7 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
                         if (++k_st == NST) k_st = 0, k_ph ^= 1u;
                     }
                 };
-                auto issue_pv = [&](int i) {  // O[row tile] += P[slot] . V[tile]
+                auto wait_pv = [&](int i) {   // the V tile of item i has landed, its probabilities are written
                     const int t = i & (MT - 1), j = MT == 1 ? i : (i >> 1);
                     if (t == 0) {
                         ok = ok && wait1(smem_u32(&bars.v_full[v_st]), v_ph);
@@ -647,8 +651,9 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
                         if (PAIR) ok = ok && wait1(smem_u32(&bars.v_peer[v_st]), v_ph);
                     }
                     ok = ok && wait1(smem_u32(&bars.p_full[i & 1]), (uint32_t)((i >> 1) & 1));
-                    if (!ok) return;
-                    tc_fence_after();
+                };
+                auto issue_pv = [&](int i) {  // O[row tile] += P[slot] . V[tile]
+                    const int t = i & (MT - 1);
                     const uint32_t d_tmem = tmem + kOCol + (uint32_t)(i & 1) * DH;  // accumulator = slot = item parity
                     const uint32_t a_tmem = tmem + (uint32_t)(i & 1) * kTK;
                     const uint32_t v_lo = v_lo0 + (uint32_t)v_st * (kVTile >> 4);
@@ -665,10 +670,20 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
                     }
                 };
                 static_assert(kSlots == 2, "slot = item & 1");
-                for (int i = 0; i < kSlots && i < n_items && ok; ++i) issue_qk(i);
+                for (int i = 0; i < kSlots && i < n_items && ok; ++i) {
+                    wait_qk(i);
+                    if (!ok) break;
+                    tc_fence_after();
+                    issue_qk(i);
+                }
                 for (int i = 0; i < n_items && ok; ++i) {
+                    const bool more = i + kSlots < n_items;
+                    wait_pv(i);
+                    if (more) wait_qk(i + kSlots);
+                    if (!ok) break;
+                    tc_fence_after();
                     issue_pv(i);
-                    if (ok && i + kSlots < n_items) issue_qk(i + kSlots);
+                    if (more) issue_qk(i + kSlots);
                 }
             }
         }
