@@ -242,6 +242,16 @@ int eagle2_tree_mask(const int32_t* sel_parent, const int32_t* sel_depth, const 
                      const int32_t* kv_len, int B, int m, uint64_t* mask_bits, uint8_t* mask_dense,
                      int32_t* pos_ids, int32_t* d_status, eagle2_stream_t stream);
 
+/*
+ * Steps 2a and 2b in one launch (paper Section 4.2): eagle2_rerank followed by eagle2_tree_mask on
+ * its selection, with the same outputs, limits and status bits as the two calls; the block that has
+ * chosen a sequence's nodes writes their mask rows and position ids itself.
+ */
+int eagle2_rerank_mask(const int32_t* tree_token, const int32_t* tree_parent, const double* tree_value,
+                       const int32_t* kv_len, int B, int k, int D, int m, int32_t* sel_index, int32_t* sel_parent,
+                       int32_t* sel_token, int32_t* sel_depth, int32_t* n_sel, uint64_t* mask_bits,
+                       uint8_t* mask_dense, int32_t* pos_ids, int32_t* d_status, eagle2_stream_t stream);
+
 /* Kernels one eagle2_tree_attention call launches at these sizes (bookkeeping for benchmarks and
  * graph builders; 0 for sizes the call would refuse): the attention kernel, a list kernel in front
  * of it when a ragged batch is served longest first, and a merge kernel behind it when the splits of

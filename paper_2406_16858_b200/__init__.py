@@ -8,4 +8,4 @@ from .binding import (  # noqa: F401
     Eagle2Error, OP_ACCEPT, OP_EXPAND, OP_KV_COMPACT, OP_RERANK, OP_TREE_ATTENTION, OP_TREE_MASK,
     STATUS_BAD_TREE, STATUS_KV_OVERFLOW, STATUS_NONFINITE_LOGIT, STATUS_NOT_CLOSED,
     EXPAND_BY_CONFIDENCE, STATUS_TIMEOUT, accept, expand, expand_static, expand_variant, kv_compact, lib, lib_path, lm_head, lm_head_expand, OP_LM_HEAD_EXPAND,
-    rerank, rerank_skipped, set_wait_limit, strerror, tree_attention, tree_attention_launches, tree_mask, version, workspace_bytes, workspace_init)
+    rerank, rerank_mask, rerank_skipped, set_wait_limit, strerror, tree_attention, tree_attention_launches, tree_mask, version, workspace_bytes, workspace_init)

@@ -23,7 +23,7 @@ EXPORTS = ("eagle2_version", "eagle2_strerror", "eagle2_workspace_bytes", "eagle
            "eagle2_expand", "eagle2_rerank", "eagle2_tree_mask", "eagle2_tree_attention",
            "eagle2_accept", "eagle2_kv_compact", "eagle2_expand_static", "eagle2_expand_variant",
            "eagle2_rerank_skipped", "eagle2_lm_head", "eagle2_set_wait_limit",
-           "eagle2_tree_attention_launches", "eagle2_lm_head_expand")
+           "eagle2_tree_attention_launches", "eagle2_lm_head_expand", "eagle2_rerank_mask")
 EXPAND_BY_CONFIDENCE = 1
 
 
@@ -72,6 +72,8 @@ def lib() -> C.CDLL:
         h.eagle2_lm_head.restype = i32
         h.eagle2_rerank_skipped.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp]
         h.eagle2_rerank_skipped.restype = i32
+        h.eagle2_rerank_mask.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+        h.eagle2_rerank_mask.restype = i32
         h.eagle2_tree_mask.argtypes = [vp, vp, vp, vp, i32, i32, vp, vp, vp, vp, vp]
         h.eagle2_tree_attention.argtypes = [vp, vp, vp, i64, vp, vp, vp, i32, i32, i32, i32, i32, i32,
                                             f32, vp, vp, vp, sz, vp, vp]
@@ -188,6 +190,15 @@ def rerank(tree_token, tree_parent, tree_value, B: int, k: int, D: int, m: int, 
         _ptr(tree_token), _ptr(tree_parent), _ptr(tree_value), B, k, D, m, _ptr(sel_index),
         _ptr(sel_parent), _ptr(sel_token), _ptr(sel_depth), _ptr(n_sel), _ptr(d_status),
         _stream(stream)))
+
+
+def rerank_mask(tree_token, tree_parent, tree_value, kv_len, B: int, k: int, D: int, m: int, sel_index, sel_parent,
+                sel_token, sel_depth, n_sel, mask_bits, mask_dense, pos_ids, d_status, stream=None) -> None:
+    """``rerank`` and ``tree_mask`` in one launch."""
+    _check("eagle2_rerank_mask", lib().eagle2_rerank_mask(
+        _ptr(tree_token), _ptr(tree_parent), _ptr(tree_value), _ptr(kv_len), B, k, D, m, _ptr(sel_index),
+        _ptr(sel_parent), _ptr(sel_token), _ptr(sel_depth), _ptr(n_sel), _ptr(mask_bits), _ptr(mask_dense),
+        _ptr(pos_ids), _ptr(d_status), _stream(stream)))
 
 
 def rerank_skipped(tree_token, tree_parent, tree_value, frontier, B: int, k: int, D: int, m: int, sel_index,

@@ -16,6 +16,41 @@ __device__ __forceinline__ unsigned long long value_code(double x) {
     return (u >> 63) ? ~u : (u | 0x8000000000000000ull);
 }
 
+// Row i of the ancestor mask (bit i and the bits of all ancestors of flat node i; a padding row has
+// only its own bit) and its position id, from the selection's parent links in shared memory.
+// Returns status bits.
+__device__ __forceinline__ int mask_row(const int32_t* s_par, int i, int ns, int m, int b, int pos,
+                                        uint64_t* __restrict__ mask_bits, uint8_t* __restrict__ mask_dense,
+                                        int32_t* __restrict__ pos_ids) {
+    const int W = (m + 63) / 64;
+    uint64_t row[(EAGLE2_MAX_M + 63) / 64] = {0, 0};
+    int status = 0;
+    row[i >> 6] |= 1ull << (i & 63);
+    if (i < ns) {
+        int a = i;
+        for (;;) {
+            const int p = s_par[a];
+            if (p < 0) {
+                if (p < -1) status |= EAGLE2_STATUS_BAD_TREE;
+                break;
+            }
+            if (p >= a) {  // parents precede children: also bounds the walk
+                status |= EAGLE2_STATUS_BAD_TREE;
+                break;
+            }
+            row[p >> 6] |= 1ull << (p & 63);
+            a = p;
+        }
+    }
+    for (int w = 0; w < W; ++w) mask_bits[((long long)b * m + i) * W + w] = row[w];
+    pos_ids[(long long)b * m + i] = pos;
+    if (mask_dense) {
+        uint8_t* d = mask_dense + ((long long)b * m + i) * m;
+        for (int j = 0; j < m; ++j) d[j] = (uint8_t)((row[j >> 6] >> (j & 63)) & 1ull);
+    }
+    return status;
+}
+
 // Values are compared as integer codes throughout (fp64 compares are slow on this part).  The
 // ranking is a bitonic sort of (code, index) pairs, padded to a power of two with code 0, which
 // sorts behind every real value.  With `frontier` given there is no ranking at all (the ablation
@@ -26,8 +61,10 @@ rerank_kernel(const int32_t* __restrict__ tree_token, const int32_t* __restrict_
               const double* __restrict__ tree_value, const int32_t* __restrict__ frontier, int k, int N,
               int P, int m, int most, int32_t* __restrict__ sel_index, int32_t* __restrict__ sel_parent,
               int32_t* __restrict__ sel_token, int32_t* __restrict__ sel_depth,
-              int32_t* __restrict__ n_sel, int32_t* d_status) {
+              int32_t* __restrict__ n_sel, const int32_t* __restrict__ kv_len, uint64_t* __restrict__ mask_bits,
+              uint8_t* __restrict__ mask_dense, int32_t* __restrict__ pos_ids, int32_t* d_status) {
     extern __shared__ __align__(16) unsigned char s_dyn[];
+    __shared__ int32_t s_selpar[EAGLE2_MAX_M], s_seldep[EAGLE2_MAX_M];  // the selection, for the mask rows
     unsigned long long* s_code = reinterpret_cast<unsigned long long*>(s_dyn);  // [N] value codes
     unsigned long long* s_key = s_code + N;                                     // [P] sort keys
     int32_t* s_idx = reinterpret_cast<int32_t*>(s_key + P);                     // [P] sort payload
@@ -181,18 +218,28 @@ rerank_kernel(const int32_t* __restrict__ tree_token, const int32_t* __restrict_
             fp = s_flat[p];
             if (fp < 0) status |= EAGLE2_STATUS_NOT_CLOSED;
         }
+        const int dep = i < k ? 0 : 1 + (i - k) / (k * k);
         o_idx[j] = i;
         o_par[j] = fp;
         o_tok[j] = tok[i];
-        o_dep[j] = i < k ? 0 : 1 + (i - k) / (k * k);
+        o_dep[j] = dep;
+        s_selpar[j] = fp;
+        s_seldep[j] = dep;
     }
     for (int j = keep + tid; j < m; j += kRerankThreads) {
         o_idx[j] = -1;
         o_par[j] = -1;
         o_tok[j] = 0;
         o_dep[j] = 0;
+        s_selpar[j] = -1;
+        s_seldep[j] = 0;
     }
     if (tid == 0) n_sel[b] = keep;
+    if (mask_bits) {  // the mask rows and position ids of this selection, in the same launch
+        __syncthreads();
+        if (tid < m) status |= mask_row(s_selpar, tid, keep, m, b, kv_len[b] + (tid < keep ? s_seldep[tid] : 0), mask_bits,
+                                        mask_dense, pos_ids);
+    }
     if (status) raise_status(d_status, status);
 }
 
@@ -205,36 +252,12 @@ tree_mask_kernel(const int32_t* __restrict__ sel_parent, const int32_t* __restri
     chain_wait();
     chain_release();
     const int b = blockIdx.x, i = threadIdx.x;
-    const int W = (m + 63) / 64;
     const int ns = n_sel[b];
     if (i < m) s_par[i] = sel_parent[(long long)b * m + i];
     __syncthreads();
     if (i >= m) return;
-    uint64_t row[(EAGLE2_MAX_M + 63) / 64] = {0, 0};
-    int status = 0;
-    row[i >> 6] |= 1ull << (i & 63);
-    if (i < ns) {
-        int a = i;
-        for (;;) {
-            const int p = s_par[a];
-            if (p < 0) {
-                if (p < -1) status |= EAGLE2_STATUS_BAD_TREE;
-                break;
-            }
-            if (p >= a) {  // parents precede children: also bounds the walk
-                status |= EAGLE2_STATUS_BAD_TREE;
-                break;
-            }
-            row[p >> 6] |= 1ull << (p & 63);
-            a = p;
-        }
-    }
-    for (int w = 0; w < W; ++w) mask_bits[((long long)b * m + i) * W + w] = row[w];
-    pos_ids[(long long)b * m + i] = kv_len[b] + (i < ns ? sel_depth[(long long)b * m + i] : 0);
-    if (mask_dense) {
-        uint8_t* d = mask_dense + ((long long)b * m + i) * m;
-        for (int j = 0; j < m; ++j) d[j] = (uint8_t)((row[j >> 6] >> (j & 63)) & 1ull);
-    }
+    const int status = mask_row(s_par, i, ns, m, b, kv_len[b] + (i < ns ? sel_depth[(long long)b * m + i] : 0), mask_bits,
+                                mask_dense, pos_ids);
     if (status) raise_status(d_status, status);
 }
 
@@ -246,6 +269,7 @@ using namespace eagle2;
 static int rerank_launch(const int32_t* tree_token, const int32_t* tree_parent, const double* tree_value,
                          const int32_t* frontier, int B, int k, int D, int m, int32_t* sel_index,
                          int32_t* sel_parent, int32_t* sel_token, int32_t* sel_depth, int32_t* n_sel,
+                         const int32_t* kv_len, uint64_t* mask_bits, uint8_t* mask_dense, int32_t* pos_ids,
                          int32_t* d_status, eagle2_stream_t stream) {
     if (!tree_token || !tree_parent || !tree_value || !sel_index || !sel_parent || !sel_token ||
         !sel_depth || !n_sel || !d_status)
@@ -267,7 +291,7 @@ static int rerank_launch(const int32_t* tree_token, const int32_t* tree_parent, 
         return EAGLE2_ERR_CUDA;
     return launch_chained(rerank_kernel, dim3(B), dim3(kRerankThreads), dyn, reinterpret_cast<cudaStream_t>(stream), 1,
                           tree_token, tree_parent, tree_value, frontier, k, N, P, m, most, sel_index, sel_parent,
-                          sel_token, sel_depth, n_sel, d_status);
+                          sel_token, sel_depth, n_sel, kv_len, mask_bits, mask_dense, pos_ids, d_status);
 }
 
 extern "C" int eagle2_rerank(const int32_t* tree_token, const int32_t* tree_parent,
@@ -275,7 +299,18 @@ extern "C" int eagle2_rerank(const int32_t* tree_token, const int32_t* tree_pare
                              int32_t* sel_parent, int32_t* sel_token, int32_t* sel_depth,
                              int32_t* n_sel, int32_t* d_status, eagle2_stream_t stream) {
     return rerank_launch(tree_token, tree_parent, tree_value, nullptr, B, k, D, m, sel_index, sel_parent,
-                         sel_token, sel_depth, n_sel, d_status, stream);
+                         sel_token, sel_depth, n_sel, nullptr, nullptr, nullptr, nullptr, d_status, stream);
+}
+
+extern "C" int eagle2_rerank_mask(const int32_t* tree_token, const int32_t* tree_parent, const double* tree_value,
+                                  const int32_t* kv_len, int B, int k, int D, int m, int32_t* sel_index,
+                                  int32_t* sel_parent, int32_t* sel_token, int32_t* sel_depth, int32_t* n_sel,
+                                  uint64_t* mask_bits, uint8_t* mask_dense, int32_t* pos_ids, int32_t* d_status,
+                                  eagle2_stream_t stream) {
+    if (!kv_len || !mask_bits || !pos_ids) return EAGLE2_ERR_NULL;
+    if (!aligned(mask_bits, 8)) return EAGLE2_ERR_ALIGN;
+    return rerank_launch(tree_token, tree_parent, tree_value, nullptr, B, k, D, m, sel_index, sel_parent,
+                         sel_token, sel_depth, n_sel, kv_len, mask_bits, mask_dense, pos_ids, d_status, stream);
 }
 
 extern "C" int eagle2_rerank_skipped(const int32_t* tree_token, const int32_t* tree_parent,
@@ -285,7 +320,7 @@ extern "C" int eagle2_rerank_skipped(const int32_t* tree_token, const int32_t* t
                                      int32_t* d_status, eagle2_stream_t stream) {
     if (!frontier) return EAGLE2_ERR_NULL;
     return rerank_launch(tree_token, tree_parent, tree_value, frontier, B, k, D, m, sel_index, sel_parent,
-                         sel_token, sel_depth, n_sel, d_status, stream);
+                         sel_token, sel_depth, n_sel, nullptr, nullptr, nullptr, nullptr, d_status, stream);
 }
 
 extern "C" int eagle2_tree_mask(const int32_t* sel_parent, const int32_t* sel_depth,

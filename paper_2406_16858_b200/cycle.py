@@ -78,11 +78,9 @@ class CycleBuffers:
 
     def rerank_and_mask(self, kv_len: torch.Tensor) -> None:
         s = self.shape
-        e2.rerank(self.tree_token, self.tree_parent, self.tree_value, s.B, s.k, s.D, s.m,
-                  self.sel_index, self.sel_parent, self.sel_token, self.sel_depth, self.n_sel,
-                  self.status)
-        e2.tree_mask(self.sel_parent, self.sel_depth, self.n_sel, kv_len, s.B, s.m, self.mask_bits,
-                     None, self.pos_ids, self.status)
+        e2.rerank_mask(self.tree_token, self.tree_parent, self.tree_value, kv_len, s.B, s.k, s.D, s.m,
+                       self.sel_index, self.sel_parent, self.sel_token, self.sel_depth, self.n_sel,
+                       self.mask_bits, None, self.pos_ids, self.status)
 
     def attention(self, q, k_cache, v_cache, kv_off, kv_len, out, scale: float) -> None:
         s = self.shape
@@ -106,7 +104,7 @@ class CycleBuffers:
         """Kernel launches of this library in one cycle (for bookkeeping in benchmarks)."""
         s = self.shape
         per_layer = e2.tree_attention_launches(s.B, s.m, s.Hq, s.Hkv, s.d, s.max_kv_len)
-        return s.D + 2 + s.n_layers * per_layer + (2 if s.temperature > 0 else 1) + 2
+        return s.D + 1 + s.n_layers * per_layer + (2 if s.temperature > 0 else 1) + 2
 
 
 def enqueue_cycle(buf: CycleBuffers, draft_rows, target_logits, u_accept, u_bonus, q_layers, k_layers,

@@ -64,21 +64,27 @@ class GpuTree:
 
 
 class GpuSelection:
-    def __init__(self, tree_token, tree_parent, tree_value, B, k, D, m, kv_len=None, dense=False):
+    def __init__(self, tree_token, tree_parent, tree_value, B, k, D, m, kv_len=None, dense=False, one_launch=False):
+        """one_launch: through eagle2_rerank_mask instead of eagle2_rerank + eagle2_tree_mask."""
         self.B, self.m = B, m
         z = lambda *shape: torch.zeros(shape, dtype=torch.int32, device=DEV)  # noqa: E731
         self.index, self.parent, self.token, self.depth = z(B, m), z(B, m), z(B, m), z(B, m)
         self.n_sel = z(B)
         self.status = new_status()
-        e2.rerank(tree_token, tree_parent, tree_value, B, k, D, m, self.index, self.parent, self.token,
-                  self.depth, self.n_sel, self.status)
         W = (m + 63) // 64
         self.mask_bits = torch.zeros((B, m, W), dtype=torch.int64, device=DEV)
         self.mask_dense = torch.zeros((B, m, m), dtype=torch.uint8, device=DEV) if dense else None
         self.pos_ids = z(B, m)
         self.kv_len = kv_len if kv_len is not None else z(B)
-        e2.tree_mask(self.parent, self.depth, self.n_sel, self.kv_len, B, m, self.mask_bits,
-                     self.mask_dense, self.pos_ids, self.status)
+        if one_launch:
+            e2.rerank_mask(tree_token, tree_parent, tree_value, self.kv_len, B, k, D, m, self.index, self.parent,
+                           self.token, self.depth, self.n_sel, self.mask_bits, self.mask_dense, self.pos_ids,
+                           self.status)
+        else:
+            e2.rerank(tree_token, tree_parent, tree_value, B, k, D, m, self.index, self.parent, self.token,
+                      self.depth, self.n_sel, self.status)
+            e2.tree_mask(self.parent, self.depth, self.n_sel, self.kv_len, B, m, self.mask_bits,
+                         self.mask_dense, self.pos_ids, self.status)
         torch.cuda.synchronize()
 
 

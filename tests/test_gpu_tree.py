@@ -249,6 +249,31 @@ def test_rerank_arbitrary_values_and_bad_parents():
     assert (host(got.index) == want.index).all() and (host(got.parent) == want.parent).all()
 
 
+@pytest.mark.parametrize("k,D,m,B", [(4, 3, 16, 3), (10, 6, 60, 2), (2, 2, 1, 1), (3, 3, 128, 2), (10, 6, 128, 1), (5, 4, 48, 4)])
+def test_selection_mask_and_position_ids_in_one_launch(k, D, m, B):
+    """eagle2_rerank_mask against eagle2_rerank + eagle2_tree_mask (which the tests above hold to the
+    oracle) and, for the mask and the position ids, against the oracle directly: random trees whose
+    values are not monotone along the edges, budgets below, at and above the number of nodes."""
+    rng = np.random.default_rng(100 * k + m)
+    N = ref.n_nodes(k, D)
+    token = rng.integers(0, 1000, (B, N)).astype(np.int32)
+    parent = np.full((B, N), -1, np.int32)
+    for b in range(B):
+        for i in range(k, N):
+            parent[b, i] = rng.integers(-1, i)
+    value = -rng.random((B, N)) * 5
+    kv_len = rng.integers(0, 5000, B).astype(np.int32)
+    args = (dev(token), dev(parent), dev(value), B, k, D, m)
+    two = GpuSelection(*args, kv_len=dev(kv_len), dense=True)
+    one = GpuSelection(*args, kv_len=dev(kv_len), dense=True, one_launch=True)
+    for name in ("index", "parent", "token", "depth", "n_sel", "mask_bits", "mask_dense", "pos_ids", "status"):
+        assert (host(getattr(one, name)) == host(getattr(two, name))).all(), name
+    want = ref.rerank(token, parent, value, k, D, m)
+    bits, dense, pos, _ = ref.tree_mask(want.parent, want.depth, want.n_sel, kv_len, m, dense=True)
+    assert (host(one.mask_bits).view(np.uint64) == bits).all()
+    assert (host(one.mask_dense) == dense).all() and (host(one.pos_ids) == pos).all()
+
+
 def test_zz_exempt_trees_stay_rare():
     """Runs after the tests above (file order).  On the seeded inputs of this module the oracle
     exempts no tree at all; the ceiling allows for one."""
