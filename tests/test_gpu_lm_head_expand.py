@@ -57,6 +57,8 @@ def _decided_by_rounding(want_logits, tree, b, k, D):
     (32, 10, 2, 128, 2049),    # 320 rows: two passes over the weights; ragged last vocabulary tile
     (9, 16, 2, 192, 3001),     # the widest list the fused path holds (k = 16), 144 rows
     (20, 7, 3, 64, 40000),     # more vocabulary tiles than blocks: every block folds two tiles or more
+    (13, 10, 2, 64, 3000),     # 130 rows: a pair pass whose instruction width (144) is no multiple of 32
+    (2, 4, 2, 64, 100),        # a vocabulary smaller than one tile
     (30, 10, 2, 64, 40000),    # 300 rows: a pass of block pairs, then 44 rows on single blocks (twice the producers per row)
 ])
 def test_fused_tree_against_the_oracle_pipeline(B, k, D, H, V):
