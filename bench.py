@@ -613,11 +613,20 @@ def run_ours(args):
                          ub=torch.from_numpy(ub_h).to(dev)))
     assert all(int(bb.status.item()) == 0 for bb in bufs), "device status raised while preparing inputs"
     buf = bufs[0]
+    # The sets read the same queries and write the same outputs, but the second set has copies of its
+    # own: the end to end region uploads a step's queries while the cycle of the step before (the other
+    # set) still reads its own, and reads a step's outputs back while the next cycle writes the other's.
+    q_alt, out_alt = q_all.clone(), torch.zeros_like(out_all)
+    for i, s in enumerate(sets):
+        s["q_all"] = q_alt if i == 1 else q_all
+        s["q_layers"] = list(s["q_all"].unbind(0))
+        s["out_all"] = out_alt if i == 1 else out_all
+        s["out_layers"] = list(s["out_all"].unbind(0))
 
     def one_cycle(s):
         kv_len.copy_(kv_len0)  # the cache length is caller state: start every cycle from the same prefix
-        enqueue_cycle(s["buf"], s["draft"], s["target"], s["ua"], s["ub"], q_layers, k_layers, v_layers,
-                      out_layers, k_ptrs, v_ptrs, kv_off, kv_len, scale)
+        enqueue_cycle(s["buf"], s["draft"], s["target"], s["ua"], s["ub"], s["q_layers"], k_layers, v_layers,
+                      s["out_layers"], k_ptrs, v_ptrs, kv_off, kv_len, scale)
 
     stream = torch.cuda.Stream(device=dev)
     graphs = []
@@ -729,7 +738,7 @@ def run_ours(args):
         # device copy per sequence and operand puts the rows behind the sequence's prefix in every layer
         host_in["tree_kv"] = torch.stack([torch.stack([c[:, r:r + cfg.m] for _, r in tree_rows], dim=1)
                                           for c in (k_all, v_all)], dim=1).cpu().pin_memory()
-        tree_kv_dev = torch.empty_like(host_in["tree_kv"], device=dev)
+        tree_kv_dev = [torch.empty_like(host_in["tree_kv"], device=dev) for _ in range(2)]  # one per alternating set
         host_out = {"acc_len": torch.zeros(cfg.B, dtype=torch.int32).pin_memory(),
                     "acc_path": torch.zeros((cfg.B, cfg.D), dtype=torch.int32).pin_memory(),
                     "bonus": torch.zeros(cfg.B, dtype=torch.int32).pin_memory(),
@@ -739,25 +748,29 @@ def run_ours(args):
         d2h = sum(t.numel() * t.element_size() for t in
                   [host_out["acc_len"], host_out["acc_path"], host_out["bonus"], host_out["o"]])
 
-        # Two input sets alternate.  A step's per-layer inputs go up on the compute stream, then the
-        # NEXT step's logits are handed to the copy stream, then the cycle runs: the one host-to-device
-        # engine serves the queues in the order the copies were issued, so this order lets the next
-        # logits travel under this cycle (issued before the per-layer inputs they would hold those
-        # up instead: 2270 us per step).  Results go down on a third stream under the next step's
-        # uploads; the next cycle waits for them, since it overwrites the buffers they are read from.
-        # Every step's copies, its own logits included, lie inside the timed region.
+        # Two input sets alternate.  All of a step's inputs - logits, uniforms, queries, the tree
+        # tokens' K/V rows (into a staging tensor) - go up on the copy stream, and the NEXT step's are
+        # handed to it before this step's cycle is replayed, so that they travel under it: the one
+        # host-to-device engine serves copies in the order they were issued (with the next logits
+        # issued in front of this step's per-layer inputs a step took 2270 us; with the per-layer
+        # inputs on the compute stream 1600 us).  The compute stream scatters the staged K/V rows into
+        # the caches and replays the cycle.  Results go down on a third stream under the next step's
+        # cycle, which writes the other set's output buffers; a set's next cycle waits for them.
+        # Every step's copies, its own inputs included, lie inside the timed region.
         copy_stream = torch.cuda.Stream(device=dev)
         down_stream = torch.cuda.Stream(device=dev)
         ev_in = [torch.cuda.Event() for _ in range(2)]    # set j's logits have arrived
         ev_free = [torch.cuda.Event() for _ in range(2)]  # the cycle that read set j has finished
         ev_done = torch.cuda.Event()                      # the cycle's results are ready on the device
-        ev_down = torch.cuda.Event()                      # ... and have reached the host buffers
+        ev_down = [torch.cuda.Event() for _ in range(2)]  # ... and set j's have reached the host buffers
         e2e_n = [0]                                       # steps of the running timed call
 
-        def upload_logits(j):
+        def upload_inputs(j):
             s = sets[j]
             with torch.cuda.stream(copy_stream):
-                copy_stream.wait_event(ev_free[j])
+                copy_stream.wait_event(ev_free[j])  # the cycle that read set j's buffers has finished
+                s["q_all"].copy_(host_in["q"], non_blocking=True)
+                tree_kv_dev[j].copy_(host_in["tree_kv"], non_blocking=True)
                 s["draft"].copy_(host_in["draft"], non_blocking=True)
                 s["target"].copy_(host_in["target"], non_blocking=True)
                 s["ua"].copy_(host_in["ua"], non_blocking=True)
@@ -770,16 +783,14 @@ def run_ours(args):
             if i == 0:
                 copy_stream.wait_stream(stream)  # nothing of the region starts before the region does
                 down_stream.wait_stream(stream)
-                upload_logits(0)
-            q_all.copy_(host_in["q"], non_blocking=True)
-            tree_kv_dev.copy_(host_in["tree_kv"], non_blocking=True)
-            for seq, (_, r) in enumerate(tree_rows):
-                k_all[:, r:r + cfg.m].copy_(tree_kv_dev[:, 0, seq])
-                v_all[:, r:r + cfg.m].copy_(tree_kv_dev[:, 1, seq])
+                upload_inputs(0)
             if i + 1 < e2e_n[0]:
-                upload_logits((i + 1) % 2)
-            stream.wait_event(ev_in[j])   # this step's logits are in place
-            stream.wait_event(ev_down)    # the previous step's results have left the buffers this cycle writes
+                upload_inputs((i + 1) % 2)
+            stream.wait_event(ev_in[j])   # this step's inputs are on the device
+            for seq, (_, r) in enumerate(tree_rows):
+                k_all[:, r:r + cfg.m].copy_(tree_kv_dev[j][:, 0, seq])
+                v_all[:, r:r + cfg.m].copy_(tree_kv_dev[j][:, 1, seq])
+            stream.wait_event(ev_down[j])  # the results of set j's last cycle have left the buffers this one writes
             graphs[j].replay()
             ev_free[j].record(stream)
             ev_done.record(stream)
@@ -788,10 +799,10 @@ def run_ours(args):
                 host_out["acc_len"].copy_(s["buf"].acc_len, non_blocking=True)
                 host_out["acc_path"].copy_(s["buf"].acc_path, non_blocking=True)
                 host_out["bonus"].copy_(s["buf"].bonus_token, non_blocking=True)
-                host_out["o"].copy_(out_all, non_blocking=True)
-                ev_down.record(down_stream)
+                host_out["o"].copy_(s["out_all"], non_blocking=True)
+                ev_down[j].record(down_stream)
             if i + 1 == e2e_n[0]:
-                stream.wait_event(ev_down)  # the region ends when the last results are on the host
+                stream.wait_event(ev_down[j])  # the region ends when the last results are on the host
 
         e2e_steps = max(5, min(K, 50))
         e2e_n[0] = 3
@@ -879,7 +890,7 @@ def run_ours(args):
         "per_replay_us": {"cycle": cycle_spread, "attention_layer": attn_spread, **breakdown_spread},
         "e2e": {"value": ms_e2e * 1e3 / (e2e_steps * world), "unit": "us", "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h,
-                "overlap": "the next step's logit upload (copy stream, alternate input set) runs under this step's cycle, the results go down (third stream) under the next step's uploads"},
+                "overlap": "the next step's inputs go up (copy stream, alternate input set) under this step's cycle, the results go down (third stream) under the next step's uploads"},
         "gpu_launches": buf.launches_per_cycle() * K,
         "roofline": {"kernel": "tree_attention_kernel + tree_attention_merge_kernel, one call per layer", "bound": "hbm",
                      "achieved": achieved, "peak": hbm_peak, "unit": "GB/s", "frac": achieved / hbm_peak,
