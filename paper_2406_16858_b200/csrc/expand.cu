@@ -27,11 +27,13 @@ constexpr int kMergeKeysMax = 1024;  // segment winners per row that the merge h
 
 // Segments per row.  A launch of up to three waves of one-tile blocks is about latency: one tile
 // per block.  Otherwise a block costs about kBlockFixed tile times of start-up and hand-over on top
-// of its tiles, blocks share an SM's issue slots, and the choice minimises (blocks per SM, rounded
-// up) x (cost of a block).  Never more segments per row than the merge can take, whole tiles per
+// of its tiles, an SM holds three blocks at once, and the choice minimises (rounds of resident blocks)
+// x (cost of a block): measured per call at 320 rows of 128256 logits, 1 / 2 / 3 / 4 segments per row
+// 54.7 / 63.4 / 71.1 / 76.1 us; at 80 rows the choice hardly matters (38-39 us for 2..8 segments).  Never more segments per row than the merge can take, whole tiles per
 // segment.
 static bool expand_plan(long long rows, int V, int k, ExpandPlan* p) {
     constexpr int kBlockFixed = 6;
+    constexpr int kResident = 3;  // streaming blocks an SM holds at once (shared memory, launch bounds)
     const long long kSMs = sm_count();
     const int tiles = (V + kTileTokens - 1) / kTileTokens;
     long long g_max = kMergeKeysMax / k;
@@ -43,7 +45,7 @@ static bool expand_plan(long long rows, int V, int k, ExpandPlan* p) {
         long long best = -1;
         for (long long c = 1; c <= g_max; ++c) {
             const long long tpb = (tiles + c - 1) / c;
-            const long long cost = ((rows * c + kSMs - 1) / kSMs) * (kBlockFixed + tpb);
+            const long long cost = ((rows * c + kResident * kSMs - 1) / (kResident * kSMs)) * (kBlockFixed + tpb);
             if (best < 0 || cost < best) best = cost, g = c;
         }
     }
