@@ -77,8 +77,13 @@ static void attention_plan(int B, int m, int Hq, int Hkv, int d, int max_kv_len,
     // Pairs pay off while the launch is short of blocks and every sequence is cut into several
     // splits (they halve the query and partial traffic); a launch that fills the device without
     // splitting is better served by independent blocks.
-    p->pair = (p->mt == 2 && p->q_tma && d == 128 && items * 2 <= tpcs) ? 1 : 0;
+    // ... and while the pair's blocks stay short: with long blocks the relay between the two blocks
+    // costs more per tile than the halved partials save (70B-shaped layer, 17 tiles per pair block
+    // against 8 per single block: 35.6 against 34.2 us; LLaMA3-8B-shaped layer, 4 against 2: 18.5
+    // against 19.7 us).
     const int tiles = (max_kv_len + m + kTK - 1) / kTK;
+    p->pair = (p->mt == 2 && p->q_tma && d == 128 && items * 2 <= tpcs &&
+               (tiles + tpcs / items - 1) / (tpcs / items) <= 8) ? 1 : 0;
     long long s = (p->pair ? tpcs : sms) / (items > 0 ? items : 1);
     if (s < 1) s = 1;
     if (s > tiles) s = tiles;
