@@ -32,7 +32,7 @@ namespace eagle2 {
 constexpr int kTK = 128;              // keys per K/V tile = N of the Q.K^T instruction
 constexpr int kRowsPerTile = 128;     // M of every tcgen05.mma
 constexpr int kMaxTilesPerSplit = 16; // sequences that would need longer blocks are served longest first (batches)
-constexpr int kMaxTilesPerSplitOrdered = 32;  // a block never streams more than 4096 keys
+constexpr int kMaxTilesPerSplitOrdered = 64;  // a block never streams more than 8192 keys
 constexpr int kTmemCols = 512;
 constexpr int kSlots = 2;             // score slots in tensor memory
 constexpr int kSoftmaxThreads = 512;  // 16 softmax warps: four per SM sub-partition
@@ -99,14 +99,20 @@ static void attention_plan(int B, int m, int Hq, int Hkv, int d, int max_kv_len,
     const int units = p->pair ? tpcs : sms;  // blocks (pairs) resident at once
     if (p->ordered) {
         // Only the longest length is known here and a ragged batch holds far fewer tiles than
-        // sequences x longest: aim at two blocks per SM by that count, within 8..32 tiles per block
+        // sequences x longest: aim at two blocks per SM by that count, from 8 tiles per block up to a cap
         // (long blocks leave a batch of a few sequences to a handful of SMs; short ones cost partials
         // and a block's start-up each).  Measured per layer at B = 8 / 16: 110 / 111 us with 32 tiles,
         // 105 / 121 us when aiming at four blocks per SM.
+        // The more items a launch has per SM, the longer a block may be before the longest ones decide the
+        // time (longer blocks: fewer partials, fewer start-ups): 32 tiles up to about one item per SM, 48
+        // at two (measured per layer with caps of 32 / 40 / 48 tiles: B = 16 110 / - / 133 us, B = 20
+        // 130 / 130 / 146, B = 24 148 / 142 / 149, B = 28 175 / 172 / 170, B = 32 189 / 181 / 177).
+        long long cap = 16 + 18 * items / sms;
+        cap = cap < 32 ? 32 : (cap > kMaxTilesPerSplitOrdered ? kMaxTilesPerSplitOrdered : cap);
         const long long want = (tiles * items + 2LL * units - 1) / (2LL * units);
-        per_split = (int)(want < 8 ? 8 : (want > kMaxTilesPerSplitOrdered ? kMaxTilesPerSplitOrdered : want));
-    } else if (per_split > kMaxTilesPerSplitOrdered) {
-        per_split = kMaxTilesPerSplitOrdered;  // more blocks than the device holds at once: several waves
+        per_split = (int)(want < 8 ? 8 : (want > cap ? cap : want));
+    } else if (per_split > 32) {
+        per_split = 32;  // more blocks than the device holds at once: several waves
     }
     if (per_split < 1) per_split = 1;
     p->per_split = per_split;
