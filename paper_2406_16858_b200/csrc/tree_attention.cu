@@ -951,9 +951,10 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
         uint32_t remote;
         asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(smem_u32(&s_ctl.abort)), "r"(rank ^ 1u));
         asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(remote), "r"(1u) : "memory");
+        asm volatile("fence.acq_rel.cluster;" ::: "memory");  // the flag is the one thing the meeting below hands over
     }
     tc_fence_before();
-    if (PAIR) cluster_sync_all();  // tensor memory is released by both blocks together
+    if (PAIR) cluster_sync_relaxed();  // tensor memory is released by both blocks together
     else __syncthreads();
     tc_fence_after();
     if (s_ctl.abort) {
@@ -982,7 +983,7 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
         else tmem_dealloc(tmem, kTmemCols);
     }
     if (tid == 0 && s_ctl.abort) raise_status(d_status, EAGLE2_STATUS_TIMEOUT);
-    if (PAIR) cluster_sync_all();  // neither block leaves while the other may still signal it
+    if (PAIR) cluster_sync_relaxed();  // neither block leaves while the other may still signal it
 }
 
 // Ordered launches: one block lists the (sequence, split) items that have tiles, most tiles first
