@@ -270,6 +270,10 @@ int eagle2_tree_attention_launches(int B, int m, int Hq, int Hkv, int d, int max
  *            128-row tiles, so it may read (and ignore) rows of the allocation that follow a
  *            sequence's last key; rows at or beyond cache_rows are never touched.
  *   kv_off   int64 [B], kv_len int32 [B], mask_bits as written by eagle2_tree_mask.
+ *            A launch for a single sequence reads kv_off and kv_len before it waits for the kernel
+ *            ahead of it in the stream: they must not be written by a kernel that lets its
+ *            dependents start before it completes (programmatic dependent launch with an early
+ *            trigger).  Ordinary kernels and copies, and eagle2_kv_compact's own update, are fine.
  *   out      bf16 [B][m][Hq][d];  lse fp32 [B][Hq][m], optional natural-log sum of exponentials.
  *   max_kv_len [host value] upper bound of kv_len[], used to size the launch and the workspace.
  * A sequence with kv_len outside [0, max_kv_len] or whose rows do not fit in cache_rows raises

@@ -51,8 +51,9 @@ kv_compact_kernel(void* const* __restrict__ k_layers, void* const* __restrict__ 
 __global__ void kv_len_advance_kernel(int32_t* __restrict__ kv_len, const int32_t* __restrict__ acc_path,
                                       const int32_t* __restrict__ acc_len, int B, int m, int D,
                                       int32_t* d_status) {
+    // No early release of the dependents here: whatever kernel follows may read the lengths before it
+    // waits for its predecessor (the attention kernel does), so it must not start before they are final.
     chain_wait();
-    chain_release();
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
     if (b >= B) return;
     const int len = acc_len[b];
