@@ -384,6 +384,77 @@ __device__ __forceinline__ void merge_row(const AttnPlan& plan, const AttnWs& ws
         lse[((long long)b * Hq + hq) * m + tok] = (mmax + log2f(l)) * 0.69314718055994531f;
 }
 
+// The same combination for R consecutive packed rows of one row block at once, when the sequence has
+// at most SB splits (R * SB <= 16): a block that merges its 128 or 256 rows by itself has few warps and
+// many rows, and one row at a time is one memory round trip per row.  Lane rr * SB + s fetches the
+// (maximum, sum) pair of row rr in split s; every lane fetches its DH/32 columns of all R * SB partial
+// rows before it uses any; the splits are added in the same order as in merge_row.
+template <int DH, int R, int SB>
+__device__ __forceinline__ void merge_rows_wide(const AttnPlan& plan, const AttnWs& ws, int b, int hk, int pr0, int n,
+                                                int S_b, int m, int Hq, int Hkv, __nv_bfloat16* __restrict__ out,
+                                                float* __restrict__ lse) {
+    static_assert(R * SB <= 16 && (SB & (SB - 1)) == 0, "sixteen partial rows in flight per lane");
+    const int lane = threadIdx.x & 31;
+    const int g = plan.g, S = plan.splits;
+    const int rb = pr0 / plan.per, r0 = pr0 % plan.per;
+    const size_t rows_per_block = (size_t)plan.mt * kRowsPerTile;
+    const size_t stride = (size_t)plan.n_rb * rows_per_block;  // rows between consecutive splits
+    const size_t first = (((size_t)b * Hkv + hk) * S) * stride + rb * rows_per_block + r0;
+    constexpr int PER = DH / 32;  // 4 or 2 consecutive columns per lane
+    const int rr_l = lane / SB, s_l = lane % SB;
+    const bool have = lane < R * SB && rr_l < n && s_l < S_b;
+    const float2 ml = have ? __ldcg(ws.ml + first + rr_l + (size_t)s_l * stride) : make_float2(-INFINITY, 0.f);
+    uint2 v[R][SB];
+#pragma unroll
+    for (int rr = 0; rr < R; ++rr)
+#pragma unroll
+        for (int sp = 0; sp < SB; ++sp) {
+            v[rr][sp] = make_uint2(0u, 0u);
+            if (rr < n && sp < S_b) {
+                const __nv_bfloat16* src = ws.o_part + (first + rr + (size_t)sp * stride) * DH + lane * PER;
+                if (PER == 4) v[rr][sp] = __ldcg(reinterpret_cast<const uint2*>(src));
+                else v[rr][sp].x = __ldcg(reinterpret_cast<const uint32_t*>(src));
+            }
+        }
+    float mx = ml.x;
+#pragma unroll
+    for (int o = SB / 2; o >= 1; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    // a split without visible keys leaves its partial row unwritten: weight 0, never multiplied
+    const float w = (have && ml.x != -INFINITY) ? exp2f(ml.x - mx) : 0.f;
+    float lw = w != 0.f ? ml.y * w : 0.f;
+#pragma unroll
+    for (int o = SB / 2; o >= 1; o >>= 1) lw += __shfl_xor_sync(0xffffffffu, lw, o);
+#pragma unroll
+    for (int rr = 0; rr < R; ++rr) {
+        if (rr >= n) break;  // uniform over the warp
+        float acc[PER];
+#pragma unroll
+        for (int e = 0; e < PER; ++e) acc[e] = 0.f;
+#pragma unroll
+        for (int sp = 0; sp < SB; ++sp) {
+            const float wu = __shfl_sync(0xffffffffu, w, rr * SB + sp);
+            if (sp < S_b && wu != 0.f) {
+                acc[0] += __uint_as_float(v[rr][sp].x << 16) * wu;
+                acc[1] += __uint_as_float(v[rr][sp].x & 0xffff0000u) * wu;
+                if (PER == 4) {
+                    acc[PER - 2] += __uint_as_float(v[rr][sp].y << 16) * wu;
+                    acc[PER - 1] += __uint_as_float(v[rr][sp].y & 0xffff0000u) * wu;
+                }
+            }
+        }
+        const float l = __shfl_sync(0xffffffffu, lw, rr * SB), mmax = __shfl_sync(0xffffffffu, mx, rr * SB);
+        const float inv = l > 0.f ? 1.f / l : 0.f;
+        const int pr = pr0 + rr;
+        const int tok = pr / g, hq = hk * g + pr % g;
+        __nv_bfloat16* dst = out + (((long long)b * m + tok) * Hq + hq) * DH + lane * PER;
+#pragma unroll
+        for (int e = 0; e < PER; e += 2)
+            *reinterpret_cast<uint32_t*>(dst + e) = pack_bf16(acc[e] * inv, acc[e + 1] * inv);
+        if (lse && lane == 0)
+            lse[((long long)b * Hq + hq) * m + tok] = (mmax + log2f(l)) * 0.69314718055994531f;
+    }
+}
+
 template <int DH, int MT, bool PAIR>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map,
@@ -950,8 +1021,22 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
         __shared__ int s_last;
         int* ticket = ws.tickets + (((size_t)b * Hkv + hk) * plan.n_rb + rb) * (PAIR ? 2 : 1) + rank;
         if (last_block_arrives(ticket, S_b, &s_last)) {
-            for (int r = warp; r < rows_here; r += kAttnThreads / 32)
-                merge_row<DH>(plan, ws, b, hk, row0 + r, S_b, m, Hq, Hkv, out, lse);
+            constexpr int NW = kAttnThreads / 32;
+            auto wide = [&](auto r_tag, auto s_tag) {
+                constexpr int R = decltype(r_tag)::value, SB = decltype(s_tag)::value;
+                for (int r = warp * R; r < rows_here; r += NW * R)
+                    merge_rows_wide<DH, R, SB>(plan, ws, b, hk, row0 + r, min(R, rows_here - r), S_b, m, Hq, Hkv, out, lse);
+            };
+            if (S_b <= 2) {
+                wide(std::integral_constant<int, 8>{}, std::integral_constant<int, 2>{});
+            } else if (S_b <= 4) {
+                wide(std::integral_constant<int, 4>{}, std::integral_constant<int, 4>{});
+            } else if (S_b <= 8) {
+                wide(std::integral_constant<int, 2>{}, std::integral_constant<int, 8>{});
+            } else {
+                for (int r = warp; r < rows_here; r += NW)
+                    merge_row<DH>(plan, ws, b, hk, row0 + r, S_b, m, Hq, Hkv, out, lse);
+            }
         }
     }
 
