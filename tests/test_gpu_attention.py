@@ -133,11 +133,15 @@ def test_ragged_batch_runs_longest_first_with_several_splits():
 @pytest.mark.parametrize("m,Hq,Hkv,d,B,longest", [
     (33, 8, 8, 64, 20, 6000),    # head_dim 64: deeper K/V ring, two splits for the longest sequences
     (40, 6, 2, 128, 80, 5000),   # three query heads per KV head: query rows copied by hand, not by TMA
+    (60, 32, 8, 128, 8, 16384),  # few long sequences on block pairs: four and five splits merged inside the kernel
+    (60, 3, 1, 128, 37, 16384),  # short blocks: eight and nine splits per long sequence (nine: one row per warp at a time)
 ])
 def test_ordered_launch_other_shapes(m, Hq, Hkv, d, B, longest):
     rng = np.random.default_rng(B + d)
     lens = rng.integers(0, 900, B)
     lens[[1, B // 2, B - 2]] = [longest, longest - 1700, longest - 300]
+    # the device-built list and the attention kernel, which merges the splits itself: no merge launch
+    assert e2.tree_attention_launches(B, m, Hq, Hkv, d, longest) == 2
     q, kc, vc, off, kl, bits = _inputs(41, B, m, Hq, Hkv, d, [int(x) for x in lens])
     n = 500
     samples = np.stack([rng.integers(0, B, n), rng.integers(0, Hq, n), rng.integers(0, m, n)], axis=1).astype(np.int32)
