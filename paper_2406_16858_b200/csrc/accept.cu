@@ -106,11 +106,11 @@ accept_greedy_kernel(const float* __restrict__ target_logits, long long t_stride
     __shared__ int s_arg[EAGLE2_MAX_M + 1];
     __shared__ int s_par[EAGLE2_MAX_M], s_tok[EAGLE2_MAX_M];
 
-    chain_wait();
-    chain_release();
     const int chunk = blockIdx.x % chunks;
     const int row = (blockIdx.x / chunks) % (m + 1);
     const int b = blockIdx.x / (chunks * (m + 1));
+    chain_wait();
+    chain_release();
     const int ns = min(n_sel[b], m);
     const size_t part = ((size_t)b * (m + 1) + row) * chunks + chunk;
 
@@ -253,13 +253,13 @@ accept_chain_kernel(const float* __restrict__ target_logits, long long t_stride,
                     const int32_t* __restrict__ sel_token, const int32_t* __restrict__ n_sel,
                     const float* __restrict__ u_accept, int V, int k, int m, int R, int slice, float inv_t,
                     AcceptWs ws, int32_t* d_status) {
-    chain_wait();
-    chain_release();
     cg::cluster_group cluster = cg::this_cluster();
     const int cs = (int)cluster.num_blocks(), me = (int)cluster.block_rank();
     const int b = blockIdx.x / cs;
     const int r = blockIdx.y;  // draft row = the expanded node whose children this cluster handles
     const int tid = threadIdx.x;
+    chain_wait();
+    chain_release();
 
     extern __shared__ __align__(16) float s_rows[];  // RESIDENT: p slice then q slice
     __shared__ double s_xchg[2 * kMaxCluster * 2];
@@ -594,11 +594,11 @@ accept_bonus_kernel(const float* __restrict__ target_logits, long long t_stride,
     __shared__ double s_scan[kScanThreads];
     __shared__ int s_flag, s_pick;
 
-    chain_wait();
-    chain_release();
     const int chunk = blockIdx.x % chunks;
     const int b = blockIdx.x / chunks;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    chain_wait();
+    chain_release();
     const int ns = min(n_sel[b], m);
     const int32_t* idx_b = sel_index + (long long)b * m;
 

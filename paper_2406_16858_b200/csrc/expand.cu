@@ -388,8 +388,7 @@ expand_kernel(const float* __restrict__ draft_logits, long long batch_stride, in
     if (lane == 0 && warp < kScanWarps) s_count[warp] = 0;
     if (STREAM && threadIdx.x < kQueue) s_queue[threadIdx.x] = 0ull;
     __syncthreads();  // the only block-wide barrier before the segment's end
-    chain_wait();
-    chain_release();
+    // (which row and tiles this block serves is worked out before it waits for the preceding kernel)
     const int chunk = blockIdx.x % chunks;
     const int row = (blockIdx.x / chunks) % n_s;
     const int b = blockIdx.x / (chunks * n_s);
@@ -428,6 +427,8 @@ expand_kernel(const float* __restrict__ draft_logits, long long batch_stride, in
         slot_issue = slot_issue == kDepth - 1 ? 0 : slot_issue + 1;
     };
     float cur[NE], nxt[NE];
+    chain_wait();
+    chain_release();
     if (VEC) {
         issue_next();
         issue_next();
@@ -617,6 +618,8 @@ expand_kernel(const float* __restrict__ draft_logits, long long batch_stride, in
     }
     } else {
     // ===== selector warp (STREAM) ==========================================================================
+    chain_wait();
+    chain_release();
     unsigned long long top = 0ull;  // the segment's best keys so far, descending over the lanes
     int head = 0;
     const long long w0 = clock64();

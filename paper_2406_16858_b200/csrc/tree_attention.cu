@@ -547,8 +547,11 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
         len_early = kv_len[b_early], off_early = kv_off[b_early];
     }
     if (plan.setup_first) set_up();
-    chain_wait();
-    chain_release();  // the merge kernel of this call (or whatever follows) may be scheduled from here on
+    // (such a launch also works out which tiles and rows the block serves before it waits: below)
+    if (!early_len) {
+        chain_wait();
+        chain_release();  // the merge kernel of this call (or whatever follows) may be scheduled from here on
+    }
 
     int bid = PAIR ? blockIdx.x >> 1 : blockIdx.x;
     int split, rb, hk, b;
@@ -593,6 +596,10 @@ tree_attention_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_co
     // a split past the sequence's last tile (never merged), or a rejected sequence: both blocks of a
     // pair take the same decision
     const bool active = nt > 0 && rows_blk > 0;
+    if (early_len) {
+        chain_wait();
+        chain_release();
+    }
     if (!plan.setup_first) {
         if (!active) return;
         set_up();
@@ -1139,17 +1146,21 @@ tree_attention_merge_kernel(const int64_t* __restrict__ kv_off, const int32_t* _
     // first row's are read while the attention kernel is still running.
     int len_first = 0;
     long long off_first = 0;
-    if (row_first < total) {
-        const int b0 = (int)(row_first / ((long long)plan.M * Hkv));
-        len_first = kv_len[b0], off_first = kv_off[b0];
+    int pr = 0, hk = 0, b = 0;
+    auto decode = [&](long long row) {
+        pr = (int)(row % plan.M);
+        hk = (int)((row / plan.M) % Hkv);
+        b = (int)(row / ((long long)plan.M * Hkv));
+    };
+    if (row_first < total) {  // ... and so is the arithmetic that says which row that is
+        decode(row_first);
+        len_first = kv_len[b], off_first = kv_off[b];
     }
     chain_wait();  // the attention kernel's partials are complete
     chain_release();
     // a large batch is walked by a grid of a few blocks per SM: most rows need no merge
     for (long long row = row_first; row < total; row += warps) {
-        const int pr = (int)(row % plan.M);
-        const int hk = (int)((row / plan.M) % Hkv);
-        const int b = (int)(row / ((long long)plan.M * Hkv));
+        if (row != row_first) decode(row);
         const int L = row == row_first ? len_first : kv_len[b];
         if (!sequence_ok(L, row == row_first ? off_first : kv_off[b], m, max_kv_len, cache_rows)) continue;
         const int tiles = (L + m + kTK - 1) / kTK;
