@@ -306,7 +306,9 @@ __device__ __forceinline__ void tile_visibility(unsigned long long mlo, unsigned
 // One warp combines the partials of one packed query row `pr` of (sequence b, KV head hk) that was
 // computed in S_b > 1 splits: the lanes fetch the splits' (maximum, sum) pairs side by side, then
 // every lane owns DH/32 columns of the row.
-template <int DH>
+// PACKED: the fetched rows stay bf16 pairs until they are used - half the registers (62 against 116 per
+// thread in the merge kernel, four blocks per SM instead of two), a little more work behind the loads.
+template <int DH, bool PACKED = false>
 __device__ __forceinline__ void merge_row(const AttnPlan& plan, const AttnWs& ws, int b, int hk, int pr, int S_b,
                                           int m, int Hq, int Hkv, __nv_bfloat16* __restrict__ out,
                                           float* __restrict__ lse) {
@@ -328,19 +330,21 @@ __device__ __forceinline__ void merge_row(const AttnPlan& plan, const AttnWs& ws
     // (maximum, sum) pairs: neither address depends on the other's data.
     auto run = [&](auto width_tag) {
         constexpr int W = decltype(width_tag)::value;
-        float v[W][PER];
+        float v[PACKED ? 1 : W][PER];
+        uint2 vp[PACKED ? W : 1];
         auto fetch = [&](int s0, int s1, int n) {
 #pragma unroll
             for (int u = 0; u < W; ++u) {
                 const int sl = min(s1 + u, n - 1);  // clamped: a repeated row gets weight 0 below
                 const __nv_bfloat16* src = ws.o_part + (first + (size_t)(s0 + sl) * stride) * DH + lane * PER;
-                if (PER == 4) {
-                    const uint2 t = __ldcg(reinterpret_cast<const uint2*>(src));
-                    v[u][0] = __uint_as_float(t.x << 16), v[u][1] = __uint_as_float(t.x & 0xffff0000u);
-                    v[u][PER - 2] = __uint_as_float(t.y << 16), v[u][PER - 1] = __uint_as_float(t.y & 0xffff0000u);
+                uint2 t = make_uint2(0u, 0u);
+                if (PER == 4) t = __ldcg(reinterpret_cast<const uint2*>(src));
+                else t.x = __ldcg(reinterpret_cast<const uint32_t*>(src));
+                if (PACKED) {
+                    vp[u] = t;
                 } else {
-                    const uint32_t t = __ldcg(reinterpret_cast<const uint32_t*>(src));
-                    v[u][0] = __uint_as_float(t << 16), v[u][1] = __uint_as_float(t & 0xffff0000u);
+                    v[u][0] = __uint_as_float(t.x << 16), v[u][1] = __uint_as_float(t.x & 0xffff0000u);
+                    if (PER == 4) v[u][PER - 2] = __uint_as_float(t.y << 16), v[u][PER - 1] = __uint_as_float(t.y & 0xffff0000u);
                 }
             }
         };
@@ -364,8 +368,19 @@ __device__ __forceinline__ void merge_row(const AttnPlan& plan, const AttnWs& ws
                     float wu = __shfl_sync(0xffffffffu, w, min(s1 + u, 31));
                     if (s1 + u >= n) wu = 0.f;
                     // a split without visible keys leaves its partial row unwritten: never multiply it
+                    if (PACKED) {
+                        if (wu != 0.f) {
+                            acc[0] += __uint_as_float(vp[u].x << 16) * wu;
+                            acc[1] += __uint_as_float(vp[u].x & 0xffff0000u) * wu;
+                            if (PER == 4) {
+                                acc[PER - 2] += __uint_as_float(vp[u].y << 16) * wu;
+                                acc[PER - 1] += __uint_as_float(vp[u].y & 0xffff0000u) * wu;
+                            }
+                        }
+                    } else {
 #pragma unroll
-                    for (int e = 0; e < PER; ++e) acc[e] += wu != 0.f ? v[u][e] * wu : 0.f;
+                        for (int e = 0; e < PER; ++e) acc[e] += wu != 0.f ? v[u][e] * wu : 0.f;
+                    }
                 }
             }
         }
@@ -1133,7 +1148,7 @@ tree_attention_schedule_kernel(const int64_t* __restrict__ kv_off, const int32_t
 
 // One warp per output row of a sequence that used several splits (launches that do not merge inside
 // the attention kernel).
-template <int DH>
+template <int DH, bool PACKED>
 __global__ void __launch_bounds__(256)
 tree_attention_merge_kernel(const int64_t* __restrict__ kv_off, const int32_t* __restrict__ kv_len, int B, int m,
                             int Hq, int Hkv, long long cache_rows, int max_kv_len, AttnPlan plan, AttnWs ws, __nv_bfloat16* __restrict__ out,
@@ -1166,7 +1181,7 @@ tree_attention_merge_kernel(const int64_t* __restrict__ kv_off, const int32_t* _
         const int tiles = (L + m + kTK - 1) / kTK;
         const int S_b = (tiles + plan.per_split - 1) / plan.per_split;
         if (S_b <= 1) continue;  // the attention kernel wrote these rows itself
-        merge_row<DH>(plan, ws, b, hk, pr, S_b, m, Hq, Hkv, out, lse);
+        merge_row<DH, PACKED>(plan, ws, b, hk, pr, S_b, m, Hq, Hkv, out, lse);
     }
 }
 
@@ -1197,7 +1212,14 @@ static int launch_attention(const CUtensorMap& k_map, const CUtensorMap& v_map, 
         const long long warps = (long long)B * Hkv * plan.M;
         long long mblocks = (warps + 7) / 8;
         if (mblocks > 8LL * sm_count()) mblocks = 8LL * sm_count();
-        if (launch_chained(tree_attention_merge_kernel<DH>, dim3((unsigned)mblocks), dim3(256), 0, st, 1, kv_off, kv_len, B, m,
+        // Two of the merge kernel's blocks fit on an SM, four of its packed variant's.  A launch that two
+        // per SM can hold runs the first (LLaMA3-8B-shaped layer, 240 blocks: 16.7 us per layer against
+        // 17.1 packed and kept to two per SM, 17.8 four per SM: the blocks then sit four deep on the SMs
+        // the attention blocks left first); a larger one runs the packed variant so that it is resident
+        // at once (70B-shaped layer, 480 blocks: 32.7 -> 31.4 us per layer).
+        const bool packed = mblocks > 2LL * sm_count();
+        auto merge = packed ? tree_attention_merge_kernel<DH, true> : tree_attention_merge_kernel<DH, false>;
+        if (launch_chained(merge, dim3((unsigned)mblocks), dim3(256), 0, st, 1, kv_off, kv_len, B, m,
                            Hq, Hkv, cache_rows, max_kv_len, plan, ws, static_cast<__nv_bfloat16*>(out), lse) != EAGLE2_OK)
             return EAGLE2_ERR_CUDA;
     }
