@@ -325,97 +325,100 @@ __device__ __forceinline__ void expand_finish(int b, int V, int k, int D, int s,
     };
     // The usual shape - at most 320 segment winners per row - takes a path written for the block that
     // runs it once per launch with none of its instructions in the cache: plain loops, no sorting
-    // network.  A lane holds ten of the row's keys; the k-th largest lane maximum is a threshold that k
-    // keys reach; the keys at or above it (a few dozen) go to the warp's list in shared memory and are
-    // ranked there by counting.  The next row's keys are requested before this row's are looked at.
-    // Returns false (nothing written) when the list would overflow: ties, rows of equal logits.
-    constexpr int kCompactBatch = 10;
-    auto merge_row_compact = [&](int r, const unsigned long long (&cand)[kCompactBatch], double2 st0) -> bool {
-        const size_t p0 = ((size_t)b * n_s + r) * chunks;
-        int parent = s ? s_parent[r] : -1;
-        const double parent_value = s ? s_pvalue[r] : 0.0;
-        if (parent < -1) {
-            status |= EAGLE2_STATUS_BAD_TREE;
-            parent = (int)(s >= 2 ? (long long)k + (long long)(s - 2) * k * k : 0);
-        }
-        // log-sum-exp of the row from the chunk partials, in double
-        double mx = st0.x;
-        for (int c = lane + 32; c < chunks; c += 32) mx = fmax(mx, ws.stats[p0 + c].x);
-        mx = warp_max_f64(mx);
-        double sum = st0.x > -INFINITY ? st0.y * exp(st0.x - mx) : 0.0;
-        for (int c = lane + 32; c < chunks; c += 32) {
-            const double2 st = ws.stats[p0 + c];
-            if (st.x > -INFINITY) sum += st.y * exp(st.x - mx);
-        }
-        sum = warp_sum_f64(sum);
-        if (!(mx > -INFINITY)) status |= EAGLE2_STATUS_NONFINITE_LOGIT;
-        const double lse = mx + log(sum);
-        // threshold: the k-th largest of the lanes' best keys (0 when fewer than k lanes hold keys)
-        unsigned long long best = 0ull;
-#pragma unroll
-        for (int t = 0; t < kCompactBatch; ++t) best = cand[t] > best ? cand[t] : best;
-        int above = 0;
-#pragma unroll 8
-        for (int l = 0; l < 32; ++l) above += __shfl_sync(0xffffffffu, best, l) > best;
-        const unsigned long long thr = warp_max_u64(above == k - 1 ? best : 0ull);
-        // the keys that reach it, packed into the warp's list
-        unsigned long long* list = s_list[warp];
-        int n_c = 0;
-#pragma unroll
-        for (int t = 0; t < kCompactBatch; ++t) {
-            const bool in = cand[t] != 0ull && cand[t] >= thr;
-            const unsigned mask = __ballot_sync(0xffffffffu, in);
-            const int pos = n_c + __popc(mask & ((1u << lane) - 1u));
-            if (in && pos < kWarpList) list[pos] = cand[t];
-            n_c += __popc(mask);
-        }
-        if (n_c > kWarpList) return false;
-        __syncwarp();
-        // rank by counting (keys differ): the ranks below k are the row's children, best first
-#pragma unroll 1
-        for (int i = lane; i < n_c; i += 32) {
-            const unsigned long long mine = list[i];
-            int rank = 0;
-#pragma unroll 4
-            for (int j = 0; j < n_c; ++j) rank += list[j] > mine;
-            if (rank < k) {
-                const long long node = base + (long long)r * k + rank;
-                const double confidence = (double)key_value(mine) - lse;  // log c_i
-                const double v = parent_value + confidence;
-                tok[node] = (int32_t)key_index(mine);
-                par[node] = parent;
-                val[node] = v;
-                s_rank[r * k + rank] = order_code_f64(by_confidence ? confidence : v);
-            }
-        }
-        __syncwarp();
-        return n_c >= k;  // fewer keys than children (tiny vocabularies): the general path pads
-    };
+    // network.  Half a warp serves a row (the ten rows of a step on eight warps in one go): a lane holds
+    // twenty of the row's keys; the k-th largest lane maximum is a threshold that k keys reach; the keys
+    // at or above it (a few dozen) go to the half-warp's list in shared memory and are ranked there by
+    // counting.  all_ok turns false (and the general path redoes the step) when a list would overflow
+    // (ties, rows of equal logits) or a row has fewer keys than children (tiny vocabularies).
+    constexpr int kCompactBatch = 20, kHalfList = kWarpList / 2;
     bool compact_done = false;
-    if (warp < kScanWarps && keys_per_row <= 32 * kCompactBatch) {
-        unsigned long long cand[kCompactBatch], nxt[kCompactBatch];
-        double2 st0 = make_double2(-INFINITY, 0.0), st0_nxt = st0;
-        auto request = [&](int r, unsigned long long (&dst)[kCompactBatch], double2& st) {
-            const size_t p0 = ((size_t)b * n_s + r) * chunks;
+    if (warp < kScanWarps && keys_per_row <= 16 * kCompactBatch) {
+        const int hw = lane >> 4, hl = lane & 15;
+        auto half_max_u64 = [](unsigned long long v) {
 #pragma unroll
-            for (int t = 0; t < kCompactBatch; ++t)
-                dst[t] = lane + 32 * t < keys_per_row ? ws.keys[p0 * k + lane + 32 * t] : 0ull;
-            st = lane < chunks ? ws.stats[p0 + lane] : make_double2(-INFINITY, 0.0);
+            for (int o = 8; o > 0; o >>= 1) {
+                const unsigned long long other = __shfl_xor_sync(0xffffffffu, v, o);
+                v = other > v ? other : v;
+            }
+            return v;
         };
         bool all_ok = true;
-        if (warp < n_s) request(warp, cand, st0);
 #pragma unroll 1
-        for (int r = warp; r < n_s; r += kScanWarps) {
-            if (r + kScanWarps < n_s) request(r + kScanWarps, nxt, st0_nxt);
-            all_ok = merge_row_compact(r, cand, st0) && all_ok;
+        for (int r0 = 0; r0 < n_s; r0 += 2 * kScanWarps) {
+            const int r = r0 + warp * 2 + hw;
+            const bool valid = r < n_s;
+            const size_t p0 = ((size_t)b * n_s + (valid ? r : 0)) * chunks;
+            unsigned long long cand[kCompactBatch];
 #pragma unroll
-            for (int t = 0; t < kCompactBatch; ++t) cand[t] = nxt[t];
-            st0 = st0_nxt;
+            for (int t = 0; t < kCompactBatch; ++t)
+                cand[t] = (valid && hl + 16 * t < keys_per_row) ? ws.keys[p0 * k + hl + 16 * t] : 0ull;
+            // log-sum-exp of the row from the chunk partials, in double
+            double mx = -INFINITY;
+            if (valid)
+                for (int c = hl; c < chunks; c += 16) mx = fmax(mx, ws.stats[p0 + c].x);
+#pragma unroll
+            for (int o = 8; o > 0; o >>= 1) mx = fmax(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+            double sum = 0.0;
+            if (valid)
+                for (int c = hl; c < chunks; c += 16) {
+                    const double2 st = ws.stats[p0 + c];
+                    if (st.x > -INFINITY) sum += st.y * exp(st.x - mx);
+                }
+#pragma unroll
+            for (int o = 8; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+            if (valid && !(mx > -INFINITY)) status |= EAGLE2_STATUS_NONFINITE_LOGIT;
+            const double lse = mx + log(sum);
+            int parent = (s && valid) ? s_parent[r] : -1;
+            const double parent_value = (s && valid) ? s_pvalue[r] : 0.0;
+            if (parent < -1) {
+                status |= EAGLE2_STATUS_BAD_TREE;
+                parent = (int)(s >= 2 ? (long long)k + (long long)(s - 2) * k * k : 0);
+            }
+            // threshold: the k-th largest of the half-warp's lane maxima (0 when fewer than k lanes hold keys)
+            unsigned long long best = 0ull;
+#pragma unroll
+            for (int t = 0; t < kCompactBatch; ++t) best = cand[t] > best ? cand[t] : best;
+            int above = 0;
+#pragma unroll 8
+            for (int l = 0; l < 16; ++l) above += __shfl_sync(0xffffffffu, best, l, 16) > best;
+            const unsigned long long thr = half_max_u64(above == k - 1 ? best : 0ull);
+            // the keys that reach it, packed into the half-warp's list
+            unsigned long long* list = s_list[warp] + hw * kHalfList;
+            int n_c = 0;
+#pragma unroll
+            for (int t = 0; t < kCompactBatch; ++t) {
+                const bool in = cand[t] != 0ull && cand[t] >= thr;
+                const unsigned mask = (__ballot_sync(0xffffffffu, in) >> (hw * 16)) & 0xffffu;
+                const int pos = n_c + __popc(mask & ((1u << hl) - 1u));
+                if (in && pos < kHalfList) list[pos] = cand[t];
+                n_c += __popc(mask);
+            }
+            __syncwarp();
+            if (valid && (n_c > kHalfList || n_c < k)) all_ok = false;
+            const int n_l = min(n_c, kHalfList);
+            // rank by counting (keys differ): the ranks below k are the row's children, best first
+#pragma unroll 1
+            for (int i = hl; i < n_l; i += 16) {
+                const unsigned long long mine = list[i];
+                int rank = 0;
+#pragma unroll 4
+                for (int j = 0; j < n_l; ++j) rank += list[j] > mine;
+                if (valid && rank < k) {
+                    const long long node = base + (long long)r * k + rank;
+                    const double confidence = (double)key_value(mine) - lse;  // log c_i
+                    const double v = parent_value + confidence;
+                    tok[node] = (int32_t)key_index(mine);
+                    par[node] = parent;
+                    val[node] = v;
+                    s_rank[r * k + rank] = order_code_f64(by_confidence ? confidence : v);
+                }
+            }
+            __syncwarp();
         }
-        compact_done = all_ok;
+        compact_done = __all_sync(0xffffffffu, all_ok);
     }
     // every warp agrees on whether the general path has to redo the step (rare: ties, tiny vocabularies)
-    compact_done = __syncthreads_and(compact_done || warp >= kScanWarps) && keys_per_row <= 32 * kCompactBatch;
+    compact_done = __syncthreads_and(compact_done || warp >= kScanWarps) && keys_per_row <= 16 * kCompactBatch;
     if (!compact_done && warp < kScanWarps) {
         using std::integral_constant;
         if (n_s > kScanWarps && n_s <= 2 * kScanWarps && keys_per_row <= 32 * 10)
