@@ -326,7 +326,7 @@ __device__ __forceinline__ void expand_finish(int b, int V, int k, int D, int s,
     // The usual shape - at most 320 segment winners per row - takes a path written for the block that
     // runs it once per launch with none of its instructions in the cache: plain loops, no sorting
     // network.  Half a warp serves a row (the ten rows of a step on eight warps in one go): a lane holds
-    // twenty of the row's keys; the k-th largest lane maximum is a threshold that k keys reach; the keys
+    // twenty of the row's keys; the k-th largest of the maxima of 32 groups of ten is a threshold that k keys reach; the keys
     // at or above it (a few dozen) go to the half-warp's list in shared memory and are ranked there by
     // counting.  all_ok turns false (and the general path redoes the step) when a list would overflow
     // (ties, rows of equal logits) or a row has fewer keys than children (tiny vocabularies).
@@ -374,14 +374,25 @@ __device__ __forceinline__ void expand_finish(int b, int V, int k, int D, int s,
                 status |= EAGLE2_STATUS_BAD_TREE;
                 parent = (int)(s >= 2 ? (long long)k + (long long)(s - 2) * k * k : 0);
             }
-            // threshold: the k-th largest of the half-warp's lane maxima (0 when fewer than k lanes hold keys)
-            unsigned long long best = 0ull;
+            // threshold: the k-th largest of 32 group maxima, two groups of ten keys per lane (0 when fewer
+            // than k groups hold keys); with 32 groups a dozen keys reach it, with 16 several dozen would
+            unsigned long long best_a = 0ull, best_b = 0ull;
 #pragma unroll
-            for (int t = 0; t < kCompactBatch; ++t) best = cand[t] > best ? cand[t] : best;
-            int above = 0;
-#pragma unroll 8
-            for (int l = 0; l < 16; ++l) above += __shfl_sync(0xffffffffu, best, l, 16) > best;
-            const unsigned long long thr = half_max_u64(above == k - 1 ? best : 0ull);
+            for (int t = 0; t < kCompactBatch / 2; ++t) {
+                best_a = cand[t] > best_a ? cand[t] : best_a;
+                best_b = cand[kCompactBatch / 2 + t] > best_b ? cand[kCompactBatch / 2 + t] : best_b;
+            }
+            int above_a = 0, above_b = 0;
+#pragma unroll 4
+            for (int l = 0; l < 16; ++l) {
+                const unsigned long long oa = __shfl_sync(0xffffffffu, best_a, l, 16);
+                const unsigned long long ob = __shfl_sync(0xffffffffu, best_b, l, 16);
+                above_a += (oa > best_a) + (ob > best_a);
+                above_b += (oa > best_b) + (ob > best_b);
+            }
+            unsigned long long pick = above_a == k - 1 ? best_a : 0ull;
+            if (above_b == k - 1 && best_b > pick) pick = best_b;
+            const unsigned long long thr = half_max_u64(pick);
             // the keys that reach it, packed into the half-warp's list
             unsigned long long* list = s_list[warp] + hw * kHalfList;
             int n_c = 0;
