@@ -32,10 +32,10 @@ from workloads import get_config  # noqa: E402
 METRIC = "us_per_draft_tree_cycle"
 N_SETS = 4  # rotating logit sets: 4 x (draft + target rows) is larger than the 126 MB L2
 
-# DRAM bytes of one tree-attention call (attention kernel 17,595,907 + merge kernel 4,618,240; the
+# DRAM bytes of one tree-attention call (attention kernel 17,596,030 + merge kernel 4,618,880; the
 # merge's are the partial rows that ncu's cache flush between captured launches pushed out of L2), from
 # the ncu capture summarised under profiles/ (None: not captured for that workload)
-NCU_DRAM_BYTES_PER_LAUNCH = {"llama3_8b": 17595907 + 4618240}
+NCU_DRAM_BYTES_PER_LAUNCH = {"llama3_8b": 17596030 + 4618880}
 
 
 def _peaks():
